@@ -1,0 +1,174 @@
+/*
+ * bnn_b200 -- run-time path of Binarized Neural Networks on one NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Plain pointers and sizes only.
+ *
+ * Conventions (hold for every call unless a call says otherwise)
+ *  - Every function returns an int status: BNN_OK (0) or a negative BNN_ERR_* code.  Nothing
+ *    throws, aborts or exits.  Argument errors are reported before anything is launched.
+ *  - Data pointers are DEVICE pointers owned by the caller.  The library never frees, keeps or
+ *    reallocates them; they must stay valid until the work enqueued by the call has finished.
+ *    Pointers marked "host" are host pointers.
+ *  - Work is enqueued on the CUDA stream bound to the context and is asynchronous with respect
+ *    to the host.  A context may be used by one host thread at a time.
+ *  - A +-1 value is stored as one bit: bit 1 <-> +1, bit 0 <-> -1 (bit = (x >= 0), Eq. 1).
+ *    Element k of a row sits in 32-bit word k/32 at bit k%32 (least significant bit first);
+ *    a 64-bit word j is words 2j and 2j+1, so both word widths are the same bytes in memory
+ *    (Section 4: 32 binary variables concatenated per register).
+ *  - "Packed matrix R x K": R rows, each ceil(K/32) words, leading dimension ld_w words with
+ *    ld_w >= ceil(K/32) and ld_w % 4 == 0, base address 16-byte aligned (BNN_ERR_ALIGNMENT
+ *    otherwise).  Bits at positions >= K of the last word and words beyond ceil(K/32) are
+ *    padding: producers write them as 0, consumers ignore them whatever they hold.
+ *  - Sizes are int64_t.  A dimension of 0 is legal: the call is a no-op (M or N == 0) or yields
+ *    the empty sum 0 (K == 0).
+ */
+#ifndef BNN_B200_H
+#define BNN_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define BNN_API __attribute__((visibility("default")))
+#else
+#define BNN_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    BNN_OK = 0,
+    BNN_ERR_INVALID_ARG = -1,   /* NULL pointer, negative size, unknown enum value, ld too small   */
+    BNN_ERR_ALIGNMENT = -2,     /* base pointer or leading dimension breaks the alignment rule     */
+    BNN_ERR_WORKSPACE = -3,     /* workspace missing or too small                                   */
+    BNN_ERR_CUDA = -4,          /* a CUDA runtime call failed; see bnn_last_cuda_error()            */
+    BNN_ERR_DEVICE_STATUS = -5  /* a kernel reported an internal error through its status word      */
+};
+
+enum { BNN_F32 = 0, BNN_F16 = 1, BNN_I8 = 2 }; /* element type of bnn_pack_signs' source */
+
+typedef struct bnn_ctx bnn_ctx;
+
+/* Context = (device, stream, optional caller-owned workspace).  `cuda_stream` is a cudaStream_t
+ * (NULL = the legacy default stream).  The context owns no device memory. */
+BNN_API int bnn_create(bnn_ctx **out, int device, void *cuda_stream);
+BNN_API int bnn_destroy(bnn_ctx *ctx);
+BNN_API const char *bnn_status_string(int status);
+/* cudaError_t of the most recent failing CUDA call made through this context (0 if none). */
+BNN_API int bnn_last_cuda_error(const bnn_ctx *ctx);
+/* Lend `bytes` of device memory (256-byte aligned) to the context for calls that need scratch
+ * (bnn_mlp_forward, bnn_mlp_forward_host).  Pass NULL, 0 to take it back. */
+BNN_API int bnn_set_workspace(bnn_ctx *ctx, void *dptr, size_t bytes);
+/* Inner loop of the tiled kernels (results are identical): 0 = library default, 1 = one POPC per
+ * word (Eq. 8 as written), 2 = carry-save: a LOP3 full adder merges two XOR words before the POPC. */
+BNN_API int bnn_set_popc_variant(bnn_ctx *ctx, int variant);
+
+/* ---------------------------------------------------------------------------------------------
+ * Sign-pack (Eq. 1 followed by the 32-per-word concatenation of Section 4).
+ *   src        rows x cols elements of `dtype`, row-major, leading dimension src_ld elements.
+ *   pack_along 0: pack along cols -> dst is a packed matrix rows x cols   (e.g. A, activations)
+ *              1: pack along rows -> dst is a packed matrix cols x rows   (a K x N weight matrix
+ *                 becomes the N x K packed operand the GEMM calls expect)
+ *   word_bits  32 or 64 (same bytes; 64 additionally needs dst_ld_w even).
+ *   dst        packed matrix, leading dimension dst_ld_w words.  All padding is written as 0.
+ * bit = (x >= 0); both zeros give 1.  NaN is not a legal input.
+ */
+BNN_API int bnn_pack_signs(bnn_ctx *ctx, const void *src, int dtype, int64_t rows, int64_t cols, int64_t src_ld,
+                   int pack_along, int word_bits, uint32_t *dst, int64_t dst_ld_w);
+
+/* ---------------------------------------------------------------------------------------------
+ * Binary matrix product (Section 4, Eq. 8).  C[m][n] = sum_k A[m][k] * B[k][n] over +-1 values
+ *   = K - 2 * popcount(Ap[m] XOR Bp[n]).
+ *   Ap packed M x K (lda_w), Bp packed N x K (ldb_w: B is given transposed, K along words),
+ *   C  M x N int32 row-major, leading dimension ldc >= N elements.
+ */
+BNN_API int bnn_xnor_gemm(bnn_ctx *ctx, const uint32_t *Ap, int64_t lda_w, const uint32_t *Bp, int64_t ldb_w,
+                  int32_t *C, int64_t ldc, int64_t M, int64_t N, int64_t K);
+
+/* ---------------------------------------------------------------------------------------------
+ * Hidden layer (Algorithm 4, step 2): binary product fused with the BatchNorm-folded integer
+ * threshold, Sign (Eq. 1) and repacking.  out_bit[m][n] = (dot[m][n] >= thr[n]) XOR flip_bit[n].
+ *   Ap packed M x K, Wp packed N x K, thr N int32 (any value), flip packed 1 x N or NULL (all 0),
+ *   out packed M x N (ldo_w words; padding written as 0).  No int32 product is written.
+ */
+BNN_API int bnn_binary_dense(bnn_ctx *ctx, const uint32_t *Ap, int64_t lda_w, const uint32_t *Wp, int64_t ldw_w,
+                     const int32_t *thr, const uint32_t *flip, uint32_t *out, int64_t ldo_w, int64_t M,
+                     int64_t N, int64_t K);
+
+/* ---------------------------------------------------------------------------------------------
+ * First layer on 8-bit inputs (Section 1.6, Eq. 6-7; Algorithm 4, step 1):
+ *   s[m][n] = sum_i X[m][i] * w[i][n] = sum_{p=1..8} 2^(p-1) * (x^p[m] . w[:,n]),  x^p in {0,1}.
+ *   X  M x K uint8 row-major (ldx elements), Wp packed N x K.
+ *   out_sums (or NULL): M x N int32, leading dimension lds.
+ *   out_bits (or NULL): packed M x N, bit = (s >= thr[n]) XOR flip_bit[n]; thr is required then.
+ * At least one output must be given.
+ */
+BNN_API int bnn_first_layer_bitplanes(bnn_ctx *ctx, const uint8_t *X, int64_t ldx, const uint32_t *Wp, int64_t ldw_w,
+                              const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, int64_t ldo_w,
+                              int32_t *out_sums, int64_t lds, int64_t M, int64_t N, int64_t K);
+
+/* ---------------------------------------------------------------------------------------------
+ * Binary 3x3 convolution, stride 1, one pixel of padding, as an implicit GEMM (Section 3.3).
+ * A tap that falls outside the image contributes 0.  Optional 2x2 / stride-2 max-pooling of the
+ * integer sums, then bit = (sum >= thr[n]) XOR flip_bit[n].
+ *   act     binary input, NHWC, channels packed: [B][H][W][C_in/32] words (C_in % 32 == 0), or
+ *   act_u8  8-bit input for a first layer, NHWC [B][H][W][C_in] bytes, 9*C_in <= 32 (bit-planes);
+ *           exactly one of act / act_u8 is non-NULL.
+ *   Wp      [C_out][3][3][C_in/32] words for a binary input; for act_u8 one word per filter with
+ *           bit (tap*C_in + c), tap = 3*(dy+1) + (dx+1).
+ *   pool    0 or 1 (H and W must be even when 1).  Output height/width are H, W or H/2, W/2.
+ *   out_bits (or NULL) [B][Ho][Wo][ceil(C_out/32)] words; out_sums (or NULL) [B][Ho][Wo][C_out] int32
+ *           (pooled sums when pool == 1).  thr is required when out_bits is given.
+ */
+BNN_API int bnn_binary_conv2d(bnn_ctx *ctx, const uint32_t *act, const uint8_t *act_u8, int64_t B, int64_t H,
+                      int64_t W, int64_t C_in, const uint32_t *Wp, int64_t C_out, int pool,
+                      const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, int32_t *out_sums);
+
+/* ---------------------------------------------------------------------------------------------
+ * Whole MLP forward (Algorithm 4): first layer on 8-bit inputs, hidden binary layers, real-valued
+ * output layer  score = gamma * ((dot - mean) / sqrt(var + eps)) + beta  (evaluated in double,
+ * stored as float32).
+ */
+typedef struct {
+    const uint32_t *Wp;  /* packed N x K weights (device) */
+    int64_t ldw_w;
+    int64_t K, N;
+    const int32_t *thr;  /* hidden layers: N thresholds (device) */
+    const uint32_t *flip; /* hidden layers: packed 1 x N or NULL (device) */
+    const float *gamma, *beta, *mean, *var; /* output layer only: N floats each (device) */
+    double eps;                             /* output layer only */
+} bnn_layer_desc;
+
+typedef struct {
+    int32_t n_layers;             /* >= 2: first layer, hidden layers..., output layer */
+    const bnn_layer_desc *layers; /* host array of n_layers entries */
+} bnn_mlp_desc;
+
+/* Scratch bytes bnn_mlp_forward (host_io = 0) or bnn_mlp_forward_host (host_io = 1) need for `batch`. */
+BNN_API size_t bnn_mlp_workspace_bytes(const bnn_mlp_desc *m, int64_t batch, int host_io);
+/* X batch x K0 uint8 (device, ldx), scores batch x N_last float32 (device, lds).
+ * If `hidden_out` is not NULL it is a host array of n_layers-1 device pointers (entries may be NULL);
+ * hidden layer k's packed activations (batch x N_k, leading dimension ceil(N_k/128)*4 words)
+ * are also copied there.  Needs a workspace (BNN_ERR_WORKSPACE otherwise). */
+BNN_API int bnn_mlp_forward(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X, int64_t ldx, int64_t batch,
+                    float *scores, int64_t lds, uint32_t *const *hidden_out);
+/* Same with HOST input and output: X_host is copied to the device, scores are copied back, both on the
+ * context's stream (pinned host memory makes the copies asynchronous).  The caller synchronises. */
+BNN_API int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X_host, int64_t ldx,
+                         int64_t batch, float *scores_host, int64_t lds);
+
+/* ---------------------------------------------------------------------------------------------
+ * Host helper (not on the timed path): fold run-time BatchNorm followed by Sign,
+ *   Sign(gamma * ((x - mean) / sqrt(var + eps)) + beta)   evaluated in double for integer x,
+ * into the integer rule (x >= thr[n]) XOR flip_bit[n] that is exact for every integer |x| <= x_max.
+ * All pointers are HOST pointers; flip is packed 1 x n (ceil(n/32) words).
+ */
+BNN_API int bnn_fold_batchnorm(const float *gamma, const float *beta, const float *mean, const float *var, double eps,
+                       int64_t n, int64_t x_max, int32_t *thr, uint32_t *flip);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BNN_B200_H */

@@ -1,0 +1,240 @@
+"""ctypes binding of libbnn_b200.so: same names as the C ABI, argument marshalling only.
+
+Tensors are torch tensors that own device (or, where the C call says so, host) memory; this module
+passes their data pointers, leading dimensions and sizes and raises on a non-zero status.  No step of
+the method is computed here.  The library is loaded on first use; if it has not been built the call
+fails with an error -- there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, c_double, c_int, c_int32, c_int64, c_size_t, c_void_p
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbnn_b200.so")
+
+BNN_F32, BNN_F16, BNN_I8 = 0, 1, 2
+VARIANT_AUTO, VARIANT_PLAIN, VARIANT_CSA = 0, 1, 2
+
+EXPORTS = (
+    "bnn_create", "bnn_destroy", "bnn_status_string", "bnn_last_cuda_error", "bnn_set_workspace",
+    "bnn_set_popc_variant", "bnn_pack_signs", "bnn_xnor_gemm", "bnn_binary_dense", "bnn_first_layer_bitplanes",
+    "bnn_binary_conv2d", "bnn_mlp_workspace_bytes", "bnn_mlp_forward", "bnn_mlp_forward_host",
+    "bnn_fold_batchnorm",
+)
+
+
+class LayerDesc(Structure):
+    _fields_ = [("Wp", c_void_p), ("ldw_w", c_int64), ("K", c_int64), ("N", c_int64), ("thr", c_void_p),
+                ("flip", c_void_p), ("gamma", c_void_p), ("beta", c_void_p), ("mean", c_void_p), ("var", c_void_p),
+                ("eps", c_double)]
+
+
+class MlpDesc(Structure):
+    _fields_ = [("n_layers", c_int32), ("layers", POINTER(LayerDesc))]
+
+
+class BnnError(RuntimeError):
+    def __init__(self, status: int, what: str, cuda_error: int = 0):
+        self.status = status
+        self.cuda_error = cuda_error
+        msg = f"{what} failed: {status} ({_status_string(status)})"
+        if cuda_error:
+            msg += f", cudaError {cuda_error}"
+        super().__init__(msg)
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C library.  Raises if it has not been built (python -m paper_1602_02830_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_1602_02830_b200.build` "
+                               "(there is no CPU or PyTorch fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        i64, vp = c_int64, c_void_p
+        L.bnn_create.argtypes = [POINTER(vp), c_int, vp]
+        L.bnn_destroy.argtypes = [vp]
+        L.bnn_status_string.argtypes = [c_int]
+        L.bnn_status_string.restype = ctypes.c_char_p
+        L.bnn_last_cuda_error.argtypes = [vp]
+        L.bnn_set_workspace.argtypes = [vp, vp, c_size_t]
+        L.bnn_set_popc_variant.argtypes = [vp, c_int]
+        L.bnn_pack_signs.argtypes = [vp, vp, c_int, i64, i64, i64, c_int, c_int, vp, i64]
+        L.bnn_xnor_gemm.argtypes = [vp, vp, i64, vp, i64, vp, i64, i64, i64, i64]
+        L.bnn_binary_dense.argtypes = [vp, vp, i64, vp, i64, vp, vp, vp, i64, i64, i64, i64]
+        L.bnn_first_layer_bitplanes.argtypes = [vp, vp, i64, vp, i64, vp, vp, vp, i64, vp, i64, i64, i64, i64]
+        L.bnn_binary_conv2d.argtypes = [vp, vp, vp, i64, i64, i64, i64, vp, i64, c_int, vp, vp, vp, vp]
+        L.bnn_mlp_workspace_bytes.argtypes = [POINTER(MlpDesc), i64, c_int]
+        L.bnn_mlp_workspace_bytes.restype = c_size_t
+        L.bnn_mlp_forward.argtypes = [vp, POINTER(MlpDesc), vp, i64, i64, vp, i64, POINTER(vp)]
+        L.bnn_mlp_forward_host.argtypes = [vp, POINTER(MlpDesc), vp, i64, i64, vp, i64]
+        L.bnn_fold_batchnorm.argtypes = [vp, vp, vp, vp, c_double, i64, i64, vp, vp]
+        _lib = L
+    return _lib
+
+
+def _status_string(status: int) -> str:
+    try:
+        return lib().bnn_status_string(status).decode()
+    except Exception:  # pragma: no cover
+        return "?"
+
+
+def _ptr(t):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def words(k: int) -> int:
+    return (k + 31) // 32
+
+
+def packed_ld(k: int) -> int:
+    """Smallest legal leading dimension (in 32-bit words) of a packed matrix with k bits per row."""
+    return ((k + 127) // 128) * 4
+
+
+class Context:
+    """bnn_ctx bound to a device and to torch's current stream on it (or to an explicit stream)."""
+
+    def __init__(self, device: int = 0, stream: "torch.cuda.Stream | None" = None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("a CUDA device is required; the library has no CPU path")
+        self.device = device
+        self.stream = stream if stream is not None else torch.cuda.current_stream(device)
+        h = c_void_p()
+        st = lib().bnn_create(ctypes.byref(h), device, c_void_p(self.stream.cuda_stream))
+        if st:
+            raise BnnError(st, "bnn_create")
+        self._h = h
+        self._ws = None
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().bnn_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    def _ck(self, st: int, what: str):
+        if st:
+            raise BnnError(st, what, lib().bnn_last_cuda_error(self._h))
+
+    def empty(self, *shape, dtype=torch.int32):
+        return torch.empty(*shape, dtype=dtype, device=f"cuda:{self.device}")
+
+    # -- plumbing ------------------------------------------------------------------------------
+    def set_workspace(self, ws: "torch.Tensor | None"):
+        self._ws = ws
+        if ws is None:
+            self._ck(lib().bnn_set_workspace(self._h, None, 0), "bnn_set_workspace")
+        else:
+            self._ck(lib().bnn_set_workspace(self._h, _ptr(ws), ws.numel() * ws.element_size()), "bnn_set_workspace")
+
+    def set_popc_variant(self, variant: int):
+        self._ck(lib().bnn_set_popc_variant(self._h, variant), "bnn_set_popc_variant")
+
+    # -- calls, one per C entry point ----------------------------------------------------------------
+    def pack_signs(self, src: torch.Tensor, pack_along: int = 0, word_bits: int = 32, dst=None, dst_ld_w=None):
+        """src: 2-D tensor (float32 / float16 / int8), row-major.  Returns the packed int32 tensor."""
+        dtype = {torch.float32: BNN_F32, torch.float16: BNN_F16, torch.int8: BNN_I8}[src.dtype]
+        rows, cols = src.shape
+        assert src.stride(1) == 1 or cols <= 1
+        out_rows, out_k = (rows, cols) if pack_along == 0 else (cols, rows)
+        ld = dst_ld_w if dst_ld_w is not None else packed_ld(out_k)
+        if dst is None:
+            dst = self.empty(out_rows, ld)
+        self._ck(lib().bnn_pack_signs(self._h, _ptr(src), dtype, rows, cols, src.stride(0) if rows > 1 else max(cols, 1),
+                                      pack_along, word_bits, _ptr(dst), ld), "bnn_pack_signs")
+        return dst
+
+    def xnor_gemm(self, Ap, Bp, M, N, K, C=None, lda_w=None, ldb_w=None, ldc=None):
+        if C is None:
+            C = self.empty(M, N)
+        self._ck(lib().bnn_xnor_gemm(self._h, _ptr(Ap), lda_w if lda_w is not None else Ap.stride(0), _ptr(Bp),
+                                     ldb_w if ldb_w is not None else Bp.stride(0), _ptr(C),
+                                     ldc if ldc is not None else (C.stride(0) if C.dim() == 2 and M > 1 else max(N, 1)),
+                                     M, N, K), "bnn_xnor_gemm")
+        return C
+
+    def binary_dense(self, Ap, Wp, thr, flip, M, N, K, out=None, ldo_w=None):
+        ld = ldo_w if ldo_w is not None else packed_ld(N)
+        if out is None:
+            out = self.empty(M, ld)
+        self._ck(lib().bnn_binary_dense(self._h, _ptr(Ap), Ap.stride(0), _ptr(Wp), Wp.stride(0), _ptr(thr), _ptr(flip),
+                                        _ptr(out), ld, M, N, K), "bnn_binary_dense")
+        return out
+
+    def first_layer_bitplanes(self, X, Wp, M, N, K, thr=None, flip=None, want_bits=True, want_sums=False):
+        ld = packed_ld(N)
+        bits = self.empty(M, ld) if want_bits else None
+        sums = self.empty(M, N) if want_sums else None
+        self._ck(lib().bnn_first_layer_bitplanes(self._h, _ptr(X), X.stride(0) if M > 1 else max(K, 1), _ptr(Wp),
+                                                 Wp.stride(0), _ptr(thr), _ptr(flip), _ptr(bits), ld, _ptr(sums), N,
+                                                 M, N, K), "bnn_first_layer_bitplanes")
+        return bits, sums
+
+    def binary_conv2d(self, act, B, H, W, C_in, Wp, C_out, pool=False, thr=None, flip=None, want_bits=True,
+                      want_sums=False):
+        """act: packed int32 [B,H,W,C_in/32] or uint8 [B,H,W,C_in] (first layer)."""
+        Ho, Wo = (H // 2, W // 2) if pool else (H, W)
+        bits = self.empty(B, Ho, Wo, words(C_out)) if want_bits else None
+        sums = self.empty(B, Ho, Wo, C_out) if want_sums else None
+        is_u8 = act.dtype == torch.uint8
+        self._ck(lib().bnn_binary_conv2d(self._h, None if is_u8 else _ptr(act), _ptr(act) if is_u8 else None, B, H, W,
+                                         C_in, _ptr(Wp), C_out, int(pool), _ptr(thr), _ptr(flip), _ptr(bits),
+                                         _ptr(sums)), "bnn_binary_conv2d")
+        return bits, sums
+
+    def make_mlp_desc(self, layers):
+        """layers: list of dicts with Wp, K, N and thr/flip (hidden) or gamma/beta/mean/var/eps (last).
+        Returns (MlpDesc, keep-alive tuple)."""
+        arr = (LayerDesc * len(layers))()
+        for d, L in zip(arr, layers):
+            d.Wp = L["Wp"].data_ptr()
+            d.ldw_w = L["Wp"].stride(0)
+            d.K, d.N = L["K"], L["N"]
+            for name in ("thr", "flip", "gamma", "beta", "mean", "var"):
+                t = L.get(name)
+                setattr(d, name, t.data_ptr() if t is not None else None)
+            d.eps = float(L.get("eps", 0.0))
+        desc = MlpDesc(len(layers), arr)
+        return desc, (arr, layers)
+
+    def mlp_workspace_bytes(self, desc, batch: int, host_io: bool = False) -> int:
+        return int(lib().bnn_mlp_workspace_bytes(ctypes.byref(desc), batch, int(host_io)))
+
+    def mlp_forward(self, desc, X, batch, scores=None, hidden_out=None):
+        n_out = desc.layers[desc.n_layers - 1].N
+        if scores is None:
+            scores = self.empty(batch, n_out, dtype=torch.float32)
+        hp = None
+        if hidden_out is not None:
+            hp = (c_void_p * (desc.n_layers - 1))(*[t.data_ptr() if t is not None else None for t in hidden_out])
+        self._ck(lib().bnn_mlp_forward(self._h, ctypes.byref(desc), _ptr(X), X.stride(0) if batch > 1 else X.shape[-1],
+                                       batch, _ptr(scores), n_out, hp), "bnn_mlp_forward")
+        return scores
+
+    def mlp_forward_host(self, desc, X_host, batch, scores_host):
+        n_out = desc.layers[desc.n_layers - 1].N
+        self._ck(lib().bnn_mlp_forward_host(self._h, ctypes.byref(desc), _ptr(X_host), X_host.stride(0), batch,
+                                            _ptr(scores_host), n_out), "bnn_mlp_forward_host")
+        return scores_host
+
+
+def fold_batchnorm(gamma, beta, mean, var, eps: float, x_max: int):
+    """Host helper bnn_fold_batchnorm: float32 CPU tensors in, (thr int32[n], flip packed int32[ceil(n/32)]) out."""
+    n = gamma.numel()
+    g, b, m, v = (t.detach().to(torch.float32).contiguous().cpu() for t in (gamma, beta, mean, var))
+    thr = torch.empty(n, dtype=torch.int32)
+    flip = torch.zeros(words(n), dtype=torch.int32)
+    st = lib().bnn_fold_batchnorm(_ptr(g), _ptr(b), _ptr(m), _ptr(v), float(eps), n, int(x_max), _ptr(thr), _ptr(flip))
+    if st:
+        raise BnnError(st, "bnn_fold_batchnorm")
+    return thr, flip

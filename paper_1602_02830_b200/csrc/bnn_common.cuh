@@ -1,0 +1,57 @@
+// Shared host-side plumbing of the bnn_b200 library: context, status codes, argument checks.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "bnn_b200.h"
+
+struct bnn_ctx {
+    int device;
+    cudaStream_t stream;
+    void *ws;
+    size_t ws_bytes;
+    int last_cuda_error;
+    int sm_count;
+    int variant;   // inner-loop choice of the tiled kernel (0 auto, 1 plain popc, 2 carry-save)
+};
+
+#define BNN_CUDA_TRY(ctx, call)                              \
+    do {                                                     \
+        cudaError_t e__ = (call);                            \
+        if (e__ != cudaSuccess) {                            \
+            if (ctx) (ctx)->last_cuda_error = (int)e__;      \
+            return BNN_ERR_CUDA;                             \
+        }                                                    \
+    } while (0)
+
+static inline int bnn_check_launch(bnn_ctx *ctx) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        ctx->last_cuda_error = (int)e;
+        return BNN_ERR_CUDA;
+    }
+    return BNN_OK;
+}
+
+static inline int64_t bnn_words(int64_t k) { return (k + 31) / 32; }
+static inline bool bnn_aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// A packed matrix R x K with leading dimension ld_w: checks of the ABI's layout rule.
+static inline int bnn_check_packed(const void *p, int64_t ld_w, int64_t K, int64_t R) {
+    if (R == 0) return BNN_OK;
+    if (p == nullptr) return BNN_ERR_INVALID_ARG;
+    if (ld_w < bnn_words(K) || ld_w < 0) return BNN_ERR_INVALID_ARG;
+    if (!bnn_aligned16(p) || (ld_w % 4) != 0) return BNN_ERR_ALIGNMENT;
+    return BNN_OK;
+}
+
+// Keeps `ctx`'s device current for the duration of a call and restores the caller's device after.
+struct bnn_device_guard {
+    int prev = -1;
+    bool ok = true;
+    explicit bnn_device_guard(bnn_ctx *ctx) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != ctx->device && cudaSetDevice(ctx->device) != cudaSuccess) ok = false;
+    }
+    ~bnn_device_guard() { if (prev >= 0) cudaSetDevice(prev); }
+};

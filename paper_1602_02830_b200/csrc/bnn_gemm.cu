@@ -1,0 +1,247 @@
+// bnn_xnor_gemm, bnn_binary_dense, bnn_first_layer_bitplanes: host-side checks and kernel selection,
+// plus the "skinny" kernel used when one operand has at most 32 rows (batch 1..32, or the 10-way output layer).
+#include "bnn_common.cuh"
+#include "bnn_tile.cuh"
+#include "bnn_internal.cuh"
+
+using namespace bnn_tile;
+
+namespace {
+
+// ------------------------------------------------------------------------------------------------
+// Skinny product.  S (small operand, RS <= 32 rows) is kept in shared memory; every warp streams rows
+// of the large operand L (one 128-bit load per lane per 128 words) and forms the RS dot products of
+// that row.  One CTA covers 32 rows of L, so that a packed output word can be assembled.
+//   MODE 0: C[s][l] int32 and/or bits out[s][l/32]         (S = activations, L = weights)
+//   MODE 1: scores[l][s] = BatchNorm(dot) as float32        (S = output-layer weights, L = activations)
+struct SkinnyArgs {
+    const uint32_t *S; int64_t lds_w; int64_t RS;
+    const uint32_t *L; int64_t ldl_w; int64_t RL;
+    int64_t K;
+    int32_t *C; int64_t ldc;
+    uint32_t *out; int64_t ldo;
+    const int32_t *thr; const uint32_t *flip;
+    float *scores; int64_t ld_scores;
+    const float *gamma, *beta, *mean, *var; double eps;
+};
+
+template <int RSMAX, int MODE>
+__global__ void __launch_bounds__(256) k_skinny(const SkinnyArgs p) {
+    extern __shared__ __align__(16) uint32_t smem[];
+    const int64_t Kw = (p.K + 31) >> 5;
+    const int64_t Kw4 = (Kw + 3) & ~int64_t(3);
+    uint32_t *Ss = smem;                                           // [RS][Kw4]
+    int32_t *res = reinterpret_cast<int32_t *>(smem + p.RS * Kw4);  // [32][RSMAX]
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t tail_mask = (p.K & 31) ? ((1u << (p.K & 31)) - 1u) : 0xffffffffu;
+
+    for (int64_t e = tid; e < p.RS * (Kw4 >> 2); e += 256) {
+        const int64_t r = e / (Kw4 >> 2), q = e % (Kw4 >> 2);
+        const uint4 v = load_row_words(p.S + r * p.lds_w, true, 4 * q, Kw, tail_mask, true);
+        *reinterpret_cast<uint4 *>(Ss + r * Kw4 + 4 * q) = v;
+    }
+    __syncthreads();
+
+    const int64_t l0 = (int64_t)blockIdx.x * 32;
+#pragma unroll 1
+    for (int cc = 0; cc < 4; ++cc) {
+        const int lcol = warp * 4 + cc;
+        const int64_t l = l0 + lcol;
+        int32_t acc[RSMAX];
+#pragma unroll
+        for (int s = 0; s < RSMAX; ++s) acc[s] = 0;
+        if (l < p.RL) {
+            for (int64_t w4 = 4 * lane; w4 < Kw4; w4 += 128) {
+                const uint4 b = load_row_words(p.L + l * p.ldl_w, true, w4, Kw, tail_mask, true);
+#pragma unroll
+                for (int s = 0; s < RSMAX; ++s) {
+                    if (s < p.RS) {
+                        const uint4 a = *reinterpret_cast<const uint4 *>(Ss + s * Kw4 + w4);
+                        acc[s] += __popc(a.x ^ b.x) + __popc(a.y ^ b.y) + __popc(a.z ^ b.z) + __popc(a.w ^ b.w);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int s = 0; s < RSMAX; ++s) {
+            int32_t v = acc[s];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            if (lane == 0) res[lcol * RSMAX + s] = (int32_t)p.K - 2 * v;
+        }
+    }
+    __syncthreads();
+
+    if (MODE == 0) {
+        if (p.C) {
+            for (int e = tid; e < 32 * (int)p.RS; e += 256) {
+                const int s = e >> 5, lc = e & 31;
+                if (l0 + lc < p.RL) p.C[(int64_t)s * p.ldc + l0 + lc] = res[lc * RSMAX + s];
+            }
+        }
+        if (p.out) {
+            if (tid < p.RS) {
+                uint32_t word = 0u;
+                const uint32_t fw = p.flip ? p.flip[blockIdx.x] : 0u;
+                for (int lc = 0; lc < 32; ++lc) {
+                    if (l0 + lc < p.RL) {
+                        const uint32_t q = res[lc * RSMAX + tid] >= p.thr[l0 + lc];
+                        word |= ((q ^ (fw >> lc)) & 1u) << lc;
+                    }
+                }
+                p.out[(int64_t)tid * p.ldo + blockIdx.x] = word;
+            }
+            if (blockIdx.x == gridDim.x - 1) {   // padding words
+                const int64_t first_pad = (p.RL + 31) >> 5, npad = p.ldo - first_pad;
+                for (int64_t e = tid; e < p.RS * npad; e += 256) p.out[(e / npad) * p.ldo + first_pad + e % npad] = 0u;
+            }
+        }
+    } else {
+        for (int e = tid; e < 32 * (int)p.RS; e += 256) {
+            const int lc = e / (int)p.RS, s = e % (int)p.RS;
+            if (l0 + lc < p.RL) {
+                const double x = (double)res[lc * RSMAX + s];
+                const double xhat = (x - (double)p.mean[s]) / sqrt((double)p.var[s] + p.eps);
+                p.scores[(l0 + lc) * p.ld_scores + s] = (float)((double)p.gamma[s] * xhat + (double)p.beta[s]);
+            }
+        }
+    }
+}
+
+template <int MODE>
+int launch_skinny(bnn_ctx *ctx, const SkinnyArgs &a) {
+    const int64_t Kw4 = (bnn_words(a.K) + 3) & ~int64_t(3);
+    const int rsmax = a.RS <= 1 ? 1 : (a.RS <= 4 ? 4 : (a.RS <= 16 ? 16 : 32));
+    const size_t smem = (size_t)a.RS * Kw4 * 4 + (size_t)32 * rsmax * 4;
+    const unsigned grid = (unsigned)((a.RL + 31) / 32);
+#define BNN_SK(R)                                                                                              \
+    do {                                                                                                       \
+        if (smem > 48 * 1024)                                                                                  \
+            BNN_CUDA_TRY(ctx, cudaFuncSetAttribute(k_skinny<R, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                                   (int)smem));                                                \
+        k_skinny<R, MODE><<<grid, 256, smem, ctx->stream>>>(a);                                                \
+    } while (0)
+    switch (rsmax) {
+        case 1: BNN_SK(1); break;
+        case 4: BNN_SK(4); break;
+        case 16: BNN_SK(16); break;
+        default: BNN_SK(32); break;
+    }
+#undef BNN_SK
+    return bnn_check_launch(ctx);
+}
+
+bool skinny_fits(int64_t RS, int64_t K) {
+    const int64_t Kw4 = (bnn_words(K) + 3) & ~int64_t(3);
+    return RS >= 1 && RS <= 32 && (RS * Kw4 * 4 + 32 * 32 * 4) <= 200 * 1024;
+}
+
+template <int AKIND>
+int launch_tile(bnn_ctx *ctx, const Args &a, int variant) {
+    const int64_t t128 = ((a.M + 127) / 128) * ((a.N + BN - 1) / BN);
+    const int64_t t64 = ((a.M + 63) / 64) * ((a.N + BN - 1) / BN);
+    const bool big = t128 >= 2 * (int64_t)ctx->sm_count;
+    const int64_t tiles = big ? t128 : t64;
+    if (tiles > 0x7fffffff) return BNN_ERR_INVALID_ARG;
+    const bool csa = (AKIND != A_PLANES) && (variant != BNN_VARIANT_PLAIN);
+    if (AKIND == A_PLANES) {
+        if (big) k_bit_tile<8, A_PLANES, false><<<(unsigned)tiles, 256, 0, ctx->stream>>>(a);
+        else k_bit_tile<4, A_PLANES, false><<<(unsigned)tiles, 128, 0, ctx->stream>>>(a);
+    } else {
+        constexpr int AK = (AKIND == A_PLANES) ? A_PACKED : AKIND;
+        if (big && csa) k_bit_tile<8, AK, true><<<(unsigned)tiles, 256, 0, ctx->stream>>>(a);
+        else if (big) k_bit_tile<8, AK, false><<<(unsigned)tiles, 256, 0, ctx->stream>>>(a);
+        else if (csa) k_bit_tile<4, AK, true><<<(unsigned)tiles, 128, 0, ctx->stream>>>(a);
+        else k_bit_tile<4, AK, false><<<(unsigned)tiles, 128, 0, ctx->stream>>>(a);
+    }
+    return bnn_check_launch(ctx);
+}
+
+}  // namespace
+
+// Used by bnn_conv.cu and bnn_mlp.cu.
+int bnn_launch_tile_packed(bnn_ctx *ctx, const Args &a) { return launch_tile<A_PACKED>(ctx, a, ctx_variant(ctx)); }
+int bnn_launch_tile_conv(bnn_ctx *ctx, const Args &a) { return launch_tile<A_CONV>(ctx, a, ctx_variant(ctx)); }
+int bnn_launch_tile_planes(bnn_ctx *ctx, const Args &a) { return launch_tile<A_PLANES>(ctx, a, ctx_variant(ctx)); }
+
+int bnn_output_scores(bnn_ctx *ctx, const uint32_t *Ap, int64_t lda_w, const uint32_t *Wp, int64_t ldw_w,
+                      const float *gamma, const float *beta, const float *mean, const float *var, double eps,
+                      float *scores, int64_t lds, int64_t M, int64_t N, int64_t K) {
+    if (M == 0 || N == 0) return BNN_OK;
+    if (!skinny_fits(N, K)) return BNN_ERR_INVALID_ARG;
+    SkinnyArgs s{};
+    s.S = Wp; s.lds_w = ldw_w; s.RS = N;
+    s.L = Ap; s.ldl_w = lda_w; s.RL = M;
+    s.K = K;
+    s.scores = scores; s.ld_scores = lds;
+    s.gamma = gamma; s.beta = beta; s.mean = mean; s.var = var; s.eps = eps;
+    return launch_skinny<1>(ctx, s);
+}
+
+static int gemm_like(bnn_ctx *ctx, const uint32_t *Ap, int64_t lda_w, const uint32_t *Bp, int64_t ldb_w, int32_t *C,
+                     int64_t ldc, const int32_t *thr, const uint32_t *flip, uint32_t *out, int64_t ldo_w, int64_t M,
+                     int64_t N, int64_t K) {
+    if (!ctx || M < 0 || N < 0 || K < 0 || K > 0x3fffffff) return BNN_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return BNN_OK;
+    if (int st = bnn_check_packed(Ap, lda_w, K, K ? M : 0)) return st;
+    if (int st = bnn_check_packed(Bp, ldb_w, K, K ? N : 0)) return st;
+    if (C) {
+        if (ldc < N) return BNN_ERR_INVALID_ARG;
+    }
+    if (out) {
+        if (!thr) return BNN_ERR_INVALID_ARG;
+        if (int st = bnn_check_packed(out, ldo_w, N, M)) return st;
+    }
+    if (!C && !out) return BNN_ERR_INVALID_ARG;
+    bnn_device_guard guard(ctx);
+    if (!guard.ok) return BNN_ERR_CUDA;
+    if (M <= 32 && skinny_fits(M, K)) {
+        SkinnyArgs s{};
+        s.S = Ap; s.lds_w = lda_w; s.RS = M;
+        s.L = Bp; s.ldl_w = ldb_w; s.RL = N;
+        s.K = K;
+        s.C = C; s.ldc = ldc; s.out = out; s.ldo = ldo_w; s.thr = thr; s.flip = flip;
+        return launch_skinny<0>(ctx, s);
+    }
+    Args a{};
+    a.A = Ap; a.lda = lda_w; a.B = Bp; a.ldb = ldb_w;
+    a.M = M; a.N = N; a.K = K;
+    a.C = C; a.ldc = ldc; a.out = out; a.ldo = ldo_w; a.thr = thr; a.flip = flip;
+    return bnn_launch_tile_packed(ctx, a);
+}
+
+extern "C" int bnn_xnor_gemm(bnn_ctx *ctx, const uint32_t *Ap, int64_t lda_w, const uint32_t *Bp, int64_t ldb_w,
+                             int32_t *C, int64_t ldc, int64_t M, int64_t N, int64_t K) {
+    if (!C && M > 0 && N > 0) return BNN_ERR_INVALID_ARG;
+    return gemm_like(ctx, Ap, lda_w, Bp, ldb_w, C, ldc, nullptr, nullptr, nullptr, 0, M, N, K);
+}
+
+extern "C" int bnn_binary_dense(bnn_ctx *ctx, const uint32_t *Ap, int64_t lda_w, const uint32_t *Wp, int64_t ldw_w,
+                                const int32_t *thr, const uint32_t *flip, uint32_t *out, int64_t ldo_w, int64_t M,
+                                int64_t N, int64_t K) {
+    if (!out && M > 0 && N > 0) return BNN_ERR_INVALID_ARG;
+    return gemm_like(ctx, Ap, lda_w, Wp, ldw_w, nullptr, 0, thr, flip, out, ldo_w, M, N, K);
+}
+
+extern "C" int bnn_first_layer_bitplanes(bnn_ctx *ctx, const uint8_t *X, int64_t ldx, const uint32_t *Wp,
+                                         int64_t ldw_w, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits,
+                                         int64_t ldo_w, int32_t *out_sums, int64_t lds, int64_t M, int64_t N,
+                                         int64_t K) {
+    if (!ctx || M < 0 || N < 0 || K < 0 || K > (0x7fffffff / 255)) return BNN_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return BNN_OK;
+    if (!out_bits && !out_sums) return BNN_ERR_INVALID_ARG;
+    if (K > 0 && (!X || ldx < K)) return BNN_ERR_INVALID_ARG;
+    if (int st = bnn_check_packed(Wp, ldw_w, K, K ? N : 0)) return st;
+    if (out_sums && lds < N) return BNN_ERR_INVALID_ARG;
+    if (out_bits) {
+        if (!thr) return BNN_ERR_INVALID_ARG;
+        if (int st = bnn_check_packed(out_bits, ldo_w, N, M)) return st;
+    }
+    bnn_device_guard guard(ctx);
+    if (!guard.ok) return BNN_ERR_CUDA;
+    Args a{};
+    a.X = X; a.ldx = ldx; a.B = Wp; a.ldb = ldw_w;
+    a.M = M; a.N = N; a.K = K;
+    a.C = out_sums; a.ldc = lds; a.out = out_bits; a.ldo = ldo_w; a.thr = thr; a.flip = flip;
+    return bnn_launch_tile_planes(ctx, a);
+}

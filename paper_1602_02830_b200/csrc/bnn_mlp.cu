@@ -1,0 +1,102 @@
+// bnn_mlp_forward: Algorithm 4 ("Running a BNN") as a sequence of stream-ordered launches:
+// bit-plane first layer -> fused binary dense layers -> real-valued output layer.
+#include "bnn_internal.cuh"
+
+namespace {
+
+inline int64_t act_ld(int64_t n) { return ((n + 127) / 128) * 4; }   // packed leading dimension, multiple of 4 words
+inline size_t round256(size_t b) { return (b + 255) & ~size_t(255); }
+
+int check_desc(const bnn_mlp_desc *m) {
+    if (!m || m->n_layers < 2 || !m->layers) return BNN_ERR_INVALID_ARG;
+    for (int k = 0; k < m->n_layers; ++k) {
+        const bnn_layer_desc &L = m->layers[k];
+        if (L.K <= 0 || L.N <= 0 || !L.Wp) return BNN_ERR_INVALID_ARG;
+        if (k > 0 && L.K != m->layers[k - 1].N) return BNN_ERR_INVALID_ARG;
+        if (k < m->n_layers - 1) {
+            if (!L.thr) return BNN_ERR_INVALID_ARG;
+        } else {
+            if (!L.gamma || !L.beta || !L.mean || !L.var) return BNN_ERR_INVALID_ARG;
+            if (L.N > 32) return BNN_ERR_INVALID_ARG;   // output layer runs on the skinny kernel
+        }
+    }
+    return BNN_OK;
+}
+
+size_t act_bytes(const bnn_mlp_desc *m, int64_t batch) {
+    int64_t widest = 0;
+    for (int k = 0; k < m->n_layers - 1; ++k) widest = m->layers[k].N > widest ? m->layers[k].N : widest;
+    return round256((size_t)batch * act_ld(widest) * 4);
+}
+
+int forward_device(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X, int64_t ldx, int64_t batch, float *scores,
+                   int64_t lds, uint32_t *const *hidden_out, char *ws) {
+    const size_t ab = act_bytes(m, batch);
+    uint32_t *bufs[2] = {reinterpret_cast<uint32_t *>(ws), reinterpret_cast<uint32_t *>(ws + ab)};
+    const int L = m->n_layers;
+    const uint32_t *cur = nullptr;
+    for (int k = 0; k < L - 1; ++k) {
+        const bnn_layer_desc &D = m->layers[k];
+        uint32_t *dst = bufs[k & 1];
+        const int64_t ldo = act_ld(D.N);
+        int st;
+        if (k == 0)
+            st = bnn_first_layer_bitplanes(ctx, X, ldx, D.Wp, D.ldw_w, D.thr, D.flip, dst, ldo, nullptr, 0, batch, D.N, D.K);
+        else
+            st = bnn_binary_dense(ctx, cur, act_ld(D.K), D.Wp, D.ldw_w, D.thr, D.flip, dst, ldo, batch, D.N, D.K);
+        if (st) return st;
+        if (hidden_out && hidden_out[k])
+            BNN_CUDA_TRY(ctx, cudaMemcpyAsync(hidden_out[k], dst, (size_t)batch * ldo * 4, cudaMemcpyDeviceToDevice,
+                                              ctx->stream));
+        cur = dst;
+    }
+    const bnn_layer_desc &O = m->layers[L - 1];
+    return bnn_output_scores(ctx, cur, act_ld(O.K), O.Wp, O.ldw_w, O.gamma, O.beta, O.mean, O.var, O.eps, scores, lds,
+                             batch, O.N, O.K);
+}
+
+}  // namespace
+
+extern "C" size_t bnn_mlp_workspace_bytes(const bnn_mlp_desc *m, int64_t batch, int host_io) {
+    if (check_desc(m) != BNN_OK || batch <= 0) return 0;
+    size_t b = 2 * act_bytes(m, batch);
+    if (host_io) {
+        b += round256((size_t)batch * m->layers[0].K);                        // staged input
+        b += round256((size_t)batch * m->layers[m->n_layers - 1].N * 4);      // staged scores
+    }
+    return b;
+}
+
+extern "C" int bnn_mlp_forward(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X, int64_t ldx, int64_t batch,
+                               float *scores, int64_t lds, uint32_t *const *hidden_out) {
+    if (!ctx || batch < 0) return BNN_ERR_INVALID_ARG;
+    if (int st = check_desc(m)) return st;
+    if (batch == 0) return BNN_OK;
+    if (!X || !scores || ldx < m->layers[0].K || lds < m->layers[m->n_layers - 1].N) return BNN_ERR_INVALID_ARG;
+    if (!ctx->ws || ctx->ws_bytes < bnn_mlp_workspace_bytes(m, batch, 0)) return BNN_ERR_WORKSPACE;
+    bnn_device_guard guard(ctx);
+    if (!guard.ok) return BNN_ERR_CUDA;
+    return forward_device(ctx, m, X, ldx, batch, scores, lds, hidden_out, static_cast<char *>(ctx->ws));
+}
+
+extern "C" int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X_host, int64_t ldx,
+                                    int64_t batch, float *scores_host, int64_t lds) {
+    if (!ctx || batch < 0) return BNN_ERR_INVALID_ARG;
+    if (int st = check_desc(m)) return st;
+    if (batch == 0) return BNN_OK;
+    const int64_t K0 = m->layers[0].K, NL = m->layers[m->n_layers - 1].N;
+    if (!X_host || !scores_host || ldx < K0 || lds < NL) return BNN_ERR_INVALID_ARG;
+    if (!ctx->ws || ctx->ws_bytes < bnn_mlp_workspace_bytes(m, batch, 1)) return BNN_ERR_WORKSPACE;
+    bnn_device_guard guard(ctx);
+    if (!guard.ok) return BNN_ERR_CUDA;
+    char *ws = static_cast<char *>(ctx->ws);
+    const size_t ab = act_bytes(m, batch);
+    uint8_t *Xd = reinterpret_cast<uint8_t *>(ws + 2 * ab);
+    float *Sd = reinterpret_cast<float *>(ws + 2 * ab + round256((size_t)batch * K0));
+    BNN_CUDA_TRY(ctx, cudaMemcpy2DAsync(Xd, (size_t)K0, X_host, (size_t)ldx, (size_t)K0, (size_t)batch,
+                                        cudaMemcpyHostToDevice, ctx->stream));
+    if (int st = forward_device(ctx, m, Xd, K0, batch, Sd, NL, nullptr, ws)) return st;
+    BNN_CUDA_TRY(ctx, cudaMemcpy2DAsync(scores_host, (size_t)lds * 4, Sd, (size_t)NL * 4, (size_t)NL * 4, (size_t)batch,
+                                        cudaMemcpyDeviceToHost, ctx->stream));
+    return BNN_OK;
+}

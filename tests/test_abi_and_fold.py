@@ -1,0 +1,107 @@
+"""CPU-side checks of the product's boundary: the shared library builds, loads and exports every function
+the header declares; status strings; and the host helper that folds BatchNorm + Sign into an integer
+threshold, compared with the oracle's double-precision Sign(BatchNorm(x)) over every integer x."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1602_02830_b200 import binding, build, workloads as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.lib()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "bnn_b200.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(bnn_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_function(lib):
+    names = declared_functions()
+    assert len(names) >= 14
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in the header but not exported"
+    assert set(binding.EXPORTS) <= set(names)
+
+
+def test_status_strings(lib):
+    assert lib.bnn_status_string(0) == b"ok"
+    seen = {lib.bnn_status_string(s) for s in range(-5, 1)}
+    assert len(seen) == 6
+
+
+def test_host_argument_errors_need_no_gpu(lib):
+    # NULL context / NULL output are rejected before any CUDA call
+    assert lib.bnn_destroy(None) == -1
+    assert lib.bnn_set_popc_variant(None, 0) == -1
+    assert lib.bnn_xnor_gemm(None, None, 0, None, 0, None, 0, 1, 1, 1) == -1
+    assert lib.bnn_fold_batchnorm(None, None, None, None, 0.0, 4, 10, None, None) == -1
+    assert lib.bnn_fold_batchnorm(None, None, None, None, 0.0, 0, 10, None, None) == 0
+
+
+def _fold_matches_oracle(bn, x_max):
+    thr, flip = binding.fold_batchnorm(*(torch.from_numpy(bn[k]) for k in ("gamma", "beta", "mean", "var")),
+                                       bn["eps"], x_max)
+    n = bn["gamma"].size
+    xs = np.arange(-x_max, x_max + 1, dtype=np.int32)
+    S = np.repeat(xs[:, None], n, axis=1)
+    want = oracle.sign_batchnorm(S, bn)                                   # double-precision definition
+    f = np.array([(int(flip[c // 32]) >> (c % 32)) & 1 for c in range(n)], dtype=np.uint8)
+    got = oracle.threshold(S, thr.numpy(), f)                             # integer rule with the folded values
+    assert np.array_equal(got, want)
+    assert thr.min() >= -x_max and thr.max() <= x_max + 1
+    return thr.numpy(), f
+
+
+def test_fold_batchnorm_random_channels():
+    rng = np.random.default_rng(5)
+    for K in (27, 784, 4096):
+        _fold_matches_oracle(wl.batchnorm_params(rng, 96, K), K)
+
+
+def test_fold_batchnorm_adversarial_channels():
+    g = np.array([1, -1, 0, 0, 0, 2, -2, 1, -1, 1e-30, -1e-30, 1, -1, 3, 0.5, -0.5], np.float32)
+    b = np.array([0, 0, -1, 0, 1, 4, 4, 1e6, 1e6, 0, 0, -1e6, -1e6, -7.5, 0.25, 0.25], np.float32)
+    m = np.array([0, 0, 0, 0, 0, 3, 3, 0, 0, 5, 5, 0, 0, 2.5, -3, -3], np.float32)
+    v = np.array([1, 1, 1, 1, 1, 4, 4, 1, 1, 1, 1, 1, 1, 9, 0.25, 0.25], np.float32)
+    bn = {"gamma": g, "beta": b, "mean": m, "var": v, "eps": 0.0}
+    thr, f = _fold_matches_oracle(bn, 40)
+    assert thr[0] == 0 and f[0] == 0            # Sign(x): tie at 0 -> +1
+    assert thr[1] == 1 and f[1] == 1            # Sign(-x): +1 iff x <= 0
+    assert (thr[2], f[2]) == (-40, 1)           # gamma = 0, beta < 0 -> always -1
+    assert (thr[3], f[3]) == (-40, 0)           # gamma = 0, beta = 0 -> always +1
+    assert (thr[7], f[7]) == (-40, 0) and (thr[11], f[11]) == (41, 0)     # saturated
+    assert (thr[8], f[8]) == (41, 1) and (thr[12], f[12]) == (-40, 1)
+    _fold_matches_oracle({**bn, "eps": 1e-4}, 40)
+
+
+def test_fold_rejects_bad_variance():
+    one = torch.ones(1)
+    with pytest.raises(binding.BnnError):
+        binding.fold_batchnorm(one, one, one, -one, 0.0, 10)
+
+
+def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "missing.so"))
+    with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
+        binding.lib()
+
+
+def test_test_side_packer_roundtrip():
+    from util import np_pack_pm1, np_unpack_pm1, padding_is_zero
+    x = wl.pm1(np.random.default_rng(0), (5, 70))
+    p = np_pack_pm1(x, 4)
+    assert p.shape == (5, 4) and np.array_equal(np_unpack_pm1(p, 70), x) and padding_is_zero(p, 70)
+    assert np_pack_pm1(np.array([[1, -1, 1]]))[0, 0] == 0b101
