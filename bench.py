@@ -1,0 +1,328 @@
+#!/usr/bin/env python
+"""Benchmark of the BNN run-time path on B200.
+
+One step = one forward pass of the MNIST-shaped BNN MLP (Algorithm 4) over a batch of 10000 synthetic
+images: bit-plane first layer, two fused binary 4096x4096 layers, real-valued 10-way output layer.
+`value` is images/s with the batch resident in HBM; `e2e` is the same through bnn_mlp_forward_host
+with pinned HOST buffers (copies inside the timed region).  The line also carries the binary-GEMM
+throughput (8192^3, Tbit-op/s), the roofline of the dominant kernel, and the CPU oracle timed on the
+host cores (`cpu_baseline`).  `--impl reference` times the oracle alone.
+
+N > 1 (under torchrun): every rank runs its own batch (independent rows, no data-path collective);
+time is the max over ranks and value the total images / that time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+BATCH = 10000
+SIZES = (784, 4096, 4096, 4096, 10)
+SEED = 1
+METRIC = "bnn_mlp_images_per_s"
+UNIT = "images/s"
+# Plain popc roofline: SMs x POPC lanes/clk/SM x 32 bit-MACs x 2 ops x max SM clock.
+POPC_PER_CLK_PER_SM = 16
+L2_FLUSH_BYTES = 256 << 20
+
+
+def popc_words_mlp(batch, sizes):
+    """popc-words (one 32-bit XOR/AND + POPC in the plain formulation) of one forward pass."""
+    w = 8 * batch * sizes[1] * ((sizes[0] + 31) // 32)
+    for k in range(1, len(sizes) - 1):
+        w += batch * sizes[k + 1] * ((sizes[k] + 31) // 32)
+    return w
+
+
+def bit_ops_mlp(batch, sizes):
+    """2 x bit-MACs of one forward pass, counting true K bits (8 planes for the first layer)."""
+    ops = 2 * 8 * batch * sizes[0] * sizes[1]
+    for k in range(1, len(sizes) - 1):
+        ops += 2 * batch * sizes[k] * sizes[k + 1]
+    return ops
+
+
+class ClockSampler:
+    """nvidia-smi sampling of SM clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, pw, reasons = [], [], [], set()
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); pw.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = [s for s, p in zip(sm, pw) if p >= 0.5 * max(pw)] or sm
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(mx), "power_w_max": max(pw),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def time_oracle_mlp(case, sample, repeats=1):
+    import oracle
+    oracle.build()
+    X = case["X"][:sample]
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        oracle.mlp_forward(X, case["weights"], case["bns"])
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return best, oracle.host_threads()
+
+
+def run_reference(args):
+    """The CPU oracle as it stands, on the host cores: each step is the MLP forward on a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from paper_1602_02830_b200 import workloads as wl
+    case = wl.mlp_case(batch=BATCH, sizes=SIZES, seed=SEED)
+    sample = 1000
+    for _ in range(max(args.warmup, 1)):
+        time_oracle_mlp(case, min(sample, 200))
+    times = []
+    cores = 0
+    for _ in range(args.steps):
+        dt, cores = time_oracle_mlp(case, sample)
+        times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    value = sample / (ms / 1e3)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int32", "data": "synthetic",
+            "config": {"workload": "MNIST-shaped BNN MLP 784-4096-4096-4096-10, seed 1; each step = %d of the 10000 images" % sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": "%d images per step, %d steps" % (sample, args.steps)},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--variant", type=int, default=0, help="tiled-kernel inner loop: 0 default, 1 plain popc, 2 carry-save")
+    ap.add_argument("--no-extras", action="store_true", help="skip the GEMM / ConvNet side measurements and the CPU baseline")
+    ap.add_argument("--gemm-size", type=int, default=8192)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    args.warmup = max(args.warmup, 3)
+
+    import torch
+    import torch.distributed as dist
+    from paper_1602_02830_b200 import binding, build, nets, workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    dev = f"cuda:{local}"
+    stream = torch.cuda.current_stream(local)
+    ctx = binding.Context(local, stream)
+    ctx.set_popc_variant(args.variant)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- workload: every rank draws the same network; rank r gets its own batch of images
+    case = wl.mlp_case(batch=BATCH, sizes=SIZES, seed=SEED)
+    if rank > 0:
+        case["X"] = wl.u8(np.random.default_rng([SEED, rank]), (BATCH, SIZES[0]))
+    net = nets.prepare_mlp(ctx, case["weights"], case["bns"])
+    desc = net["desc"]
+    ws = torch.empty(ctx.mlp_workspace_bytes(desc, BATCH, True), dtype=torch.uint8, device=dev)
+    ctx.set_workspace(ws)
+    X = torch.from_numpy(case["X"]).to(dev)
+    scores = torch.empty(BATCH, SIZES[-1], dtype=torch.float32, device=dev)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    launches_per_step = len(SIZES) - 1
+
+    def timed_steps(fn, steps, warmup):
+        """CUDA events on the launch stream around each step; L2 flushed (untimed) before each step."""
+        for _ in range(warmup):
+            flush.fill_(1)
+            fn()
+        sync_all()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, b in ev:
+            flush.fill_(1)
+            a.record(stream)
+            fn()
+            b.record(stream)
+        sync_all()
+        return [a.elapsed_time(b) for a, b in ev]
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.start()
+    times = timed_steps(lambda: ctx.mlp_forward(desc, X, BATCH, scores=scores), args.steps, args.warmup)
+    total_ms = sum(times)
+
+    # ---- end to end: pinned host buffers, copies inside the timed region
+    Xh = torch.from_numpy(case["X"]).pin_memory()
+    Sh = torch.empty(BATCH, SIZES[-1], dtype=torch.float32).pin_memory()
+    e2e_times = timed_steps(lambda: ctx.mlp_forward_host(desc, Xh, BATCH, Sh), args.steps, args.warmup)
+    e2e_total_ms = sum(e2e_times)
+
+    # ---- dominant kernel of the step, timed alone on the same stream: the fused 4096x4096 binary dense layer
+    hid = net["layers"][1]
+    act_in = torch.randint(-2**31, 2**31 - 1, (BATCH, binding.packed_ld(SIZES[1])), dtype=torch.int32, device=dev)
+    act_out = torch.empty(BATCH, binding.packed_ld(SIZES[2]), dtype=torch.int32, device=dev)
+    dense_times = timed_steps(lambda: ctx.binary_dense(act_in, hid["Wp"], hid["thr"], hid["flip"], BATCH, SIZES[2], SIZES[1],
+                                                       out=act_out), args.steps, args.warmup)
+    first = net["layers"][0]
+    first_times = timed_steps(lambda: ctx.first_layer_bitplanes(X, first["Wp"], BATCH, SIZES[1], SIZES[0], thr=first["thr"],
+                                                                flip=first["flip"]), max(args.steps // 2, 3), 3)
+    clocks = sampler.stop() if sampler else None
+
+    if world > 1:
+        t = torch.tensor([total_ms, e2e_total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_total_ms = t.tolist()
+
+    ms_per_step = total_ms / args.steps
+    value = world * BATCH / (ms_per_step / 1e3)
+    e2e_value = world * BATCH / (e2e_total_ms / args.steps / 1e3)
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return 0
+
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except OSError:
+        pass
+    sm_count = torch.cuda.get_device_properties(local).multi_processor_count
+    sm_max_mhz = float(peaks.get("sm_max_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0)
+    popc_peak_tbitops = sm_count * POPC_PER_CLK_PER_SM * 32 * 2 * sm_max_mhz * 1e6 / 1e12
+
+    dense_ms = sum(dense_times) / len(dense_times)
+    dense_ops = 2.0 * BATCH * SIZES[1] * SIZES[2]
+    dense_ach = dense_ops / (dense_ms / 1e3) / 1e12
+    first_ms = sum(first_times) / len(first_times)
+    first_ach = 2.0 * 8 * BATCH * SIZES[0] * SIZES[1] / (first_ms / 1e3) / 1e12
+    mlp_ach = bit_ops_mlp(BATCH, SIZES) / (ms_per_step / 1e3) / 1e12
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32", "data": "synthetic",
+        "config": {"workload": "MNIST-shaped BNN MLP forward 784-4096-4096-4096-10 (8 bit-planes, 2 fused binary dense, float output), "
+                               "batch 10000 per GPU, seed 1", "batch_per_gpu": BATCH, "parallelism": "replicas x%d" % world,
+                   "l2": "256 MiB written between timed steps (inputs fit in L2)", "popc_variant": args.variant},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": BATCH * SIZES[0], "d2h_bytes_per_step": BATCH * SIZES[-1] * 4,
+                "ms_per_step": e2e_total_ms / args.steps},
+        "gpu_launches": launches_per_step * args.steps,
+        "roofline": {"bound": "alu", "kernel": "k_bit_tile (fused binary dense 10000x4096x4096)", "achieved": dense_ach,
+                     "peak": popc_peak_tbitops, "unit": "Tbit-op/s", "frac": dense_ach / popc_peak_tbitops, "traffic": None,
+                     "peak_kind": "derived: %d SMs x 16 POPC/clk/SM x 32 bit-MAC x 2 x %.0f MHz (one POPC per 32-bit word); "
+                                  "carry-save kernels may exceed it" % (sm_count, sm_max_mhz),
+                     "ms_per_launch": dense_ms},
+        "mlp_step": {"achieved_tbitops": mlp_ach, "frac_of_popc_peak": mlp_ach / popc_peak_tbitops,
+                     "first_layer_ms": first_ms, "first_layer_tbitops": first_ach, "dense_layer_ms": dense_ms},
+    }
+
+    if not args.no_extras and world == 1:
+        line["gemm"] = bench_gemm(ctx, args.gemm_size, popc_peak_tbitops, timed_steps)
+        line["convnet"] = bench_convnet(ctx, timed_steps)
+        dt, cores = time_oracle_mlp(case, 2000)
+        line["cpu_baseline"] = {"value": 2000 / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": "first 2000 of the 10000 images, one pass (%.1f s)" % dt}
+    else:
+        line["cpu_baseline"] = None
+    print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+def bench_gemm(ctx, n, peak, timed_steps):
+    """Binary GEMM n^3 (the paper's 8192^3 by default): Tbit-op/s = 2 n^3 / t."""
+    import torch
+    words = n // 32
+    g = torch.Generator(device="cuda").manual_seed(2)
+    Ap = torch.randint(-2**31, 2**31 - 1, (n, words), dtype=torch.int32, device="cuda", generator=g)
+    Bp = torch.randint(-2**31, 2**31 - 1, (n, words), dtype=torch.int32, device="cuda", generator=g)
+    C = torch.empty(n, n, dtype=torch.int32, device="cuda")
+    t = timed_steps(lambda: ctx.xnor_gemm(Ap, Bp, n, n, n, C=C), 5, 3)
+    ms = sum(t) / len(t)
+    tb = 2.0 * n ** 3 / (ms / 1e3) / 1e12
+    return {"shape": [n, n, n], "ms": ms, "tbitops": tb, "frac_of_popc_peak": tb / peak}
+
+
+def bench_convnet(ctx, timed_steps):
+    """CIFAR-shaped ConvNet forward, batch 256: images/s."""
+    import torch
+    from paper_1602_02830_b200 import nets, workloads as wl
+    case = wl.convnet_case()
+    net = nets.prepare_convnet(ctx, case["layers"])
+    X = torch.from_numpy(case["X"]).cuda()
+    t = timed_steps(lambda: nets.convnet_forward(ctx, net, X), 5, 3)
+    ms = sum(t) / len(t)
+    return {"batch": case["batch"], "ms": ms, "images_per_s": case["batch"] / (ms / 1e3)}
+
+
+if __name__ == "__main__":
+    sys.exit(main())
