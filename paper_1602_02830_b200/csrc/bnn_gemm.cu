@@ -137,23 +137,20 @@ bool skinny_fits(int64_t RS, int64_t K) {
 }
 
 template <int AKIND>
-int launch_tile(bnn_ctx *ctx, const Args &a, int variant) {
-    const int64_t t128 = ((a.M + 127) / 128) * ((a.N + BN - 1) / BN);
-    const int64_t t64 = ((a.M + 63) / 64) * ((a.N + BN - 1) / BN);
+int launch_tile(bnn_ctx *ctx, const Args &a_in, int variant) {
+    Args a = a_in;
+    a.one = 1u;
+    const int64_t rows = (AKIND == A_PLANES) ? 8 * a.M : a.M;     // operand rows (8 bit-plane rows per image)
+    const int64_t t128 = ((rows + 127) / 128) * ((a.N + BN - 1) / BN);
+    const int64_t t64 = ((rows + 63) / 64) * ((a.N + BN - 1) / BN);
     const bool big = t128 >= 2 * (int64_t)ctx->sm_count;
     const int64_t tiles = big ? t128 : t64;
     if (tiles > 0x7fffffff) return BNN_ERR_INVALID_ARG;
-    const bool csa = (AKIND != A_PLANES) && (variant != BNN_VARIANT_PLAIN);
-    if (AKIND == A_PLANES) {
-        if (big) k_bit_tile<8, A_PLANES, false><<<(unsigned)tiles, 256, 0, ctx->stream>>>(a);
-        else k_bit_tile<4, A_PLANES, false><<<(unsigned)tiles, 128, 0, ctx->stream>>>(a);
-    } else {
-        constexpr int AK = (AKIND == A_PLANES) ? A_PACKED : AKIND;
-        if (big && csa) k_bit_tile<8, AK, true><<<(unsigned)tiles, 256, 0, ctx->stream>>>(a);
-        else if (big) k_bit_tile<8, AK, false><<<(unsigned)tiles, 256, 0, ctx->stream>>>(a);
-        else if (csa) k_bit_tile<4, AK, true><<<(unsigned)tiles, 128, 0, ctx->stream>>>(a);
-        else k_bit_tile<4, AK, false><<<(unsigned)tiles, 128, 0, ctx->stream>>>(a);
-    }
+    const bool csa = (variant != BNN_VARIANT_PLAIN);
+    if (big && csa) k_bit_tile<8, AKIND, true><<<(unsigned)tiles, 256, 0, ctx->stream>>>(a);
+    else if (big) k_bit_tile<8, AKIND, false><<<(unsigned)tiles, 256, 0, ctx->stream>>>(a);
+    else if (csa) k_bit_tile<4, AKIND, true><<<(unsigned)tiles, 128, 0, ctx->stream>>>(a);
+    else k_bit_tile<4, AKIND, false><<<(unsigned)tiles, 128, 0, ctx->stream>>>(a);
     return bnn_check_launch(ctx);
 }
 

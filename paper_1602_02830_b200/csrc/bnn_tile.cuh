@@ -13,10 +13,13 @@
 //   CSA     (ones, carry) = full_add(ones, a0 ^ b0, a1 ^ b1); acc2 += popc(carry)
 //           1 POPC per TWO words; the POPC pipe (16 lanes/clk/SM on sm_100) is the bottleneck and
 //           the two extra LOP3 go to the 64-lane integer pipe.  Total = 2 * acc2 + popc(ones).
-//   PLANES  acc += popc(x_plane_p & w) << p   for the 8 bit-planes of an 8-bit input (Eq. 6-7)
+// The accumulate is written as popc * one + acc with `one` a run-time 1, so that it is issued as an integer
+// multiply-add on the FMA pipe instead of competing with the LOP3s for the integer pipe.
 //
-// A-operand sources: a packed matrix, an implicit im2col view of a packed NHWC activation map
-// (3x3, pad 1), or an 8-bit matrix split into bit-planes on the fly.
+// A-operand sources: a packed matrix; an implicit im2col view of a packed NHWC activation map (3x3, pad 1);
+// or an 8-bit matrix split into bit-planes on the fly (Eq. 6-7): each image contributes 8 operand rows, one
+// per bit-plane x^p in {0,1}, combined with AND instead of XOR, and the epilogue forms
+// s = 2 * sum_p 2^p popc(x^p & w_plus) - sum(x)  (w_plus = the +1 mask of the weights).
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -45,6 +48,7 @@ struct Args {
     const int32_t *thr;
     const uint32_t *flip;
     int H, W, Cw, pool;  // A_CONV geometry: image height/width, C_in/32, 2x2 pooling flag
+    uint32_t one;        // always 1; a run-time value so that "popc * one + acc" stays an IMAD
 };
 
 __device__ __forceinline__ uint32_t lop3_xor3(uint32_t a, uint32_t b, uint32_t c) {
@@ -89,28 +93,30 @@ __device__ __forceinline__ uint32_t plane_nibble(uint32_t w, int p) {
 
 template <int NWARPS, int AKIND, bool CSA>
 __global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile(const Args p) {
-    constexpr int BM = NWARPS * TM;
+    constexpr int BM = NWARPS * TM;        // operand rows per tile (A_PLANES: 8 rows per image)
     constexpr int NT = NWARPS * 32;
     static_assert(2 * BM == NT, "one A load item per thread");
-    static_assert(!(CSA && AKIND == A_PLANES), "bit-plane mode has its own inner loop");
+    constexpr bool PLANES = (AKIND == A_PLANES);
+    constexpr int IMGS = BM / 8;           // A_PLANES: images per tile
 
     __shared__ __align__(16) uint32_t As[2][BKW][BM];
     __shared__ __align__(16) uint32_t Bs[2][BKW][BN];
-    __shared__ int32_t aux[(AKIND == A_CONV) ? 9 * BN : ((AKIND == A_PLANES) ? 2 * BM : 1)];
+    __shared__ int32_t aux[(AKIND == A_CONV) ? 9 * BN : (PLANES ? IMGS : 1)];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int64_t tiles_m = (p.M + BM - 1) / BM;
+    const int64_t rows_total = PLANES ? 8 * p.M : p.M;      // operand rows
+    const int64_t tiles_m = (rows_total + BM - 1) / BM;
     const int64_t tile_m = blockIdx.x % tiles_m, tile_n = blockIdx.x / tiles_m;
-    const int64_t m0 = tile_m * BM, n0 = tile_n * BN;
-    const int64_t Kw = (AKIND == A_PLANES) ? ((p.K + 31) >> 5) : ((p.K + 31) >> 5);
-    const int64_t nchunks = (AKIND == A_PLANES) ? Kw : (Kw + BKW - 1) / BKW;
+    const int64_t m0 = tile_m * BM, n0 = tile_n * BN;       // m0 in operand rows
+    const int64_t Kw = (p.K + 31) >> 5;
+    const int64_t nchunks = (Kw + BKW - 1) / BKW;
     const uint32_t tail_mask = (p.K & 31) ? ((1u << (p.K & 31)) - 1u) : 0xffffffffu;
 
     // ---- loader roles: one A item per thread, (2*BN)/NT B items per thread
-    const int a_row = tid % BM, a_half = tid / BM;
-    const int64_t am = m0 + a_row;
+    const int a_row = tid % BM, a_half = tid / BM;          // A_PACKED / A_CONV: row and which 4 of the 8 words
+    const int a_img = tid >> 4, a_seg = tid & 15;           // A_PLANES: image in tile and 16-byte segment of the chunk
+    const int64_t am = PLANES ? (m0 >> 3) + a_img : m0 + a_row;
     const bool a_ok = am < p.M;
-    // A_CONV: pixel of this loader's row
     int pix_y = 0, pix_x = 0;
     int64_t pix_b = 0;
     if (AKIND == A_CONV && a_ok) {
@@ -124,7 +130,7 @@ __global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile
         pix_b = idx / Hd;
         if (p.pool) { pix_y = 2 * pix_y + (q >> 1); pix_x = 2 * pix_x + (q & 1); }
     }
-    const bool a_vec = (AKIND == A_PACKED) ? true : ((p.Cw & 3) == 0);
+    const bool a_vec = (AKIND == A_CONV) ? ((p.Cw & 3) == 0) : true;
     const bool b_vec = (AKIND == A_CONV) ? ((p.Cw & 3) == 0) : true;
     int32_t x_sum = 0;   // A_PLANES: running sum of this loader's bytes
 
@@ -158,9 +164,9 @@ __global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile
                     ra = make_uint4(w[0], w[1], w[2], w[3]);
                 }
             }
-        } else {   // A_PLANES: 16 bytes of input group c
+        } else {   // A_PLANES: 16 bytes (inputs 256c + 16*seg ...) of image `am`
             ra = make_uint4(0u, 0u, 0u, 0u);
-            const int64_t k0 = c * 32 + 16 * a_half;
+            const int64_t k0 = c * (32 * BKW) + 16 * a_seg;
             if (a_ok && k0 < p.K) {
                 const uint8_t *src = p.X + am * p.ldx + k0;
                 if (k0 + 16 <= p.K && ((reinterpret_cast<uintptr_t>(src) & 15u) == 0)) {
@@ -178,25 +184,19 @@ __global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile
             const int idx = tid + it * NT;
             const int b_row = idx % BN, b_half = idx / BN;
             const int64_t bn = n0 + b_row;
-            if (AKIND == A_PLANES) {
-                uint32_t w = 0u;
-                if (b_half == 0 && bn < p.N) w = p.B[bn * p.ldb + c];
-                rb[it] = make_uint4(w, 0u, 0u, 0u);
-            } else {
-                rb[it] = load_row_words(p.B + bn * p.ldb, bn < p.N, c * BKW + 4 * b_half, Kw, tail_mask, b_vec);
-            }
+            rb[it] = load_row_words(p.B + bn * p.ldb, bn < p.N, c * BKW + 4 * b_half, Kw, tail_mask, b_vec);
         }
     };
 
     auto store_chunk = [&](int buf) {
-        if (AKIND == A_PLANES) {
+        if (PLANES) {
             const uint32_t w[4] = {ra.x, ra.y, ra.z, ra.w};
             x_sum += (int32_t)(__vsadu4(ra.x, 0u) + __vsadu4(ra.y, 0u) + __vsadu4(ra.z, 0u) + __vsadu4(ra.w, 0u));
 #pragma unroll
             for (int pl = 0; pl < 8; ++pl) {
                 const uint32_t h = plane_nibble(w[0], pl) | (plane_nibble(w[1], pl) << 4) |
                                    (plane_nibble(w[2], pl) << 8) | (plane_nibble(w[3], pl) << 12);
-                reinterpret_cast<uint16_t *>(&As[buf][pl][a_row])[a_half] = (uint16_t)h;
+                reinterpret_cast<uint16_t *>(&As[buf][a_seg >> 1][8 * a_img + pl])[a_seg & 1] = (uint16_t)h;
             }
         } else {
             As[buf][4 * a_half + 0][a_row] = ra.x;
@@ -208,19 +208,15 @@ __global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile
         for (int it = 0; it < B_ITEMS; ++it) {
             const int idx = tid + it * NT;
             const int b_row = idx % BN, b_half = idx / BN;
-            if (AKIND == A_PLANES) {
-                if (b_half == 0) Bs[buf][0][b_row] = rb[it].x;
-            } else {
-                Bs[buf][4 * b_half + 0][b_row] = rb[it].x;
-                Bs[buf][4 * b_half + 1][b_row] = rb[it].y;
-                Bs[buf][4 * b_half + 2][b_row] = rb[it].z;
-                Bs[buf][4 * b_half + 3][b_row] = rb[it].w;
-            }
+            Bs[buf][4 * b_half + 0][b_row] = rb[it].x;
+            Bs[buf][4 * b_half + 1][b_row] = rb[it].y;
+            Bs[buf][4 * b_half + 2][b_row] = rb[it].z;
+            Bs[buf][4 * b_half + 3][b_row] = rb[it].w;
         }
     };
 
-    // ---- A_CONV prologue: popcount of every filter's weights per tap (correction for skipped taps)
-    if (AKIND == A_CONV) {
+    // ---- prologues
+    if (AKIND == A_CONV) {   // popcount of every filter's weights per tap (correction for skipped taps)
         for (int e = tid; e < 9 * BN; e += NT) {
             const int tap = e / BN, col = e % BN;
             int32_t s = 0;
@@ -230,6 +226,9 @@ __global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile
             }
             aux[e] = s;
         }
+    }
+    if (PLANES) {
+        if (tid < IMGS) aux[tid] = 0;
     }
 
     uint32_t acc[TM][TN];
@@ -246,6 +245,7 @@ __global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile
     }
 
     const int wr = warp * TM;
+    const uint32_t one = p.one;
     if (nchunks > 0) {
         load_chunk(0);
         store_chunk(0);
@@ -255,63 +255,53 @@ __global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile
     for (int64_t c = 0; c < nchunks; ++c) {
         const int buf = (int)(c & 1);
         if (c + 1 < nchunks) load_chunk(c + 1);
+        // words of this chunk that can be non-zero (rounded up to a pair); the rest of the chunk is skipped
+        const int kw_lim = (int)min((int64_t)BKW, ((Kw - c * BKW) + 1) & ~int64_t(1));
 
-        if (AKIND == A_PLANES) {
-            uint32_t b[TN];
-#pragma unroll
-            for (int j = 0; j < TN; ++j) b[j] = Bs[buf][0][lane + 32 * j];
-#pragma unroll
-            for (int pl = 0; pl < 8; ++pl) {
-                uint32_t a[TM];
-#pragma unroll
-                for (int q = 0; q < TM / 4; ++q) {
-                    const uint4 v = *reinterpret_cast<const uint4 *>(&As[buf][pl][wr + 4 * q]);
-                    a[4 * q] = v.x; a[4 * q + 1] = v.y; a[4 * q + 2] = v.z; a[4 * q + 3] = v.w;
-                }
-#pragma unroll
-                for (int i = 0; i < TM; ++i)
-#pragma unroll
-                    for (int j = 0; j < TN; ++j) acc[i][j] += (uint32_t)__popc(a[i] & b[j]) << pl;
-            }
-        } else if (!CSA) {
+        if (!CSA) {
 #pragma unroll
             for (int kw = 0; kw < BKW; ++kw) {
-                uint32_t a[TM], b[TN];
+                if (kw < kw_lim) {
+                    uint32_t a[TM], b[TN];
 #pragma unroll
-                for (int q = 0; q < TM / 4; ++q) {
-                    const uint4 v = *reinterpret_cast<const uint4 *>(&As[buf][kw][wr + 4 * q]);
-                    a[4 * q] = v.x; a[4 * q + 1] = v.y; a[4 * q + 2] = v.z; a[4 * q + 3] = v.w;
+                    for (int q = 0; q < TM / 4; ++q) {
+                        const uint4 v = *reinterpret_cast<const uint4 *>(&As[buf][kw][wr + 4 * q]);
+                        a[4 * q] = v.x; a[4 * q + 1] = v.y; a[4 * q + 2] = v.z; a[4 * q + 3] = v.w;
+                    }
+#pragma unroll
+                    for (int j = 0; j < TN; ++j) b[j] = Bs[buf][kw][lane + 32 * j];
+#pragma unroll
+                    for (int i = 0; i < TM; ++i)
+#pragma unroll
+                        for (int j = 0; j < TN; ++j)
+                            acc[i][j] += (uint32_t)__popc(PLANES ? (a[i] & b[j]) : (a[i] ^ b[j]));
                 }
-#pragma unroll
-                for (int j = 0; j < TN; ++j) b[j] = Bs[buf][kw][lane + 32 * j];
-#pragma unroll
-                for (int i = 0; i < TM; ++i)
-#pragma unroll
-                    for (int j = 0; j < TN; ++j) acc[i][j] += (uint32_t)__popc(a[i] ^ b[j]);
             }
         } else {
 #pragma unroll
             for (int kw = 0; kw < BKW; kw += 2) {
-                uint32_t b0[TN], b1[TN];
+                if (kw < kw_lim) {
+                    uint32_t b0[TN], b1[TN];
 #pragma unroll
-                for (int j = 0; j < TN; ++j) { b0[j] = Bs[buf][kw][lane + 32 * j]; b1[j] = Bs[buf][kw + 1][lane + 32 * j]; }
+                    for (int j = 0; j < TN; ++j) { b0[j] = Bs[buf][kw][lane + 32 * j]; b1[j] = Bs[buf][kw + 1][lane + 32 * j]; }
 #pragma unroll
-                for (int q = 0; q < TM / 4; ++q) {
-                    const uint4 v0 = *reinterpret_cast<const uint4 *>(&As[buf][kw][wr + 4 * q]);
-                    const uint4 v1 = *reinterpret_cast<const uint4 *>(&As[buf][kw + 1][wr + 4 * q]);
-                    const uint32_t a0[4] = {v0.x, v0.y, v0.z, v0.w};
-                    const uint32_t a1[4] = {v1.x, v1.y, v1.z, v1.w};
+                    for (int q = 0; q < TM / 4; ++q) {
+                        const uint4 v0 = *reinterpret_cast<const uint4 *>(&As[buf][kw][wr + 4 * q]);
+                        const uint4 v1 = *reinterpret_cast<const uint4 *>(&As[buf][kw + 1][wr + 4 * q]);
+                        const uint32_t a0[4] = {v0.x, v0.y, v0.z, v0.w};
+                        const uint32_t a1[4] = {v1.x, v1.y, v1.z, v1.w};
 #pragma unroll
-                    for (int ii = 0; ii < 4; ++ii)
+                        for (int ii = 0; ii < 4; ++ii)
 #pragma unroll
-                        for (int j = 0; j < TN; ++j) {
-                            const int i = 4 * q + ii;
-                            const uint32_t x0 = a0[ii] ^ b0[j];
-                            const uint32_t x1 = a1[ii] ^ b1[j];
-                            const uint32_t o = ones[CSA ? i : 0][CSA ? j : 0];
-                            ones[CSA ? i : 0][CSA ? j : 0] = lop3_xor3(o, x0, x1);
-                            acc[i][j] += (uint32_t)__popc(lop3_maj(o, x0, x1));
-                        }
+                            for (int j = 0; j < TN; ++j) {
+                                const int i = 4 * q + ii;
+                                const uint32_t x0 = PLANES ? (a0[ii] & b0[j]) : (a0[ii] ^ b0[j]);
+                                const uint32_t x1 = PLANES ? (a1[ii] & b1[j]) : (a1[ii] ^ b1[j]);
+                                const uint32_t o = ones[CSA ? i : 0][CSA ? j : 0];
+                                ones[CSA ? i : 0][CSA ? j : 0] = lop3_xor3(o, x0, x1);
+                                acc[i][j] = (uint32_t)__popc(lop3_maj(o, x0, x1)) * one + acc[i][j];
+                            }
+                    }
                 }
             }
         }
@@ -320,13 +310,12 @@ __global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile
         __syncthreads();
     }
 
-    if (AKIND == A_PLANES) {
-        aux[a_half * BM + a_row] = x_sum;
+    if (PLANES) {
+        atomicAdd(&aux[a_img], x_sum);
         __syncthreads();
     }
 
     // ---- epilogue: integer result per output, then optional int32 store and optional Sign + repack
-    const int64_t Ktrue = p.K;
     int32_t thr_r[TN];
     uint32_t flip_r[TN];
 #pragma unroll
@@ -335,84 +324,109 @@ __global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile
         thr_r[j] = (p.out && col < p.N) ? p.thr[col] : 0;
         flip_r[j] = (p.out && p.flip && col < p.N) ? ((p.flip[col >> 5] >> (col & 31)) & 1u) : 0u;
     }
-
+    // total popcount of output (i, j)
+    auto total = [&](int i, int j) -> int32_t {
+        int32_t P = (int32_t)acc[i][j];
+        if (CSA) P = 2 * P + __popc(ones[CSA ? i : 0][CSA ? j : 0]);
+        return P;
+    };
     uint32_t keep = 0u;   // packed word this lane will store
-    int32_t pooled[TN];
-    uint32_t pooled_bit[TN];
+
+    if (PLANES) {
+        // this thread holds the 8 plane rows of 2 images: rows wr + 8*mi + pl
 #pragma unroll
-    for (int i = 0; i < TM; ++i) {
-        const int64_t row = m0 + wr + i;
-        int32_t base;      // dot = base - 2 * (P - corr)  (XOR modes)  or  2 * acc - x_sum (planes)
-        int inval = 0;     // A_CONV: bit t set if tap t falls outside the image
-        if (AKIND == A_PACKED) {
-            base = (int32_t)Ktrue;
-        } else if (AKIND == A_CONV) {
-            int64_t idx = row < p.M ? row : 0;
-            int q = 0, Wd = p.W, Hd = p.H;
-            if (p.pool) { q = (int)(idx & 3); idx >>= 2; Wd >>= 1; Hd >>= 1; }
-            int x = (int)(idx % Wd);
-            int y = (int)((idx / Wd) % Hd);
-            if (p.pool) { y = 2 * y + (q >> 1); x = 2 * x + (q & 1); }
-            if (y == 0) inval |= 0x007;
-            if (y == p.H - 1) inval |= 0x1c0;
-            if (x == 0) inval |= 0x049;
-            if (x == p.W - 1) inval |= 0x124;
-            base = (int32_t)(p.Cw * 32) * (9 - __popc(inval));
-        } else {
-            base = -(aux[wr + i] + aux[BM + wr + i]);
+        for (int mi = 0; mi < 2; ++mi) {
+            const int64_t img = (m0 >> 3) + 2 * warp + mi;
+            const int32_t xs = aux[2 * warp + mi];
+#pragma unroll
+            for (int j = 0; j < TN; ++j) {
+                const int64_t col = n0 + lane + 32 * j;
+                int32_t wsum = 0;
+#pragma unroll
+                for (int pl = 0; pl < 8; ++pl) wsum += total(8 * mi + pl, j) << pl;
+                const int32_t dot = 2 * wsum - xs;
+                const bool in = img < p.M && col < p.N;
+                if (p.C && in) p.C[img * p.ldc + col] = dot;
+                if (p.out) {
+                    const bool bit = in && ((((uint32_t)(dot >= thr_r[j])) ^ flip_r[j]) & 1u);
+                    const uint32_t word = __ballot_sync(0xffffffffu, bit);
+                    if (lane == mi * TN + j) keep = word;
+                }
+            }
         }
+        if (p.out && lane < 2 * TN) {
+            const int64_t img = (m0 >> 3) + 2 * warp + (lane >> 2);
+            const int64_t ow = (n0 >> 5) + (lane & 3);
+            if (img < p.M && ow * 32 < p.N) p.out[img * p.ldo + ow] = keep;
+        }
+    } else {
+        int32_t pooled[TN];
+        uint32_t pooled_bit[TN];
+        const bool pooled_mode = (AKIND == A_CONV) && p.pool;
 #pragma unroll
-        for (int j = 0; j < TN; ++j) {
-            const int64_t col = n0 + lane + 32 * j;
-            int32_t P = (int32_t)acc[i][j];
-            if (CSA) P = 2 * P + __popc(ones[CSA ? i : 0][CSA ? j : 0]);
-            int32_t dot;
-            if (AKIND == A_PLANES) {
-                dot = 2 * P + base;
-            } else {
+        for (int i = 0; i < TM; ++i) {
+            const int64_t row = m0 + wr + i;
+            int32_t base = (int32_t)p.K;
+            int inval = 0;     // A_CONV: bit t set if tap t falls outside the image
+            if (AKIND == A_CONV) {
+                int64_t idx = row < p.M ? row : 0;
+                int q = 0, Wd = p.W, Hd = p.H;
+                if (p.pool) { q = (int)(idx & 3); idx >>= 2; Wd >>= 1; Hd >>= 1; }
+                int x = (int)(idx % Wd);
+                int y = (int)((idx / Wd) % Hd);
+                if (p.pool) { y = 2 * y + (q >> 1); x = 2 * x + (q & 1); }
+                if (y == 0) inval |= 0x007;
+                if (y == p.H - 1) inval |= 0x1c0;
+                if (x == 0) inval |= 0x049;
+                if (x == p.W - 1) inval |= 0x124;
+                base = (int32_t)(p.Cw * 32) * (9 - __popc(inval));
+            }
+#pragma unroll
+            for (int j = 0; j < TN; ++j) {
+                const int64_t col = n0 + lane + 32 * j;
+                int32_t P = total(i, j);
                 if (AKIND == A_CONV && inval) {
                     for (int t = 0; t < 9; ++t)
                         if ((inval >> t) & 1) P -= aux[t * BN + lane + 32 * j];
                 }
-                dot = base - 2 * P;
-            }
-            const bool in = row < p.M && col < p.N;
-            const bool q = in && (dot >= thr_r[j]);
-            if (AKIND == A_CONV && p.pool) {
-                // rows 4w..4w+3 of a thread are one pooling window
-                if ((i & 3) == 0) { pooled[j] = dot; pooled_bit[j] = q; }
-                else { pooled[j] = max(pooled[j], dot); pooled_bit[j] |= (uint32_t)q; }
-                if ((i & 3) == 3) {
-                    if (p.C && in) p.C[(row >> 2) * p.ldc + col] = pooled[j];
+                const int32_t dot = base - 2 * P;
+                const bool in = row < p.M && col < p.N;
+                const bool q = in && (dot >= thr_r[j]);
+                if (pooled_mode) {
+                    // rows 4w..4w+3 of a thread are one pooling window
+                    if ((i & 3) == 0) { pooled[j] = dot; pooled_bit[j] = q; }
+                    else { pooled[j] = max(pooled[j], dot); pooled_bit[j] |= (uint32_t)q; }
+                    if ((i & 3) == 3) {
+                        if (p.C && in) p.C[(row >> 2) * p.ldc + col] = pooled[j];
+                        if (p.out) {
+                            const bool bit = in && ((pooled_bit[j] ^ flip_r[j]) & 1u);
+                            const uint32_t word = __ballot_sync(0xffffffffu, bit);
+                            if (lane == (((i >> 2) * TN + j) & 31)) keep = word;
+                        }
+                    }
+                } else {
+                    if (p.C && in) p.C[row * p.ldc + col] = dot;
                     if (p.out) {
-                        const bool bit = col < p.N && row < p.M && ((pooled_bit[j] ^ flip_r[j]) & 1u);
+                        const bool bit = in && (((uint32_t)q ^ flip_r[j]) & 1u);
                         const uint32_t word = __ballot_sync(0xffffffffu, bit);
-                        if (lane == (((i >> 2) * TN + j) & 31)) keep = word;
+                        if (lane == ((i * TN + j) & 31)) keep = word;
                     }
                 }
-            } else {
-                if (p.C && in) p.C[row * p.ldc + col] = dot;
-                if (p.out) {
-                    const bool bit = in && (((uint32_t)q ^ flip_r[j]) & 1u);
-                    const uint32_t word = __ballot_sync(0xffffffffu, bit);
-                    if (lane == ((i * TN + j) & 31)) keep = word;
+            }
+            // flush the 32 words gathered over the last 8 rows (or the 16 words of 4 pooled windows)
+            if (p.out) {
+                if (!pooled_mode && (i & 7) == 7) {
+                    const int ri = (i & ~7) + (lane >> 2), j = lane & 3;
+                    const int64_t orow = m0 + wr + ri;
+                    const int64_t ow = (n0 >> 5) + j;
+                    if (orow < p.M && ow * 32 < p.N) p.out[orow * p.ldo + ow] = keep;
                 }
-            }
-        }
-        // flush the 32 words gathered over the last 8 rows (or the 16 words of 4 pooled windows)
-        if (p.out) {
-            const bool pooled_mode = (AKIND == A_CONV) && p.pool;
-            if (!pooled_mode && (i & 7) == 7) {
-                const int ri = (i & ~7) + (lane >> 2), j = lane & 3;
-                const int64_t orow = m0 + wr + ri;
-                const int64_t ow = (n0 >> 5) + j;
-                if (orow < p.M && ow * 32 < p.N) p.out[orow * p.ldo + ow] = keep;
-            }
-            if (pooled_mode && i == TM - 1 && lane < 16) {
-                const int wi = lane >> 2, j = lane & 3;
-                const int64_t orow = ((m0 + wr) >> 2) + wi;
-                const int64_t ow = (n0 >> 5) + j;
-                if (orow * 4 < p.M && ow * 32 < p.N) p.out[orow * p.ldo + ow] = keep;
+                if (pooled_mode && i == TM - 1 && lane < 16) {
+                    const int wi = lane >> 2, j = lane & 3;
+                    const int64_t orow = ((m0 + wr) >> 2) + wi;
+                    const int64_t ow = (n0 >> 5) + j;
+                    if (orow * 4 < p.M && ow * 32 < p.N) p.out[orow * p.ldo + ow] = keep;
+                }
             }
         }
     }
@@ -423,9 +437,10 @@ __global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile
         const int64_t npad = p.ldo - first_pad;
         if (npad > 0) {
             const bool pooled_mode = (AKIND == A_CONV) && p.pool;
+            const int sh = PLANES ? 3 : (pooled_mode ? 2 : 0);   // operand rows per output row, log2
             const int64_t rows_out = pooled_mode ? (p.M >> 2) : p.M;
-            const int64_t r0 = pooled_mode ? (m0 >> 2) : m0;
-            const int64_t nrows = pooled_mode ? (BM >> 2) : BM;
+            const int64_t r0 = m0 >> sh;
+            const int64_t nrows = BM >> sh;
             for (int64_t e = tid; e < nrows * npad; e += NT) {
                 const int64_t r = r0 + e / npad;
                 if (r < rows_out) p.out[r * p.ldo + first_pad + e % npad] = 0u;
