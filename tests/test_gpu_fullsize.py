@@ -1,0 +1,146 @@
+"""GPU parity at the full sizes of the benchmark configurations, in the launch configuration bench.py
+times (library-default inner loop).  Where the oracle cannot finish the whole problem in seconds it checks
+sampled rows (first, last, tile-boundary and random ones) over all columns, and the complete output is
+compared on the GPU with torch.matmul / conv2d of the +-1 values (exact: every partial sum is an integer
+below 2^24)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1602_02830_b200 import binding, build, nets, workloads as wl
+from util import np_unpack_pm1, padding_is_zero
+
+pytestmark = pytest.mark.gpu
+torch.backends.cuda.matmul.allow_tf32 = False
+torch.backends.cudnn.allow_tf32 = False
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    build.build()
+    c = binding.Context(0)
+    yield c
+    torch.cuda.synchronize()
+    c.close()
+
+
+def sample_rows(M, n_random, rng):
+    fixed = [0, 1, M - 1, M - 2]
+    for t in (63, 64, 127, 128, 255, 256, M // 2 - 1, M // 2, M - 128, M - 129):
+        if 0 <= t < M:
+            fixed.append(t)
+    rows = np.unique(np.concatenate([np.array(fixed), rng.integers(0, M, n_random)]))
+    return rows[(rows >= 0) & (rows < M)]
+
+
+def unpack_bits_gpu(words: torch.Tensor, n: int) -> torch.Tensor:
+    """Packed int32 [R, ld] -> bool [R, n] on the GPU (test-side decoding of the ABI's bit layout)."""
+    sh = torch.arange(32, device=words.device, dtype=torch.int32)
+    bits = (words.unsqueeze(-1) >> sh) & 1
+    return bits.reshape(words.shape[0], -1)[:, :n].bool()
+
+
+@pytest.mark.parametrize("M,N,K", wl.GEMM_SWEEP)
+def test_gemm_sweep_full_size(ctx, M, N, K):
+    A, B = wl.gemm_case(M, N, K, seed=2)
+    Ad, Bd = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
+    Ap = ctx.pack_signs(Ad)
+    Bp = ctx.pack_signs(Bd, pack_along=1)
+    assert Ap.shape[1] % 4 == 0 and Ap.shape[1] >= (K + 31) // 32
+    if K % 32:   # "padded bits must not count": fill the padding of both operands with ones
+        Ap[:, K // 32] |= torch.tensor(-1 << (K % 32), dtype=torch.int32, device="cuda")
+        Bp[:, K // 32] |= torch.tensor(-1 << (K % 32), dtype=torch.int32, device="cuda")
+        Ap[:, K // 32 + 1:] = -1
+        Bp[:, K // 32 + 1:] = -1
+    C = ctx.xnor_gemm(Ap, Bp, M, N, K)
+    torch.cuda.synchronize()
+    # (a) complete output against the library matmul of the +-1 values, on the GPU
+    ref = torch.matmul(Ad.float(), Bd.float())          # fp32, TF32 off: exact
+    assert torch.equal(C.float(), ref)
+    del ref
+    # (b) sampled rows against the oracle
+    rows = sample_rows(M, 48, np.random.default_rng(K))
+    want = oracle.gemm(A[rows], B)
+    assert np.array_equal(C[torch.from_numpy(rows).cuda()].cpu().numpy(), want)
+    # (c) invariants at any size: parity and bound
+    assert bool(((C - K) % 2 == 0).all()) and int(C.abs().max()) <= K
+
+
+def test_mlp_config_full_batch(ctx):
+    case = wl.mlp_case()           # batch 10000, 784-4096-4096-4096-10, seed 1
+    want_scores, want_hidden = oracle.mlp_forward(case["X"], case["weights"], case["bns"])
+    net = nets.prepare_mlp(ctx, case["weights"], case["bns"])
+    batch, sizes = case["batch"], case["sizes"]
+    ws = torch.empty(ctx.mlp_workspace_bytes(net["desc"], batch, True), dtype=torch.uint8, device="cuda")
+    ctx.set_workspace(ws)
+    hidden = [torch.empty(batch, binding.packed_ld(n), dtype=torch.int32, device="cuda") for n in sizes[1:-1]]
+    scores = ctx.mlp_forward(net["desc"], torch.from_numpy(case["X"]).cuda(), batch, hidden_out=hidden)
+    torch.cuda.synchronize()
+    for k, (g, w) in enumerate(zip(hidden, want_hidden)):
+        gh = g.cpu().numpy()
+        assert np.array_equal(np_unpack_pm1(gh, w.shape[1]), w), f"hidden layer {k}"
+        assert padding_is_zero(gh, w.shape[1])
+    got = scores.cpu().numpy().astype(np.float64)
+    tol = 1e-5 * np.abs(want_scores) + 1e-6 * np.abs(want_scores).max()
+    assert (np.abs(got - want_scores) <= tol).all()
+    assert np.array_equal(got.argmax(1), want_scores.argmax(1))
+    # the host-buffer entry point gives the same scores
+    Xh = torch.from_numpy(case["X"]).pin_memory()
+    Sh = torch.empty(batch, sizes[-1], dtype=torch.float32).pin_memory()
+    ctx.mlp_forward_host(net["desc"], Xh, batch, Sh)
+    torch.cuda.synchronize()
+    assert np.array_equal(Sh.numpy(), scores.cpu().numpy())
+    ctx.set_workspace(None)
+
+
+def test_convnet_config_full_batch(ctx):
+    case = wl.convnet_case()       # batch 256, 32x32x3, 128-128-256-256-512-512, seed 3
+    net = nets.prepare_convnet(ctx, case["layers"])
+    Xd = torch.from_numpy(case["X"]).cuda()
+    outs = nets.convnet_forward(ctx, net, Xd, keep_all=True)
+    torch.cuda.synchronize()
+    # (a) oracle, every layer, on the first and last images of the batch
+    pick = np.r_[0:12, 244:256]
+    want = oracle.convnet_forward(case["X"][pick], case["layers"])
+    for k, (g, w) in enumerate(zip(outs, want)):
+        gh = g[torch.from_numpy(pick).cuda()].cpu().numpy()
+        assert np.array_equal(np_unpack_pm1(gh, w.shape[-1]), w), f"conv layer {k}"
+    # (b) every image, layer by layer, against torch conv2d on the GPU fed with the library's own previous layer
+    B = case["batch"]
+    a = Xd.float().permute(0, 3, 1, 2)
+    for k, (L, P) in enumerate(zip(case["layers"], net)):
+        w = torch.from_numpy(L["wgt"]).cuda().float().permute(0, 3, 1, 2)
+        s = torch.round(torch.nn.functional.conv2d(a, w, padding=1))   # integers; cuDNN may pick a transform-based algorithm
+        if L["pool"]:
+            s = torch.nn.functional.max_pool2d(s, 2)
+        s = s.permute(0, 2, 3, 1).contiguous()                       # B, H, W, Cout  (exact integers in fp32)
+        Cout = s.shape[-1]
+        thr = P["thr"].float()
+        flipw = P["flip"]
+        flip = unpack_bits_gpu(flipw.reshape(1, -1), Cout)[0]
+        want_bits = (s >= thr) ^ flip
+        got_bits = unpack_bits_gpu(outs[k].reshape(-1, outs[k].shape[-1]), Cout).reshape(want_bits.shape)
+        assert torch.equal(got_bits, want_bits), f"conv layer {k} (all {B} images)"
+        a = (got_bits.float() * 2 - 1).permute(0, 3, 1, 2)
+
+
+@pytest.mark.parametrize("batch", wl.DENSE_BATCHES)
+def test_dense_batch_sweep(ctx, batch):
+    case = wl.dense_case(batch)
+    K = N = 4096
+    Ad, Wd = torch.from_numpy(case["A"]).cuda(), torch.from_numpy(case["W"]).cuda()
+    Ap = ctx.pack_signs(Ad)
+    Wp = ctx.pack_signs(Wd, pack_along=1)
+    thr = torch.from_numpy(case["thr"]).cuda()
+    out = ctx.binary_dense(Ap, Wp, thr, None, batch, N, K)
+    torch.cuda.synchronize()
+    # complete output against the library matmul on the GPU
+    ref = torch.matmul(Ad.float(), Wd.float())          # fp32, TF32 off: exact
+    assert torch.equal(unpack_bits_gpu(out, N), ref >= thr.float())
+    # oracle on (sampled) rows
+    rows = np.arange(batch) if batch <= 4096 else sample_rows(batch, 1000, np.random.default_rng(batch))
+    want = oracle.threshold(oracle.gemm(case["A"][rows], case["W"]), case["thr"])
+    got = out[torch.from_numpy(rows).cuda()].cpu().numpy()
+    assert np.array_equal(np_unpack_pm1(got, N), want)
+    assert padding_is_zero(got, N)
