@@ -44,7 +44,8 @@ enum {
     BNN_ERR_ALIGNMENT = -2,     /* base pointer or leading dimension breaks the alignment rule     */
     BNN_ERR_WORKSPACE = -3,     /* workspace missing or too small                                   */
     BNN_ERR_CUDA = -4,          /* a CUDA runtime call failed; see bnn_last_cuda_error()            */
-    BNN_ERR_DEVICE_STATUS = -5  /* a kernel reported an internal error through its status word      */
+    BNN_ERR_DEVICE_STATUS = -5, /* a kernel reported an internal error through its status word      */
+    BNN_ERR_TOO_LARGE = -6      /* bnn_mlp_forward_noalloc: the problem does not fit the built-in scratch */
 };
 
 enum { BNN_F32 = 0, BNN_F16 = 1, BNN_I8 = 2 }; /* element type of bnn_pack_signs' source */
@@ -158,6 +159,33 @@ BNN_API int bnn_mlp_forward(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *
  * context's stream (pinned host memory makes the copies asynchronous).  The caller synchronises. */
 BNN_API int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X_host, int64_t ldx,
                          int64_t batch, float *scores_host, int64_t lds);
+
+/* ---------------------------------------------------------------------------------------------
+ * bnn_mlp_forward for callers that cannot allocate device memory.  (The paper has no counterpart: this
+ * is a deployment convenience of the library, not a step of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a serving loop whose device memory was
+ * sized and handed out at start-up and whose policy forbids further allocation (an allocation can
+ * synchronise the device, fail under memory pressure, or fragment a pool someone else owns), a plug-in
+ * that is handed pointers but owns no allocator, or a process that simply has no memory budget left for a
+ * workspace.  Such a caller still passes its input and output buffers; only the scratch between the layers
+ * is supplied by the library, from an array that is part of the library image.
+ *
+ * Same arguments and results as bnn_mlp_forward (device X and scores; no hidden_out), no workspace needed
+ * and none used.  Limits and rules:
+ *  - batch * ceil(widest hidden layer / 128) * 16 bytes must not exceed bnn_mlp_noalloc_max_bytes()
+ *    (512 KiB: e.g. batch 1024 at 4096 units); beyond that the call returns BNN_ERR_TOO_LARGE and does nothing.
+ *    Every GPU that loads the library holds 1 MiB for this array until the process exits.
+ *  - The first call on each device looks up the array's device address (one cudaGetSymbolAddress, no
+ *    allocation); make that first call before starting any stream capture on that device.
+ *  - The call itself never calls cudaMalloc, cudaFree or any allocating routine.
+ *  - All calls on one device share the one array: calls whose GPU work can overlap (different streams,
+ *    different contexts, different threads) race on it and must be serialised by the caller.  The array
+ *    keeps whatever the last call left; no call depends on its previous contents.
+ */
+BNN_API size_t bnn_mlp_noalloc_max_bytes(void);
+BNN_API int bnn_mlp_forward_noalloc(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X, int64_t ldx,
+                                    int64_t batch, float *scores, int64_t lds);
 
 /* ---------------------------------------------------------------------------------------------
  * Host helper (not on the timed path): fold run-time BatchNorm followed by Sign,

@@ -23,7 +23,7 @@ EXPORTS = (
     "bnn_create", "bnn_destroy", "bnn_status_string", "bnn_last_cuda_error", "bnn_set_workspace",
     "bnn_set_popc_variant", "bnn_pack_signs", "bnn_xnor_gemm", "bnn_binary_dense", "bnn_first_layer_bitplanes",
     "bnn_binary_conv2d", "bnn_mlp_workspace_bytes", "bnn_mlp_forward", "bnn_mlp_forward_host",
-    "bnn_fold_batchnorm",
+    "bnn_fold_batchnorm", "bnn_mlp_noalloc_max_bytes", "bnn_mlp_forward_noalloc",
 )
 
 
@@ -76,6 +76,9 @@ def lib() -> ctypes.CDLL:
         L.bnn_mlp_forward.argtypes = [vp, POINTER(MlpDesc), vp, i64, i64, vp, i64, POINTER(vp)]
         L.bnn_mlp_forward_host.argtypes = [vp, POINTER(MlpDesc), vp, i64, i64, vp, i64]
         L.bnn_fold_batchnorm.argtypes = [vp, vp, vp, vp, c_double, i64, i64, vp, vp]
+        L.bnn_mlp_noalloc_max_bytes.argtypes = []
+        L.bnn_mlp_noalloc_max_bytes.restype = c_size_t
+        L.bnn_mlp_forward_noalloc.argtypes = [vp, POINTER(MlpDesc), vp, i64, i64, vp, i64]
         _lib = L
     return _lib
 
@@ -219,6 +222,14 @@ class Context:
             hp = (c_void_p * (desc.n_layers - 1))(*[t.data_ptr() if t is not None else None for t in hidden_out])
         self._ck(lib().bnn_mlp_forward(self._h, ctypes.byref(desc), _ptr(X), X.stride(0) if batch > 1 else X.shape[-1],
                                        batch, _ptr(scores), n_out, hp), "bnn_mlp_forward")
+        return scores
+
+    def mlp_forward_noalloc(self, desc, X, batch, scores):
+        """bnn_mlp_forward_noalloc: the caller passes the output too, so that nothing is allocated here either."""
+        n_out = desc.layers[desc.n_layers - 1].N
+        self._ck(lib().bnn_mlp_forward_noalloc(self._h, ctypes.byref(desc), _ptr(X),
+                                               X.stride(0) if batch > 1 else X.shape[-1], batch, _ptr(scores), n_out),
+                 "bnn_mlp_forward_noalloc")
         return scores
 
     def mlp_forward_host(self, desc, X_host, batch, scores_host):

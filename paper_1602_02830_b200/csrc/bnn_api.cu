@@ -39,6 +39,7 @@ extern "C" const char *bnn_status_string(int status) {
         case BNN_ERR_WORKSPACE: return "workspace missing or too small";
         case BNN_ERR_CUDA: return "CUDA runtime error";
         case BNN_ERR_DEVICE_STATUS: return "kernel reported an internal error";
+        case BNN_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }

@@ -1,6 +1,7 @@
 // bnn_mlp_forward: Algorithm 4 ("Running a BNN") as a sequence of stream-ordered launches:
 // bit-plane first layer -> fused binary dense layers -> real-valued output layer.
 #include "bnn_internal.cuh"
+#include <mutex>
 
 namespace {
 
@@ -99,4 +100,59 @@ extern "C" int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const u
     BNN_CUDA_TRY(ctx, cudaMemcpy2DAsync(scores_host, (size_t)lds * 4, Sd, (size_t)NL * 4, (size_t)NL * 4, (size_t)batch,
                                         cudaMemcpyDeviceToHost, ctx->stream));
     return BNN_OK;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// bnn_mlp_forward_noalloc: the same forward pass for callers that must not allocate device memory.
+//
+// The two activation buffers that bnn_mlp_forward takes from the caller's workspace live here in a
+// file-scope device array instead.  It is part of the library image: every GPU that loads the library
+// holds these bytes until the process exits, which is why the limit is kept modest.
+//
+// In host code the array's name is only a host-side stand-in for the symbol, not a device address, so the
+// address is obtained once per device with cudaGetSymbolAddress (with that device current) and that
+// pointer is what the kernels receive.
+namespace {
+
+constexpr size_t kNoAllocBufferBytes = 512u * 1024u;   // per activation buffer; two buffers
+constexpr int kNoAllocMaxDevices = 64;
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[2 * kNoAllocBufferBytes];
+
+std::mutex g_noalloc_mutex;
+void *g_noalloc_ptr[kNoAllocMaxDevices] = {};
+
+// Device address of the scratch array on ctx's device (which the caller has made current).
+int noalloc_scratch(bnn_ctx *ctx, char **out) {
+    if (ctx->device < 0 || ctx->device >= kNoAllocMaxDevices) return BNN_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[ctx->device]) {
+        void *ptr = nullptr;
+        BNN_CUDA_TRY(ctx, cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+        if (!ptr) return BNN_ERR_CUDA;
+        g_noalloc_ptr[ctx->device] = ptr;
+    }
+    *out = static_cast<char *>(g_noalloc_ptr[ctx->device]);
+    return BNN_OK;
+}
+
+}  // namespace
+
+extern "C" size_t bnn_mlp_noalloc_max_bytes(void) { return kNoAllocBufferBytes; }
+
+extern "C" int bnn_mlp_forward_noalloc(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X, int64_t ldx,
+                                       int64_t batch, float *scores, int64_t lds) {
+    if (!ctx || batch < 0) return BNN_ERR_INVALID_ARG;
+    if (int st = check_desc(m)) return st;
+    if (batch == 0) return BNN_OK;
+    if (!X || !scores || ldx < m->layers[0].K || lds < m->layers[m->n_layers - 1].N) return BNN_ERR_INVALID_ARG;
+    // one activation buffer = batch rows of the widest hidden layer, packed; it must fit the built-in array
+    if (act_bytes(m, batch) > kNoAllocBufferBytes) return BNN_ERR_TOO_LARGE;
+    bnn_device_guard guard(ctx);
+    if (!guard.ok) return BNN_ERR_CUDA;
+    char *scratch = nullptr;
+    if (int st = noalloc_scratch(ctx, &scratch)) return st;
+    // Nothing in the scratch has to start at zero: every layer writes all words of its output rows, padding
+    // included, before the next layer reads them; what an earlier call left behind is never read.
+    return forward_device(ctx, m, X, ldx, batch, scores, lds, nullptr, scratch);
 }
