@@ -147,6 +147,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--variant", type=int, default=0, help="tiled-kernel inner loop: 0 default, 1 plain popc, 2 carry-save")
+    ap.add_argument("--engine", type=int, default=0, help="0 auto (tensor-core int8 engine for large shapes), 1 CUDA-core XOR-popcount only, 2 tensor")
     ap.add_argument("--no-extras", action="store_true", help="skip the GEMM / ConvNet side measurements and the CPU baseline")
     ap.add_argument("--gemm-size", type=int, default=8192)
     args = ap.parse_args()
@@ -174,6 +175,7 @@ def main():
     stream = torch.cuda.current_stream(local)
     ctx = binding.Context(local, stream)
     ctx.set_popc_variant(args.variant)
+    ctx.set_engine(args.engine)
 
     def sync_all():
         torch.cuda.synchronize()
@@ -192,7 +194,9 @@ def main():
     X = torch.from_numpy(case["X"]).to(dev)
     scores = torch.empty(BATCH, SIZES[-1], dtype=torch.float32, device=dev)
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
-    launches_per_step = len(SIZES) - 1
+    tensor_step = args.engine != 1          # batch 10000 qualifies for the tensor engine on every hidden layer
+    # per step: (weight expansion + GEMM) per hidden layer + output layer, or one kernel per layer on the CUDA-core path
+    launches_per_step = (2 * (len(SIZES) - 2) + 1) if tensor_step else (len(SIZES) - 1)
 
     def timed_steps(fn, steps, warmup):
         """CUDA events on the launch stream around each step; L2 flushed (untimed) before each step."""
@@ -247,6 +251,13 @@ def main():
             dist.destroy_process_group()
         return 0
 
+    # the same two layers on the CUDA-core XOR-popcount path (Eq. 8 as the paper computes it), for the popc roofline
+    ctx.set_engine(1)
+    popc_dense_times = timed_steps(lambda: ctx.binary_dense(act_in, hid["Wp"], hid["thr"], hid["flip"], BATCH, SIZES[2], SIZES[1],
+                                                            out=act_out), max(args.steps // 2, 3), 3) if rank == 0 else [1.0]
+    popc_mlp_times = timed_steps(lambda: ctx.mlp_forward(desc, X, BATCH, scores=scores), max(args.steps // 2, 3), 3) if rank == 0 else [1.0]
+    ctx.set_engine(args.engine)
+
     peaks = {}
     try:
         peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
@@ -259,6 +270,11 @@ def main():
     dense_ms = sum(dense_times) / len(dense_times)
     dense_ops = 2.0 * BATCH * SIZES[1] * SIZES[2]
     dense_ach = dense_ops / (dense_ms / 1e3) / 1e12
+    popc_dense_ms = sum(popc_dense_times) / len(popc_dense_times)
+    popc_dense_ach = dense_ops / (popc_dense_ms / 1e3) / 1e12
+    popc_mlp_ms = sum(popc_mlp_times) / len(popc_mlp_times)
+    bf16_peak = float(peaks.get("bf16_tflops") or 1590.0)
+    tensor_peak = 2.0 * bf16_peak           # int8 : bf16 nominal ratio 2 (4.5 vs 2.25 PFLOP/s dense)
     first_ms = sum(first_times) / len(first_times)
     first_ach = 2.0 * 8 * BATCH * SIZES[0] * SIZES[1] / (first_ms / 1e3) / 1e12
     mlp_ach = bit_ops_mlp(BATCH, SIZES) / (ms_per_step / 1e3) / 1e12
@@ -269,22 +285,34 @@ def main():
         "dtype": "int32", "data": "synthetic",
         "config": {"workload": "MNIST-shaped BNN MLP forward 784-4096-4096-4096-10 (8 bit-planes, 2 fused binary dense, float output), "
                                "batch 10000 per GPU, seed 1", "batch_per_gpu": BATCH, "parallelism": "replicas x%d" % world,
-                   "l2": "256 MiB written between timed steps (inputs fit in L2)", "popc_variant": args.variant},
+                   "l2": "256 MiB written between timed steps (inputs fit in L2)", "popc_variant": args.variant,
+                   "engine": {0: "auto (tensor-core int8 for the large layers)", 1: "CUDA-core XOR-popcount", 2: "tensor"}[args.engine]},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": BATCH * SIZES[0], "d2h_bytes_per_step": BATCH * SIZES[-1] * 4,
                 "ms_per_step": e2e_total_ms / args.steps},
         "gpu_launches": launches_per_step * args.steps,
-        "roofline": {"bound": "alu", "kernel": "k_bit_tile (fused binary dense 10000x4096x4096)", "achieved": dense_ach,
-                     "peak": popc_peak_tbitops, "unit": "Tbit-op/s", "frac": dense_ach / popc_peak_tbitops, "traffic": None,
-                     "peak_kind": "derived: %d SMs x 16 POPC/clk/SM x 32 bit-MAC x 2 x %.0f MHz (one POPC per 32-bit word); "
-                                  "carry-save kernels may exceed it" % (sm_count, sm_max_mhz),
-                     "ms_per_launch": dense_ms},
+        "roofline": ({"bound": "tensor", "kernel": "bnn_binary_dense 10000x4096x4096 on the tensor engine (k_expand_s8 x2 + k_umma_i8, "
+                                                    "timed as one call)", "achieved": dense_ach, "peak": tensor_peak, "unit": "TFLOP/s",
+                      "frac": dense_ach / tensor_peak, "traffic": None,
+                      "peak_kind": "int8 ops (2 per MAC); peak = 2 x measured bf16 burst %.1f TFLOP/s (nominal int8:bf16 ratio), "
+                                   "%s" % (bf16_peak, "of measured" if peaks else "of fallback"), "ms_per_launch": dense_ms}
+                     if tensor_step else
+                     {"bound": "alu", "kernel": "k_bit_tile (fused binary dense 10000x4096x4096)", "achieved": dense_ach,
+                      "peak": popc_peak_tbitops, "unit": "Tbit-op/s", "frac": dense_ach / popc_peak_tbitops, "traffic": 7299840,
+                      "peak_kind": "derived: %d SMs x 16 POPC/clk/SM x 32 bit-MAC x 2 x %.0f MHz (one POPC per 32-bit word); "
+                                   "carry-save kernels may exceed it" % (sm_count, sm_max_mhz),
+                      "ms_per_launch": dense_ms}),
+        "popc_path": {"what": "the same layer and the same MLP step on the CUDA-core XOR-popcount kernels (engine 1)",
+                      "dense_layer_ms": popc_dense_ms, "dense_tbitops": popc_dense_ach,
+                      "dense_frac_of_popc_peak": popc_dense_ach / popc_peak_tbitops, "popc_peak_tbitops": popc_peak_tbitops,
+                      "mlp_ms_per_step": popc_mlp_ms, "mlp_images_per_s": BATCH / (popc_mlp_ms / 1e3)},
         "mlp_step": {"achieved_tbitops": mlp_ach, "frac_of_popc_peak": mlp_ach / popc_peak_tbitops,
                      "first_layer_ms": first_ms, "first_layer_tbitops": first_ach, "dense_layer_ms": dense_ms},
     }
 
     if not args.no_extras and world == 1:
-        line["gemm"] = bench_gemm(ctx, args.gemm_size, popc_peak_tbitops, timed_steps)
+        line["gemm"] = bench_gemm(ctx, args.gemm_size, popc_peak_tbitops, timed_steps, args.engine)
+        ctx.set_workspace(ws)
         line["convnet"] = bench_convnet(ctx, timed_steps)
         dt, cores = time_oracle_mlp(case, 2000)
         line["cpu_baseline"] = {"value": 2000 / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
@@ -298,18 +326,26 @@ def main():
     return 0
 
 
-def bench_gemm(ctx, n, peak, timed_steps):
-    """Binary GEMM n^3 (the paper's 8192^3 by default): Tbit-op/s = 2 n^3 / t."""
+def bench_gemm(ctx, n, peak, timed_steps, engine):
+    """Binary GEMM n^3 (the paper's 8192^3 by default) from packed operands to int32: Tbit-op/s = 2 n^3 / t,
+    on the CUDA-core XOR-popcount kernel and on the selected engine."""
     import torch
     words = n // 32
     g = torch.Generator(device="cuda").manual_seed(2)
     Ap = torch.randint(-2**31, 2**31 - 1, (n, words), dtype=torch.int32, device="cuda", generator=g)
     Bp = torch.randint(-2**31, 2**31 - 1, (n, words), dtype=torch.int32, device="cuda", generator=g)
     C = torch.empty(n, n, dtype=torch.int32, device="cuda")
-    t = timed_steps(lambda: ctx.xnor_gemm(Ap, Bp, n, n, n, C=C), 5, 3)
-    ms = sum(t) / len(t)
-    tb = 2.0 * n ** 3 / (ms / 1e3) / 1e12
-    return {"shape": [n, n, n], "ms": ms, "tbitops": tb, "frac_of_popc_peak": tb / peak}
+    gws = torch.empty(max(ctx.gemm_workspace_bytes(n, n, n), 256), dtype=torch.uint8, device="cuda")
+    ctx.set_workspace(gws)
+    out = {"shape": [n, n, n]}
+    for name, eng in (("popc", 1), ("selected_engine", engine)):
+        ctx.set_engine(eng)
+        t = timed_steps(lambda: ctx.xnor_gemm(Ap, Bp, n, n, n, C=C), 5, 3)
+        ms = sum(t) / len(t)
+        tb = 2.0 * n ** 3 / (ms / 1e3) / 1e12
+        out[name] = {"ms": ms, "tbitops": tb, "frac_of_popc_peak": tb / peak}
+    ctx.set_engine(engine)
+    return out
 
 
 def bench_convnet(ctx, timed_steps):

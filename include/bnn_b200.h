@@ -66,6 +66,22 @@ BNN_API int bnn_set_workspace(bnn_ctx *ctx, void *dptr, size_t bytes);
  * word (Eq. 8 as written), 2 = carry-save: a LOP3 full adder merges two XOR words before the POPC. */
 BNN_API int bnn_set_popc_variant(bnn_ctx *ctx, int variant);
 
+/* Which kernels evaluate the large products (results are the same integers either way):
+ *   0 = automatic: the tensor-core engine for large shapes when the context's workspace is big enough
+ *       (bnn_gemm_workspace_bytes / bnn_mlp_workspace_bytes), otherwise the CUDA-core kernels;
+ *   1 = CUDA-core XOR-popcount kernels only (Eq. 8 as the paper computes it);
+ *   2 = tensor-core engine wherever the shape qualifies; BNN_ERR_WORKSPACE if the workspace is too small.
+ * The tensor-core engine expands the packed operands to one signed byte per value in the workspace and
+ * multiplies them with int8 tensor-core instructions (Section 4: on +-1 inputs the binary kernel and an ordinary
+ * matrix product return identical outputs). */
+BNN_API int bnn_set_engine(bnn_ctx *ctx, int engine);
+/* Workspace bytes bnn_xnor_gemm / bnn_binary_dense need to run M x N x K on the tensor-core engine
+ * (0 if the shape does not qualify for it). */
+BNN_API size_t bnn_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
+/* Synchronises the context's stream and returns BNN_ERR_DEVICE_STATUS if a kernel gave up on one of its
+ * bounded waits since the last call (its outputs are then undefined), BNN_OK otherwise. */
+BNN_API int bnn_device_status(bnn_ctx *ctx);
+
 /* ---------------------------------------------------------------------------------------------
  * Sign-pack (Eq. 1 followed by the 32-per-word concatenation of Section 4).
  *   src        rows x cols elements of `dtype`, row-major, leading dimension src_ld elements.

@@ -18,12 +18,14 @@ LIB_PATH = os.path.join(_HERE, "libbnn_b200.so")
 
 BNN_F32, BNN_F16, BNN_I8 = 0, 1, 2
 VARIANT_AUTO, VARIANT_PLAIN, VARIANT_CSA = 0, 1, 2
+ENGINE_AUTO, ENGINE_POPC, ENGINE_TENSOR = 0, 1, 2
 
 EXPORTS = (
     "bnn_create", "bnn_destroy", "bnn_status_string", "bnn_last_cuda_error", "bnn_set_workspace",
     "bnn_set_popc_variant", "bnn_pack_signs", "bnn_xnor_gemm", "bnn_binary_dense", "bnn_first_layer_bitplanes",
     "bnn_binary_conv2d", "bnn_mlp_workspace_bytes", "bnn_mlp_forward", "bnn_mlp_forward_host",
-    "bnn_fold_batchnorm", "bnn_mlp_noalloc_max_bytes", "bnn_mlp_forward_noalloc",
+    "bnn_fold_batchnorm", "bnn_mlp_noalloc_max_bytes", "bnn_mlp_forward_noalloc", "bnn_set_engine",
+    "bnn_gemm_workspace_bytes", "bnn_device_status",
 )
 
 
@@ -66,6 +68,10 @@ def lib() -> ctypes.CDLL:
         L.bnn_last_cuda_error.argtypes = [vp]
         L.bnn_set_workspace.argtypes = [vp, vp, c_size_t]
         L.bnn_set_popc_variant.argtypes = [vp, c_int]
+        L.bnn_set_engine.argtypes = [vp, c_int]
+        L.bnn_gemm_workspace_bytes.argtypes = [i64, i64, i64]
+        L.bnn_gemm_workspace_bytes.restype = c_size_t
+        L.bnn_device_status.argtypes = [vp]
         L.bnn_pack_signs.argtypes = [vp, vp, c_int, i64, i64, i64, c_int, c_int, vp, i64]
         L.bnn_xnor_gemm.argtypes = [vp, vp, i64, vp, i64, vp, i64, i64, i64, i64]
         L.bnn_binary_dense.argtypes = [vp, vp, i64, vp, i64, vp, vp, vp, i64, i64, i64, i64]
@@ -139,6 +145,16 @@ class Context:
             self._ck(lib().bnn_set_workspace(self._h, None, 0), "bnn_set_workspace")
         else:
             self._ck(lib().bnn_set_workspace(self._h, _ptr(ws), ws.numel() * ws.element_size()), "bnn_set_workspace")
+
+    def set_engine(self, engine: int):
+        self._ck(lib().bnn_set_engine(self._h, engine), "bnn_set_engine")
+
+    def gemm_workspace_bytes(self, M: int, N: int, K: int) -> int:
+        return int(lib().bnn_gemm_workspace_bytes(M, N, K))
+
+    def device_status(self):
+        """Synchronises the stream; raises if a kernel reported that one of its bounded waits gave up."""
+        self._ck(lib().bnn_device_status(self._h), "bnn_device_status")
 
     def set_popc_variant(self, variant: int):
         self._ck(lib().bnn_set_popc_variant(self._h, variant), "bnn_set_popc_variant")

@@ -17,6 +17,7 @@ extern "C" int bnn_create(bnn_ctx **out, int device, void *cuda_stream) {
     c->last_cuda_error = 0;
     c->sm_count = 0;
     c->variant = 0;
+    c->engine = 0;
     if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
         delete c;
         return BNN_ERR_CUDA;
@@ -47,6 +48,12 @@ extern "C" const char *bnn_status_string(int status) {
 extern "C" int bnn_set_popc_variant(bnn_ctx *ctx, int variant) {
     if (!ctx || variant < 0 || variant > 2) return BNN_ERR_INVALID_ARG;
     ctx->variant = variant;
+    return BNN_OK;
+}
+
+extern "C" int bnn_set_engine(bnn_ctx *ctx, int engine) {
+    if (!ctx || engine < 0 || engine > 2) return BNN_ERR_INVALID_ARG;
+    ctx->engine = engine;
     return BNN_OK;
 }
 

@@ -192,6 +192,19 @@ static int gemm_like(bnn_ctx *ctx, const uint32_t *Ap, int64_t lda_w, const uint
     if (!C && !out) return BNN_ERR_INVALID_ARG;
     bnn_device_guard guard(ctx);
     if (!guard.ok) return BNN_ERR_CUDA;
+    if (ctx->engine != BNN_ENGINE_POPC && bnn_umma_shape_ok(M, N, K)) {
+        // tensor-core engine: both packed operands are expanded to signed bytes in the workspace first
+        const size_t need = bnn_umma_operand_bytes(M, K) + bnn_umma_operand_bytes(N, K);
+        if (ctx->ws && ctx->ws_bytes >= need) {
+            int8_t *A8 = static_cast<int8_t *>(ctx->ws);
+            int8_t *B8 = A8 + bnn_umma_operand_bytes(M, K);
+            const int64_t ld8 = bnn_umma_operand_ld(K);
+            if (int st = bnn_umma_expand(ctx, Ap, lda_w, M, K, A8)) return st;
+            if (int st = bnn_umma_expand(ctx, Bp, ldb_w, N, K, B8)) return st;
+            return bnn_umma_gemm(ctx, A8, ld8, false, B8, ld8, M, N, K, C, ldc, thr, flip, out, ldo_w, nullptr, 0);
+        }
+        if (ctx->engine == BNN_ENGINE_TENSOR) return BNN_ERR_WORKSPACE;
+    }
     if (M <= 32 && skinny_fits(M, K)) {
         SkinnyArgs s{};
         s.S = Ap; s.lds_w = lda_w; s.RS = M;
@@ -236,9 +249,26 @@ extern "C" int bnn_first_layer_bitplanes(bnn_ctx *ctx, const uint8_t *X, int64_t
     }
     bnn_device_guard guard(ctx);
     if (!guard.ok) return BNN_ERR_CUDA;
+    if (ctx->engine != BNN_ENGINE_POPC && bnn_umma_shape_ok(M, N, K) && (ldx % 16) == 0 && bnn_aligned16(X)) {
+        // tensor-core engine: the 8-bit inputs are used as they are (unsigned bytes), only the weights are expanded;
+        // the 8 bit-plane products of Eq. 7 collapse into the byte product the tensor core forms in one step
+        const size_t need = bnn_umma_operand_bytes(N, K);
+        if (ctx->ws && ctx->ws_bytes >= need) {
+            int8_t *W8 = static_cast<int8_t *>(ctx->ws);
+            if (int st = bnn_umma_expand(ctx, Wp, ldw_w, N, K, W8)) return st;
+            return bnn_umma_gemm(ctx, X, ldx, true, W8, bnn_umma_operand_ld(K), M, N, K, out_sums, lds, thr, flip, out_bits,
+                                 ldo_w, nullptr, 0);
+        }
+        if (ctx->engine == BNN_ENGINE_TENSOR) return BNN_ERR_WORKSPACE;
+    }
     Args a{};
     a.X = X; a.ldx = ldx; a.B = Wp; a.ldb = ldw_w;
     a.M = M; a.N = N; a.K = K;
     a.C = out_sums; a.ldc = lds; a.out = out_bits; a.ldo = ldo_w; a.thr = thr; a.flip = flip;
     return bnn_launch_tile_planes(ctx, a);
+}
+
+extern "C" size_t bnn_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+    if (M <= 0 || N <= 0 || K <= 0 || !bnn_umma_shape_ok(M, N, K)) return 0;
+    return bnn_umma_operand_bytes(M, K) + bnn_umma_operand_bytes(N, K);
 }

@@ -12,3 +12,16 @@ int bnn_launch_tile_planes(bnn_ctx *ctx, const bnn_tile::Args &a);
 int bnn_output_scores(bnn_ctx *ctx, const uint32_t *Ap, int64_t lda_w, const uint32_t *Wp, int64_t ldw_w,
                       const float *gamma, const float *beta, const float *mean, const float *var, double eps,
                       float *scores, int64_t lds, int64_t M, int64_t N, int64_t K);
+
+// ---- tensor-core int8 engine (bnn_umma.cu)
+enum { BNN_ENGINE_AUTO = 0, BNN_ENGINE_POPC = 1, BNN_ENGINE_TENSOR = 2 };
+size_t bnn_umma_operand_bytes(int64_t rows, int64_t K);   // bytes of an expanded (one byte per value) operand
+int64_t bnn_umma_operand_ld(int64_t K);                   // its row pitch in bytes (multiple of 128)
+int bnn_umma_expand(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t rows, int64_t K, int8_t *dst);
+int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, const int8_t *B8, int64_t ldb8, int64_t M,
+                  int64_t N, int64_t K, int32_t *C, int64_t ldc, const int32_t *thr, const uint32_t *flip, uint32_t *out,
+                  int64_t ldo, int8_t *out8, int64_t ldo8);
+// Shapes for which the tensor engine is worth its expansion pass.
+static inline bool bnn_umma_shape_ok(int64_t M, int64_t N, int64_t K) {
+    return M >= 256 && N >= 128 && K >= 128 && (double)M * (double)N * (double)K >= 1.0e9;
+}

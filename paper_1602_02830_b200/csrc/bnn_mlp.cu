@@ -56,11 +56,80 @@ int forward_device(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X, int64_
                              batch, O.N, O.K);
 }
 
+// Bytes the tensor-core engine adds: two byte-per-value activation buffers and one expanded weight matrix.
+size_t tensor_act8_bytes(const bnn_mlp_desc *m, int64_t batch) {
+    int64_t widest = 0;
+    for (int k = 0; k < m->n_layers - 1; ++k) widest = m->layers[k].N > widest ? m->layers[k].N : widest;
+    return bnn_umma_operand_bytes(batch, widest);
+}
+size_t tensor_w8_bytes(const bnn_mlp_desc *m) {
+    size_t w = 0;
+    for (int k = 0; k < m->n_layers - 1; ++k) {
+        const size_t b = bnn_umma_operand_bytes(m->layers[k].N, m->layers[k].K);
+        w = b > w ? b : w;
+    }
+    return w;
+}
+bool tensor_applies(const bnn_ctx *ctx, const bnn_mlp_desc *m, int64_t batch) {
+    if (ctx->engine == BNN_ENGINE_POPC) return false;
+    for (int k = 0; k < m->n_layers - 1; ++k)
+        if (!bnn_umma_shape_ok(batch, m->layers[k].N, m->layers[k].K)) return false;
+    return true;
+}
+
+// The same layer sequence on the tensor-core engine.  Every hidden layer writes its signs twice: packed (the
+// ABI's activation format, read by the output layer and by hidden_out) and as +-1 bytes (next layer's operand).
+int forward_device_tensor(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X, int64_t ldx, int64_t batch, float *scores,
+                          int64_t lds, uint32_t *const *hidden_out, char *ws) {
+    const size_t ab = act_bytes(m, batch), a8 = tensor_act8_bytes(m, batch);
+    uint32_t *bits[2] = {reinterpret_cast<uint32_t *>(ws), reinterpret_cast<uint32_t *>(ws + ab)};
+    int8_t *act8[2] = {reinterpret_cast<int8_t *>(ws + 2 * ab), reinterpret_cast<int8_t *>(ws + 2 * ab + a8)};
+    int8_t *W8 = reinterpret_cast<int8_t *>(ws + 2 * ab + 2 * a8);
+    const int L = m->n_layers;
+    const uint32_t *cur = nullptr;
+    const int8_t *cur8 = nullptr;
+    for (int k = 0; k < L - 1; ++k) {
+        const bnn_layer_desc &D = m->layers[k];
+        uint32_t *dst = bits[k & 1];
+        int8_t *dst8 = act8[k & 1];
+        const int64_t ldo = act_ld(D.N);
+        if (int st = bnn_umma_expand(ctx, D.Wp, D.ldw_w, D.N, D.K, W8)) return st;
+        const bool need8 = (k < L - 2);
+        int st;
+        if (k == 0)
+            st = bnn_umma_gemm(ctx, X, ldx, true, W8, bnn_umma_operand_ld(D.K), batch, D.N, D.K, nullptr, 0, D.thr, D.flip, dst,
+                               ldo, need8 ? dst8 : nullptr, bnn_umma_operand_ld(D.N));
+        else
+            st = bnn_umma_gemm(ctx, cur8, bnn_umma_operand_ld(D.K), false, W8, bnn_umma_operand_ld(D.K), batch, D.N, D.K, nullptr,
+                               0, D.thr, D.flip, dst, ldo, need8 ? dst8 : nullptr, bnn_umma_operand_ld(D.N));
+        if (st) return st;
+        if (hidden_out && hidden_out[k])
+            BNN_CUDA_TRY(ctx, cudaMemcpyAsync(hidden_out[k], dst, (size_t)batch * ldo * 4, cudaMemcpyDeviceToDevice,
+                                              ctx->stream));
+        cur = dst;
+        cur8 = dst8;
+    }
+    const bnn_layer_desc &O = m->layers[L - 1];
+    return bnn_output_scores(ctx, cur, act_ld(O.K), O.Wp, O.ldw_w, O.gamma, O.beta, O.mean, O.var, O.eps, scores, lds,
+                             batch, O.N, O.K);
+}
+
+size_t tensor_extra_bytes(const bnn_mlp_desc *m, int64_t batch) {
+    return 2 * tensor_act8_bytes(m, batch) + tensor_w8_bytes(m);
+}
+
 }  // namespace
 
 extern "C" size_t bnn_mlp_workspace_bytes(const bnn_mlp_desc *m, int64_t batch, int host_io) {
     if (check_desc(m) != BNN_OK || batch <= 0) return 0;
     size_t b = 2 * act_bytes(m, batch);
+    // room for the tensor-core engine when the shapes qualify for it (whatever engine is selected later)
+    {
+        bool all = true;
+        for (int k = 0; k < m->n_layers - 1; ++k)
+            if (!bnn_umma_shape_ok(batch, m->layers[k].N, m->layers[k].K)) all = false;
+        if (all) b += tensor_extra_bytes(m, batch);
+    }
     if (host_io) {
         b += round256((size_t)batch * m->layers[0].K);                        // staged input
         b += round256((size_t)batch * m->layers[m->n_layers - 1].N * 4);      // staged scores
@@ -77,6 +146,8 @@ extern "C" int bnn_mlp_forward(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_
     if (!ctx->ws || ctx->ws_bytes < bnn_mlp_workspace_bytes(m, batch, 0)) return BNN_ERR_WORKSPACE;
     bnn_device_guard guard(ctx);
     if (!guard.ok) return BNN_ERR_CUDA;
+    if (tensor_applies(ctx, m, batch) && (ldx % 16) == 0 && bnn_aligned16(X))
+        return forward_device_tensor(ctx, m, X, ldx, batch, scores, lds, hidden_out, static_cast<char *>(ctx->ws));
     return forward_device(ctx, m, X, ldx, batch, scores, lds, hidden_out, static_cast<char *>(ctx->ws));
 }
 
@@ -91,12 +162,16 @@ extern "C" int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const u
     bnn_device_guard guard(ctx);
     if (!guard.ok) return BNN_ERR_CUDA;
     char *ws = static_cast<char *>(ctx->ws);
-    const size_t ab = act_bytes(m, batch);
-    uint8_t *Xd = reinterpret_cast<uint8_t *>(ws + 2 * ab);
-    float *Sd = reinterpret_cast<float *>(ws + 2 * ab + round256((size_t)batch * K0));
+    const bool tensor = tensor_applies(ctx, m, batch) && (K0 % 16) == 0;
+    // staging buffers sit behind everything the device-side forward may use
+    const size_t fwd = bnn_mlp_workspace_bytes(m, batch, 0);
+    uint8_t *Xd = reinterpret_cast<uint8_t *>(ws + fwd);
+    float *Sd = reinterpret_cast<float *>(ws + fwd + round256((size_t)batch * K0));
     BNN_CUDA_TRY(ctx, cudaMemcpy2DAsync(Xd, (size_t)K0, X_host, (size_t)ldx, (size_t)K0, (size_t)batch,
                                         cudaMemcpyHostToDevice, ctx->stream));
-    if (int st = forward_device(ctx, m, Xd, K0, batch, Sd, NL, nullptr, ws)) return st;
+    if (int st = tensor ? forward_device_tensor(ctx, m, Xd, K0, batch, Sd, NL, nullptr, ws)
+                        : forward_device(ctx, m, Xd, K0, batch, Sd, NL, nullptr, ws))
+        return st;
     BNN_CUDA_TRY(ctx, cudaMemcpy2DAsync(scores_host, (size_t)lds * 4, Sd, (size_t)NL * 4, (size_t)NL * 4, (size_t)batch,
                                         cudaMemcpyDeviceToHost, ctx->stream));
     return BNN_OK;

@@ -1,0 +1,395 @@
+// Tensor-core engine for the large products: the +-1 (or 8-bit x +-1) product evaluated EXACTLY by the
+// 5th-generation tensor cores as an int8 GEMM with int32 accumulation in tensor memory.
+//
+//   Section 4 states that the binary kernel and an ordinary matrix product return identical outputs on +-1
+//   inputs.  On sm_100a the ordinary product has a far higher ceiling than the POPC pipe (8192 int8 MACs vs
+//   512 bit-MACs per clock per SM), so for large shapes the packed operands are expanded to one signed byte
+//   per value (a streaming pass) and multiplied with tcgen05.mma kind::i8.  Results are the same integers.
+//
+// Kernel k_umma_i8 (one 128 x 256 output tile per CTA, 192 threads):
+//   warp 0    TMA producer: cp.async.bulk.tensor 2-D loads of 128-byte-wide K slices (128B swizzle) of both
+//             operands into a 4-stage shared-memory ring, completion on mbarriers;
+//   warp 1    allocates 256 TMEM columns, then one lane issues tcgen05.mma (M=128, N=256, K=32) four times per
+//             stage and releases the stage with tcgen05.commit;
+//   warps 2-5 epilogue: tcgen05.ld of the int32 accumulators (each thread owns one output row, 32 columns at
+//             a time), then either int32 stores, or the BatchNorm-folded threshold + Sign + repack to one
+//             32-bit word per 32 columns (and, for the next layer, the same signs as bytes).
+// Every wait is bounded: after the limit the kernel records an error code and runs to its end without
+// touching the accumulators, so a failure surfaces as BNN_ERR_DEVICE_STATUS instead of a hang.
+#include "bnn_internal.cuh"
+#include <cuda.h>
+#include <mutex>
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 128;     // BK in bytes = int8 elements
+constexpr int STAGES = 4;
+constexpr int NTHREADS = 192;
+constexpr uint32_t A_BYTES = BM * BK, B_BYTES = BN * BK;
+constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr uint32_t TMEM_COLS = 256;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // a wait gives up after 2 s of wall clock
+
+__device__ int g_umma_error;                    // 0 = fine; otherwise a code saying which wait gave up
+
+struct UmmaArgs {
+    int64_t M, N;
+    int k_iters;            // ceil(K_bytes / BK)
+    uint32_t idesc;
+    int32_t *C; int64_t ldc;                     // optional int32 output
+    uint32_t *out; int64_t ldo;                  // optional packed sign output
+    int8_t *out8; int64_t ldo8;                  // optional +-1 byte output (next layer's operand)
+    const int32_t *thr; const uint32_t *flip;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait on a phase parity.  Returns false if the limit ran out.
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    unsigned long long t0 = 0;
+    for (uint32_t i = 0;; ++i) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+        if ((i & 63u) == 63u) {
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) return false;
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+// Shared-memory matrix descriptor: K-major tile, rows of 128 bytes, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = (uint64_t)((addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)(1024u >> 4) << 32;   // stride byte offset
+    d |= 1ull << 46;                      // descriptor version of sm_100
+    d |= 2ull << 61;                      // SWIZZLE_128B
+    return d;
+}
+__device__ __forceinline__ void umma_i8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+struct __align__(8) Control {
+    uint64_t full[STAGES];
+    uint64_t empty[STAGES];
+    uint64_t accum;
+    uint32_t tmem_base;
+    uint32_t failed;
+    int32_t thr[BN];
+    uint32_t flip[BN / 32];
+};
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const UmmaArgs p) {
+    extern __shared__ uint8_t smem_raw[];
+    // operand tiles need 1024-byte alignment for the 128-byte swizzle pattern
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    Control *ctl = reinterpret_cast<Control *>(tiles + STAGES * STAGE_BYTES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t tiles_m = (p.M + BM - 1) / BM;
+    const int64_t tile_m = blockIdx.x % tiles_m, tile_n = blockIdx.x / tiles_m;
+    const int64_t m0 = tile_m * BM, n0 = tile_n * BN;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
+        mbar_init(smem_u32(&ctl->accum), 1);
+        ctl->failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (warp >= 2 && p.out) {
+        for (int e = threadIdx.x - 64; e < BN; e += 128) ctl->thr[e] = (n0 + e < p.N) ? p.thr[n0 + e] : 0x7fffffff;
+        if (threadIdx.x - 64 < BN / 32) {
+            const int64_t w = (n0 >> 5) + (threadIdx.x - 64);
+            ctl->flip[threadIdx.x - 64] = (p.flip && w * 32 < p.N) ? p.flip[w] : 0u;
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ---------------- TMA producer
+        if (lane == 0) {
+            for (int it = 0; it < p.k_iters; ++it) {
+                const int s = it % STAGES;
+                if (it >= STAGES) {
+                    if (!mbar_wait(smem_u32(&ctl->empty[s]), ((it / STAGES) - 1) & 1)) { ctl->failed = 1; atomicExch(&g_umma_error, 1); break; }
+                }
+                const uint32_t bar = smem_u32(&ctl->full[s]);
+                mbar_expect_tx(bar, STAGE_BYTES);
+                tma_load_2d(smem_u32(tiles + s * STAGE_BYTES), &mapA, it * BK, (int)m0, bar);
+                tma_load_2d(smem_u32(tiles + s * STAGE_BYTES + A_BYTES), &mapB, it * BK, (int)n0, bar);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer
+        if (lane == 0) {
+            bool ok = true;
+            for (int it = 0; it < p.k_iters && ok; ++it) {
+                const int s = it % STAGES;
+                if (!mbar_wait(smem_u32(&ctl->full[s]), (it / STAGES) & 1)) { ctl->failed = 2; atomicExch(&g_umma_error, 2); ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint64_t adesc = smem_desc_sw128(smem_u32(tiles + s * STAGE_BYTES));
+                const uint64_t bdesc = smem_desc_sw128(smem_u32(tiles + s * STAGE_BYTES + A_BYTES));
+#pragma unroll
+                for (int k = 0; k < BK / 32; ++k)   // 32 bytes of K per instruction: start address advances by 32 B (>> 4 = 2)
+                    umma_i8(tmem_base, adesc + 2 * k, bdesc + 2 * k, p.idesc, (it > 0 || k > 0) ? 1u : 0u);
+                umma_commit(smem_u32(&ctl->empty[s]));      // stage may be refilled once these MMAs have read it
+            }
+            umma_commit(smem_u32(&ctl->accum));             // accumulators complete (arrives even after a failure)
+        }
+    } else {
+        // ---------------- epilogue: warps 2..5 own TMEM lanes 32*(warp%4) .. +31
+        const int q = warp & 3;
+        const int row_in_tile = 32 * q + lane;
+        const int64_t row = m0 + row_in_tile;
+        bool ok = mbar_wait(smem_u32(&ctl->accum), 0);
+        if (!ok) { ctl->failed = 3; atomicExch(&g_umma_error, 3); }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        ok = ok && (ctl->failed == 0);
+        if (ok && p.k_iters > 0) {
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                const int64_t col0 = n0 + 32 * c;
+                if (col0 >= p.N) break;                      // uniform over the warp
+                uint32_t r[32];
+                tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * c), r);
+                if (row < p.M) {
+                    if (p.C) {
+                        int32_t *dst = p.C + row * p.ldc + col0;
+                        if (col0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4)
+                                *reinterpret_cast<int4 *>(dst + j) = make_int4((int)r[j], (int)r[j + 1], (int)r[j + 2], (int)r[j + 3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + j < p.N) dst[j] = (int32_t)r[j];
+                        }
+                    }
+                    if (p.out) {
+                        uint32_t word = 0u;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) word |= (uint32_t)((int32_t)r[j] >= ctl->thr[32 * c + j]) << j;
+                        word ^= ctl->flip[c];
+                        if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;      // columns beyond N stay 0
+                        p.out[row * p.ldo + (col0 >> 5)] = word;
+                        if (p.out8) {
+                            int8_t *d8 = p.out8 + row * p.ldo8 + col0;
+                            uint32_t b[8];
+#pragma unroll
+                            for (int g = 0; g < 8; ++g) {
+                                // 4 sign bits -> 4 bytes of +1 (0x01) / -1 (0xff)
+                                const uint32_t t = (((word >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u;
+                                b[g] = ~(t * 0xfeu);
+                            }
+                            if (col0 + 32 <= p.N) {
+                                *reinterpret_cast<uint4 *>(d8) = make_uint4(b[0], b[1], b[2], b[3]);
+                                *reinterpret_cast<uint4 *>(d8 + 16) = make_uint4(b[4], b[5], b[6], b[7]);
+                            } else {
+                                for (int j = 0; j < 32; ++j)
+                                    if (col0 + j < p.N) d8[j] = ((word >> j) & 1u) ? (int8_t)1 : (int8_t)-1;
+                                    else if (col0 + j < p.ldo8) d8[j] = 0;
+                            }
+                        }
+                    }
+                }
+            }
+        }
+        // K == 0: the empty sum
+        if (ok && p.k_iters == 0 && row < p.M) {
+            for (int64_t col = n0; col < min(n0 + (int64_t)BN, p.N); ++col) {
+                if (p.C) p.C[row * p.ldc + col] = 0;
+            }
+        }
+        // padding words of the packed output
+        if (p.out && row < p.M && n0 + BN >= p.N) {
+            for (int64_t w = (p.N + 31) >> 5; w < p.ldo; ++w) p.out[row * p.ldo + w] = 0u;
+        }
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Packed signs -> one signed byte per value (+1 = 0x01, -1 = 0xff); bytes at or beyond K are 0.
+// One thread per 32-bit word = 32 output bytes (two 128-bit stores).
+__global__ void __launch_bounds__(256) k_expand_s8(const uint32_t *__restrict__ src, int64_t ld_w, int64_t rows, int64_t K,
+                                                   int8_t *__restrict__ dst, int64_t ld8) {
+    const int64_t wpr = ld8 >> 5;            // words per output row (ld8 is a multiple of 32)
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= rows * wpr) return;
+    const int64_t r = idx / wpr, w = idx - r * wpr;
+    const int64_t Kw = (K + 31) >> 5;
+    uint32_t bits = 0u, valid = 0u;
+    if (w < Kw) {
+        bits = src[r * ld_w + w];
+        valid = (w == Kw - 1 && (K & 31)) ? ((1u << (K & 31)) - 1u) : 0xffffffffu;
+    }
+    uint32_t b[8];
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+        const uint32_t t = (((bits >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u;      // 0/1 bytes
+        const uint32_t v = (((valid >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u;
+        b[g] = (~(t * 0xfeu)) & (v * 0xffu);
+    }
+    uint4 *d = reinterpret_cast<uint4 *>(dst + r * ld8 + 32 * w);
+    d[0] = make_uint4(b[0], b[1], b[2], b[3]);
+    d[1] = make_uint4(b[4], b[5], b[6], b[7]);
+}
+
+typedef CUresult (*encode_fn_t)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+std::mutex g_encode_mutex;
+encode_fn_t g_encode = nullptr;
+
+int get_encode(bnn_ctx *ctx, encode_fn_t *out) {
+    std::lock_guard<std::mutex> lock(g_encode_mutex);
+    if (!g_encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        BNN_CUDA_TRY(ctx, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+        if (!fn || qres != cudaDriverEntryPointSuccess) return BNN_ERR_CUDA;
+        g_encode = reinterpret_cast<encode_fn_t>(fn);
+    }
+    *out = g_encode;
+    return BNN_OK;
+}
+
+// 2-D byte tensor rows x kbytes (row pitch ld bytes), box 128 bytes x box_rows, 128-byte swizzle, zero fill outside.
+int make_map(bnn_ctx *ctx, CUtensorMap *map, const void *base, int64_t rows, int64_t kbytes, int64_t ld, int box_rows) {
+    encode_fn_t enc;
+    if (int st = get_encode(ctx, &enc)) return st;
+    cuuint64_t dims[2] = {(cuuint64_t)kbytes, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld};
+    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { ctx->last_cuda_error = (int)r; return BNN_ERR_CUDA; }
+    return BNN_OK;
+}
+
+}  // namespace
+
+size_t bnn_umma_operand_bytes(int64_t rows, int64_t K) {
+    const int64_t ld8 = ((K + 127) / 128) * 128;
+    return ((size_t)rows * ld8 + 255) & ~size_t(255);
+}
+int64_t bnn_umma_operand_ld(int64_t K) { return ((K + 127) / 128) * 128; }
+
+int bnn_umma_expand(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t rows, int64_t K, int8_t *dst) {
+    const int64_t ld8 = bnn_umma_operand_ld(K);
+    const int64_t total = rows * (ld8 >> 5);
+    if (total == 0) return BNN_OK;
+    const int64_t blocks = (total + 255) / 256;
+    if (blocks > 0x7fffffff) return BNN_ERR_INVALID_ARG;
+    k_expand_s8<<<(unsigned)blocks, 256, 0, ctx->stream>>>(src, ld_w, rows, K, dst, ld8);
+    return bnn_check_launch(ctx);
+}
+
+// C / bits = A8 (M x K bytes, pitch lda8; unsigned if a_unsigned) times B8^T (N x K signed bytes, pitch ldb8).
+int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, const int8_t *B8, int64_t ldb8, int64_t M,
+                  int64_t N, int64_t K, int32_t *C, int64_t ldc, const int32_t *thr, const uint32_t *flip, uint32_t *out,
+                  int64_t ldo, int8_t *out8, int64_t ldo8) {
+    if (M == 0 || N == 0) return BNN_OK;
+    if ((lda8 & 15) || (ldb8 & 15) || !bnn_aligned16(A8) || !bnn_aligned16(B8)) return BNN_ERR_ALIGNMENT;
+    if (M > 0x7fffffff || N > 0x7fffffff) return BNN_ERR_INVALID_ARG;
+    CUtensorMap mapA, mapB;
+    const int64_t kb = ((K + 15) / 16) * 16;      // extent along K in bytes; beyond it TMA fills zeros
+    if (K > 0) {
+        if (int st = make_map(ctx, &mapA, A8, M, kb <= lda8 ? kb : lda8, lda8, BM)) return st;
+        if (int st = make_map(ctx, &mapB, B8, N, kb <= ldb8 ? kb : ldb8, ldb8, BN)) return st;
+    } else {
+        memset(&mapA, 0, sizeof(mapA));
+        memset(&mapB, 0, sizeof(mapB));
+    }
+    UmmaArgs a{};
+    a.M = M; a.N = N;
+    a.k_iters = (int)((K + BK - 1) / BK);
+    a.idesc = (2u << 4) | ((a_unsigned ? 0u : 1u) << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+    a.C = C; a.ldc = ldc; a.out = out; a.ldo = ldo; a.out8 = out8; a.ldo8 = ldo8; a.thr = thr; a.flip = flip;
+    const size_t smem = (size_t)STAGES * STAGE_BYTES + sizeof(Control) + 1024;
+    static std::mutex attr_mutex;
+    static bool attr_set[64] = {};
+    {
+        std::lock_guard<std::mutex> lock(attr_mutex);
+        if (ctx->device < 64 && !attr_set[ctx->device]) {
+            BNN_CUDA_TRY(ctx, cudaFuncSetAttribute(k_umma_i8, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            attr_set[ctx->device] = true;
+        }
+    }
+    const int64_t tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
+    if (tiles > 0x7fffffff) return BNN_ERR_INVALID_ARG;
+    k_umma_i8<<<(unsigned)tiles, NTHREADS, smem, ctx->stream>>>(mapA, mapB, a);
+    return bnn_check_launch(ctx);
+}
+
+// Reads (and clears) the error word the tensor-core kernel sets when one of its bounded waits gives up.
+// Synchronises the context's stream.
+extern "C" int bnn_device_status(bnn_ctx *ctx) {
+    if (!ctx) return BNN_ERR_INVALID_ARG;
+    bnn_device_guard guard(ctx);
+    if (!guard.ok) return BNN_ERR_CUDA;
+    BNN_CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream));
+    int code = 0;
+    BNN_CUDA_TRY(ctx, cudaMemcpyFromSymbol(&code, g_umma_error, sizeof(int)));
+    if (code != 0) {
+        const int zero = 0;
+        BNN_CUDA_TRY(ctx, cudaMemcpyToSymbol(g_umma_error, &zero, sizeof(int)));
+        return BNN_ERR_DEVICE_STATUS;
+    }
+    return BNN_OK;
+}

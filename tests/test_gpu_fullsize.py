@@ -16,13 +16,22 @@ torch.backends.cuda.matmul.allow_tf32 = False
 torch.backends.cudnn.allow_tf32 = False
 
 
-@pytest.fixture(scope="module")
-def ctx():
+@pytest.fixture(scope="module", params=[binding.ENGINE_POPC, binding.ENGINE_AUTO], ids=["popc", "auto"])
+def ctx(request):
+    """Both engines bench.py can time: the CUDA-core XOR-popcount kernels, and "auto" (the tensor-core int8
+    engine wherever the shape qualifies and a workspace is set)."""
     build.build()
     c = binding.Context(0)
+    c.set_engine(request.param)
     yield c
     torch.cuda.synchronize()
     c.close()
+
+
+def give_gemm_workspace(ctx, M, N, K):
+    ws = torch.empty(max(ctx.gemm_workspace_bytes(M, N, K), 256), dtype=torch.uint8, device="cuda")
+    ctx.set_workspace(ws)
+    return ws
 
 
 def sample_rows(M, n_random, rng):
@@ -53,8 +62,9 @@ def test_gemm_sweep_full_size(ctx, M, N, K):
         Bp[:, K // 32] |= torch.tensor(-1 << (K % 32), dtype=torch.int32, device="cuda")
         Ap[:, K // 32 + 1:] = -1
         Bp[:, K // 32 + 1:] = -1
+    ws = give_gemm_workspace(ctx, M, N, K)
     C = ctx.xnor_gemm(Ap, Bp, M, N, K)
-    torch.cuda.synchronize()
+    ctx.device_status()
     # (a) complete output against the library matmul of the +-1 values, on the GPU
     ref = torch.matmul(Ad.float(), Bd.float())          # fp32, TF32 off: exact
     assert torch.equal(C.float(), ref)
@@ -76,7 +86,7 @@ def test_mlp_config_full_batch(ctx):
     ctx.set_workspace(ws)
     hidden = [torch.empty(batch, binding.packed_ld(n), dtype=torch.int32, device="cuda") for n in sizes[1:-1]]
     scores = ctx.mlp_forward(net["desc"], torch.from_numpy(case["X"]).cuda(), batch, hidden_out=hidden)
-    torch.cuda.synchronize()
+    ctx.device_status()
     for k, (g, w) in enumerate(zip(hidden, want_hidden)):
         gh = g.cpu().numpy()
         assert np.array_equal(np_unpack_pm1(gh, w.shape[1]), w), f"hidden layer {k}"
@@ -133,8 +143,9 @@ def test_dense_batch_sweep(ctx, batch):
     Ap = ctx.pack_signs(Ad)
     Wp = ctx.pack_signs(Wd, pack_along=1)
     thr = torch.from_numpy(case["thr"]).cuda()
+    ws = give_gemm_workspace(ctx, batch, N, K)
     out = ctx.binary_dense(Ap, Wp, thr, None, batch, N, K)
-    torch.cuda.synchronize()
+    ctx.device_status()
     # complete output against the library matmul on the GPU
     ref = torch.matmul(Ad.float(), Wd.float())          # fp32, TF32 off: exact
     assert torch.equal(unpack_bits_gpu(out, N), ref >= thr.float())

@@ -1,0 +1,135 @@
+"""GPU parity of the tensor-core engine (int8 tcgen05 path) against the oracle: the same calls as the
+CUDA-core path, forced onto the tensor engine through bnn_set_engine, on shapes that span several
+128 x 256 tiles with ragged edges in M, N and K."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1602_02830_b200 import binding, build, nets, workloads as wl
+from util import np_pack_pm1, np_unpack_pm1, padding_is_zero
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    build.build()
+    c = binding.Context(0)
+    c.set_engine(binding.ENGINE_TENSOR)
+    yield c
+    torch.cuda.synchronize()
+    c.close()
+
+
+def dev(a, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    return (t if dtype is None else t.to(dtype)).cuda()
+
+
+def with_ws(ctx, nbytes):
+    ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+    ctx.set_workspace(ws)
+    return ws
+
+
+@pytest.mark.parametrize("M,N,K", [(1000, 1100, 1000), (300, 4096, 1024), (512, 640, 4100), (257, 129, 32768),
+                                   (2048, 2048, 2048)])
+def test_xnor_gemm_tensor_engine(ctx, M, N, K):
+    A, B = wl.gemm_case(M, N, K, seed=M + N + K)
+    Ap = ctx.pack_signs(dev(A, torch.int8))
+    Bp = ctx.pack_signs(dev(B, torch.int8), pack_along=1)
+    need = ctx.gemm_workspace_bytes(M, N, K)
+    assert need > 0
+    with pytest.raises(binding.BnnError) as e:          # forced engine without workspace is an error, not a fallback
+        ctx.set_workspace(None)
+        ctx.xnor_gemm(Ap, Bp, M, N, K)
+    assert e.value.status == -3
+    ws = with_ws(ctx, need)
+    if K % 32:
+        Ap[:, K // 32] |= torch.tensor(-1 << (K % 32), dtype=torch.int32, device="cuda")   # garbage in the padding
+        Bp[:, K // 32] |= torch.tensor(-1 << (K % 32), dtype=torch.int32, device="cuda")
+    ldc = N + 3
+    big = torch.full((M + 2, ldc), 12345, dtype=torch.int32, device="cuda")
+    ctx.xnor_gemm(Ap, Bp, M, N, K, C=big[1:], ldc=ldc)
+    ctx.device_status()
+    out = big.cpu().numpy()
+    assert np.array_equal(out[1:M + 1, :N], oracle.gemm(A, B))
+    assert (out[0] == 12345).all() and (out[M + 1] == 12345).all() and (out[:, N:] == 12345).all()
+    ctx.set_workspace(None)
+    del ws
+
+
+@pytest.mark.parametrize("M,N,K", [(700, 1500, 1000), (1000, 4096, 300), (300, 130, 30000)])
+def test_binary_dense_tensor_engine(ctx, M, N, K):
+    rng = np.random.default_rng(M + N)
+    A, W = wl.gemm_case(M, N, K, seed=M * N)
+    S = oracle.gemm(A, W)
+    thr = rng.integers(-40, 41, N).astype(np.int32)
+    d = min(M, N)
+    thr[:d] = S[np.arange(d), np.arange(d)]            # exact ties
+    thr[-1], thr[-2] = K + 1, -K
+    flip = rng.integers(0, 2, N).astype(np.uint8)
+    flip_p = dev(np_pack_pm1(2 * flip.astype(np.int8)[None, :] - 1)[0].view(np.int32))
+    Ap = ctx.pack_signs(dev(A, torch.int8))
+    Wp = ctx.pack_signs(dev(W, torch.int8), pack_along=1)
+    ws = with_ws(ctx, ctx.gemm_workspace_bytes(M, N, K))
+    ld = binding.packed_ld(N) + 4
+    out = torch.full((M, ld), -1, dtype=torch.int32, device="cuda")
+    ctx.binary_dense(Ap, Wp, dev(thr), flip_p, M, N, K, out=out, ldo_w=ld)
+    ctx.device_status()
+    got = out.cpu().numpy()
+    assert np.array_equal(np_unpack_pm1(got, N), oracle.threshold(S, thr, flip))
+    assert padding_is_zero(got, N)
+    ctx.set_workspace(None)
+    del ws
+
+
+@pytest.mark.parametrize("M,N,K", [(700, 2048, 784), (1300, 1000, 784), (600, 2000, 1008)])
+def test_first_layer_tensor_engine(ctx, M, N, K):
+    rng = np.random.default_rng(M)
+    X = wl.u8(rng, (M, K))
+    X[0, :] = 255
+    X[1, :] = 0
+    W = wl.pm1(rng, (K, N))
+    S = oracle.first_layer(X, W)
+    thr = rng.integers(-3000, 3000, N).astype(np.int32)
+    thr[0] = S[0, 0]
+    Wp = ctx.pack_signs(dev(W, torch.int8), pack_along=1)
+    ws = with_ws(ctx, ctx.gemm_workspace_bytes(M, N, K))
+    bits, sums = ctx.first_layer_bitplanes(dev(X), Wp, M, N, K, thr=dev(thr), want_sums=True)
+    ctx.device_status()
+    assert np.array_equal(sums.cpu().numpy(), S)
+    got = bits.cpu().numpy()
+    assert np.array_equal(np_unpack_pm1(got, N), oracle.threshold(S, thr))
+    assert padding_is_zero(got, N)
+    ctx.set_workspace(None)
+    del ws
+
+
+@pytest.mark.parametrize("host_io", [False, True])
+def test_mlp_forward_tensor_engine(ctx, host_io):
+    batch, sizes = 2000, (784, 1024, 1100, 1024, 10)
+    case = wl.mlp_case(batch=batch, sizes=sizes, seed=77)
+    want_scores, want_hidden = oracle.mlp_forward(case["X"], case["weights"], case["bns"])
+    net = nets.prepare_mlp(ctx, case["weights"], case["bns"])
+    ws = with_ws(ctx, ctx.mlp_workspace_bytes(net["desc"], batch, host_io))
+    if host_io:
+        Xh = torch.from_numpy(case["X"]).pin_memory()
+        Sh = torch.empty(batch, sizes[-1], dtype=torch.float32).pin_memory()
+        ctx.mlp_forward_host(net["desc"], Xh, batch, Sh)
+        ctx.device_status()
+        got = Sh.numpy().astype(np.float64)
+    else:
+        hidden = [torch.empty(batch, binding.packed_ld(n), dtype=torch.int32, device="cuda") for n in sizes[1:-1]]
+        scores = ctx.mlp_forward(net["desc"], dev(case["X"]), batch, hidden_out=hidden)
+        ctx.device_status()
+        for k, (g, w) in enumerate(zip(hidden, want_hidden)):
+            gh = g.cpu().numpy()
+            assert np.array_equal(np_unpack_pm1(gh, w.shape[1]), w), f"hidden layer {k}"
+            assert padding_is_zero(gh, w.shape[1])
+        got = scores.cpu().numpy().astype(np.float64)
+    tol = 1e-5 * np.abs(want_scores) + 1e-6 * np.abs(want_scores).max()
+    assert (np.abs(got - want_scores) <= tol).all()
+    ctx.set_workspace(None)
+    del ws
