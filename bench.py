@@ -65,7 +65,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -143,8 +143,8 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--variant", type=int, default=0, help="tiled-kernel inner loop: 0 default, 1 plain popc, 2 carry-save")
     ap.add_argument("--engine", type=int, default=0, help="0 auto (tensor-core int8 engine for large shapes), 1 CUDA-core XOR-popcount only, 2 tensor")
@@ -230,10 +230,10 @@ def main():
     act_in = torch.randint(-2**31, 2**31 - 1, (BATCH, binding.packed_ld(SIZES[1])), dtype=torch.int32, device=dev)
     act_out = torch.empty(BATCH, binding.packed_ld(SIZES[2]), dtype=torch.int32, device=dev)
     dense_times = timed_steps(lambda: ctx.binary_dense(act_in, hid["Wp"], hid["thr"], hid["flip"], BATCH, SIZES[2], SIZES[1],
-                                                       out=act_out), args.steps, args.warmup)
+                                                       out=act_out), min(args.steps, 50), 3)
     first = net["layers"][0]
     first_times = timed_steps(lambda: ctx.first_layer_bitplanes(X, first["Wp"], BATCH, SIZES[1], SIZES[0], thr=first["thr"],
-                                                                flip=first["flip"]), max(args.steps // 2, 3), 3)
+                                                                flip=first["flip"]), min(args.steps, 50), 3)
     clocks = sampler.stop() if sampler else None
 
     if world > 1:
@@ -254,8 +254,8 @@ def main():
     # the same two layers on the CUDA-core XOR-popcount path (Eq. 8 as the paper computes it), for the popc roofline
     ctx.set_engine(1)
     popc_dense_times = timed_steps(lambda: ctx.binary_dense(act_in, hid["Wp"], hid["thr"], hid["flip"], BATCH, SIZES[2], SIZES[1],
-                                                            out=act_out), max(args.steps // 2, 3), 3) if rank == 0 else [1.0]
-    popc_mlp_times = timed_steps(lambda: ctx.mlp_forward(desc, X, BATCH, scores=scores), max(args.steps // 2, 3), 3) if rank == 0 else [1.0]
+                                                            out=act_out), min(args.steps, 20), 3) if rank == 0 else [1.0]
+    popc_mlp_times = timed_steps(lambda: ctx.mlp_forward(desc, X, BATCH, scores=scores), min(args.steps, 20), 3) if rank == 0 else [1.0]
     ctx.set_engine(args.engine)
 
     peaks = {}

@@ -167,13 +167,19 @@ extern "C" int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const u
     const size_t fwd = bnn_mlp_workspace_bytes(m, batch, 0);
     uint8_t *Xd = reinterpret_cast<uint8_t *>(ws + fwd);
     float *Sd = reinterpret_cast<float *>(ws + fwd + round256((size_t)batch * K0));
-    BNN_CUDA_TRY(ctx, cudaMemcpy2DAsync(Xd, (size_t)K0, X_host, (size_t)ldx, (size_t)K0, (size_t)batch,
-                                        cudaMemcpyHostToDevice, ctx->stream));
+    if (ldx == K0)   // contiguous: one linear copy
+        BNN_CUDA_TRY(ctx, cudaMemcpyAsync(Xd, X_host, (size_t)K0 * batch, cudaMemcpyHostToDevice, ctx->stream));
+    else
+        BNN_CUDA_TRY(ctx, cudaMemcpy2DAsync(Xd, (size_t)K0, X_host, (size_t)ldx, (size_t)K0, (size_t)batch,
+                                            cudaMemcpyHostToDevice, ctx->stream));
     if (int st = tensor ? forward_device_tensor(ctx, m, Xd, K0, batch, Sd, NL, nullptr, ws)
                         : forward_device(ctx, m, Xd, K0, batch, Sd, NL, nullptr, ws))
         return st;
-    BNN_CUDA_TRY(ctx, cudaMemcpy2DAsync(scores_host, (size_t)lds * 4, Sd, (size_t)NL * 4, (size_t)NL * 4, (size_t)batch,
-                                        cudaMemcpyDeviceToHost, ctx->stream));
+    if (lds == NL)
+        BNN_CUDA_TRY(ctx, cudaMemcpyAsync(scores_host, Sd, (size_t)NL * 4 * batch, cudaMemcpyDeviceToHost, ctx->stream));
+    else
+        BNN_CUDA_TRY(ctx, cudaMemcpy2DAsync(scores_host, (size_t)lds * 4, Sd, (size_t)NL * 4, (size_t)NL * 4, (size_t)batch,
+                                            cudaMemcpyDeviceToHost, ctx->stream));
     return BNN_OK;
 }
 

@@ -6,11 +6,11 @@
 //   512 bit-MACs per clock per SM), so for large shapes the packed operands are expanded to one signed byte
 //   per value (a streaming pass) and multiplied with tcgen05.mma kind::i8.  Results are the same integers.
 //
-// Kernel k_umma_i8 (one 128 x 256 output tile per CTA, 192 threads):
+// Kernel k_umma_i8 (persistent, one CTA per SM walking 128 x 256 output tiles, 192 threads):
 //   warp 0    TMA producer: cp.async.bulk.tensor 2-D loads of 128-byte-wide K slices (128B swizzle) of both
 //             operands into a 4-stage shared-memory ring, completion on mbarriers;
-//   warp 1    allocates 256 TMEM columns, then one lane issues tcgen05.mma (M=128, N=256, K=32) four times per
-//             stage and releases the stage with tcgen05.commit;
+//   warp 1    allocates all 512 TMEM columns (two accumulator buffers), then one lane issues tcgen05.mma
+//             (M=128, N=256, K=32) four times per stage and releases the stage with tcgen05.commit;
 //   warps 2-5 epilogue: tcgen05.ld of the int32 accumulators (each thread owns one output row, 32 columns at
 //             a time), then either int32 stores, or the BatchNorm-folded threshold + Sign + repack to one
 //             32-bit word per 32 columns (and, for the next layer, the same signs as bytes).
@@ -27,7 +27,8 @@ constexpr int STAGES = 4;
 constexpr int NTHREADS = 192;
 constexpr uint32_t A_BYTES = BM * BK, B_BYTES = BN * BK;
 constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr uint32_t TMEM_COLS = 256;
+constexpr int ACC_BUFS = 2;
+constexpr uint32_t TMEM_COLS = 512;       // two accumulator buffers of BN columns
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // a wait gives up after 2 s of wall clock
 
 __device__ int g_umma_error;                    // 0 = fine; otherwise a code saying which wait gave up
@@ -111,13 +112,25 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 struct __align__(8) Control {
     uint64_t full[STAGES];
     uint64_t empty[STAGES];
-    uint64_t accum;
+    uint64_t acc_full[ACC_BUFS];
+    uint64_t acc_empty[ACC_BUFS];
     uint32_t tmem_base;
     uint32_t failed;
-    int32_t thr[BN];
-    uint32_t flip[BN / 32];
+    int32_t thr[ACC_BUFS][BN];
+    uint32_t flip[ACC_BUFS][BN / 32];
 };
 
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void fail(Control *ctl, int code) {
+    ctl->failed = (uint32_t)code;
+    atomicExch(&g_umma_error, code);
+}
+
+// Persistent: gridDim.x CTAs (one per SM) walk the tile list with stride gridDim.x.  The shared-memory ring
+// runs on across tiles; the accumulator is double-buffered in tensor memory (2 x 256 columns), so the
+// epilogue of tile i overlaps the main loop of tile i+1.
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const UmmaArgs p) {
     extern __shared__ uint8_t smem_raw[];
@@ -127,25 +140,18 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t tiles_m = (p.M + BM - 1) / BM;
-    const int64_t tile_m = blockIdx.x % tiles_m, tile_n = blockIdx.x / tiles_m;
-    const int64_t m0 = tile_m * BM, n0 = tile_n * BN;
+    const int64_t tiles_n = (p.N + BN - 1) / BN;
+    const int64_t ntiles = tiles_m * tiles_n;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
-        mbar_init(smem_u32(&ctl->accum), 1);
+        for (int b = 0; b < ACC_BUFS; ++b) { mbar_init(smem_u32(&ctl->acc_full[b]), 1); mbar_init(smem_u32(&ctl->acc_empty[b]), 4); }
         ctl->failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    if (warp >= 2 && p.out) {
-        for (int e = threadIdx.x - 64; e < BN; e += 128) ctl->thr[e] = (n0 + e < p.N) ? p.thr[n0 + e] : 0x7fffffff;
-        if (threadIdx.x - 64 < BN / 32) {
-            const int64_t w = (n0 >> 5) + (threadIdx.x - 64);
-            ctl->flip[threadIdx.x - 64] = (p.flip && w * 32 < p.N) ? p.flip[w] : 0u;
-        }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -155,101 +161,122 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
     if (warp == 0) {
         // ---------------- TMA producer
         if (lane == 0) {
-            for (int it = 0; it < p.k_iters; ++it) {
-                const int s = it % STAGES;
-                if (it >= STAGES) {
-                    if (!mbar_wait(smem_u32(&ctl->empty[s]), ((it / STAGES) - 1) & 1)) { ctl->failed = 1; atomicExch(&g_umma_error, 1); break; }
+            uint32_t it = 0;
+            bool ok = true;
+            for (int64_t t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+                const int m0 = (int)((t % tiles_m) * BM), n0 = (int)((t / tiles_m) * BN);
+                for (int kit = 0; kit < p.k_iters; ++kit, ++it) {
+                    const uint32_t s = it % STAGES;
+                    if (it >= STAGES && !mbar_wait(smem_u32(&ctl->empty[s]), ((it / STAGES) - 1) & 1)) { fail(ctl, 1); ok = false; break; }
+                    const uint32_t bar = smem_u32(&ctl->full[s]);
+                    mbar_expect_tx(bar, STAGE_BYTES);
+                    tma_load_2d(smem_u32(tiles + s * STAGE_BYTES), &mapA, kit * BK, m0, bar);
+                    tma_load_2d(smem_u32(tiles + s * STAGE_BYTES + A_BYTES), &mapB, kit * BK, n0, bar);
                 }
-                const uint32_t bar = smem_u32(&ctl->full[s]);
-                mbar_expect_tx(bar, STAGE_BYTES);
-                tma_load_2d(smem_u32(tiles + s * STAGE_BYTES), &mapA, it * BK, (int)m0, bar);
-                tma_load_2d(smem_u32(tiles + s * STAGE_BYTES + A_BYTES), &mapB, it * BK, (int)n0, bar);
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer
         if (lane == 0) {
+            uint32_t it = 0, tc = 0;
             bool ok = true;
-            for (int it = 0; it < p.k_iters && ok; ++it) {
-                const int s = it % STAGES;
-                if (!mbar_wait(smem_u32(&ctl->full[s]), (it / STAGES) & 1)) { ctl->failed = 2; atomicExch(&g_umma_error, 2); ok = false; break; }
+            for (int64_t t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++tc) {
+                const uint32_t buf = tc & 1;
+                if (tc >= ACC_BUFS && !mbar_wait(smem_u32(&ctl->acc_empty[buf]), ((tc / ACC_BUFS) - 1) & 1)) { fail(ctl, 4); ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint64_t adesc = smem_desc_sw128(smem_u32(tiles + s * STAGE_BYTES));
-                const uint64_t bdesc = smem_desc_sw128(smem_u32(tiles + s * STAGE_BYTES + A_BYTES));
+                const uint32_t tmem_d = tmem_base + buf * BN;
+                for (int kit = 0; kit < p.k_iters; ++kit, ++it) {
+                    const uint32_t s = it % STAGES;
+                    if (!mbar_wait(smem_u32(&ctl->full[s]), (it / STAGES) & 1)) { fail(ctl, 2); ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint64_t adesc = smem_desc_sw128(smem_u32(tiles + s * STAGE_BYTES));
+                    const uint64_t bdesc = smem_desc_sw128(smem_u32(tiles + s * STAGE_BYTES + A_BYTES));
 #pragma unroll
-                for (int k = 0; k < BK / 32; ++k)   // 32 bytes of K per instruction: start address advances by 32 B (>> 4 = 2)
-                    umma_i8(tmem_base, adesc + 2 * k, bdesc + 2 * k, p.idesc, (it > 0 || k > 0) ? 1u : 0u);
-                umma_commit(smem_u32(&ctl->empty[s]));      // stage may be refilled once these MMAs have read it
+                    for (int k = 0; k < BK / 32; ++k)   // 32 bytes of K per instruction: start address advances by 32 B (>> 4 = 2)
+                        umma_i8(tmem_d, adesc + 2 * k, bdesc + 2 * k, p.idesc, (kit > 0 || k > 0) ? 1u : 0u);
+                    umma_commit(smem_u32(&ctl->empty[s]));      // stage may be refilled once these MMAs have read it
+                }
+                umma_commit(smem_u32(&ctl->acc_full[buf]));     // accumulators of this tile complete (also after a failure)
             }
-            umma_commit(smem_u32(&ctl->accum));             // accumulators complete (arrives even after a failure)
         }
     } else {
         // ---------------- epilogue: warps 2..5 own TMEM lanes 32*(warp%4) .. +31
         const int q = warp & 3;
-        const int row_in_tile = 32 * q + lane;
-        const int64_t row = m0 + row_in_tile;
-        bool ok = mbar_wait(smem_u32(&ctl->accum), 0);
-        if (!ok) { ctl->failed = 3; atomicExch(&g_umma_error, 3); }
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        ok = ok && (ctl->failed == 0);
-        if (ok && p.k_iters > 0) {
+        const int et = threadIdx.x - 64;                 // 0..127 among the epilogue threads
+        uint32_t tc = 0;
+        bool ok = true;
+        for (int64_t t = blockIdx.x; t < ntiles; t += gridDim.x, ++tc) {
+            const uint32_t buf = tc & 1;
+            const int64_t m0 = (t % tiles_m) * BM, n0 = (t / tiles_m) * BN;
+            const int64_t row = m0 + 32 * q + lane;
+            if (p.out) {
+                for (int e = et; e < BN; e += 128) ctl->thr[buf][e] = (n0 + e < p.N) ? p.thr[n0 + e] : 0x7fffffff;
+                if (et < BN / 32) {
+                    const int64_t w = (n0 >> 5) + et;
+                    ctl->flip[buf][et] = (p.flip && w * 32 < p.N) ? p.flip[w] : 0u;
+                }
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps only
+            if (ok && !mbar_wait(smem_u32(&ctl->acc_full[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 3); ok = false; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            ok = ok && (ctl->failed == 0);
+            if (ok) {
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                const int64_t col0 = n0 + 32 * c;
-                if (col0 >= p.N) break;                      // uniform over the warp
-                uint32_t r[32];
-                tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * c), r);
-                if (row < p.M) {
-                    if (p.C) {
-                        int32_t *dst = p.C + row * p.ldc + col0;
-                        if (col0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
+                for (int c = 0; c < BN / 32; ++c) {
+                    const int64_t col0 = n0 + 32 * c;
+                    if (col0 >= p.N) break;                      // uniform over the warp
+                    uint32_t r[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + buf * BN + (uint32_t)(32 * c), r);
+                    if (row < p.M) {
+                        if (p.C) {
+                            int32_t *dst = p.C + row * p.ldc + col0;
+                            if (col0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4)
-                                *reinterpret_cast<int4 *>(dst + j) = make_int4((int)r[j], (int)r[j + 1], (int)r[j + 2], (int)r[j + 3]);
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (col0 + j < p.N) dst[j] = (int32_t)r[j];
-                        }
-                    }
-                    if (p.out) {
-                        uint32_t word = 0u;
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) word |= (uint32_t)((int32_t)r[j] >= ctl->thr[32 * c + j]) << j;
-                        word ^= ctl->flip[c];
-                        if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;      // columns beyond N stay 0
-                        p.out[row * p.ldo + (col0 >> 5)] = word;
-                        if (p.out8) {
-                            int8_t *d8 = p.out8 + row * p.ldo8 + col0;
-                            uint32_t b[8];
-#pragma unroll
-                            for (int g = 0; g < 8; ++g) {
-                                // 4 sign bits -> 4 bytes of +1 (0x01) / -1 (0xff)
-                                const uint32_t t = (((word >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u;
-                                b[g] = ~(t * 0xfeu);
-                            }
-                            if (col0 + 32 <= p.N) {
-                                *reinterpret_cast<uint4 *>(d8) = make_uint4(b[0], b[1], b[2], b[3]);
-                                *reinterpret_cast<uint4 *>(d8 + 16) = make_uint4(b[4], b[5], b[6], b[7]);
+                                for (int j = 0; j < 32; j += 4)
+                                    *reinterpret_cast<int4 *>(dst + j) = make_int4((int)r[j], (int)r[j + 1], (int)r[j + 2], (int)r[j + 3]);
                             } else {
+#pragma unroll
                                 for (int j = 0; j < 32; ++j)
-                                    if (col0 + j < p.N) d8[j] = ((word >> j) & 1u) ? (int8_t)1 : (int8_t)-1;
-                                    else if (col0 + j < p.ldo8) d8[j] = 0;
+                                    if (col0 + j < p.N) dst[j] = (int32_t)r[j];
+                            }
+                        }
+                        if (p.out) {
+                            uint32_t word = 0u;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) word |= (uint32_t)((int32_t)r[j] >= ctl->thr[buf][32 * c + j]) << j;
+                            word ^= ctl->flip[buf][c];
+                            if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;      // columns beyond N stay 0
+                            p.out[row * p.ldo + (col0 >> 5)] = word;
+                            if (p.out8) {
+                                int8_t *d8 = p.out8 + row * p.ldo8 + col0;
+                                uint32_t b[8];
+#pragma unroll
+                                for (int g = 0; g < 8; ++g) {
+                                    // 4 sign bits -> 4 bytes of +1 (0x01) / -1 (0xff)
+                                    const uint32_t t4 = (((word >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u;
+                                    b[g] = ~(t4 * 0xfeu);
+                                }
+                                if (col0 + 32 <= p.N) {
+                                    *reinterpret_cast<uint4 *>(d8) = make_uint4(b[0], b[1], b[2], b[3]);
+                                    *reinterpret_cast<uint4 *>(d8 + 16) = make_uint4(b[4], b[5], b[6], b[7]);
+                                } else {
+                                    for (int j = 0; j < 32; ++j)
+                                        if (col0 + j < p.N) d8[j] = ((word >> j) & 1u) ? (int8_t)1 : (int8_t)-1;
+                                        else if (col0 + j < p.ldo8) d8[j] = 0;
+                                }
                             }
                         }
                     }
                 }
+                // padding words of the packed output
+                if (p.out && row < p.M && n0 + BN >= p.N) {
+                    for (int64_t w = (p.N + 31) >> 5; w < p.ldo; ++w) p.out[row * p.ldo + w] = 0u;
+                }
             }
-        }
-        // K == 0: the empty sum
-        if (ok && p.k_iters == 0 && row < p.M) {
-            for (int64_t col = n0; col < min(n0 + (int64_t)BN, p.N); ++col) {
-                if (p.C) p.C[row * p.ldc + col] = 0;
-            }
-        }
-        // padding words of the packed output
-        if (p.out && row < p.M && n0 + BN >= p.N) {
-            for (int64_t w = (p.N + 31) >> 5; w < p.ldo; ++w) p.out[row * p.ldo + w] = 0u;
+            // hand the accumulator buffer back to the MMA warp
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[buf]));
         }
     }
 
@@ -371,9 +398,10 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
             attr_set[ctx->device] = true;
         }
     }
+    if (K <= 0) return BNN_ERR_INVALID_ARG;      // callers route the empty product elsewhere
     const int64_t tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
-    if (tiles > 0x7fffffff) return BNN_ERR_INVALID_ARG;
-    k_umma_i8<<<(unsigned)tiles, NTHREADS, smem, ctx->stream>>>(mapA, mapB, a);
+    const int64_t grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+    k_umma_i8<<<(unsigned)grid, NTHREADS, smem, ctx->stream>>>(mapA, mapB, a);
     return bnn_check_launch(ctx);
 }
 
