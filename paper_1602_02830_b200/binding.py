@@ -25,7 +25,7 @@ EXPORTS = (
     "bnn_set_popc_variant", "bnn_pack_signs", "bnn_xnor_gemm", "bnn_binary_dense", "bnn_first_layer_bitplanes",
     "bnn_binary_conv2d", "bnn_mlp_workspace_bytes", "bnn_mlp_forward", "bnn_mlp_forward_host",
     "bnn_fold_batchnorm", "bnn_mlp_noalloc_max_bytes", "bnn_mlp_forward_noalloc", "bnn_set_engine",
-    "bnn_gemm_workspace_bytes", "bnn_device_status",
+    "bnn_gemm_workspace_bytes", "bnn_device_status", "bnn_conv_workspace_bytes",
 )
 
 
@@ -72,6 +72,8 @@ def lib() -> ctypes.CDLL:
         L.bnn_gemm_workspace_bytes.argtypes = [i64, i64, i64]
         L.bnn_gemm_workspace_bytes.restype = c_size_t
         L.bnn_device_status.argtypes = [vp]
+        L.bnn_conv_workspace_bytes.argtypes = [i64, i64, i64, i64, i64, c_int]
+        L.bnn_conv_workspace_bytes.restype = c_size_t
         L.bnn_pack_signs.argtypes = [vp, vp, c_int, i64, i64, i64, c_int, c_int, vp, i64]
         L.bnn_xnor_gemm.argtypes = [vp, vp, i64, vp, i64, vp, i64, i64, i64, i64]
         L.bnn_binary_dense.argtypes = [vp, vp, i64, vp, i64, vp, vp, vp, i64, i64, i64, i64]
@@ -151,6 +153,9 @@ class Context:
 
     def gemm_workspace_bytes(self, M: int, N: int, K: int) -> int:
         return int(lib().bnn_gemm_workspace_bytes(M, N, K))
+
+    def conv_workspace_bytes(self, B, H, W, C_in, C_out, pool) -> int:
+        return int(lib().bnn_conv_workspace_bytes(B, H, W, C_in, C_out, int(pool)))
 
     def device_status(self):
         """Synchronises the stream; raises if a kernel reported that one of its bounded waits gave up."""

@@ -104,6 +104,24 @@ extern "C" int bnn_binary_conv2d(bnn_ctx *ctx, const uint32_t *act, const uint8_
     if (!bnn_aligned16(act) && (Cw % 4) == 0) return BNN_ERR_ALIGNMENT;
     if (!bnn_aligned16(Wp) && (Cw % 4) == 0) return BNN_ERR_ALIGNMENT;
     if (out_bits && !bnn_aligned16(out_bits)) return BNN_ERR_ALIGNMENT;
+    {
+        // tensor-core engine: activations and weights are expanded to +-1 bytes in the workspace and the convolution
+        // runs as 9 * C_in/128 K steps of TMA 4-D loads whose out-of-image halo arrives as zeros
+        int TH, TB;
+        const bool shape_ok = (C_in % 128) == 0 && bnn_umma_conv_tiling(H, W, pool, &TH, &TB) && !(pool && out_sums) &&
+                              bnn_umma_shape_ok(B * H * W, C_out, 9 * C_in);
+        if (ctx->engine != BNN_ENGINE_POPC && shape_ok) {
+            const size_t a_bytes = bnn_umma_operand_bytes(B * H * W, C_in), w_bytes = bnn_umma_operand_bytes(C_out, 9 * C_in);
+            if (ctx->ws && ctx->ws_bytes >= a_bytes + w_bytes) {
+                int8_t *act8 = static_cast<int8_t *>(ctx->ws);
+                int8_t *W8 = act8 + a_bytes;
+                if (int st = bnn_umma_expand(ctx, act, Cw, B * H * W, C_in, act8)) return st;
+                if (int st = bnn_umma_expand(ctx, Wp, 9 * Cw, C_out, 9 * C_in, W8)) return st;
+                return bnn_umma_conv(ctx, act8, W8, B, H, W, C_in, C_out, pool, thr, flip, out_bits, out_sums);
+            }
+            if (ctx->engine == BNN_ENGINE_TENSOR) return BNN_ERR_WORKSPACE;
+        }
+    }
     Args a{};
     a.A = act; a.lda = 0;
     a.B = Wp; a.ldb = 9 * Cw;
@@ -114,4 +132,11 @@ extern "C" int bnn_binary_conv2d(bnn_ctx *ctx, const uint32_t *act, const uint8_
     a.thr = thr; a.flip = flip;
     a.H = (int)H; a.W = (int)W; a.Cw = (int)Cw; a.pool = pool;
     return bnn_launch_tile_conv(ctx, a);
+}
+
+extern "C" size_t bnn_conv_workspace_bytes(int64_t B, int64_t H, int64_t W, int64_t C_in, int64_t C_out, int pool) {
+    int TH, TB;
+    if (B <= 0 || H <= 0 || W <= 0 || C_in <= 0 || C_out <= 0 || (C_in % 128) != 0) return 0;
+    if (!bnn_umma_conv_tiling(H, W, pool, &TH, &TB) || !bnn_umma_shape_ok(B * H * W, C_out, 9 * C_in)) return 0;
+    return bnn_umma_operand_bytes(B * H * W, C_in) + bnn_umma_operand_bytes(C_out, 9 * C_in);
 }

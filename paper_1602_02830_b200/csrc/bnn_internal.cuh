@@ -25,3 +25,6 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
 static inline bool bnn_umma_shape_ok(int64_t M, int64_t N, int64_t K) {
     return M >= 256 && N >= 128 && K >= 128 && (double)M * (double)N * (double)K >= 1.0e9;
 }
+bool bnn_umma_conv_tiling(int64_t H, int64_t W, int pool, int *TH, int *TB);
+int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B, int64_t H, int64_t W, int64_t C_in,
+                  int64_t C_out, int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, int32_t *out_sums);

@@ -41,6 +41,11 @@ struct UmmaArgs {
     uint32_t *out; int64_t ldo;                  // optional packed sign output
     int8_t *out8; int64_t ldo8;                  // optional +-1 byte output (next layer's operand)
     const int32_t *thr; const uint32_t *flip;
+    // convolution mode (3x3, pad 1): A is a 4-D byte tensor [B][H][W][C_in]; one K step = (tap, 128-channel slice)
+    int conv;               // 0 = plain GEMM
+    int H, W, TH, TB;       // image size; a 128-pixel tile = TB images x TH rows x W columns
+    int c_chunks;           // C_in / 128
+    int pool;               // 2x2 max-pool (as OR of the sign bits) before the packed store
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -78,6 +83,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, int c3, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
 }
 // Shared-memory matrix descriptor: K-major tile, rows of 128 bytes, 128-byte swizzle, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
@@ -118,6 +128,7 @@ struct __align__(8) Control {
     uint32_t failed;
     int32_t thr[ACC_BUFS][BN];
     uint32_t flip[ACC_BUFS][BN / 32];
+    uint32_t poolw[BM][BN / 32 + 1];   // convolution with pooling: the sign words of every pixel of the tile
 };
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
@@ -170,7 +181,18 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                     if (it >= STAGES && !mbar_wait(smem_u32(&ctl->empty[s]), ((it / STAGES) - 1) & 1)) { fail(ctl, 1); ok = false; break; }
                     const uint32_t bar = smem_u32(&ctl->full[s]);
                     mbar_expect_tx(bar, STAGE_BYTES);
-                    tma_load_2d(smem_u32(tiles + s * STAGE_BYTES), &mapA, kit * BK, m0, bar);
+                    if (p.conv) {
+                        // tile -> (first image, first row); K step -> (tap, channel slice); halo rows/columns and
+                        // images beyond the batch are outside the tensor and arrive as zeros
+                        const int tm = m0 / BM;
+                        const int tiles_per_img = p.H / p.TH;
+                        const int b0 = (p.TB > 1) ? tm * p.TB : tm / tiles_per_img;
+                        const int y0 = (p.TB > 1) ? 0 : (tm % tiles_per_img) * p.TH;
+                        const int tap = kit / p.c_chunks, cc = kit % p.c_chunks;
+                        tma_load_4d(smem_u32(tiles + s * STAGE_BYTES), &mapA, cc * BK, tap % 3 - 1, y0 + tap / 3 - 1, b0, bar);
+                    } else {
+                        tma_load_2d(smem_u32(tiles + s * STAGE_BYTES), &mapA, kit * BK, m0, bar);
+                    }
                     tma_load_2d(smem_u32(tiles + s * STAGE_BYTES + A_BYTES), &mapB, kit * BK, n0, bar);
                 }
             }
@@ -246,7 +268,8 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                             for (int j = 0; j < 32; ++j) word |= (uint32_t)((int32_t)r[j] >= ctl->thr[buf][32 * c + j]) << j;
                             word ^= ctl->flip[buf][c];
                             if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;      // columns beyond N stay 0
-                            p.out[row * p.ldo + (col0 >> 5)] = word;
+                            if (p.pool) ctl->poolw[32 * q + lane][c] = word ^ ctl->flip[buf][c];   // un-flipped (dot >= thr) bits
+                            else p.out[row * p.ldo + (col0 >> 5)] = word;
                             if (p.out8) {
                                 int8_t *d8 = p.out8 + row * p.ldo8 + col0;
                                 uint32_t b[8];
@@ -269,8 +292,36 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                     }
                 }
                 // padding words of the packed output
-                if (p.out && row < p.M && n0 + BN >= p.N) {
+                if (p.out && !p.pool && row < p.M && n0 + BN >= p.N) {
                     for (int64_t w = (p.N + 31) >> 5; w < p.ldo; ++w) p.out[row * p.ldo + w] = 0u;
+                }
+            }
+            if (p.pool) {
+                // 2x2 max-pool then threshold == OR of the four thresholded bits, then flip.  The tile holds TB images
+                // x TH rows x W columns (TH, W even), i.e. 32 whole windows; 256 (window, word) items for 128 threads.
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (ok) {
+                    const int Wo = p.W >> 1, nwords = (int)((min((int64_t)BN, p.N - n0) + 31) >> 5);
+                    for (int e = et; e < (BM / 4) * (BN / 32); e += 128) {
+                        const int win = e / (BN / 32), c = e % (BN / 32);
+                        if (c >= nwords) continue;
+                        const int wx = win % Wo, wy = win / Wo;                 // wy counts window rows over the tile's TB*TH/2 rows
+                        const int r0 = (2 * wy) * p.W + 2 * wx;                 // top-left pixel of the window inside the tile
+                        const int64_t pix = m0 + r0;                            // its linear pixel index b*H*W + y*W + x
+                        if (pix >= p.M) continue;
+                        uint32_t word = ctl->poolw[r0][c] | ctl->poolw[r0 + 1][c] | ctl->poolw[r0 + p.W][c] | ctl->poolw[r0 + p.W + 1][c];
+                        word ^= ctl->flip[buf][c];
+                        const int64_t col0 = n0 + 32 * c;
+                        if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;
+                        // output pixel: same image, (y/2, x/2)
+                        const int64_t img = pix / ((int64_t)p.H * p.W);
+                        const int64_t rem = pix - img * (int64_t)p.H * p.W;
+                        const int64_t oy = (rem / p.W) >> 1, ox = (rem % p.W) >> 1;
+                        const int64_t opix = (img * (p.H >> 1) + oy) * Wo + ox;
+                        p.out[opix * p.ldo + (col0 >> 5)] = word;
+                        if (n0 + BN >= p.N && c == nwords - 1)
+                            for (int64_t w = (p.N + 31) >> 5; w < p.ldo; ++w) p.out[opix * p.ldo + w] = 0u;
+                    }
                 }
             }
             // hand the accumulator buffer back to the MMA warp
@@ -351,6 +402,20 @@ int make_map(bnn_ctx *ctx, CUtensorMap *map, const void *base, int64_t rows, int
 
 }  // namespace
 
+static size_t umma_smem_bytes() { return (size_t)STAGES * STAGE_BYTES + sizeof(Control) + 1024; }
+// Opt in to the large dynamic shared memory once per device.
+static int umma_prepare(bnn_ctx *ctx) {
+    static std::mutex attr_mutex;
+    static bool attr_set[64] = {};
+    std::lock_guard<std::mutex> lock(attr_mutex);
+    if (ctx->device < 0 || ctx->device >= 64) return BNN_ERR_INVALID_ARG;
+    if (!attr_set[ctx->device]) {
+        BNN_CUDA_TRY(ctx, cudaFuncSetAttribute(k_umma_i8, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes()));
+        attr_set[ctx->device] = true;
+    }
+    return BNN_OK;
+}
+
 size_t bnn_umma_operand_bytes(int64_t rows, int64_t K) {
     const int64_t ld8 = ((K + 127) / 128) * 128;
     return ((size_t)rows * ld8 + 255) & ~size_t(255);
@@ -388,20 +453,67 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
     a.k_iters = (int)((K + BK - 1) / BK);
     a.idesc = (2u << 4) | ((a_unsigned ? 0u : 1u) << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
     a.C = C; a.ldc = ldc; a.out = out; a.ldo = ldo; a.out8 = out8; a.ldo8 = ldo8; a.thr = thr; a.flip = flip;
-    const size_t smem = (size_t)STAGES * STAGE_BYTES + sizeof(Control) + 1024;
-    static std::mutex attr_mutex;
-    static bool attr_set[64] = {};
-    {
-        std::lock_guard<std::mutex> lock(attr_mutex);
-        if (ctx->device < 64 && !attr_set[ctx->device]) {
-            BNN_CUDA_TRY(ctx, cudaFuncSetAttribute(k_umma_i8, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            attr_set[ctx->device] = true;
-        }
-    }
+    const size_t smem = umma_smem_bytes();
+    if (int st = umma_prepare(ctx)) return st;
     if (K <= 0) return BNN_ERR_INVALID_ARG;      // callers route the empty product elsewhere
     const int64_t tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
     const int64_t grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
     k_umma_i8<<<(unsigned)grid, NTHREADS, smem, ctx->stream>>>(mapA, mapB, a);
+    return bnn_check_launch(ctx);
+}
+
+namespace {
+int make_map_nhwc(bnn_ctx *ctx, CUtensorMap *map, const void *base, int64_t B, int64_t H, int64_t W, int64_t C, int TW, int TH,
+                  int TB) {
+    encode_fn_t enc;
+    if (int st = get_encode(ctx, &enc)) return st;
+    cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)B};
+    cuuint64_t strides[3] = {(cuuint64_t)C, (cuuint64_t)(W * C), (cuuint64_t)(H * W * C)};
+    cuuint32_t box[4] = {(cuuint32_t)BK, (cuuint32_t)TW, (cuuint32_t)TH, (cuuint32_t)TB};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { ctx->last_cuda_error = (int)r; return BNN_ERR_CUDA; }
+    return BNN_OK;
+}
+}  // namespace
+
+// How a 128-pixel tile is cut out of H x W images: TB images x TH rows x W columns.  Returns false if the
+// geometry does not tile that way (the caller then uses the CUDA-core kernel).
+bool bnn_umma_conv_tiling(int64_t H, int64_t W, int pool, int *TH, int *TB) {
+    if (W < 1 || W > BM || (BM % W) != 0) return false;
+    const int64_t rows = BM / W;                 // image rows per tile if one image were tall enough
+    if (H >= rows) {
+        if (H % rows) return false;
+        *TH = (int)rows; *TB = 1;
+    } else {
+        if (rows % H) return false;
+        *TH = (int)H; *TB = (int)(rows / H);
+    }
+    if (pool && ((*TH & 1) || (W & 1))) return false;
+    return true;
+}
+
+// 3x3 / pad 1 convolution on the tensor engine.  act8: [B][H][W][C_in] +-1 bytes (C_in % 128 == 0);
+// W8: [C_out][9 * C_in] +-1 bytes.  Outputs as bnn_binary_conv2d (sums only without pooling).
+int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B, int64_t H, int64_t W, int64_t C_in,
+                  int64_t C_out, int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, int32_t *out_sums) {
+    int TH, TB;
+    if (!bnn_umma_conv_tiling(H, W, pool, &TH, &TB) || (C_in % BK) != 0 || (pool && out_sums)) return BNN_ERR_INVALID_ARG;
+    CUtensorMap mapA, mapB;
+    if (int st = make_map_nhwc(ctx, &mapA, act8, B, H, W, C_in, (int)W, TH, TB)) return st;
+    if (int st = make_map(ctx, &mapB, W8, C_out, 9 * C_in, 9 * C_in, BN)) return st;
+    UmmaArgs a{};
+    a.M = B * H * W; a.N = C_out;
+    a.k_iters = (int)(9 * (C_in / BK));
+    a.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+    a.C = out_sums; a.ldc = C_out; a.out = out_bits; a.ldo = (C_out + 31) / 32; a.thr = thr; a.flip = flip;
+    a.conv = 1; a.H = (int)H; a.W = (int)W; a.TH = TH; a.TB = TB; a.c_chunks = (int)(C_in / BK); a.pool = pool;
+    if (int st = umma_prepare(ctx)) return st;
+    const int64_t tiles = ((a.M + BM - 1) / BM) * ((C_out + BN - 1) / BN);
+    const int64_t grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+    k_umma_i8<<<(unsigned)grid, NTHREADS, umma_smem_bytes(), ctx->stream>>>(mapA, mapB, a);
     return bnn_check_launch(ctx);
 }
 

@@ -77,3 +77,13 @@ def convnet_forward(ctx, net, X_u8: torch.Tensor, keep_all: bool = False):
         if keep_all:
             outs.append(act)
     return outs if keep_all else act
+
+
+def convnet_workspace_bytes(ctx, net, B: int, H: int, W: int) -> int:
+    """Largest workspace any layer of `net` asks for on the tensor-core engine (0 if none qualifies)."""
+    need = 0
+    for L in net:
+        need = max(need, ctx.conv_workspace_bytes(B, H, W, L["Cin"], L["Cout"], L["pool"]))
+        if L["pool"]:
+            H, W = H // 2, W // 2
+    return need

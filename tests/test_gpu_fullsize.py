@@ -108,8 +108,11 @@ def test_convnet_config_full_batch(ctx):
     case = wl.convnet_case()       # batch 256, 32x32x3, 128-128-256-256-512-512, seed 3
     net = nets.prepare_convnet(ctx, case["layers"])
     Xd = torch.from_numpy(case["X"]).cuda()
+    ws = torch.empty(max(nets.convnet_workspace_bytes(ctx, net, case["batch"], case["hw"], case["hw"]), 256),
+                     dtype=torch.uint8, device="cuda")
+    ctx.set_workspace(ws)
     outs = nets.convnet_forward(ctx, net, Xd, keep_all=True)
-    torch.cuda.synchronize()
+    ctx.device_status()
     # (a) oracle, every layer, on the first and last images of the batch
     pick = np.r_[0:12, 244:256]
     want = oracle.convnet_forward(case["X"][pick], case["layers"])

@@ -133,3 +133,33 @@ def test_mlp_forward_tensor_engine(ctx, host_io):
     assert (np.abs(got - want_scores) <= tol).all()
     ctx.set_workspace(None)
     del ws
+
+
+@pytest.mark.parametrize("B,H,W,Cin,Cout,pool", [(8, 32, 32, 128, 128, False), (8, 32, 32, 128, 200, True),
+                                                 (16, 16, 16, 256, 256, True), (33, 8, 8, 512, 512, True),
+                                                 (35, 8, 8, 256, 300, False), (3, 64, 64, 128, 128, True)])
+def test_binary_conv2d_tensor_engine(ctx, B, H, W, Cin, Cout, pool):
+    rng = np.random.default_rng(B + H + Cin + Cout)
+    act = wl.pm1(rng, (B, H, W, Cin))
+    wgt = wl.pm1(rng, (Cout, 3, 3, Cin))
+    S = oracle.conv3x3(act, wgt)
+    thr = rng.integers(-40, 41, Cout).astype(np.int32)
+    thr[0] = S[0, 0, 0, 0]                       # a tie on a corner pixel (only 4 valid taps)
+    flip = rng.integers(0, 2, Cout).astype(np.uint8)
+    P = oracle.maxpool2x2(S) if pool else S
+    want = oracle.threshold(P, thr, flip)
+    actp = dev(np_pack_pm1(act).view(np.int32))
+    Wp = dev(np_pack_pm1(wgt.reshape(Cout, 9, Cin)).reshape(Cout, -1).view(np.int32))
+    flip_p = dev(np_pack_pm1(2 * flip.astype(np.int8)[None, :] - 1)[0].view(np.int32))
+    need = ctx.conv_workspace_bytes(B, H, W, Cin, Cout, pool)
+    assert need > 0
+    ws = with_ws(ctx, need)
+    bits, sums = ctx.binary_conv2d(actp, B, H, W, Cin, Wp, Cout, pool=pool, thr=dev(thr), flip=flip_p, want_sums=not pool)
+    ctx.device_status()
+    if not pool:
+        assert np.array_equal(sums.cpu().numpy(), S)
+    got = bits.cpu().numpy()
+    assert np.array_equal(np_unpack_pm1(got, Cout), want)
+    assert padding_is_zero(got, Cout)
+    ctx.set_workspace(None)
+    del ws
