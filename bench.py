@@ -156,21 +156,16 @@ def main():
     args.warmup = max(args.warmup, 3)
 
     import torch
-    import torch.distributed as dist
-    from paper_1602_02830_b200 import binding, build, nets, workloads as wl
+    from paper_1602_02830_b200 import binding, build, nets, replicas, workloads as wl
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local = replicas.world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    replicas.init("nccl", torch.device("cuda", local))
     if rank == 0:
         build.build()
-    if world > 1:
-        dist.barrier()
+    replicas.barrier()
     dev = f"cuda:{local}"
     stream = torch.cuda.current_stream(local)
     ctx = binding.Context(local, stream)
@@ -180,13 +175,13 @@ def main():
     def sync_all():
         torch.cuda.synchronize()
         if world > 1:
-            dist.barrier()
+            replicas.barrier()
             torch.cuda.synchronize()
 
     # ---- workload: every rank draws the same network; rank r gets its own batch of images
     case = wl.mlp_case(batch=BATCH, sizes=SIZES, seed=SEED)
     if rank > 0:
-        case["X"] = wl.u8(np.random.default_rng([SEED, rank]), (BATCH, SIZES[0]))
+        case["X"] = wl.u8(np.random.default_rng(replicas.rank_seed(SEED, rank)), (BATCH, SIZES[0]))
     net = nets.prepare_mlp(ctx, case["weights"], case["bns"])
     desc = net["desc"]
     ws = torch.empty(ctx.mlp_workspace_bytes(desc, BATCH, True), dtype=torch.uint8, device=dev)
@@ -236,19 +231,13 @@ def main():
                                                                 flip=first["flip"]), min(args.steps, 50), 3)
     clocks = sampler.stop() if sampler else None
 
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_total_ms = t.tolist()
-
+    total_ms, e2e_total_ms = replicas.max_over_ranks([total_ms, e2e_total_ms], device=dev)
     ms_per_step = total_ms / args.steps
-    value = world * BATCH / (ms_per_step / 1e3)
-    e2e_value = world * BATCH / (e2e_total_ms / args.steps / 1e3)
+    value = replicas.job_throughput(BATCH, ms_per_step, world)
+    e2e_value = replicas.job_throughput(BATCH, e2e_total_ms / args.steps, world)
 
     if rank != 0:
-        if world > 1:
-            dist.barrier()
-            dist.destroy_process_group()
+        replicas.finish()
         return 0
 
     # the same two layers on the CUDA-core XOR-popcount path (Eq. 8 as the paper computes it), for the popc roofline
@@ -314,6 +303,7 @@ def main():
         line["gemm"] = bench_gemm(ctx, args.gemm_size, popc_peak_tbitops, timed_steps, args.engine)
         ctx.set_workspace(ws)
         line["convnet"] = bench_convnet(ctx, timed_steps, args.engine)
+        line["dense_sweep"] = bench_dense_sweep(ctx, timed_steps, args.engine)
         ctx.set_workspace(ws)
         t0 = time.perf_counter()
         dt, cores = time_oracle_mlp(case, BATCH, repeats=4)
@@ -323,10 +313,35 @@ def main():
     else:
         line["cpu_baseline"] = None
     print(json.dumps(line))
-    if world > 1:
-        dist.barrier()
-        dist.destroy_process_group()
+    replicas.finish()
     return 0
+
+
+def bench_dense_sweep(ctx, timed_steps, engine):
+    """One fused 4096 -> 4096 binary dense layer at batch 1 .. 65536 (thresholds uniform in [-64, 64])."""
+    import torch
+    from paper_1602_02830_b200 import workloads as wl
+    K = N = 4096
+    g = torch.Generator(device="cuda").manual_seed(4)
+    Wp = torch.randint(-2**31, 2**31 - 1, (N, K // 32), dtype=torch.int32, device="cuda", generator=g)
+    thr = torch.randint(-64, 65, (N,), dtype=torch.int32, device="cuda", generator=g)
+    out = {}
+    for batch in wl.DENSE_BATCHES:
+        Ap = torch.randint(-2**31, 2**31 - 1, (batch, K // 32), dtype=torch.int32, device="cuda", generator=g)
+        O = torch.empty(batch, N // 32, dtype=torch.int32, device="cuda")
+        dws = torch.empty(max(ctx.gemm_workspace_bytes(batch, N, K), 256), dtype=torch.uint8, device="cuda")
+        ctx.set_workspace(dws)
+        row = {}
+        for name, eng in (("popc", 1), ("selected_engine", engine)):
+            ctx.set_engine(eng)
+            t = timed_steps(lambda: ctx.binary_dense(Ap, Wp, thr, None, batch, N, K, out=O), 20, 3)
+            ms = sorted(t)[len(t) // 2]
+            row[name] = {"ms": ms, "tbitops": 2.0 * batch * N * K / (ms / 1e3) / 1e12}
+        out[str(batch)] = row
+        ctx.set_workspace(None)
+        del dws
+    ctx.set_engine(engine)
+    return out
 
 
 def bench_gemm(ctx, n, peak, timed_steps, engine):
