@@ -148,6 +148,7 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--variant", type=int, default=0, help="tiled-kernel inner loop: 0 default, 1 plain popc, 2 carry-save")
     ap.add_argument("--engine", type=int, default=0, help="0 auto (tensor-core int8 engine for large shapes), 1 CUDA-core XOR-popcount only, 2 tensor")
+    ap.add_argument("--tile-rows", type=int, default=0, help="accumulator rows per thread of the CUDA-core tile kernel (8 or 16; 0 = library default)")
     ap.add_argument("--no-extras", action="store_true", help="skip the GEMM / ConvNet side measurements and the CPU baseline")
     ap.add_argument("--gemm-size", type=int, default=8192)
     args = ap.parse_args()
@@ -171,6 +172,8 @@ def main():
     ctx = binding.Context(local, stream)
     ctx.set_popc_variant(args.variant)
     ctx.set_engine(args.engine)
+    if args.tile_rows:
+        ctx.set_tile_rows(args.tile_rows)
 
     def sync_all():
         torch.cuda.synchronize()

@@ -65,6 +65,9 @@ BNN_API int bnn_set_workspace(bnn_ctx *ctx, void *dptr, size_t bytes);
 /* Inner loop of the tiled kernels (results are identical): 0 = library default, 1 = one POPC per
  * word (Eq. 8 as written), 2 = carry-save: a LOP3 full adder merges two XOR words before the POPC. */
 BNN_API int bnn_set_popc_variant(bnn_ctx *ctx, int variant);
+/* Accumulator rows per thread of the tiled CUDA-core kernel: 16 (one CTA of 8 warps per SM) or 8 (two CTAs per
+ * SM, more warps per scheduler; the default, faster on B200).  A tuning knob; results are identical. */
+BNN_API int bnn_set_tile_rows(bnn_ctx *ctx, int rows);
 
 /* Which kernels evaluate the large products (results are the same integers either way):
  *   0 = automatic: the tensor-core engine for large shapes when the context's workspace is big enough

@@ -18,6 +18,7 @@ extern "C" int bnn_create(bnn_ctx **out, int device, void *cuda_stream) {
     c->sm_count = 0;
     c->variant = 0;
     c->engine = 0;
+    c->tile_rows = 8;
     if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
         delete c;
         return BNN_ERR_CUDA;
@@ -48,6 +49,12 @@ extern "C" const char *bnn_status_string(int status) {
 extern "C" int bnn_set_popc_variant(bnn_ctx *ctx, int variant) {
     if (!ctx || variant < 0 || variant > 2) return BNN_ERR_INVALID_ARG;
     ctx->variant = variant;
+    return BNN_OK;
+}
+
+extern "C" int bnn_set_tile_rows(bnn_ctx *ctx, int rows) {
+    if (!ctx || (rows != 8 && rows != 16)) return BNN_ERR_INVALID_ARG;
+    ctx->tile_rows = rows;
     return BNN_OK;
 }
 

@@ -13,6 +13,7 @@ struct bnn_ctx {
     int last_cuda_error;
     int sm_count;
     int variant;   // inner-loop choice of the tiled kernel (0 auto, 1 plain popc, 2 carry-save)
+    int tile_rows; // accumulator rows per thread of the tiled popc kernel: 16 or 8
     int engine;    // 0 auto, 1 CUDA-core XOR-popcount kernels only, 2 tensor-core int8 engine where it applies
 };
 

@@ -141,16 +141,22 @@ int launch_tile(bnn_ctx *ctx, const Args &a_in, int variant) {
     Args a = a_in;
     a.one = 1u;
     const int64_t rows = (AKIND == A_PLANES) ? 8 * a.M : a.M;     // operand rows (8 bit-plane rows per image)
-    const int64_t t128 = ((rows + 127) / 128) * ((a.N + BN - 1) / BN);
-    const int64_t t64 = ((rows + 63) / 64) * ((a.N + BN - 1) / BN);
+    const int64_t tn = (a.N + BN - 1) / BN;
+    const int64_t t128 = ((rows + 127) / 128) * tn, t64 = ((rows + 63) / 64) * tn;
+    const bool csa = (variant != BNN_VARIANT_PLAIN);
+    if (t64 > 0x7fffffff) return BNN_ERR_INVALID_ARG;
+    if (ctx->tile_rows == 8) {
+        // 8 accumulator rows per thread: 64 x 128 tiles, 8 warps, two CTAs per SM
+        if (csa) k_bit_tile<8, AKIND, true, 8><<<(unsigned)t64, 256, 0, ctx->stream>>>(a);
+        else k_bit_tile<8, AKIND, false, 8><<<(unsigned)t64, 256, 0, ctx->stream>>>(a);
+        return bnn_check_launch(ctx);
+    }
     const bool big = t128 >= 2 * (int64_t)ctx->sm_count;
     const int64_t tiles = big ? t128 : t64;
-    if (tiles > 0x7fffffff) return BNN_ERR_INVALID_ARG;
-    const bool csa = (variant != BNN_VARIANT_PLAIN);
-    if (big && csa) k_bit_tile<8, AKIND, true><<<(unsigned)tiles, 256, 0, ctx->stream>>>(a);
-    else if (big) k_bit_tile<8, AKIND, false><<<(unsigned)tiles, 256, 0, ctx->stream>>>(a);
-    else if (csa) k_bit_tile<4, AKIND, true><<<(unsigned)tiles, 128, 0, ctx->stream>>>(a);
-    else k_bit_tile<4, AKIND, false><<<(unsigned)tiles, 128, 0, ctx->stream>>>(a);
+    if (big && csa) k_bit_tile<8, AKIND, true, 16><<<(unsigned)tiles, 256, 0, ctx->stream>>>(a);
+    else if (big) k_bit_tile<8, AKIND, false, 16><<<(unsigned)tiles, 256, 0, ctx->stream>>>(a);
+    else if (csa) k_bit_tile<4, AKIND, true, 16><<<(unsigned)tiles, 128, 0, ctx->stream>>>(a);
+    else k_bit_tile<4, AKIND, false, 16><<<(unsigned)tiles, 128, 0, ctx->stream>>>(a);
     return bnn_check_launch(ctx);
 }
 

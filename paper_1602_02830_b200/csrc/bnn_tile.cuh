@@ -28,7 +28,6 @@ namespace bnn_tile {
 
 constexpr int BN = 128;   // tile columns
 constexpr int BKW = 8;    // words of K per chunk
-constexpr int TM = 16;    // rows per warp (= per thread)
 constexpr int TN = 4;     // columns per lane
 
 enum { A_PACKED = 0, A_CONV = 1, A_PLANES = 2 };
@@ -91,11 +90,14 @@ __device__ __forceinline__ uint32_t plane_nibble(uint32_t w, int p) {
     return ((((w >> p) & 0x01010101u) * 0x01020408u) >> 24) & 0xfu;
 }
 
-template <int NWARPS, int AKIND, bool CSA>
-__global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile(const Args p) {
+// TM = rows per warp (= accumulator rows per thread): 16 (243 registers, one 8-warp CTA per SM) or
+// 8 (two CTAs per SM, twice the warps per scheduler to hide the POPC / LOP3 pipe latencies).
+template <int NWARPS, int AKIND, bool CSA, int TM>
+__global__ void __launch_bounds__(NWARPS * 32, (TM == 8) ? (512 / (NWARPS * 32)) : ((NWARPS == 8) ? 1 : 2)) k_bit_tile(const Args p) {
     constexpr int BM = NWARPS * TM;        // operand rows per tile (A_PLANES: 8 rows per image)
     constexpr int NT = NWARPS * 32;
-    static_assert(2 * BM == NT, "one A load item per thread");
+    static_assert(2 * BM <= NT && (TM == 8 || TM == 16), "at most one A load item per thread");
+    constexpr int A_THREADS = 2 * BM;      // threads that load A
     constexpr bool PLANES = (AKIND == A_PLANES);
     constexpr int IMGS = BM / 8;           // A_PLANES: images per tile
 
@@ -113,10 +115,11 @@ __global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile
     const uint32_t tail_mask = (p.K & 31) ? ((1u << (p.K & 31)) - 1u) : 0xffffffffu;
 
     // ---- loader roles: one A item per thread, (2*BN)/NT B items per thread
-    const int a_row = tid % BM, a_half = tid / BM;          // A_PACKED / A_CONV: row and which 4 of the 8 words
-    const int a_img = tid >> 4, a_seg = tid & 15;           // A_PLANES: image in tile and 16-byte segment of the chunk
+    const bool a_thread = tid < A_THREADS;
+    const int a_row = tid % BM, a_half = (tid / BM) & 1;    // A_PACKED / A_CONV: row and which 4 of the 8 words
+    const int a_img = (tid >> 4) % IMGS, a_seg = tid & 15;  // A_PLANES: image in tile and 16-byte segment of the chunk
     const int64_t am = PLANES ? (m0 >> 3) + a_img : m0 + a_row;
-    const bool a_ok = am < p.M;
+    const bool a_ok = a_thread && am < p.M;
     int pix_y = 0, pix_x = 0;
     int64_t pix_b = 0;
     if (AKIND == A_CONV && a_ok) {
@@ -189,7 +192,8 @@ __global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile
     };
 
     auto store_chunk = [&](int buf) {
-        if (PLANES) {
+        if (!a_thread) {
+        } else if (PLANES) {
             const uint32_t w[4] = {ra.x, ra.y, ra.z, ra.w};
             x_sum += (int32_t)(__vsadu4(ra.x, 0u) + __vsadu4(ra.y, 0u) + __vsadu4(ra.z, 0u) + __vsadu4(ra.w, 0u));
 #pragma unroll
@@ -311,7 +315,7 @@ __global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile
     }
 
     if (PLANES) {
-        atomicAdd(&aux[a_img], x_sum);
+        if (a_thread) atomicAdd(&aux[a_img], x_sum);
         __syncthreads();
     }
 
@@ -333,11 +337,12 @@ __global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile
     uint32_t keep = 0u;   // packed word this lane will store
 
     if (PLANES) {
-        // this thread holds the 8 plane rows of 2 images: rows wr + 8*mi + pl
+        // this thread holds the 8 plane rows of TM/8 images: rows wr + 8*mi + pl
+        constexpr int IPT = TM / 8;
 #pragma unroll
-        for (int mi = 0; mi < 2; ++mi) {
-            const int64_t img = (m0 >> 3) + 2 * warp + mi;
-            const int32_t xs = aux[2 * warp + mi];
+        for (int mi = 0; mi < IPT; ++mi) {
+            const int64_t img = (m0 >> 3) + IPT * warp + mi;
+            const int32_t xs = aux[IPT * warp + mi];
 #pragma unroll
             for (int j = 0; j < TN; ++j) {
                 const int64_t col = n0 + lane + 32 * j;
@@ -354,8 +359,8 @@ __global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile
                 }
             }
         }
-        if (p.out && lane < 2 * TN) {
-            const int64_t img = (m0 >> 3) + 2 * warp + (lane >> 2);
+        if (p.out && lane < IPT * TN) {
+            const int64_t img = (m0 >> 3) + IPT * warp + (lane >> 2);
             const int64_t ow = (n0 >> 5) + (lane & 3);
             if (img < p.M && ow * 32 < p.N) p.out[img * p.ldo + ow] = keep;
         }
@@ -421,7 +426,7 @@ __global__ void __launch_bounds__(NWARPS * 32, (NWARPS == 8) ? 1 : 2) k_bit_tile
                     const int64_t ow = (n0 >> 5) + j;
                     if (orow < p.M && ow * 32 < p.N) p.out[orow * p.ldo + ow] = keep;
                 }
-                if (pooled_mode && i == TM - 1 && lane < 16) {
+                if (pooled_mode && i == TM - 1 && lane < TM) {
                     const int wi = lane >> 2, j = lane & 3;
                     const int64_t orow = ((m0 + wr) >> 2) + wi;
                     const int64_t ow = (n0 >> 5) + j;

@@ -13,10 +13,12 @@ pytestmark = pytest.mark.gpu
 VARIANTS = [binding.VARIANT_PLAIN, binding.VARIANT_CSA]
 
 
-@pytest.fixture(scope="module")
-def ctx():
+@pytest.fixture(scope="module", params=[16, 8], ids=["rows16", "rows8"])
+def ctx(request):
+    """The CUDA-core kernels in both register-tile shapes (no workspace is set, so nothing goes to the tensor engine)."""
     build.build()
     c = binding.Context(0)
+    c.set_tile_rows(request.param)
     yield c
     torch.cuda.synchronize()
     c.close()
