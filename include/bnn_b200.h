@@ -81,8 +81,8 @@ BNN_API int bnn_set_engine(bnn_ctx *ctx, int engine);
 /* Workspace bytes bnn_xnor_gemm / bnn_binary_dense need to run M x N x K on the tensor-core engine
  * (0 if the shape does not qualify for it). */
 BNN_API size_t bnn_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
-/* The same for bnn_binary_conv2d with a binary input (0 if the tensor-core engine does not apply: it needs
- * C_in % 128 == 0 and a width that divides 128). */
+/* The same for bnn_binary_conv2d (0 if the tensor-core engine does not apply: a binary input needs
+ * C_in % 128 == 0 and a width that divides 128; 9 * C_in <= 32 means the 8-bit first layer). */
 BNN_API size_t bnn_conv_workspace_bytes(int64_t B, int64_t H, int64_t W, int64_t C_in, int64_t C_out, int pool);
 /* Synchronises the context's stream and returns BNN_ERR_DEVICE_STATUS if a kernel gave up on one of its
  * bounded waits since the last call (its outputs are then undefined), BNN_OK otherwise. */

@@ -91,6 +91,27 @@ extern "C" int bnn_binary_conv2d(bnn_ctx *ctx, const uint32_t *act, const uint8_
 
     if (act_u8) {
         if (C_in < 1 || 9 * C_in > 32 || C_out > 8192) return BNN_ERR_INVALID_ARG;
+        {
+            // tensor-core engine: im2col of the image to 32-byte rows (unsigned bytes) times the filters as +-1 bytes
+            int TH, TB;
+            const bool tiling = bnn_umma_conv_tiling(H, W, pool, &TH, &TB);
+            if (ctx->engine != BNN_ENGINE_POPC && bnn_umma_first_conv_ok(B * H * W, C_out) && (tiling || !pool) &&
+                !(pool && out_sums)) {
+                const size_t a_bytes = ((size_t)B * H * W * 32 + 255) & ~size_t(255);
+                const size_t w_bytes = bnn_umma_operand_bytes(C_out, 9 * C_in);
+                // the one-word-per-filter operand must be readable as a packed matrix row: 4-byte stride is not 16-byte
+                // aligned, so the filters are expanded with a leading dimension of one word
+                if (ctx->ws && ctx->ws_bytes >= a_bytes + w_bytes) {
+                    uint8_t *A8 = static_cast<uint8_t *>(ctx->ws);
+                    int8_t *W8 = reinterpret_cast<int8_t *>(A8 + a_bytes);
+                    if (int st = bnn_umma_im2col_u8(ctx, act_u8, B, H, W, C_in, A8)) return st;
+                    if (int st = bnn_umma_expand(ctx, Wp, 1, C_out, 9 * C_in, W8)) return st;
+                    return bnn_umma_gemm(ctx, A8, 32, true, W8, bnn_umma_operand_ld(9 * C_in), B * H * W, C_out, 9 * C_in, out_sums,
+                                         C_out, thr, flip, out_bits, (C_out + 31) / 32, nullptr, 0, pool, H, W);
+                }
+                if (ctx->engine == BNN_ENGINE_TENSOR) return BNN_ERR_WORKSPACE;
+            }
+        }
         ConvU8Args a{act_u8, B, (int)H, (int)W, (int)C_in, Wp, C_out, pool, thr, flip, out_bits, out_sums};
         const int64_t total = B * (pool ? H / 2 : H) * (pool ? W / 2 : W);
         const int64_t blocks = (total + 127) / 128;
@@ -136,7 +157,12 @@ extern "C" int bnn_binary_conv2d(bnn_ctx *ctx, const uint32_t *act, const uint8_
 
 extern "C" size_t bnn_conv_workspace_bytes(int64_t B, int64_t H, int64_t W, int64_t C_in, int64_t C_out, int pool) {
     int TH, TB;
-    if (B <= 0 || H <= 0 || W <= 0 || C_in <= 0 || C_out <= 0 || (C_in % 128) != 0) return 0;
+    if (B <= 0 || H <= 0 || W <= 0 || C_in <= 0 || C_out <= 0) return 0;
+    if (9 * C_in <= 32) {   // first layer on 8-bit input: im2col rows + expanded filters
+        if (!bnn_umma_first_conv_ok(B * H * W, C_out) || (pool && !bnn_umma_conv_tiling(H, W, pool, &TH, &TB))) return 0;
+        return (((size_t)B * H * W * 32 + 255) & ~size_t(255)) + bnn_umma_operand_bytes(C_out, 9 * C_in);
+    }
+    if ((C_in % 128) != 0) return 0;
     if (!bnn_umma_conv_tiling(H, W, pool, &TH, &TB) || !bnn_umma_shape_ok(B * H * W, C_out, 9 * C_in)) return 0;
     return bnn_umma_operand_bytes(B * H * W, C_in) + bnn_umma_operand_bytes(C_out, 9 * C_in);
 }

@@ -366,6 +366,29 @@ __global__ void __launch_bounds__(256) k_expand_s8(const uint32_t *__restrict__ 
     d[1] = make_uint4(b[4], b[5], b[6], b[7]);
 }
 
+// First convolution: the 3x3 neighbourhood of every pixel of an 8-bit NHWC image (9 * C_in <= 32 bytes, taps
+// outside the image as zeros) written as one 32-byte row, byte (tap * C_in + c).  One thread per pixel.
+__global__ void __launch_bounds__(256) k_im2col_u8(const uint8_t *__restrict__ act, int64_t B, int H, int W, int Cin,
+                                                   uint8_t *__restrict__ dst) {
+    const int64_t pix = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (pix >= B * H * W) return;
+    const int x = (int)(pix % W), y = (int)((pix / W) % H);
+    const int64_t b = pix / ((int64_t)W * H);
+    uint32_t w[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+    for (int tap = 0; tap < 9; ++tap) {
+        const int yy = y + tap / 3 - 1, xx = x + tap % 3 - 1;
+        if (yy < 0 || yy >= H || xx < 0 || xx >= W) continue;
+        const uint8_t *px = act + ((b * H + yy) * W + xx) * Cin;
+        for (int c = 0; c < Cin; ++c) {
+            const int k = tap * Cin + c;
+            w[k >> 2] |= (uint32_t)px[c] << (8 * (k & 3));
+        }
+    }
+    uint4 *d = reinterpret_cast<uint4 *>(dst + pix * 32);
+    d[0] = make_uint4(w[0], w[1], w[2], w[3]);
+    d[1] = make_uint4(w[4], w[5], w[6], w[7]);
+}
+
 typedef CUresult (*encode_fn_t)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
                                 const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -435,8 +458,12 @@ int bnn_umma_expand(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t row
 // C / bits = A8 (M x K bytes, pitch lda8; unsigned if a_unsigned) times B8^T (N x K signed bytes, pitch ldb8).
 int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, const int8_t *B8, int64_t ldb8, int64_t M,
                   int64_t N, int64_t K, int32_t *C, int64_t ldc, const int32_t *thr, const uint32_t *flip, uint32_t *out,
-                  int64_t ldo, int8_t *out8, int64_t ldo8) {
+                  int64_t ldo, int8_t *out8, int64_t ldo8, int pool, int64_t H, int64_t W) {
     if (M == 0 || N == 0) return BNN_OK;
+    if (pool) {   // rows are pixels of H x W images in (b, y, x) order; 128-row tiles must hold whole 2x2 windows
+        int TH, TB;
+        if (!bnn_umma_conv_tiling(H, W, 1, &TH, &TB) || C || out8) return BNN_ERR_INVALID_ARG;
+    }
     if ((lda8 & 15) || (ldb8 & 15) || !bnn_aligned16(A8) || !bnn_aligned16(B8)) return BNN_ERR_ALIGNMENT;
     if (M > 0x7fffffff || N > 0x7fffffff) return BNN_ERR_INVALID_ARG;
     CUtensorMap mapA, mapB;
@@ -453,6 +480,7 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
     a.k_iters = (int)((K + BK - 1) / BK);
     a.idesc = (2u << 4) | ((a_unsigned ? 0u : 1u) << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
     a.C = C; a.ldc = ldc; a.out = out; a.ldo = ldo; a.out8 = out8; a.ldo8 = ldo8; a.thr = thr; a.flip = flip;
+    a.pool = pool; a.H = (int)H; a.W = (int)W;
     const size_t smem = umma_smem_bytes();
     if (int st = umma_prepare(ctx)) return st;
     if (K <= 0) return BNN_ERR_INVALID_ARG;      // callers route the empty product elsewhere
@@ -478,6 +506,15 @@ int make_map_nhwc(bnn_ctx *ctx, CUtensorMap *map, const void *base, int64_t B, i
     return BNN_OK;
 }
 }  // namespace
+
+int bnn_umma_im2col_u8(bnn_ctx *ctx, const uint8_t *act, int64_t B, int64_t H, int64_t W, int64_t C_in, uint8_t *dst) {
+    const int64_t total = B * H * W;
+    if (total == 0) return BNN_OK;
+    const int64_t blocks = (total + 255) / 256;
+    if (blocks > 0x7fffffff || 9 * C_in > 32) return BNN_ERR_INVALID_ARG;
+    k_im2col_u8<<<(unsigned)blocks, 256, 0, ctx->stream>>>(act, B, (int)H, (int)W, (int)C_in, dst);
+    return bnn_check_launch(ctx);
+}
 
 // How a 128-pixel tile is cut out of H x W images: TB images x TH rows x W columns.  Returns false if the
 // geometry does not tile that way (the caller then uses the CUDA-core kernel).

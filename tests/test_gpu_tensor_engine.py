@@ -163,3 +163,30 @@ def test_binary_conv2d_tensor_engine(ctx, B, H, W, Cin, Cout, pool):
     assert padding_is_zero(got, Cout)
     ctx.set_workspace(None)
     del ws
+
+
+@pytest.mark.parametrize("B,H,W,Cin,Cout,pool", [(20, 32, 32, 3, 128, False), (17, 32, 32, 3, 100, True), (70, 16, 16, 1, 64, True),
+                                                 (300, 8, 8, 2, 300, False)])
+def test_first_conv_u8_tensor_engine(ctx, B, H, W, Cin, Cout, pool):
+    rng = np.random.default_rng(B + Cout)
+    X = wl.u8(rng, (B, H, W, Cin))
+    X[0] = 255
+    wgt = wl.pm1(rng, (Cout, 3, 3, Cin))
+    thr = rng.integers(-500, 500, Cout).astype(np.int32)
+    flip = rng.integers(0, 2, Cout).astype(np.uint8)
+    S = oracle.conv3x3(X, wgt)
+    P = oracle.maxpool2x2(S) if pool else S
+    Wp = dev(np_pack_pm1(wgt.reshape(Cout, 9 * Cin)).reshape(-1).view(np.int32))
+    flip_p = dev(np_pack_pm1(2 * flip.astype(np.int8)[None, :] - 1)[0].view(np.int32))
+    need = ctx.conv_workspace_bytes(B, H, W, Cin, Cout, pool)
+    assert need > 0
+    ws = with_ws(ctx, need)
+    bits, sums = ctx.binary_conv2d(dev(X), B, H, W, Cin, Wp, Cout, pool=pool, thr=dev(thr), flip=flip_p, want_sums=not pool)
+    ctx.device_status()
+    if not pool:
+        assert np.array_equal(sums.cpu().numpy(), S)
+    got = bits.cpu().numpy()
+    assert np.array_equal(np_unpack_pm1(got, Cout), oracle.threshold(P, thr, flip))
+    assert padding_is_zero(got, Cout)
+    ctx.set_workspace(None)
+    del ws
