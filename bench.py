@@ -151,6 +151,8 @@ def main():
     ap.add_argument("--tile-rows", type=int, default=0, help="accumulator rows per thread of the CUDA-core tile kernel (8 or 16; 0 = library default)")
     ap.add_argument("--no-extras", action="store_true", help="skip the GEMM / ConvNet side measurements and the CPU baseline")
     ap.add_argument("--gemm-size", type=int, default=8192)
+    ap.add_argument("--section", default="all", choices=["all", "gemm", "convnet", "sweep"],
+                    help="side measurements to run after the MLP step (a single one keeps profiler captures small)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -303,13 +305,15 @@ def main():
     }
 
     if not args.no_extras and world == 1:
-        line["gemm"] = bench_gemm(ctx, args.gemm_size, popc_peak_tbitops, timed_steps, args.engine)
-        ctx.set_workspace(ws)
-        line["convnet"] = bench_convnet(ctx, timed_steps, args.engine)
-        line["dense_sweep"] = bench_dense_sweep(ctx, timed_steps, args.engine)
+        if args.section in ("all", "gemm"):
+            line["gemm"] = bench_gemm(ctx, args.gemm_size, popc_peak_tbitops, timed_steps, args.engine)
+        if args.section in ("all", "convnet"):
+            line["convnet"] = bench_convnet(ctx, timed_steps, args.engine)
+        if args.section in ("all", "sweep"):
+            line["dense_sweep"] = bench_dense_sweep(ctx, timed_steps, args.engine)
         ctx.set_workspace(ws)
         t0 = time.perf_counter()
-        dt, cores = time_oracle_mlp(case, BATCH, repeats=4)
+        dt, cores = time_oracle_mlp(case, BATCH, repeats=4 if args.section == "all" else 1)
         line["cpu_baseline"] = {"value": BATCH / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": "the whole batch of 10000 images, best of 4 passes (%.1f s of CPU work in total)"
                                           % (time.perf_counter() - t0)}

@@ -11,8 +11,9 @@
 //             operands into a 4-stage shared-memory ring, completion on mbarriers;
 //   warp 1    allocates all 512 TMEM columns (two accumulator buffers), then one lane issues tcgen05.mma
 //             (M=128, N=256, K=32) four times per stage and releases the stage with tcgen05.commit;
-//   warps 2-5 epilogue: tcgen05.ld of the int32 accumulators (each thread owns one output row, 32 columns at
-//             a time), then either int32 stores, or the BatchNorm-folded threshold + Sign + repack to one
+//   warps 2-9 epilogue (two warps per TMEM lane quadrant, each half of the columns): tcgen05.ld of the int32
+//             accumulators (each thread owns one output row, 32 columns at a time, the next chunk in flight while
+//             the current one is processed), then either int32 stores, or the BatchNorm-folded threshold + Sign + repack to one
 //             32-bit word per 32 columns (and, for the next layer, the same signs as bytes).
 // Every wait is bounded: after the limit the kernel records an error code and runs to its end without
 // touching the accumulators, so a failure surfaces as BNN_ERR_DEVICE_STATUS instead of a hang.
@@ -22,13 +23,20 @@
 
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 128;     // BK in bytes = int8 elements
-constexpr int STAGES = 4;
-constexpr int NTHREADS = 192;
-constexpr uint32_t A_BYTES = BM * BK, B_BYTES = BN * BK;
-constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int BM = 128, BK = 128;               // BK in bytes = int8 elements
+constexpr int BN_MAX = 256;                     // tile width: 256, or 128 for narrow outputs (template parameter)
+constexpr int EPI_WARPS = 8;                    // two per TMEM lane quadrant, each takes half of the tile's columns
+constexpr int EPI_THREADS = EPI_WARPS * 32;
+constexpr int NTHREADS = 64 + EPI_THREADS;
+constexpr uint32_t A_BYTES = BM * BK;
 constexpr int ACC_BUFS = 2;
-constexpr uint32_t TMEM_COLS = 512;       // two accumulator buffers of BN columns
+template <int BN> struct Cfg {
+    static constexpr uint32_t B_BYTES = BN * BK;
+    static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int STAGES = (BN == 256) ? 4 : 6;          // 192 KB of operand stages either way
+    static constexpr uint32_t TMEM_COLS = 2 * BN;               // two accumulator buffers of BN columns
+};
+constexpr int STAGES_MAX = 6;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // a wait gives up after 2 s of wall clock
 
 __device__ int g_umma_error;                    // 0 = fine; otherwise a code saying which wait gave up
@@ -116,19 +124,28 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
           "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// Completes every tcgen05.ld issued so far.  The registers are passed through so that no use of them can be
+// scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+          "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),
+          "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
+          "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+        :: "memory");
 }
 
 struct __align__(8) Control {
-    uint64_t full[STAGES];
-    uint64_t empty[STAGES];
+    uint64_t full[STAGES_MAX];
+    uint64_t empty[STAGES_MAX];
     uint64_t acc_full[ACC_BUFS];
     uint64_t acc_empty[ACC_BUFS];
     uint32_t tmem_base;
     uint32_t failed;
-    int32_t thr[ACC_BUFS][BN];
-    uint32_t flip[ACC_BUFS][BN / 32];
-    uint32_t poolw[BM][BN / 32 + 1];   // convolution with pooling: the sign words of every pixel of the tile
+    int32_t thr[ACC_BUFS][BN_MAX];
+    uint32_t flip[ACC_BUFS][BN_MAX / 32];
+    uint32_t poolw[BM][BN_MAX / 32 + 1];   // convolution with pooling: the sign words of every pixel of the tile
 };
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
@@ -142,8 +159,12 @@ __device__ __forceinline__ void fail(Control *ctl, int code) {
 // Persistent: gridDim.x CTAs (one per SM) walk the tile list with stride gridDim.x.  The shared-memory ring
 // runs on across tiles; the accumulator is double-buffered in tensor memory (2 x 256 columns), so the
 // epilogue of tile i overlaps the main loop of tile i+1.
+template <int BN>
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const UmmaArgs p) {
+    constexpr int STAGES = Cfg<BN>::STAGES;
+    constexpr uint32_t STAGE_BYTES = Cfg<BN>::STAGE_BYTES;
+    constexpr uint32_t TMEM_COLS = Cfg<BN>::TMEM_COLS;
     extern __shared__ uint8_t smem_raw[];
     // operand tiles need 1024-byte alignment for the 128-byte swizzle pattern
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -156,7 +177,7 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
-        for (int b = 0; b < ACC_BUFS; ++b) { mbar_init(smem_u32(&ctl->acc_full[b]), 1); mbar_init(smem_u32(&ctl->acc_empty[b]), 4); }
+        for (int b = 0; b < ACC_BUFS; ++b) { mbar_init(smem_u32(&ctl->acc_full[b]), 1); mbar_init(smem_u32(&ctl->acc_empty[b]), EPI_WARPS); }
         ctl->failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -215,16 +236,19 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                     const uint64_t bdesc = smem_desc_sw128(smem_u32(tiles + s * STAGE_BYTES + A_BYTES));
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k)   // 32 bytes of K per instruction: start address advances by 32 B (>> 4 = 2)
-                        umma_i8(tmem_d, adesc + 2 * k, bdesc + 2 * k, p.idesc, (kit > 0 || k > 0) ? 1u : 0u);
+                        umma_i8(tmem_d, adesc + 2 * k, bdesc + 2 * k, p.idesc | ((uint32_t)(BN >> 3) << 17), (kit > 0 || k > 0) ? 1u : 0u);
                     umma_commit(smem_u32(&ctl->empty[s]));      // stage may be refilled once these MMAs have read it
                 }
                 umma_commit(smem_u32(&ctl->acc_full[buf]));     // accumulators of this tile complete (also after a failure)
             }
         }
     } else {
-        // ---------------- epilogue: warps 2..5 own TMEM lanes 32*(warp%4) .. +31
+        // ---------------- epilogue: warps 2..9; warp w may only touch TMEM lanes 32*(w%4) .. +31, so two warps share
+        // each lane quadrant and split the tile's columns between them
         const int q = warp & 3;
-        const int et = threadIdx.x - 64;                 // 0..127 among the epilogue threads
+        const int half = (warp - 2) >> 2;
+        constexpr int CHUNKS = BN / 32, CPW = CHUNKS / 2;   // 32-column chunks per tile and per warp
+        const int et = threadIdx.x - 64;                 // 0 .. EPI_THREADS-1 among the epilogue threads
         uint32_t tc = 0;
         bool ok = true;
         for (int64_t t = blockIdx.x; t < ntiles; t += gridDim.x, ++tc) {
@@ -232,23 +256,31 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
             const int64_t m0 = (t % tiles_m) * BM, n0 = (t / tiles_m) * BN;
             const int64_t row = m0 + 32 * q + lane;
             if (p.out) {
-                for (int e = et; e < BN; e += 128) ctl->thr[buf][e] = (n0 + e < p.N) ? p.thr[n0 + e] : 0x7fffffff;
+                for (int e = et; e < BN; e += EPI_THREADS) ctl->thr[buf][e] = (n0 + e < p.N) ? p.thr[n0 + e] : 0x7fffffff;
                 if (et < BN / 32) {
                     const int64_t w = (n0 >> 5) + et;
                     ctl->flip[buf][et] = (p.flip && w * 32 < p.N) ? p.flip[w] : 0u;
                 }
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps only
+            asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");   // the epilogue warps only
             if (ok && !mbar_wait(smem_u32(&ctl->acc_full[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 3); ok = false; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             ok = ok && (ctl->failed == 0);
             if (ok) {
+                // chunk c+1 is fetched from tensor memory while chunk c is processed
+                const uint32_t tbase = tmem_base + ((uint32_t)(32 * q) << 16) + buf * BN;
+                uint32_t ra[32], rb[32];
+                const int c_first = half * CPW;
+                if (n0 + 32 * c_first < p.N) { tmem_ld32(tbase + (uint32_t)(32 * c_first), ra); tmem_ld_wait(ra); }
 #pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
+                for (int cc = 0; cc < CPW; ++cc) {
+                    const int c = c_first + cc;
                     const int64_t col0 = n0 + 32 * c;
                     if (col0 >= p.N) break;                      // uniform over the warp
-                    uint32_t r[32];
-                    tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + buf * BN + (uint32_t)(32 * c), r);
+                    const bool more = (cc + 1 < CPW) && (col0 + 32 < p.N);
+                    uint32_t (&r)[32] = (cc & 1) ? rb : ra;
+                    uint32_t (&rn)[32] = (cc & 1) ? ra : rb;
+                    if (more) tmem_ld32(tbase + (uint32_t)(32 * (c + 1)), rn);
                     if (row < p.M) {
                         if (p.C) {
                             int32_t *dst = p.C + row * p.ldc + col0;
@@ -290,19 +322,20 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                             }
                         }
                     }
+                    if (more) tmem_ld_wait(rn);
                 }
                 // padding words of the packed output
-                if (p.out && !p.pool && row < p.M && n0 + BN >= p.N) {
+                if (half == 0 && p.out && !p.pool && row < p.M && n0 + BN >= p.N) {
                     for (int64_t w = (p.N + 31) >> 5; w < p.ldo; ++w) p.out[row * p.ldo + w] = 0u;
                 }
             }
             if (p.pool) {
                 // 2x2 max-pool then threshold == OR of the four thresholded bits, then flip.  The tile holds TB images
                 // x TH rows x W columns (TH, W even), i.e. 32 whole windows; 256 (window, word) items for 128 threads.
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
                 if (ok) {
                     const int Wo = p.W >> 1, nwords = (int)((min((int64_t)BN, p.N - n0) + 31) >> 5);
-                    for (int e = et; e < (BM / 4) * (BN / 32); e += 128) {
+                    for (int e = et; e < (BM / 4) * (BN / 32); e += EPI_THREADS) {
                         const int win = e / (BN / 32), c = e % (BN / 32);
                         if (c >= nwords) continue;
                         const int wx = win % Wo, wy = win / Wo;                 // wy counts window rows over the tile's TB*TH/2 rows
@@ -425,7 +458,7 @@ int make_map(bnn_ctx *ctx, CUtensorMap *map, const void *base, int64_t rows, int
 
 }  // namespace
 
-static size_t umma_smem_bytes() { return (size_t)STAGES * STAGE_BYTES + sizeof(Control) + 1024; }
+template <int BN> static size_t umma_smem_bytes() { return (size_t)Cfg<BN>::STAGES * Cfg<BN>::STAGE_BYTES + sizeof(Control) + 1024; }
 // Opt in to the large dynamic shared memory once per device.
 static int umma_prepare(bnn_ctx *ctx) {
     static std::mutex attr_mutex;
@@ -433,10 +466,21 @@ static int umma_prepare(bnn_ctx *ctx) {
     std::lock_guard<std::mutex> lock(attr_mutex);
     if (ctx->device < 0 || ctx->device >= 64) return BNN_ERR_INVALID_ARG;
     if (!attr_set[ctx->device]) {
-        BNN_CUDA_TRY(ctx, cudaFuncSetAttribute(k_umma_i8, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes()));
+        BNN_CUDA_TRY(ctx, cudaFuncSetAttribute(k_umma_i8<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes<256>()));
+        BNN_CUDA_TRY(ctx, cudaFuncSetAttribute(k_umma_i8<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes<128>()));
         attr_set[ctx->device] = true;
     }
     return BNN_OK;
+}
+// Tile width for N output columns: 128 when that leaves no (or less) idle MMA columns.
+static int umma_tile_n(int64_t N) { return (((N + 127) / 128) & 1) ? 128 : 256; }
+static int umma_launch(bnn_ctx *ctx, const CUtensorMap &mapA, const CUtensorMap &mapB, const UmmaArgs &a, int bn) {
+    if (int st = umma_prepare(ctx)) return st;
+    const int64_t tiles = ((a.M + BM - 1) / BM) * ((a.N + bn - 1) / bn);
+    const int64_t grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+    if (bn == 256) k_umma_i8<256><<<(unsigned)grid, NTHREADS, umma_smem_bytes<256>(), ctx->stream>>>(mapA, mapB, a);
+    else k_umma_i8<128><<<(unsigned)grid, NTHREADS, umma_smem_bytes<128>(), ctx->stream>>>(mapA, mapB, a);
+    return bnn_check_launch(ctx);
 }
 
 size_t bnn_umma_operand_bytes(int64_t rows, int64_t K) {
@@ -466,28 +510,19 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
     }
     if ((lda8 & 15) || (ldb8 & 15) || !bnn_aligned16(A8) || !bnn_aligned16(B8)) return BNN_ERR_ALIGNMENT;
     if (M > 0x7fffffff || N > 0x7fffffff) return BNN_ERR_INVALID_ARG;
+    if (K <= 0) return BNN_ERR_INVALID_ARG;      // callers route the empty product elsewhere
     CUtensorMap mapA, mapB;
+    const int bn = umma_tile_n(N);
     const int64_t kb = ((K + 15) / 16) * 16;      // extent along K in bytes; beyond it TMA fills zeros
-    if (K > 0) {
-        if (int st = make_map(ctx, &mapA, A8, M, kb <= lda8 ? kb : lda8, lda8, BM)) return st;
-        if (int st = make_map(ctx, &mapB, B8, N, kb <= ldb8 ? kb : ldb8, ldb8, BN)) return st;
-    } else {
-        memset(&mapA, 0, sizeof(mapA));
-        memset(&mapB, 0, sizeof(mapB));
-    }
+    if (int st = make_map(ctx, &mapA, A8, M, kb <= lda8 ? kb : lda8, lda8, BM)) return st;
+    if (int st = make_map(ctx, &mapB, B8, N, kb <= ldb8 ? kb : ldb8, ldb8, bn)) return st;
     UmmaArgs a{};
     a.M = M; a.N = N;
     a.k_iters = (int)((K + BK - 1) / BK);
-    a.idesc = (2u << 4) | ((a_unsigned ? 0u : 1u) << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+    a.idesc = (2u << 4) | ((a_unsigned ? 0u : 1u) << 7) | (1u << 10) | ((uint32_t)(BM >> 4) << 24);   // N field added by the kernel
     a.C = C; a.ldc = ldc; a.out = out; a.ldo = ldo; a.out8 = out8; a.ldo8 = ldo8; a.thr = thr; a.flip = flip;
     a.pool = pool; a.H = (int)H; a.W = (int)W;
-    const size_t smem = umma_smem_bytes();
-    if (int st = umma_prepare(ctx)) return st;
-    if (K <= 0) return BNN_ERR_INVALID_ARG;      // callers route the empty product elsewhere
-    const int64_t tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
-    const int64_t grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
-    k_umma_i8<<<(unsigned)grid, NTHREADS, smem, ctx->stream>>>(mapA, mapB, a);
-    return bnn_check_launch(ctx);
+    return umma_launch(ctx, mapA, mapB, a, bn);
 }
 
 namespace {
@@ -539,19 +574,16 @@ int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B,
     int TH, TB;
     if (!bnn_umma_conv_tiling(H, W, pool, &TH, &TB) || (C_in % BK) != 0 || (pool && out_sums)) return BNN_ERR_INVALID_ARG;
     CUtensorMap mapA, mapB;
+    const int bn = umma_tile_n(C_out);
     if (int st = make_map_nhwc(ctx, &mapA, act8, B, H, W, C_in, (int)W, TH, TB)) return st;
-    if (int st = make_map(ctx, &mapB, W8, C_out, 9 * C_in, 9 * C_in, BN)) return st;
+    if (int st = make_map(ctx, &mapB, W8, C_out, 9 * C_in, 9 * C_in, bn)) return st;
     UmmaArgs a{};
     a.M = B * H * W; a.N = C_out;
     a.k_iters = (int)(9 * (C_in / BK));
-    a.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+    a.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BM >> 4) << 24);
     a.C = out_sums; a.ldc = C_out; a.out = out_bits; a.ldo = (C_out + 31) / 32; a.thr = thr; a.flip = flip;
     a.conv = 1; a.H = (int)H; a.W = (int)W; a.TH = TH; a.TB = TB; a.c_chunks = (int)(C_in / BK); a.pool = pool;
-    if (int st = umma_prepare(ctx)) return st;
-    const int64_t tiles = ((a.M + BM - 1) / BM) * ((C_out + BN - 1) / BN);
-    const int64_t grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
-    k_umma_i8<<<(unsigned)grid, NTHREADS, umma_smem_bytes(), ctx->stream>>>(mapA, mapB, a);
-    return bnn_check_launch(ctx);
+    return umma_launch(ctx, mapA, mapB, a, bn);
 }
 
 // Reads (and clears) the error word the tensor-core kernel sets when one of its bounded waits gives up.
