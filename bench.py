@@ -149,6 +149,7 @@ def main():
     ap.add_argument("--variant", type=int, default=0, help="tiled-kernel inner loop: 0 default, 1 plain popc, 2 carry-save")
     ap.add_argument("--engine", type=int, default=0, help="0 auto (tensor-core int8 engine for large shapes), 1 CUDA-core XOR-popcount only, 2 tensor")
     ap.add_argument("--tile-rows", type=int, default=0, help="accumulator rows per thread of the CUDA-core tile kernel (8 or 16; 0 = library default)")
+    ap.add_argument("--pair-mode", type=int, default=0, help="tensor engine CTA pairs (cta_group::2): 0 = for very large outputs, 1 = never, 2 = wherever possible")
     ap.add_argument("--no-extras", action="store_true", help="skip the GEMM / ConvNet side measurements and the CPU baseline")
     ap.add_argument("--gemm-size", type=int, default=8192)
     ap.add_argument("--section", default="all", choices=["all", "gemm", "convnet", "sweep"],
@@ -176,6 +177,7 @@ def main():
     ctx.set_engine(args.engine)
     if args.tile_rows:
         ctx.set_tile_rows(args.tile_rows)
+    ctx.set_pair_mode(args.pair_mode)
 
     def sync_all():
         torch.cuda.synchronize()

@@ -78,6 +78,10 @@ BNN_API int bnn_set_tile_rows(bnn_ctx *ctx, int rows);
  * multiplies them with int8 tensor-core instructions (Section 4: on +-1 inputs the binary kernel and an ordinary
  * matrix product return identical outputs). */
 BNN_API int bnn_set_engine(bnn_ctx *ctx, int engine);
+/* Tensor-core engine only: plain products can run on pairs of SMs (thread-block clusters of two, tcgen05
+ * cta_group::2) that share the B operand.  0 (default) = for outputs of 2^26 elements and more, where it measured
+ * faster; 1 = never; 2 = wherever the kernel allows (M >= 512, 256-wide tiles).  Results are identical. */
+BNN_API int bnn_set_pair_mode(bnn_ctx *ctx, int mode);
 /* Workspace bytes bnn_xnor_gemm / bnn_binary_dense need to run M x N x K on the tensor-core engine
  * (0 if the shape does not qualify for it). */
 BNN_API size_t bnn_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);

@@ -25,7 +25,7 @@ EXPORTS = (
     "bnn_set_popc_variant", "bnn_pack_signs", "bnn_xnor_gemm", "bnn_binary_dense", "bnn_first_layer_bitplanes",
     "bnn_binary_conv2d", "bnn_mlp_workspace_bytes", "bnn_mlp_forward", "bnn_mlp_forward_host",
     "bnn_fold_batchnorm", "bnn_mlp_noalloc_max_bytes", "bnn_mlp_forward_noalloc", "bnn_set_engine",
-    "bnn_gemm_workspace_bytes", "bnn_device_status", "bnn_conv_workspace_bytes", "bnn_set_tile_rows",
+    "bnn_gemm_workspace_bytes", "bnn_device_status", "bnn_conv_workspace_bytes", "bnn_set_tile_rows", "bnn_set_pair_mode",
 )
 
 
@@ -70,6 +70,7 @@ def lib() -> ctypes.CDLL:
         L.bnn_set_popc_variant.argtypes = [vp, c_int]
         L.bnn_set_engine.argtypes = [vp, c_int]
         L.bnn_set_tile_rows.argtypes = [vp, c_int]
+        L.bnn_set_pair_mode.argtypes = [vp, c_int]
         L.bnn_gemm_workspace_bytes.argtypes = [i64, i64, i64]
         L.bnn_gemm_workspace_bytes.restype = c_size_t
         L.bnn_device_status.argtypes = [vp]
@@ -148,6 +149,9 @@ class Context:
             self._ck(lib().bnn_set_workspace(self._h, None, 0), "bnn_set_workspace")
         else:
             self._ck(lib().bnn_set_workspace(self._h, _ptr(ws), ws.numel() * ws.element_size()), "bnn_set_workspace")
+
+    def set_pair_mode(self, mode: int):
+        self._ck(lib().bnn_set_pair_mode(self._h, mode), "bnn_set_pair_mode")
 
     def set_tile_rows(self, rows: int):
         self._ck(lib().bnn_set_tile_rows(self._h, rows), "bnn_set_tile_rows")

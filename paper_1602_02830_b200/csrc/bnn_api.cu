@@ -19,6 +19,7 @@ extern "C" int bnn_create(bnn_ctx **out, int device, void *cuda_stream) {
     c->variant = 0;
     c->engine = 0;
     c->tile_rows = 8;
+    c->pair_mode = 0;
     if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
         delete c;
         return BNN_ERR_CUDA;
@@ -55,6 +56,12 @@ extern "C" int bnn_set_popc_variant(bnn_ctx *ctx, int variant) {
 extern "C" int bnn_set_tile_rows(bnn_ctx *ctx, int rows) {
     if (!ctx || (rows != 8 && rows != 16)) return BNN_ERR_INVALID_ARG;
     ctx->tile_rows = rows;
+    return BNN_OK;
+}
+
+extern "C" int bnn_set_pair_mode(bnn_ctx *ctx, int mode) {
+    if (!ctx || mode < 0 || mode > 2) return BNN_ERR_INVALID_ARG;
+    ctx->pair_mode = mode;
     return BNN_OK;
 }
 

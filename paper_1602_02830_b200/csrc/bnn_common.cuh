@@ -14,6 +14,7 @@ struct bnn_ctx {
     int sm_count;
     int variant;   // inner-loop choice of the tiled kernel (0 auto, 1 plain popc, 2 carry-save)
     int tile_rows; // accumulator rows per thread of the tiled popc kernel: 16 or 8
+    int pair_mode; // tensor engine: 0 = CTA pairs (cta_group::2) for very large outputs, 1 = never, 2 = wherever the kernel allows
     int engine;    // 0 auto, 1 CUDA-core XOR-popcount kernels only, 2 tensor-core int8 engine where it applies
 };
 

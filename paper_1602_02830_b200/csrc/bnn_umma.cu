@@ -156,6 +156,117 @@ __device__ __forceinline__ void fail(Control *ctl, int code) {
     atomicExch(&g_umma_error, code);
 }
 
+// One tile's epilogue for the calling epilogue warp: stage the tile's thresholds, wait for the accumulators in
+// buffer `buf`, and turn them into the requested outputs.  `ok` turns false once a wait has given up.
+template <int BN>
+__device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, uint32_t tmem_base, uint32_t buf, uint32_t tc,
+                                              int64_t m0, int64_t n0, int q, int half, int lane, int et, bool &ok) {
+    constexpr int CHUNKS = BN / 32, CPW = CHUNKS / 2;   // 32-column chunks per tile and per warp
+    const int64_t row = m0 + 32 * q + lane;
+    if (p.out) {
+        for (int e = et; e < BN; e += EPI_THREADS) ctl->thr[buf][e] = (n0 + e < p.N) ? p.thr[n0 + e] : 0x7fffffff;
+        if (et < BN / 32) {
+            const int64_t w = (n0 >> 5) + et;
+            ctl->flip[buf][et] = (p.flip && w * 32 < p.N) ? p.flip[w] : 0u;
+        }
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");   // the epilogue warps only
+    if (ok && !mbar_wait(smem_u32(&ctl->acc_full[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 3); ok = false; }
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    ok = ok && (ctl->failed == 0);
+    if (ok) {
+        // chunk c+1 is fetched from tensor memory while chunk c is processed
+        const uint32_t tbase = tmem_base + ((uint32_t)(32 * q) << 16) + buf * BN;
+        uint32_t ra[32], rb[32];
+        const int c_first = half * CPW;
+        if (n0 + 32 * c_first < p.N) { tmem_ld32(tbase + (uint32_t)(32 * c_first), ra); tmem_ld_wait(ra); }
+#pragma unroll 1
+        for (int cc = 0; cc < CPW; ++cc) {
+            const int c = c_first + cc;
+            const int64_t col0 = n0 + 32 * c;
+            if (col0 >= p.N) break;                      // uniform over the warp
+            const bool more = (cc + 1 < CPW) && (col0 + 32 < p.N);
+            uint32_t (&r)[32] = (cc & 1) ? rb : ra;
+            uint32_t (&rn)[32] = (cc & 1) ? ra : rb;
+            if (more) tmem_ld32(tbase + (uint32_t)(32 * (c + 1)), rn);
+            if (row < p.M) {
+                if (p.C) {
+                    int32_t *dst = p.C + row * p.ldc + col0;
+                    if (col0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<int4 *>(dst + j) = make_int4((int)r[j], (int)r[j + 1], (int)r[j + 2], (int)r[j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (col0 + j < p.N) dst[j] = (int32_t)r[j];
+                    }
+                }
+                if (p.out) {
+                    uint32_t word = 0u;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) word |= (uint32_t)((int32_t)r[j] >= ctl->thr[buf][32 * c + j]) << j;
+                    word ^= ctl->flip[buf][c];
+                    if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;      // columns beyond N stay 0
+                    if (p.pool) ctl->poolw[32 * q + lane][c] = word ^ ctl->flip[buf][c];   // un-flipped (dot >= thr) bits
+                    else p.out[row * p.ldo + (col0 >> 5)] = word;
+                    if (p.out8) {
+                        int8_t *d8 = p.out8 + row * p.ldo8 + col0;
+                        uint32_t b[8];
+#pragma unroll
+                        for (int g = 0; g < 8; ++g) {
+                            // 4 sign bits -> 4 bytes of +1 (0x01) / -1 (0xff)
+                            const uint32_t t4 = (((word >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u;
+                            b[g] = ~(t4 * 0xfeu);
+                        }
+                        if (col0 + 32 <= p.N) {
+                            *reinterpret_cast<uint4 *>(d8) = make_uint4(b[0], b[1], b[2], b[3]);
+                            *reinterpret_cast<uint4 *>(d8 + 16) = make_uint4(b[4], b[5], b[6], b[7]);
+                        } else {
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + j < p.N) d8[j] = ((word >> j) & 1u) ? (int8_t)1 : (int8_t)-1;
+                                else if (col0 + j < p.ldo8) d8[j] = 0;
+                        }
+                    }
+                }
+            }
+            if (more) tmem_ld_wait(rn);
+        }
+        // padding words of the packed output
+        if (half == 0 && p.out && !p.pool && row < p.M && n0 + BN >= p.N) {
+            for (int64_t w = (p.N + 31) >> 5; w < p.ldo; ++w) p.out[row * p.ldo + w] = 0u;
+        }
+    }
+    if (p.pool) {
+        // 2x2 max-pool then threshold == OR of the four thresholded bits, then flip.  The tile holds TB images
+        // x TH rows x W columns (TH, W even), i.e. 32 whole windows; 256 (window, word) items for 128 threads.
+        asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
+        if (ok) {
+            const int Wo = p.W >> 1, nwords = (int)((min((int64_t)BN, p.N - n0) + 31) >> 5);
+            for (int e = et; e < (BM / 4) * (BN / 32); e += EPI_THREADS) {
+                const int win = e / (BN / 32), c = e % (BN / 32);
+                if (c >= nwords) continue;
+                const int wx = win % Wo, wy = win / Wo;                 // wy counts window rows over the tile's TB*TH/2 rows
+                const int r0 = (2 * wy) * p.W + 2 * wx;                 // top-left pixel of the window inside the tile
+                const int64_t pix = m0 + r0;                            // its linear pixel index b*H*W + y*W + x
+                if (pix >= p.M) continue;
+                uint32_t word = ctl->poolw[r0][c] | ctl->poolw[r0 + 1][c] | ctl->poolw[r0 + p.W][c] | ctl->poolw[r0 + p.W + 1][c];
+                word ^= ctl->flip[buf][c];
+                const int64_t col0 = n0 + 32 * c;
+                if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;
+                // output pixel: same image, (y/2, x/2)
+                const int64_t img = pix / ((int64_t)p.H * p.W);
+                const int64_t rem = pix - img * (int64_t)p.H * p.W;
+                const int64_t oy = (rem / p.W) >> 1, ox = (rem % p.W) >> 1;
+                const int64_t opix = (img * (p.H >> 1) + oy) * Wo + ox;
+                p.out[opix * p.ldo + (col0 >> 5)] = word;
+                if (n0 + BN >= p.N && c == nwords - 1)
+                    for (int64_t w = (p.N + 31) >> 5; w < p.ldo; ++w) p.out[opix * p.ldo + w] = 0u;
+            }
+        }
+    }
+}
+
 // Persistent: gridDim.x CTAs (one per SM) walk the tile list with stride gridDim.x.  The shared-memory ring
 // runs on across tiles; the accumulator is double-buffered in tensor memory (2 x 256 columns), so the
 // epilogue of tile i overlaps the main loop of tile i+1.
@@ -247,116 +358,13 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
         // each lane quadrant and split the tile's columns between them
         const int q = warp & 3;
         const int half = (warp - 2) >> 2;
-        constexpr int CHUNKS = BN / 32, CPW = CHUNKS / 2;   // 32-column chunks per tile and per warp
         const int et = threadIdx.x - 64;                 // 0 .. EPI_THREADS-1 among the epilogue threads
         uint32_t tc = 0;
         bool ok = true;
         for (int64_t t = blockIdx.x; t < ntiles; t += gridDim.x, ++tc) {
             const uint32_t buf = tc & 1;
             const int64_t m0 = (t % tiles_m) * BM, n0 = (t / tiles_m) * BN;
-            const int64_t row = m0 + 32 * q + lane;
-            if (p.out) {
-                for (int e = et; e < BN; e += EPI_THREADS) ctl->thr[buf][e] = (n0 + e < p.N) ? p.thr[n0 + e] : 0x7fffffff;
-                if (et < BN / 32) {
-                    const int64_t w = (n0 >> 5) + et;
-                    ctl->flip[buf][et] = (p.flip && w * 32 < p.N) ? p.flip[w] : 0u;
-                }
-            }
-            asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");   // the epilogue warps only
-            if (ok && !mbar_wait(smem_u32(&ctl->acc_full[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 3); ok = false; }
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            ok = ok && (ctl->failed == 0);
-            if (ok) {
-                // chunk c+1 is fetched from tensor memory while chunk c is processed
-                const uint32_t tbase = tmem_base + ((uint32_t)(32 * q) << 16) + buf * BN;
-                uint32_t ra[32], rb[32];
-                const int c_first = half * CPW;
-                if (n0 + 32 * c_first < p.N) { tmem_ld32(tbase + (uint32_t)(32 * c_first), ra); tmem_ld_wait(ra); }
-#pragma unroll 1
-                for (int cc = 0; cc < CPW; ++cc) {
-                    const int c = c_first + cc;
-                    const int64_t col0 = n0 + 32 * c;
-                    if (col0 >= p.N) break;                      // uniform over the warp
-                    const bool more = (cc + 1 < CPW) && (col0 + 32 < p.N);
-                    uint32_t (&r)[32] = (cc & 1) ? rb : ra;
-                    uint32_t (&rn)[32] = (cc & 1) ? ra : rb;
-                    if (more) tmem_ld32(tbase + (uint32_t)(32 * (c + 1)), rn);
-                    if (row < p.M) {
-                        if (p.C) {
-                            int32_t *dst = p.C + row * p.ldc + col0;
-                            if (col0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
-#pragma unroll
-                                for (int j = 0; j < 32; j += 4)
-                                    *reinterpret_cast<int4 *>(dst + j) = make_int4((int)r[j], (int)r[j + 1], (int)r[j + 2], (int)r[j + 3]);
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j)
-                                    if (col0 + j < p.N) dst[j] = (int32_t)r[j];
-                            }
-                        }
-                        if (p.out) {
-                            uint32_t word = 0u;
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) word |= (uint32_t)((int32_t)r[j] >= ctl->thr[buf][32 * c + j]) << j;
-                            word ^= ctl->flip[buf][c];
-                            if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;      // columns beyond N stay 0
-                            if (p.pool) ctl->poolw[32 * q + lane][c] = word ^ ctl->flip[buf][c];   // un-flipped (dot >= thr) bits
-                            else p.out[row * p.ldo + (col0 >> 5)] = word;
-                            if (p.out8) {
-                                int8_t *d8 = p.out8 + row * p.ldo8 + col0;
-                                uint32_t b[8];
-#pragma unroll
-                                for (int g = 0; g < 8; ++g) {
-                                    // 4 sign bits -> 4 bytes of +1 (0x01) / -1 (0xff)
-                                    const uint32_t t4 = (((word >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u;
-                                    b[g] = ~(t4 * 0xfeu);
-                                }
-                                if (col0 + 32 <= p.N) {
-                                    *reinterpret_cast<uint4 *>(d8) = make_uint4(b[0], b[1], b[2], b[3]);
-                                    *reinterpret_cast<uint4 *>(d8 + 16) = make_uint4(b[4], b[5], b[6], b[7]);
-                                } else {
-                                    for (int j = 0; j < 32; ++j)
-                                        if (col0 + j < p.N) d8[j] = ((word >> j) & 1u) ? (int8_t)1 : (int8_t)-1;
-                                        else if (col0 + j < p.ldo8) d8[j] = 0;
-                                }
-                            }
-                        }
-                    }
-                    if (more) tmem_ld_wait(rn);
-                }
-                // padding words of the packed output
-                if (half == 0 && p.out && !p.pool && row < p.M && n0 + BN >= p.N) {
-                    for (int64_t w = (p.N + 31) >> 5; w < p.ldo; ++w) p.out[row * p.ldo + w] = 0u;
-                }
-            }
-            if (p.pool) {
-                // 2x2 max-pool then threshold == OR of the four thresholded bits, then flip.  The tile holds TB images
-                // x TH rows x W columns (TH, W even), i.e. 32 whole windows; 256 (window, word) items for 128 threads.
-                asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
-                if (ok) {
-                    const int Wo = p.W >> 1, nwords = (int)((min((int64_t)BN, p.N - n0) + 31) >> 5);
-                    for (int e = et; e < (BM / 4) * (BN / 32); e += EPI_THREADS) {
-                        const int win = e / (BN / 32), c = e % (BN / 32);
-                        if (c >= nwords) continue;
-                        const int wx = win % Wo, wy = win / Wo;                 // wy counts window rows over the tile's TB*TH/2 rows
-                        const int r0 = (2 * wy) * p.W + 2 * wx;                 // top-left pixel of the window inside the tile
-                        const int64_t pix = m0 + r0;                            // its linear pixel index b*H*W + y*W + x
-                        if (pix >= p.M) continue;
-                        uint32_t word = ctl->poolw[r0][c] | ctl->poolw[r0 + 1][c] | ctl->poolw[r0 + p.W][c] | ctl->poolw[r0 + p.W + 1][c];
-                        word ^= ctl->flip[buf][c];
-                        const int64_t col0 = n0 + 32 * c;
-                        if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;
-                        // output pixel: same image, (y/2, x/2)
-                        const int64_t img = pix / ((int64_t)p.H * p.W);
-                        const int64_t rem = pix - img * (int64_t)p.H * p.W;
-                        const int64_t oy = (rem / p.W) >> 1, ox = (rem % p.W) >> 1;
-                        const int64_t opix = (img * (p.H >> 1) + oy) * Wo + ox;
-                        p.out[opix * p.ldo + (col0 >> 5)] = word;
-                        if (n0 + BN >= p.N && c == nwords - 1)
-                            for (int64_t w = (p.N + 31) >> 5; w < p.ldo; ++w) p.out[opix * p.ldo + w] = 0u;
-                    }
-                }
-            }
+            epilogue_tile<BN>(ctl, p, tmem_base, buf, tc, m0, n0, q, half, lane, et, ok);
             // hand the accumulator buffer back to the MMA warp
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
@@ -369,6 +377,151 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Two-SM variant (GEMM mode): a cluster of two CTAs computes a 256 x 256 tile with tcgen05.mma cta_group::2.
+// Each CTA loads its own 128 rows of A and its own 128 of the tile's 256 B rows (32 KB per K step instead of
+// 48 KB, six stages), so the L2 -> shared-memory traffic per MAC drops by a third; the pair's tensor cores read
+// both halves of B.  CTA 0 of the pair issues the MMAs; completion of every CTA's TMA loads is counted on CTA 0's
+// "full" barrier, stages and accumulators are released to both CTAs with multicast tcgen05.commit, and the
+// epilogue warps of both CTAs hand their accumulator buffer back by arriving on CTA 0's barrier.
+constexpr int STAGES2 = 6;
+constexpr uint32_t STAGE2_BYTES = 2 * A_BYTES;           // A half-tile + B half-tile, 128 rows x 128 bytes each
+constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;              // clears the CTA-rank bit of a shared::cluster address -> CTA 0 of the pair
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_2d_2sm(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void umma_i8_2sm(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrives on the barrier at this shared-memory offset in both CTAs of the pair once the MMAs issued so far are done.
+__device__ __forceinline__ void umma_commit_2sm(uint32_t bar) {
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask) : "memory");
+}
+// Arrive on the barrier at the same offset in CTA 0 of the cluster.
+__device__ __forceinline__ void mbar_arrive_cta0(uint32_t bar) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(remote) : "r"(bar));
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
+k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const UmmaArgs p) {
+    constexpr int BN = 256;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    Control *ctl = reinterpret_cast<Control *>(tiles + STAGES2 * STAGE2_BYTES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();                // 0 = leader of the pair
+    const int64_t pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+    const int64_t tiles_m = (p.M + 2 * BM - 1) / (2 * BM);  // 256-row tiles
+    const int64_t tiles_n = (p.N + BN - 1) / BN;
+    const int64_t ntiles = tiles_m * tiles_n;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES2; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
+        for (int b = 0; b < ACC_BUFS; ++b) { mbar_init(smem_u32(&ctl->acc_full[b]), 1); mbar_init(smem_u32(&ctl->acc_empty[b]), 2 * EPI_WARPS); }
+        ctl->failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(2u * BN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    cluster_sync_all();                                     // both CTAs' barriers exist before anyone signals them
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ---------------- TMA producer (both CTAs): own A rows, own half of the tile's B rows
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int64_t t = pair; t < ntiles && ok; t += npairs) {
+                const int m0 = (int)((t % tiles_m) * (2 * BM) + rank * BM);
+                const int nb0 = (int)((t / tiles_m) * BN + rank * (BN / 2));
+                for (int kit = 0; kit < p.k_iters; ++kit, ++it) {
+                    const uint32_t s = it % STAGES2;
+                    if (it >= STAGES2 && !mbar_wait(smem_u32(&ctl->empty[s]), ((it / STAGES2) - 1) & 1)) { fail(ctl, 11); ok = false; break; }
+                    if (rank == 0) mbar_expect_tx(smem_u32(&ctl->full[s]), 2 * STAGE2_BYTES);   // the bytes of both CTAs
+                    const uint32_t bar0 = smem_u32(&ctl->full[s]) & PEER_MASK;
+                    tma_load_2d_2sm(smem_u32(tiles + s * STAGE2_BYTES), &mapA, kit * BK, m0, bar0);
+                    tma_load_2d_2sm(smem_u32(tiles + s * STAGE2_BYTES + A_BYTES), &mapB, kit * BK, nb0, bar0);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer: the leader CTA only, for both tensor cores
+        if (lane == 0 && rank == 0) {
+            uint32_t it = 0, tc = 0;
+            bool ok = true;
+            // the host's descriptor carries M = 128 in bits [24,29); the pair multiplies M = 256
+            const uint32_t idesc = (p.idesc & ~(0x1fu << 24)) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+            for (int64_t t = pair; t < ntiles && ok; t += npairs, ++tc) {
+                const uint32_t buf = tc & 1;
+                if (tc >= ACC_BUFS && !mbar_wait(smem_u32(&ctl->acc_empty[buf]), ((tc / ACC_BUFS) - 1) & 1)) { fail(ctl, 14); ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tmem_d = tmem_base + buf * BN;
+                for (int kit = 0; kit < p.k_iters; ++kit, ++it) {
+                    const uint32_t s = it % STAGES2;
+                    if (!mbar_wait(smem_u32(&ctl->full[s]), (it / STAGES2) & 1)) { fail(ctl, 12); ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint64_t adesc = smem_desc_sw128(smem_u32(tiles + s * STAGE2_BYTES));
+                    const uint64_t bdesc = smem_desc_sw128(smem_u32(tiles + s * STAGE2_BYTES + A_BYTES));
+#pragma unroll
+                    for (int k = 0; k < BK / 32; ++k)
+                        umma_i8_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u);
+                    umma_commit_2sm(smem_u32(&ctl->empty[s]));
+                }
+                umma_commit_2sm(smem_u32(&ctl->acc_full[buf]));
+            }
+        }
+    } else {
+        // ---------------- epilogue (both CTAs): this CTA's 128 rows of the pair's tile
+        const int q = warp & 3;
+        const int half = (warp - 2) >> 2;
+        const int et = threadIdx.x - 64;
+        uint32_t tc = 0;
+        bool ok = true;
+        for (int64_t t = pair; t < ntiles; t += npairs, ++tc) {
+            const uint32_t buf = tc & 1;
+            const int64_t m0 = (t % tiles_m) * (2 * BM) + rank * BM, n0 = (t / tiles_m) * BN;
+            epilogue_tile<BN>(ctl, p, tmem_base, buf, tc, m0, n0, q, half, lane, et, ok);
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cta0(smem_u32(&ctl->acc_empty[buf]));
+        }
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    cluster_sync_all();                                     // nobody leaves while the peer may still read its shared memory
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2u * BN) : "memory");
     }
 }
 
@@ -474,6 +627,33 @@ static int umma_prepare(bnn_ctx *ctx) {
 }
 // Tile width for N output columns: 128 when that leaves no (or less) idle MMA columns.
 static int umma_tile_n(int64_t N) { return (((N + 127) / 128) & 1) ? 128 : 256; }
+static size_t umma2_smem_bytes() { return (size_t)STAGES2 * STAGE2_BYTES + sizeof(Control) + 1024; }
+// Pairs of CTAs that can be resident at once for the two-SM kernel on this device (0 = cannot be used).
+static int umma2_max_pairs(bnn_ctx *ctx) {
+    static std::mutex m;
+    static int cached[64];
+    static bool have[64] = {};
+    std::lock_guard<std::mutex> lock(m);
+    if (ctx->device < 0 || ctx->device >= 64) return 0;
+    if (!have[ctx->device]) {
+        int pairs = 0;
+        if (cudaFuncSetAttribute(k_umma_i8_2sm, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma2_smem_bytes()) == cudaSuccess) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(2 * ctx->sm_count, 1, 1);
+            cfg.blockDim = dim3(NTHREADS, 1, 1);
+            cfg.dynamicSmemBytes = umma2_smem_bytes();
+            cudaLaunchAttribute attr;
+            attr.id = cudaLaunchAttributeClusterDimension;
+            attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+            cfg.attrs = &attr; cfg.numAttrs = 1;
+            if (cudaOccupancyMaxActiveClusters(&pairs, k_umma_i8_2sm, &cfg) != cudaSuccess) pairs = 0;
+        }
+        (void)cudaGetLastError();
+        cached[ctx->device] = pairs;
+        have[ctx->device] = true;
+    }
+    return cached[ctx->device];
+}
 static int umma_launch(bnn_ctx *ctx, const CUtensorMap &mapA, const CUtensorMap &mapB, const UmmaArgs &a, int bn) {
     if (int st = umma_prepare(ctx)) return st;
     const int64_t tiles = ((a.M + BM - 1) / BM) * ((a.N + bn - 1) / bn);
@@ -514,14 +694,25 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
     CUtensorMap mapA, mapB;
     const int bn = umma_tile_n(N);
     const int64_t kb = ((K + 15) / 16) * 16;      // extent along K in bytes; beyond it TMA fills zeros
+    // two-SM kernel: 256-wide tiles, at least two 256-row tiles, plain GEMM epilogues
+    // (auto: only where it measured faster -- outputs of 2^26 elements and more, e.g. 8192 x 8192 or 65536 x 4096)
+    const bool pair_shape = bn == 256 && M >= 512 && !pool;
+    const bool pair_want = ctx->pair_mode == 2 || (ctx->pair_mode == 0 && (double)M * (double)N >= 67108864.0);
+    const int pairs = (pair_shape && pair_want) ? umma2_max_pairs(ctx) : 0;
     if (int st = make_map(ctx, &mapA, A8, M, kb <= lda8 ? kb : lda8, lda8, BM)) return st;
-    if (int st = make_map(ctx, &mapB, B8, N, kb <= ldb8 ? kb : ldb8, ldb8, bn)) return st;
+    if (int st = make_map(ctx, &mapB, B8, N, kb <= ldb8 ? kb : ldb8, ldb8, pairs > 0 ? 128 : bn)) return st;
     UmmaArgs a{};
     a.M = M; a.N = N;
     a.k_iters = (int)((K + BK - 1) / BK);
     a.idesc = (2u << 4) | ((a_unsigned ? 0u : 1u) << 7) | (1u << 10) | ((uint32_t)(BM >> 4) << 24);   // N field added by the kernel
     a.C = C; a.ldc = ldc; a.out = out; a.ldo = ldo; a.out8 = out8; a.ldo8 = ldo8; a.thr = thr; a.flip = flip;
     a.pool = pool; a.H = (int)H; a.W = (int)W;
+    if (pairs > 0) {
+        const int64_t tiles2 = ((M + 2 * BM - 1) / (2 * BM)) * ((N + 255) / 256);
+        const int64_t use = tiles2 < pairs ? tiles2 : pairs;
+        k_umma_i8_2sm<<<(unsigned)(2 * use), NTHREADS, umma2_smem_bytes(), ctx->stream>>>(mapA, mapB, a);
+        return bnn_check_launch(ctx);
+    }
     return umma_launch(ctx, mapA, mapB, a, bn);
 }
 

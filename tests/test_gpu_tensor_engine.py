@@ -12,11 +12,13 @@ from util import np_pack_pm1, np_unpack_pm1, padding_is_zero
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module")
-def ctx():
+@pytest.fixture(scope="module", params=[2, 1], ids=["pairs", "single"])
+def ctx(request):
+    """Tensor engine forced; with CTA pairs (cta_group::2) wherever the kernel allows, and with the single-SM kernel only."""
     build.build()
     c = binding.Context(0)
     c.set_engine(binding.ENGINE_TENSOR)
+    c.set_pair_mode(request.param)
     yield c
     torch.cuda.synchronize()
     c.close()
@@ -34,7 +36,7 @@ def with_ws(ctx, nbytes):
 
 
 @pytest.mark.parametrize("M,N,K", [(1000, 1100, 1000), (300, 4096, 1024), (512, 640, 4100), (257, 129, 32768),
-                                   (2048, 2048, 2048)])
+                                   (2048, 2048, 2048), (1111, 512, 2100), (513, 300, 7000), (3000, 1024, 400)])
 def test_xnor_gemm_tensor_engine(ctx, M, N, K):
     A, B = wl.gemm_case(M, N, K, seed=M + N + K)
     Ap = ctx.pack_signs(dev(A, torch.int8))
