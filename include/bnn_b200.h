@@ -88,6 +88,13 @@ BNN_API size_t bnn_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
 /* The same for bnn_binary_conv2d (0 if the tensor-core engine does not apply: a binary input needs
  * C_in % 128 == 0 and a width that divides 128; 9 * C_in <= 32 means the 8-bit first layer). */
 BNN_API size_t bnn_conv_workspace_bytes(int64_t B, int64_t H, int64_t W, int64_t C_in, int64_t C_out, int pool);
+/* Packed signs -> one signed byte per value (+1 -> 0x01, -1 -> 0xff), the operand format of the tensor-core engine.
+ *   src packed rows x K (ld_w words); dst rows x bnn_expanded_ld(K) bytes, bytes at positions >= K written as 0;
+ *   dst must be 16-byte aligned and hold bnn_expanded_bytes(rows, K).  Weights can be expanded once and handed to
+ *   bnn_mlp_forward through bnn_layer_desc.W8. */
+BNN_API int64_t bnn_expanded_ld(int64_t K);
+BNN_API size_t bnn_expanded_bytes(int64_t rows, int64_t K);
+BNN_API int bnn_expand_signs(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t rows, int64_t K, int8_t *dst);
 /* Synchronises the context's stream and returns BNN_ERR_DEVICE_STATUS if a kernel gave up on one of its
  * bounded waits since the last call (its outputs are then undefined), BNN_OK otherwise. */
 BNN_API int bnn_device_status(bnn_ctx *ctx);
@@ -166,6 +173,8 @@ typedef struct {
     const uint32_t *flip; /* hidden layers: packed 1 x N or NULL (device) */
     const float *gamma, *beta, *mean, *var; /* output layer only: N floats each (device) */
     double eps;                             /* output layer only */
+    const int8_t *W8; /* optional (device, may be NULL): the same weights as written by bnn_expand_signs, used by the
+                         tensor-core engine; when NULL that engine expands Wp into the workspace on every call */
 } bnn_layer_desc;
 
 typedef struct {

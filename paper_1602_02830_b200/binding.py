@@ -25,14 +25,15 @@ EXPORTS = (
     "bnn_set_popc_variant", "bnn_pack_signs", "bnn_xnor_gemm", "bnn_binary_dense", "bnn_first_layer_bitplanes",
     "bnn_binary_conv2d", "bnn_mlp_workspace_bytes", "bnn_mlp_forward", "bnn_mlp_forward_host",
     "bnn_fold_batchnorm", "bnn_mlp_noalloc_max_bytes", "bnn_mlp_forward_noalloc", "bnn_set_engine",
-    "bnn_gemm_workspace_bytes", "bnn_device_status", "bnn_conv_workspace_bytes", "bnn_set_tile_rows", "bnn_set_pair_mode",
+    "bnn_gemm_workspace_bytes", "bnn_device_status", "bnn_conv_workspace_bytes", "bnn_set_tile_rows", "bnn_set_pair_mode", "bnn_expanded_ld",
+    "bnn_expanded_bytes", "bnn_expand_signs",
 )
 
 
 class LayerDesc(Structure):
     _fields_ = [("Wp", c_void_p), ("ldw_w", c_int64), ("K", c_int64), ("N", c_int64), ("thr", c_void_p),
                 ("flip", c_void_p), ("gamma", c_void_p), ("beta", c_void_p), ("mean", c_void_p), ("var", c_void_p),
-                ("eps", c_double)]
+                ("eps", c_double), ("W8", c_void_p)]
 
 
 class MlpDesc(Structure):
@@ -71,6 +72,11 @@ def lib() -> ctypes.CDLL:
         L.bnn_set_engine.argtypes = [vp, c_int]
         L.bnn_set_tile_rows.argtypes = [vp, c_int]
         L.bnn_set_pair_mode.argtypes = [vp, c_int]
+        L.bnn_expanded_ld.argtypes = [i64]
+        L.bnn_expanded_ld.restype = i64
+        L.bnn_expanded_bytes.argtypes = [i64, i64]
+        L.bnn_expanded_bytes.restype = c_size_t
+        L.bnn_expand_signs.argtypes = [vp, vp, i64, i64, i64, vp]
         L.bnn_gemm_workspace_bytes.argtypes = [i64, i64, i64]
         L.bnn_gemm_workspace_bytes.restype = c_size_t
         L.bnn_device_status.argtypes = [vp]
@@ -149,6 +155,13 @@ class Context:
             self._ck(lib().bnn_set_workspace(self._h, None, 0), "bnn_set_workspace")
         else:
             self._ck(lib().bnn_set_workspace(self._h, _ptr(ws), ws.numel() * ws.element_size()), "bnn_set_workspace")
+
+    def expand_signs(self, packed, rows: int, K: int):
+        """bnn_expand_signs: packed rows x K -> int8 tensor [rows, bnn_expanded_ld(K)] of +1 / -1 (0 beyond K)."""
+        ld = int(lib().bnn_expanded_ld(K))
+        dst = self.empty(rows, ld, dtype=torch.int8)
+        self._ck(lib().bnn_expand_signs(self._h, _ptr(packed), packed.stride(0), rows, K, _ptr(dst)), "bnn_expand_signs")
+        return dst
 
     def set_pair_mode(self, mode: int):
         self._ck(lib().bnn_set_pair_mode(self._h, mode), "bnn_set_pair_mode")
@@ -232,7 +245,7 @@ class Context:
             d.Wp = L["Wp"].data_ptr()
             d.ldw_w = L["Wp"].stride(0)
             d.K, d.N = L["K"], L["N"]
-            for name in ("thr", "flip", "gamma", "beta", "mean", "var"):
+            for name in ("thr", "flip", "gamma", "beta", "mean", "var", "W8"):
                 t = L.get(name)
                 setattr(d, name, t.data_ptr() if t is not None else None)
             d.eps = float(L.get("eps", 0.0))

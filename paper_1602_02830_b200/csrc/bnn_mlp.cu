@@ -13,6 +13,7 @@ int check_desc(const bnn_mlp_desc *m) {
     for (int k = 0; k < m->n_layers; ++k) {
         const bnn_layer_desc &L = m->layers[k];
         if (L.K <= 0 || L.N <= 0 || !L.Wp) return BNN_ERR_INVALID_ARG;
+        if (L.W8 && !bnn_aligned16(L.W8)) return BNN_ERR_ALIGNMENT;
         if (k > 0 && L.K != m->layers[k - 1].N) return BNN_ERR_INVALID_ARG;
         if (k < m->n_layers - 1) {
             if (!L.thr) return BNN_ERR_INVALID_ARG;
@@ -93,14 +94,18 @@ int forward_device_tensor(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X,
         uint32_t *dst = bits[k & 1];
         int8_t *dst8 = act8[k & 1];
         const int64_t ldo = act_ld(D.N);
-        if (int st = bnn_umma_expand(ctx, D.Wp, D.ldw_w, D.N, D.K, W8)) return st;
+        const int8_t *Wk8 = D.W8;                      // expanded once by the caller, or here on every call
+        if (!Wk8) {
+            if (int st = bnn_umma_expand(ctx, D.Wp, D.ldw_w, D.N, D.K, W8)) return st;
+            Wk8 = W8;
+        }
         const bool need8 = (k < L - 2);
         int st;
         if (k == 0)
-            st = bnn_umma_gemm(ctx, X, ldx, true, W8, bnn_umma_operand_ld(D.K), batch, D.N, D.K, nullptr, 0, D.thr, D.flip, dst,
+            st = bnn_umma_gemm(ctx, X, ldx, true, Wk8, bnn_umma_operand_ld(D.K), batch, D.N, D.K, nullptr, 0, D.thr, D.flip, dst,
                                ldo, need8 ? dst8 : nullptr, bnn_umma_operand_ld(D.N));
         else
-            st = bnn_umma_gemm(ctx, cur8, bnn_umma_operand_ld(D.K), false, W8, bnn_umma_operand_ld(D.K), batch, D.N, D.K, nullptr,
+            st = bnn_umma_gemm(ctx, cur8, bnn_umma_operand_ld(D.K), false, Wk8, bnn_umma_operand_ld(D.K), batch, D.N, D.K, nullptr,
                                0, D.thr, D.flip, dst, ldo, need8 ? dst8 : nullptr, bnn_umma_operand_ld(D.N));
         if (st) return st;
         if (hidden_out && hidden_out[k])

@@ -777,6 +777,18 @@ int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B,
     return umma_launch(ctx, mapA, mapB, a, bn);
 }
 
+extern "C" int64_t bnn_expanded_ld(int64_t K) { return K > 0 ? bnn_umma_operand_ld(K) : 0; }
+extern "C" size_t bnn_expanded_bytes(int64_t rows, int64_t K) { return (rows > 0 && K > 0) ? bnn_umma_operand_bytes(rows, K) : 0; }
+extern "C" int bnn_expand_signs(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t rows, int64_t K, int8_t *dst) {
+    if (!ctx || rows < 0 || K < 0) return BNN_ERR_INVALID_ARG;
+    if (rows == 0 || K == 0) return BNN_OK;
+    if (!src || !dst || ld_w < bnn_words(K)) return BNN_ERR_INVALID_ARG;
+    if (!bnn_aligned16(dst)) return BNN_ERR_ALIGNMENT;
+    bnn_device_guard guard(ctx);
+    if (!guard.ok) return BNN_ERR_CUDA;
+    return bnn_umma_expand(ctx, src, ld_w, rows, K, dst);
+}
+
 // Reads (and clears) the error word the tensor-core kernel sets when one of its bounded waits gives up.
 // Synchronises the context's stream.
 extern "C" int bnn_device_status(bnn_ctx *ctx) {

@@ -27,8 +27,10 @@ def fold(ctx, bn: dict, x_max: int):
     return thr.to(f"cuda:{ctx.device}"), flip.to(f"cuda:{ctx.device}")
 
 
-def prepare_mlp(ctx, weights, bns):
-    """Algorithm 4's inputs (binary weights W^b and BatchNorm parameters theta) -> device layer list."""
+def prepare_mlp(ctx, weights, bns, expand_weights: bool = True):
+    """Algorithm 4's inputs (binary weights W^b and BatchNorm parameters theta) -> device layer list.
+    With expand_weights the hidden layers' weights are also stored as +-1 bytes (bnn_expand_signs) once, so the
+    tensor-core engine does not have to expand them on every forward call."""
     layers = []
     L = len(weights)
     for k, (W, bn) in enumerate(zip(weights, bns)):
@@ -36,6 +38,8 @@ def prepare_mlp(ctx, weights, bns):
         d = {"Wp": pack_weight(ctx, W), "K": K, "N": N}
         if k < L - 1:
             d["thr"], d["flip"] = fold(ctx, bn, 255 * K if k == 0 else K)
+            if expand_weights:
+                d["W8"] = ctx.expand_signs(d["Wp"], N, K)
         else:
             for name in ("gamma", "beta", "mean", "var"):
                 d[name] = _dev(ctx, bn[name], torch.float32)

@@ -109,12 +109,20 @@ def test_first_layer_tensor_engine(ctx, M, N, K):
     del ws
 
 
+def test_expand_signs(ctx):
+    x = wl.pm1(np.random.default_rng(3), (37, 300))
+    p = ctx.pack_signs(dev(x, torch.int8))
+    e = ctx.expand_signs(p, 37, 300).cpu().numpy()
+    assert e.shape == (37, 384) and np.array_equal(e[:, :300], x) and not e[:, 300:].any()
+
+
+@pytest.mark.parametrize("pre_expanded", [True, False])
 @pytest.mark.parametrize("host_io", [False, True])
-def test_mlp_forward_tensor_engine(ctx, host_io):
+def test_mlp_forward_tensor_engine(ctx, host_io, pre_expanded):
     batch, sizes = 2000, (784, 1024, 1100, 1024, 10)
     case = wl.mlp_case(batch=batch, sizes=sizes, seed=77)
     want_scores, want_hidden = oracle.mlp_forward(case["X"], case["weights"], case["bns"])
-    net = nets.prepare_mlp(ctx, case["weights"], case["bns"])
+    net = nets.prepare_mlp(ctx, case["weights"], case["bns"], expand_weights=pre_expanded)
     ws = with_ws(ctx, ctx.mlp_workspace_bytes(net["desc"], batch, host_io))
     if host_io:
         Xh = torch.from_numpy(case["X"]).pin_memory()
