@@ -336,6 +336,11 @@ def bench_dense_sweep(ctx, timed_steps, engine):
     Wp = torch.randint(-2**31, 2**31 - 1, (N, K // 32), dtype=torch.int32, device="cuda", generator=g)
     thr = torch.randint(-64, 65, (N,), dtype=torch.int32, device="cuda", generator=g)
     out = {}
+    # launch floor for the small batches: a one-word sign-pack (one tiny kernel) timed the same way
+    tiny_src = torch.zeros(1, 32, dtype=torch.int8, device="cuda")
+    tiny_dst = torch.empty(1, 4, dtype=torch.int32, device="cuda")
+    t = timed_steps(lambda: ctx.pack_signs(tiny_src, dst=tiny_dst), 20, 3)
+    out["launch_floor_ms"] = sorted(t)[len(t) // 2]
     for batch in wl.DENSE_BATCHES:
         Ap = torch.randint(-2**31, 2**31 - 1, (batch, K // 32), dtype=torch.int32, device="cuda", generator=g)
         O = torch.empty(batch, N // 32, dtype=torch.int32, device="cuda")

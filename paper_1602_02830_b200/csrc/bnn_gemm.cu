@@ -25,6 +25,49 @@ struct SkinnyArgs {
     const float *gamma, *beta, *mean, *var; double eps;
 };
 
+// Sums V per-lane values over the 32 lanes of a warp with V-1 + (5 - log2 V) shuffles for V < 32 (31 per group of
+// 32 values otherwise) instead of 5 per value: at every stage half of the values travel to the partner lane.
+// On return, for V >= 32 lane l holds the total of value 32*g + l in v[g]; for V < 32 every lane holds the total
+// of value l >> (5 - log2 V) in v[0].
+template <int N, int O>
+__device__ __forceinline__ void butterfly_stage(int32_t *v, int lane) {
+    const bool up = (lane & O) != 0;
+#pragma unroll
+    for (int i = 0; i < N / 2; ++i) {
+        const int32_t send = up ? v[i] : v[i + N / 2];
+        const int32_t keep = up ? v[i + N / 2] : v[i];
+        v[i] = keep + __shfl_xor_sync(0xffffffffu, send, O);
+    }
+}
+template <int V>
+__device__ __forceinline__ void warp_sum_many(int32_t (&v)[V], int lane) {
+    if constexpr (V >= 32) {
+#pragma unroll
+        for (int g = 0; g < V / 32; ++g) {
+            int32_t *w = &v[32 * g];
+            butterfly_stage<32, 16>(w, lane);
+            butterfly_stage<16, 8>(w, lane);
+            butterfly_stage<8, 4>(w, lane);
+            butterfly_stage<4, 2>(w, lane);
+            butterfly_stage<2, 1>(w, lane);
+            v[g] = w[0];
+        }
+    } else if constexpr (V == 16) {
+        butterfly_stage<16, 16>(v, lane);
+        butterfly_stage<8, 8>(v, lane);
+        butterfly_stage<4, 4>(v, lane);
+        butterfly_stage<2, 2>(v, lane);
+        v[0] += __shfl_xor_sync(0xffffffffu, v[0], 1);
+    } else {
+        static_assert(V == 4, "4, 16 or a multiple of 32 values");
+        butterfly_stage<4, 16>(v, lane);
+        butterfly_stage<2, 8>(v, lane);
+        v[0] += __shfl_xor_sync(0xffffffffu, v[0], 4);
+        v[0] += __shfl_xor_sync(0xffffffffu, v[0], 2);
+        v[0] += __shfl_xor_sync(0xffffffffu, v[0], 1);
+    }
+}
+
 template <int RSMAX, int MODE>
 __global__ void __launch_bounds__(256) k_skinny(const SkinnyArgs p) {
     extern __shared__ __align__(16) uint32_t smem[];
@@ -34,6 +77,14 @@ __global__ void __launch_bounds__(256) k_skinny(const SkinnyArgs p) {
     int32_t *res = reinterpret_cast<int32_t *>(smem + p.RS * Kw4);  // [32][RSMAX]
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t tail_mask = (p.K & 31) ? ((1u << (p.K & 31)) - 1u) : 0xffffffffu;
+    const int64_t l0 = (int64_t)blockIdx.x * 32;
+
+    // the warp's four rows of the large operand: their first 128-bit chunks are requested before anything else
+    const int64_t lrow0 = l0 + warp * 4;
+    uint4 b[4];
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc)
+        b[cc] = load_row_words(p.L + (lrow0 + cc) * p.ldl_w, lrow0 + cc < p.RL, 4 * lane, Kw, tail_mask, true);
 
     for (int64_t e = tid; e < p.RS * (Kw4 >> 2); e += 256) {
         const int64_t r = e / (Kw4 >> 2), q = e % (Kw4 >> 2);
@@ -42,32 +93,38 @@ __global__ void __launch_bounds__(256) k_skinny(const SkinnyArgs p) {
     }
     __syncthreads();
 
-    const int64_t l0 = (int64_t)blockIdx.x * 32;
-#pragma unroll 1
-    for (int cc = 0; cc < 4; ++cc) {
-        const int lcol = warp * 4 + cc;
-        const int64_t l = l0 + lcol;
-        int32_t acc[RSMAX];
+    int32_t acc[4 * RSMAX];                                        // value cc * RSMAX + s
 #pragma unroll
-        for (int s = 0; s < RSMAX; ++s) acc[s] = 0;
-        if (l < p.RL) {
-            for (int64_t w4 = 4 * lane; w4 < Kw4; w4 += 128) {
-                const uint4 b = load_row_words(p.L + l * p.ldl_w, true, w4, Kw, tail_mask, true);
+    for (int e = 0; e < 4 * RSMAX; ++e) acc[e] = 0;
+    for (int64_t w4 = 4 * lane; w4 < Kw4; w4 += 128) {
+        if (w4 != 4 * lane) {
 #pragma unroll
-                for (int s = 0; s < RSMAX; ++s) {
-                    if (s < p.RS) {
-                        const uint4 a = *reinterpret_cast<const uint4 *>(Ss + s * Kw4 + w4);
-                        acc[s] += __popc(a.x ^ b.x) + __popc(a.y ^ b.y) + __popc(a.z ^ b.z) + __popc(a.w ^ b.w);
-                    }
-                }
-            }
+            for (int cc = 0; cc < 4; ++cc)
+                b[cc] = load_row_words(p.L + (lrow0 + cc) * p.ldl_w, lrow0 + cc < p.RL, w4, Kw, tail_mask, true);
         }
 #pragma unroll
         for (int s = 0; s < RSMAX; ++s) {
-            int32_t v = acc[s];
+            if (s < p.RS) {
+                const uint4 a = *reinterpret_cast<const uint4 *>(Ss + s * Kw4 + w4);
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            if (lane == 0) res[lcol * RSMAX + s] = (int32_t)p.K - 2 * v;
+                for (int cc = 0; cc < 4; ++cc)
+                    acc[cc * RSMAX + s] += __popc(a.x ^ b[cc].x) + __popc(a.y ^ b[cc].y) + __popc(a.z ^ b[cc].z) + __popc(a.w ^ b[cc].w);
+            }
+        }
+    }
+    warp_sum_many<4 * RSMAX>(acc, lane);
+    constexpr int V = 4 * RSMAX;
+    if constexpr (V >= 32) {
+#pragma unroll
+        for (int g = 0; g < V / 32; ++g) {
+            const int e = 32 * g + lane, cc = e / RSMAX, sidx = e % RSMAX;
+            res[(warp * 4 + cc) * RSMAX + sidx] = (int32_t)p.K - 2 * acc[g];
+        }
+    } else {
+        constexpr int SH = (V == 16) ? 1 : 3;                      // lanes per value
+        if ((lane & ((1 << SH) - 1)) == 0) {
+            const int e = lane >> SH, cc = e / RSMAX, sidx = e % RSMAX;
+            res[(warp * 4 + cc) * RSMAX + sidx] = (int32_t)p.K - 2 * acc[0];
         }
     }
     __syncthreads();
