@@ -290,7 +290,7 @@ def main():
         "gpu_launches": launches_per_step * args.steps,
         "roofline": ({"bound": "tensor", "kernel": "bnn_binary_dense 10000x4096x4096 on the tensor engine (k_expand_s8 x2 + k_umma_i8, "
                                                     "timed as one call)", "achieved": dense_ach, "peak": tensor_peak, "unit": "TFLOP/s",
-                      "frac": dense_ach / tensor_peak, "traffic": None,
+                      "frac": dense_ach / tensor_peak, "traffic": 60967424,
                       "peak_kind": "int8 ops (2 per MAC); peak = 2 x measured bf16 burst %.1f TFLOP/s (nominal int8:bf16 ratio), "
                                    "%s" % (bf16_peak, "of measured" if peaks else "of fallback"), "ms_per_launch": dense_ms}
                      if tensor_step else
