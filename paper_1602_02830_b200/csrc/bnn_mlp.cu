@@ -31,8 +31,19 @@ size_t act_bytes(const bnn_mlp_desc *m, int64_t batch) {
     return round256((size_t)batch * act_ld(widest) * 4);
 }
 
+// Restores the context's engine choice on scope exit.
+struct engine_pin {
+    bnn_ctx *ctx;
+    int saved;
+    engine_pin(bnn_ctx *c, int engine) : ctx(c), saved(c->engine) { c->engine = engine; }
+    ~engine_pin() { ctx->engine = saved; }
+};
+
 int forward_device(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X, int64_t ldx, int64_t batch, float *scores,
                    int64_t lds, uint32_t *const *hidden_out, char *ws) {
+    // The layer calls below must stay on the CUDA-core kernels: the tensor engine would expand operands into the
+    // context's workspace, which may be the very memory `ws` points into.
+    engine_pin pin(ctx, BNN_ENGINE_POPC);
     const size_t ab = act_bytes(m, batch);
     uint32_t *bufs[2] = {reinterpret_cast<uint32_t *>(ws), reinterpret_cast<uint32_t *>(ws + ab)};
     const int L = m->n_layers;

@@ -200,3 +200,24 @@ def test_first_conv_u8_tensor_engine(ctx, B, H, W, Cin, Cout, pool):
     assert padding_is_zero(got, Cout)
     ctx.set_workspace(None)
     del ws
+
+
+def test_mlp_forward_unaligned_input_falls_back_cleanly(ctx):
+    """An input whose rows are not 16-byte aligned cannot be fed to the tensor engine's TMA loads: the forward pass
+    must run on the CUDA-core kernels without touching the activations it keeps in the same workspace."""
+    batch, sizes = 2000, (790, 1024, 1024, 10)          # 790-byte rows: not a multiple of 16
+    case = wl.mlp_case(batch=batch, sizes=sizes, seed=5)
+    want_scores, want_hidden = oracle.mlp_forward(case["X"], case["weights"], case["bns"])
+    net = nets.prepare_mlp(ctx, case["weights"], case["bns"])
+    ws = with_ws(ctx, ctx.mlp_workspace_bytes(net["desc"], batch, False))
+    ctx.set_engine(binding.ENGINE_AUTO)
+    hidden = [torch.empty(batch, binding.packed_ld(n), dtype=torch.int32, device="cuda") for n in sizes[1:-1]]
+    scores = ctx.mlp_forward(net["desc"], dev(case["X"]), batch, hidden_out=hidden)
+    ctx.device_status()
+    ctx.set_engine(binding.ENGINE_TENSOR)
+    for k, (g, w) in enumerate(zip(hidden, want_hidden)):
+        assert np.array_equal(np_unpack_pm1(g.cpu().numpy(), w.shape[1]), w), f"hidden layer {k}"
+    got = scores.cpu().numpy().astype(np.float64)
+    assert (np.abs(got - want_scores) <= 1e-5 * np.abs(want_scores) + 1e-6 * np.abs(want_scores).max()).all()
+    ctx.set_workspace(None)
+    del ws
