@@ -152,7 +152,7 @@ def main():
     ap.add_argument("--pair-mode", type=int, default=0, help="tensor engine CTA pairs (cta_group::2): 0 = for very large outputs, 1 = never, 2 = wherever possible")
     ap.add_argument("--no-extras", action="store_true", help="skip the GEMM / ConvNet side measurements and the CPU baseline")
     ap.add_argument("--gemm-size", type=int, default=8192)
-    ap.add_argument("--section", default="all", choices=["all", "gemm", "convnet", "sweep"],
+    ap.add_argument("--section", default="all", choices=["all", "gemm", "convnet", "sweep", "fig3"],
                     help="side measurements to run after the MLP step (a single one keeps profiler captures small)")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -314,6 +314,8 @@ def main():
             line["convnet"] = bench_convnet(ctx, timed_steps, args.engine)
         if args.section in ("all", "sweep"):
             line["dense_sweep"] = bench_dense_sweep(ctx, timed_steps, args.engine)
+        if args.section in ("all", "fig3"):
+            line["fig3_context"] = bench_fig3(ctx, timed_steps, args.engine, popc_mlp_ms, ms_per_step)
         ctx.set_workspace(ws)
         t0 = time.perf_counter()
         dt, cores = time_oracle_mlp(case, BATCH, repeats=4 if args.section == "all" else 1)
@@ -325,6 +327,52 @@ def main():
     print(json.dumps(line))
     replicas.finish()
     return 0
+
+
+def bench_fig3(ctx, timed_steps, engine, popc_mlp_ms, mlp_ms):
+    """The paper's Fig. 3 on this GPU (context, not a target): 8192^3 product of +-1 matrices with (a) a deliberately
+    unoptimized float32 kernel, (b) the XNOR-popcount kernel, (c) cuBLAS via torch.matmul; and the MLP with the
+    unoptimized kernel in place of the binary one.  The paper reports XNOR 23x faster than its baseline kernel and
+    3.4x faster than cuBLAS, and the MLP 7x faster, on a GTX750."""
+    import torch
+    n = 8192
+    g = torch.Generator(device="cuda").manual_seed(2)
+    A = (torch.randint(0, 2, (n, n), device="cuda", generator=g, dtype=torch.int8) * 2 - 1)
+    B = (torch.randint(0, 2, (n, n), device="cuda", generator=g, dtype=torch.int8) * 2 - 1)
+    Af, Bf = A.float(), B.float()
+    C = torch.empty(n, n, dtype=torch.float32, device="cuda")
+    base = timed_steps(lambda: ctx.baseline_gemm_f32(Af, Bf, C), 2, 1)
+    base_ms = min(base)
+    torch.backends.cuda.matmul.allow_tf32 = False
+    cublas_f32 = min(timed_steps(lambda: torch.matmul(Af, Bf, out=C), 3, 2))
+    Ab, Bb = A.to(torch.bfloat16), B.to(torch.bfloat16)
+    Cb = torch.empty(n, n, dtype=torch.bfloat16, device="cuda")
+    cublas_bf16 = min(timed_steps(lambda: torch.matmul(Ab, Bb, out=Cb), 5, 3))
+    try:
+        cublas_i8 = min(timed_steps(lambda: torch._int_mm(A, B), 5, 3))
+    except Exception:  # pragma: no cover - library support varies
+        cublas_i8 = None
+    Ap = ctx.pack_signs(A)
+    Bp = ctx.pack_signs(B, pack_along=1)
+    Ci = torch.empty(n, n, dtype=torch.int32, device="cuda")
+    ctx.set_engine(1)
+    xnor_ms = min(timed_steps(lambda: ctx.xnor_gemm(Ap, Bp, n, n, n, C=Ci), 5, 3))
+    ctx.set_engine(engine)
+    assert torch.equal(Ci.float(), torch.matmul(Af, Bf)), "XNOR kernel and float product differ"   # fp32 is exact here
+    del Ab, Bb, Cb, Ci
+    # MLP with the unoptimized float kernel standing in for every layer's product (batch 10000, same shapes)
+    mlp_base = 0.0
+    for K, N in zip(SIZES[:-1], SIZES[1:]):
+        X = torch.ones(BATCH, K, dtype=torch.float32, device="cuda")
+        W = torch.ones(K, N, dtype=torch.float32, device="cuda")
+        O = torch.empty(BATCH, N, dtype=torch.float32, device="cuda")
+        mlp_base += min(timed_steps(lambda: ctx.baseline_gemm_f32(X, W, O), 2, 1))
+    return {"shape": [n, n, n], "baseline_f32_ms": base_ms, "xnor_popc_ms": xnor_ms, "cublas_f32_ms": cublas_f32,
+            "cublas_bf16_ms": cublas_bf16, "cublas_int8_ms": cublas_i8,
+            "xnor_vs_baseline": base_ms / xnor_ms, "xnor_vs_cublas_f32": cublas_f32 / xnor_ms,
+            "mlp_baseline_kernel_ms": mlp_base, "mlp_xnor_vs_baseline": mlp_base / popc_mlp_ms,
+            "mlp_selected_engine_vs_baseline": mlp_base / mlp_ms,
+            "paper_gtx750": {"xnor_vs_baseline": 23, "xnor_vs_cublas": 3.4, "mlp_xnor_vs_baseline": 7}}
 
 
 def bench_dense_sweep(ctx, timed_steps, engine):

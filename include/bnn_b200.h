@@ -196,6 +196,13 @@ BNN_API int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint
                          int64_t batch, float *scores_host, int64_t lds);
 
 /* ---------------------------------------------------------------------------------------------
+ * Context only (Section 4, Fig. 3): the paper's comparison point, a deliberately unoptimized matrix product of the
+ * +-1 values held as float32 (one thread per output).  A is M x K, B is K x N, C is M x N, all row-major device
+ * float32.  Not used by any other call. */
+BNN_API int bnn_baseline_gemm_f32(bnn_ctx *ctx, const float *A, const float *B, float *C, int64_t M, int64_t N,
+                                  int64_t K);
+
+/* ---------------------------------------------------------------------------------------------
  * bnn_mlp_forward for callers that cannot allocate device memory.  (The paper has no counterpart: this
  * is a deployment convenience of the library, not a step of the method.)
  *

@@ -26,7 +26,7 @@ EXPORTS = (
     "bnn_binary_conv2d", "bnn_mlp_workspace_bytes", "bnn_mlp_forward", "bnn_mlp_forward_host",
     "bnn_fold_batchnorm", "bnn_mlp_noalloc_max_bytes", "bnn_mlp_forward_noalloc", "bnn_set_engine",
     "bnn_gemm_workspace_bytes", "bnn_device_status", "bnn_conv_workspace_bytes", "bnn_set_tile_rows", "bnn_set_pair_mode", "bnn_expanded_ld",
-    "bnn_expanded_bytes", "bnn_expand_signs",
+    "bnn_expanded_bytes", "bnn_expand_signs", "bnn_baseline_gemm_f32",
 )
 
 
@@ -77,6 +77,7 @@ def lib() -> ctypes.CDLL:
         L.bnn_expanded_bytes.argtypes = [i64, i64]
         L.bnn_expanded_bytes.restype = c_size_t
         L.bnn_expand_signs.argtypes = [vp, vp, i64, i64, i64, vp]
+        L.bnn_baseline_gemm_f32.argtypes = [vp, vp, vp, vp, i64, i64, i64]
         L.bnn_gemm_workspace_bytes.argtypes = [i64, i64, i64]
         L.bnn_gemm_workspace_bytes.restype = c_size_t
         L.bnn_device_status.argtypes = [vp]
@@ -162,6 +163,15 @@ class Context:
         dst = self.empty(rows, ld, dtype=torch.int8)
         self._ck(lib().bnn_expand_signs(self._h, _ptr(packed), packed.stride(0), rows, K, _ptr(dst)), "bnn_expand_signs")
         return dst
+
+    def baseline_gemm_f32(self, A, B, C=None):
+        """bnn_baseline_gemm_f32: the paper's unoptimized float32 comparison kernel (context only)."""
+        M, K = A.shape
+        N = B.shape[1]
+        if C is None:
+            C = self.empty(M, N, dtype=torch.float32)
+        self._ck(lib().bnn_baseline_gemm_f32(self._h, _ptr(A), _ptr(B), _ptr(C), M, N, K), "bnn_baseline_gemm_f32")
+        return C
 
     def set_pair_mode(self, mode: int):
         self._ck(lib().bnn_set_pair_mode(self._h, mode), "bnn_set_pair_mode")
