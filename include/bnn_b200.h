@@ -190,8 +190,11 @@ BNN_API size_t bnn_mlp_workspace_bytes(const bnn_mlp_desc *m, int64_t batch, int
  * are also copied there.  Needs a workspace (BNN_ERR_WORKSPACE otherwise). */
 BNN_API int bnn_mlp_forward(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X, int64_t ldx, int64_t batch,
                     float *scores, int64_t lds, uint32_t *const *hidden_out);
-/* Same with HOST input and output: X_host is copied to the device, scores are copied back, both on the
- * context's stream (pinned host memory makes the copies asynchronous).  The caller synchronises. */
+/* Same with HOST input and output: X_host is copied to the device and the scores are copied back (pinned host
+ * memory makes the copies asynchronous).  For large batches the input travels in row chunks on an internal stream
+ * so that later chunks are copied while earlier ones are already being computed; all of it is ordered after the work
+ * already queued on the context's stream and completes before anything queued on it afterwards, so the caller just
+ * synchronises the context's stream. */
 BNN_API int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X_host, int64_t ldx,
                          int64_t batch, float *scores_host, int64_t lds);
 

@@ -20,6 +20,9 @@ extern "C" int bnn_create(bnn_ctx **out, int device, void *cuda_stream) {
     c->engine = 0;
     c->tile_rows = 8;
     c->pair_mode = 0;
+    c->copy_stream = nullptr;
+    c->copy_ready = false;
+    for (int i = 0; i < 5; ++i) c->ev[i] = nullptr;
     if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
         delete c;
         return BNN_ERR_CUDA;
@@ -30,6 +33,14 @@ extern "C" int bnn_create(bnn_ctx **out, int device, void *cuda_stream) {
 
 extern "C" int bnn_destroy(bnn_ctx *ctx) {
     if (!ctx) return BNN_ERR_INVALID_ARG;
+    if (ctx->copy_ready) {
+        bnn_device_guard guard(ctx);
+        if (guard.ok) {
+            cudaStreamSynchronize(ctx->copy_stream);
+            for (int i = 0; i < 5; ++i) cudaEventDestroy(ctx->ev[i]);
+            cudaStreamDestroy(ctx->copy_stream);
+        }
+    }
     delete ctx;
     return BNN_OK;
 }

@@ -183,14 +183,43 @@ extern "C" int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const u
     const size_t fwd = bnn_mlp_workspace_bytes(m, batch, 0);
     uint8_t *Xd = reinterpret_cast<uint8_t *>(ws + fwd);
     float *Sd = reinterpret_cast<float *>(ws + fwd + round256((size_t)batch * K0));
-    if (ldx == K0)   // contiguous: one linear copy
-        BNN_CUDA_TRY(ctx, cudaMemcpyAsync(Xd, X_host, (size_t)K0 * batch, cudaMemcpyHostToDevice, ctx->stream));
-    else
-        BNN_CUDA_TRY(ctx, cudaMemcpy2DAsync(Xd, (size_t)K0, X_host, (size_t)ldx, (size_t)K0, (size_t)batch,
-                                            cudaMemcpyHostToDevice, ctx->stream));
-    if (int st = tensor ? forward_device_tensor(ctx, m, Xd, K0, batch, Sd, NL, nullptr, ws)
-                        : forward_device(ctx, m, Xd, K0, batch, Sd, NL, nullptr, ws))
-        return st;
+
+    // Row chunks are independent through every layer, so for a large batch on the tensor engine the input is copied
+    // in up to three chunks on an internal stream while the previous chunk is already running through the layers.
+    // Chunk sizes are multiples of 128 rows (whole tiles).
+    int nchunks = 1;
+    int64_t rows_per = batch;
+    if (tensor && batch >= 6144) {
+        nchunks = 3;
+        rows_per = (((batch + nchunks - 1) / nchunks + 127) / 128) * 128;
+        if (!tensor_applies(ctx, m, batch - 2 * rows_per > 0 ? batch - 2 * rows_per : 1)) nchunks = 1, rows_per = batch;
+    }
+    if (nchunks > 1 && !ctx->copy_ready) {
+        BNN_CUDA_TRY(ctx, cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+        for (int i = 0; i < 5; ++i) BNN_CUDA_TRY(ctx, cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming));
+        ctx->copy_ready = true;
+    }
+    cudaStream_t cs = nchunks > 1 ? ctx->copy_stream : ctx->stream;
+    if (nchunks > 1) {   // the copies may not overtake work that is already queued on the context's stream
+        BNN_CUDA_TRY(ctx, cudaEventRecord(ctx->ev[0], ctx->stream));
+        BNN_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->ev[0], 0));
+    }
+    for (int c = 0; c < nchunks; ++c) {
+        const int64_t r0 = c * rows_per, rows = (r0 + rows_per <= batch) ? rows_per : batch - r0;
+        if (ldx == K0)   // contiguous: one linear copy
+            BNN_CUDA_TRY(ctx, cudaMemcpyAsync(Xd + r0 * K0, X_host + r0 * ldx, (size_t)K0 * rows, cudaMemcpyHostToDevice, cs));
+        else
+            BNN_CUDA_TRY(ctx, cudaMemcpy2DAsync(Xd + r0 * K0, (size_t)K0, X_host + r0 * ldx, (size_t)ldx, (size_t)K0, (size_t)rows,
+                                                cudaMemcpyHostToDevice, cs));
+        if (nchunks > 1) BNN_CUDA_TRY(ctx, cudaEventRecord(ctx->ev[1 + c], cs));
+    }
+    for (int c = 0; c < nchunks; ++c) {
+        const int64_t r0 = c * rows_per, rows = (r0 + rows_per <= batch) ? rows_per : batch - r0;
+        if (nchunks > 1) BNN_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev[1 + c], 0));
+        if (int st = tensor ? forward_device_tensor(ctx, m, Xd + r0 * K0, K0, rows, Sd + r0 * NL, NL, nullptr, ws)
+                            : forward_device(ctx, m, Xd + r0 * K0, K0, rows, Sd + r0 * NL, NL, nullptr, ws))
+            return st;
+    }
     if (lds == NL)
         BNN_CUDA_TRY(ctx, cudaMemcpyAsync(scores_host, Sd, (size_t)NL * 4 * batch, cudaMemcpyDeviceToHost, ctx->stream));
     else
