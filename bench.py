@@ -447,21 +447,23 @@ def bench_gemm(ctx, n, peak, timed_steps, engine):
 
 
 def bench_convnet(ctx, timed_steps, engine):
-    """CIFAR-shaped ConvNet forward, batch 256: images/s."""
+    """CIFAR-shaped ConvNet forward, batch 256, through bnn_convnet_forward: images/s on both engines."""
     import torch
     from paper_1602_02830_b200 import nets, workloads as wl
     case = wl.convnet_case()
+    B, hw = case["batch"], case["hw"]
     net = nets.prepare_convnet(ctx, case["layers"])
+    desc, keep = ctx.make_convnet_desc(net)
     X = torch.from_numpy(case["X"]).cuda()
-    cws = torch.empty(max(nets.convnet_workspace_bytes(ctx, net, case["batch"], case["hw"], case["hw"]), 256),
-                      dtype=torch.uint8, device="cuda")
+    cws = torch.empty(max(ctx.convnet_workspace_bytes(desc, B, hw, hw), 256), dtype=torch.uint8, device="cuda")
     ctx.set_workspace(cws)
-    out = {"batch": case["batch"]}
+    final = torch.empty(nets.convnet_output_shape(net, B, hw, hw), dtype=torch.int32, device="cuda")
+    out = {"batch": B}
     for name, eng in (("popc", 1), ("selected_engine", engine)):
         ctx.set_engine(eng)
-        t = timed_steps(lambda: nets.convnet_forward(ctx, net, X), 10, 3)
+        t = timed_steps(lambda: ctx.convnet_forward(desc, X, B, hw, hw, final), 20, 3)
         ms = sum(t) / len(t)
-        out[name] = {"ms": ms, "images_per_s": case["batch"] / (ms / 1e3)}
+        out[name] = {"ms": ms, "images_per_s": B / (ms / 1e3)}
     ctx.set_engine(engine)
     return out
 

@@ -161,6 +161,33 @@ BNN_API int bnn_binary_conv2d(bnn_ctx *ctx, const uint32_t *act, const uint8_t *
                       const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, int32_t *out_sums);
 
 /* ---------------------------------------------------------------------------------------------
+ * Whole ConvNet forward: a stack of 3x3 / pad-1 layers, each  conv -> optional 2x2 max-pool -> threshold -> Sign
+ * (Algorithm 4 with convolutions in place of the dense products, Section 3.3).  Layer 0 takes the 8-bit image
+ * (9 * C_in <= 32, bit-plane layer of Section 1.6); every other layer takes the previous layer's binary map.
+ * The activations stay on the device between layers (packed, plus one byte per value for the tensor-core engine).
+ */
+typedef struct {
+    const uint32_t *Wp;   /* as for bnn_binary_conv2d (device) */
+    int64_t C_in, C_out;
+    int32_t pool;         /* 0 or 1 */
+    const int32_t *thr;   /* C_out thresholds (device) */
+    const uint32_t *flip; /* packed 1 x C_out or NULL (device) */
+    const int8_t *W8;     /* optional (device, may be NULL): bnn_expand_signs(Wp viewed as C_out rows of 9*C_in bits) */
+} bnn_conv_layer_desc;
+
+typedef struct {
+    int32_t n_layers;
+    const bnn_conv_layer_desc *layers; /* host array */
+} bnn_convnet_desc;
+
+BNN_API size_t bnn_convnet_workspace_bytes(const bnn_convnet_desc *net, int64_t B, int64_t H, int64_t W);
+/* X: [B][H][W][C_in of layer 0] bytes (device).  out_bits: the last layer's packed map [B][Ho][Wo][ceil(C_out/32)].
+ * layer_out: NULL, or a host array of n_layers device pointers (entries may be NULL) that receive every layer's packed
+ * map.  Needs a workspace of bnn_convnet_workspace_bytes (BNN_ERR_WORKSPACE otherwise). */
+BNN_API int bnn_convnet_forward(bnn_ctx *ctx, const bnn_convnet_desc *net, const uint8_t *X, int64_t B, int64_t H, int64_t W,
+                                uint32_t *out_bits, uint32_t *const *layer_out);
+
+/* ---------------------------------------------------------------------------------------------
  * Whole MLP forward (Algorithm 4): first layer on 8-bit inputs, hidden binary layers, real-valued
  * output layer  score = gamma * ((dot - mean) / sqrt(var + eps)) + beta  (evaluated in double,
  * stored as float32).

@@ -26,7 +26,8 @@ EXPORTS = (
     "bnn_binary_conv2d", "bnn_mlp_workspace_bytes", "bnn_mlp_forward", "bnn_mlp_forward_host",
     "bnn_fold_batchnorm", "bnn_mlp_noalloc_max_bytes", "bnn_mlp_forward_noalloc", "bnn_set_engine",
     "bnn_gemm_workspace_bytes", "bnn_device_status", "bnn_conv_workspace_bytes", "bnn_set_tile_rows", "bnn_set_pair_mode", "bnn_expanded_ld",
-    "bnn_expanded_bytes", "bnn_expand_signs", "bnn_baseline_gemm_f32",
+    "bnn_expanded_bytes", "bnn_expand_signs", "bnn_baseline_gemm_f32", "bnn_convnet_workspace_bytes",
+    "bnn_convnet_forward",
 )
 
 
@@ -38,6 +39,15 @@ class LayerDesc(Structure):
 
 class MlpDesc(Structure):
     _fields_ = [("n_layers", c_int32), ("layers", POINTER(LayerDesc))]
+
+
+class ConvLayerDesc(Structure):
+    _fields_ = [("Wp", c_void_p), ("C_in", c_int64), ("C_out", c_int64), ("pool", c_int32), ("thr", c_void_p),
+                ("flip", c_void_p), ("W8", c_void_p)]
+
+
+class ConvNetDesc(Structure):
+    _fields_ = [("n_layers", c_int32), ("layers", POINTER(ConvLayerDesc))]
 
 
 class BnnError(RuntimeError):
@@ -78,6 +88,9 @@ def lib() -> ctypes.CDLL:
         L.bnn_expanded_bytes.restype = c_size_t
         L.bnn_expand_signs.argtypes = [vp, vp, i64, i64, i64, vp]
         L.bnn_baseline_gemm_f32.argtypes = [vp, vp, vp, vp, i64, i64, i64]
+        L.bnn_convnet_workspace_bytes.argtypes = [POINTER(ConvNetDesc), i64, i64, i64]
+        L.bnn_convnet_workspace_bytes.restype = c_size_t
+        L.bnn_convnet_forward.argtypes = [vp, POINTER(ConvNetDesc), vp, i64, i64, i64, vp, POINTER(vp)]
         L.bnn_gemm_workspace_bytes.argtypes = [i64, i64, i64]
         L.bnn_gemm_workspace_bytes.restype = c_size_t
         L.bnn_device_status.argtypes = [vp]
@@ -261,6 +274,28 @@ class Context:
             d.eps = float(L.get("eps", 0.0))
         desc = MlpDesc(len(layers), arr)
         return desc, (arr, layers)
+
+    def make_convnet_desc(self, layers):
+        """layers: list of dicts with Wp, Cin, Cout, pool, thr, flip and optionally W8.  Returns (ConvNetDesc, keep-alive)."""
+        arr = (ConvLayerDesc * len(layers))()
+        for d, L in zip(arr, layers):
+            d.Wp = L["Wp"].data_ptr()
+            d.C_in, d.C_out, d.pool = L["Cin"], L["Cout"], int(L["pool"])
+            d.thr = L["thr"].data_ptr()
+            d.flip = L["flip"].data_ptr() if L.get("flip") is not None else None
+            d.W8 = L["W8"].data_ptr() if L.get("W8") is not None else None
+        return ConvNetDesc(len(layers), arr), (arr, layers)
+
+    def convnet_workspace_bytes(self, desc, B: int, H: int, W: int) -> int:
+        return int(lib().bnn_convnet_workspace_bytes(ctypes.byref(desc), B, H, W))
+
+    def convnet_forward(self, desc, X, B: int, H: int, W: int, out_bits, layer_out=None):
+        hp = None
+        if layer_out is not None:
+            hp = (c_void_p * desc.n_layers)(*[t.data_ptr() if t is not None else None for t in layer_out])
+        self._ck(lib().bnn_convnet_forward(self._h, ctypes.byref(desc), _ptr(X), B, H, W, _ptr(out_bits), hp),
+                 "bnn_convnet_forward")
+        return out_bits
 
     def mlp_workspace_bytes(self, desc, batch: int, host_io: bool = False) -> int:
         return int(lib().bnn_mlp_workspace_bytes(ctypes.byref(desc), batch, int(host_io)))

@@ -166,3 +166,137 @@ extern "C" size_t bnn_conv_workspace_bytes(int64_t B, int64_t H, int64_t W, int6
     if (!bnn_umma_conv_tiling(H, W, pool, &TH, &TB) || !bnn_umma_shape_ok(B * H * W, C_out, 9 * C_in)) return 0;
     return bnn_umma_operand_bytes(B * H * W, C_in) + bnn_umma_operand_bytes(C_out, 9 * C_in);
 }
+
+// ---------------------------------------------------------------------------------------------------------
+// bnn_convnet_forward
+namespace {
+
+inline size_t r256(size_t b) { return (b + 255) & ~size_t(255); }
+
+struct ConvPlan {
+    bool chain;            // every layer runs on the tensor engine and hands +-1 bytes to the next one
+    size_t bits_bytes;     // one packed activation buffer (two of them)
+    size_t act8_bytes;     // one byte activation buffer (two of them, chain only)
+    size_t im2col_bytes;   // first layer's 32-byte rows (chain only)
+    size_t w8_bytes;       // scratch for one layer's expanded weights (chain only)
+};
+
+int plan_convnet(const bnn_ctx *ctx, const bnn_convnet_desc *net, int64_t B, int64_t H, int64_t W, ConvPlan *plan) {
+    if (!net || net->n_layers < 1 || !net->layers || B <= 0 || H <= 0 || W <= 0) return BNN_ERR_INVALID_ARG;
+    ConvPlan p{};
+    p.chain = !ctx || ctx->engine != BNN_ENGINE_POPC;
+    int64_t h = H, w = W;
+    for (int k = 0; k < net->n_layers; ++k) {
+        const bnn_conv_layer_desc &L = net->layers[k];
+        if (L.C_in <= 0 || L.C_out <= 0 || !L.Wp || !L.thr || (L.pool != 0 && L.pool != 1)) return BNN_ERR_INVALID_ARG;
+        if (k == 0 ? (9 * L.C_in > 32) : (L.C_in != net->layers[k - 1].C_out || (L.C_in % 32) != 0)) return BNN_ERR_INVALID_ARG;
+        if (L.pool && ((h & 1) || (w & 1))) return BNN_ERR_INVALID_ARG;
+        int TH, TB;
+        const bool tiling = bnn_umma_conv_tiling(h, w, L.pool, &TH, &TB);
+        if (k == 0) {
+            if (!tiling || !bnn_umma_first_conv_ok(B * h * w, L.C_out)) p.chain = false;
+            p.im2col_bytes = r256((size_t)B * h * w * 32);
+        } else {
+            if (!tiling || (L.C_in % 128) != 0 || !bnn_umma_shape_ok(B * h * w, L.C_out, 9 * L.C_in)) p.chain = false;
+        }
+        if (k < net->n_layers - 1 && (L.C_out % 128) != 0) p.chain = false;      // the next layer reads these bytes with TMA
+        const size_t w8 = bnn_umma_operand_bytes(L.C_out, 9 * L.C_in);
+        p.w8_bytes = w8 > p.w8_bytes ? w8 : p.w8_bytes;
+        const int64_t ho = L.pool ? h / 2 : h, wo = L.pool ? w / 2 : w;
+        const size_t bits = r256((size_t)B * ho * wo * ((L.C_out + 31) / 32) * 4);
+        const size_t a8 = r256((size_t)B * ho * wo * L.C_out);
+        p.bits_bytes = bits > p.bits_bytes ? bits : p.bits_bytes;
+        p.act8_bytes = a8 > p.act8_bytes ? a8 : p.act8_bytes;
+        h = ho; w = wo;
+    }
+    *plan = p;
+    return BNN_OK;
+}
+
+size_t plan_bytes(const ConvPlan &p) {
+    // sized for the tensor engine whenever the shapes allow it, whatever engine is selected later
+    return 2 * p.bits_bytes + (p.chain ? 2 * p.act8_bytes + p.im2col_bytes + p.w8_bytes : 0);
+}
+
+}  // namespace
+
+extern "C" size_t bnn_convnet_workspace_bytes(const bnn_convnet_desc *net, int64_t B, int64_t H, int64_t W) {
+    ConvPlan p;
+    if (plan_convnet(nullptr, net, B, H, W, &p) != BNN_OK) return 0;
+    return plan_bytes(p);
+}
+
+extern "C" int bnn_convnet_forward(bnn_ctx *ctx, const bnn_convnet_desc *net, const uint8_t *X, int64_t B, int64_t H, int64_t W,
+                                   uint32_t *out_bits, uint32_t *const *layer_out) {
+    if (!ctx || B < 0 || H < 0 || W < 0) return BNN_ERR_INVALID_ARG;
+    if (B == 0 || H == 0 || W == 0) return (net && net->n_layers >= 1 && net->layers) ? BNN_OK : BNN_ERR_INVALID_ARG;
+    ConvPlan full, plan;
+    if (int st = plan_convnet(nullptr, net, B, H, W, &full)) return st;
+    if (int st = plan_convnet(ctx, net, B, H, W, &plan)) return st;
+    if (!X || !out_bits) return BNN_ERR_INVALID_ARG;
+    if (!ctx->ws || ctx->ws_bytes < plan_bytes(full)) return BNN_ERR_WORKSPACE;
+    if (ctx->engine == BNN_ENGINE_TENSOR && !plan.chain) return BNN_ERR_INVALID_ARG;   // forced engine, unsuitable shapes
+    bnn_device_guard guard(ctx);
+    if (!guard.ok) return BNN_ERR_CUDA;
+
+    char *ws = static_cast<char *>(ctx->ws);
+    uint32_t *bits[2] = {reinterpret_cast<uint32_t *>(ws), reinterpret_cast<uint32_t *>(ws + full.bits_bytes)};
+    int8_t *act8[2] = {reinterpret_cast<int8_t *>(ws + 2 * full.bits_bytes),
+                       reinterpret_cast<int8_t *>(ws + 2 * full.bits_bytes + full.act8_bytes)};
+    uint8_t *im2col = reinterpret_cast<uint8_t *>(ws + 2 * full.bits_bytes + 2 * full.act8_bytes);
+    int8_t *w8_scratch = reinterpret_cast<int8_t *>(ws + 2 * full.bits_bytes + 2 * full.act8_bytes + full.im2col_bytes);
+    const int L = net->n_layers;
+    int64_t h = H, w = W;
+
+    if (!plan.chain) {
+        // one bnn_binary_conv2d per layer on the CUDA-core kernels (they must not expand into the workspace the
+        // activations live in, so the engine is pinned for the duration)
+        const int saved = ctx->engine;
+        ctx->engine = BNN_ENGINE_POPC;
+        int st = BNN_OK;
+        const uint32_t *cur = nullptr;
+        for (int k = 0; k < L && st == BNN_OK; ++k) {
+            const bnn_conv_layer_desc &D = net->layers[k];
+            uint32_t *dst = (k == L - 1) ? out_bits : bits[k & 1];
+            st = bnn_binary_conv2d(ctx, k == 0 ? nullptr : cur, k == 0 ? X : nullptr, B, h, w, D.C_in, D.Wp, D.C_out, D.pool,
+                                   D.thr, D.flip, dst, nullptr);
+            if (D.pool) { h /= 2; w /= 2; }
+            if (st == BNN_OK && layer_out && layer_out[k] && layer_out[k] != dst) {
+                cudaError_t e = cudaMemcpyAsync(layer_out[k], dst, (size_t)B * h * w * ((D.C_out + 31) / 32) * 4,
+                                                cudaMemcpyDeviceToDevice, ctx->stream);
+                if (e != cudaSuccess) { ctx->last_cuda_error = (int)e; st = BNN_ERR_CUDA; }
+            }
+            cur = dst;
+        }
+        ctx->engine = saved;
+        return st;
+    }
+
+    const int8_t *cur8 = nullptr;
+    for (int k = 0; k < L; ++k) {
+        const bnn_conv_layer_desc &D = net->layers[k];
+        uint32_t *dst = (k == L - 1) ? out_bits : bits[k & 1];
+        int8_t *dst8 = (k < L - 1) ? act8[k & 1] : nullptr;
+        const int8_t *W8 = D.W8;
+        if (!W8) {
+            // first layer: one word per filter; others: C_out rows of 9 * C_in bits
+            if (int st = bnn_umma_expand(ctx, D.Wp, k == 0 ? 1 : 9 * (D.C_in / 32), D.C_out, 9 * D.C_in, w8_scratch)) return st;
+            W8 = w8_scratch;
+        }
+        int st;
+        if (k == 0) {
+            if ((st = bnn_umma_im2col_u8(ctx, X, B, h, w, D.C_in, im2col))) return st;
+            st = bnn_umma_gemm(ctx, im2col, 32, true, W8, bnn_umma_operand_ld(9 * D.C_in), B * h * w, D.C_out, 9 * D.C_in, nullptr, 0,
+                               D.thr, D.flip, dst, (D.C_out + 31) / 32, dst8, D.C_out, D.pool, h, w);
+        } else {
+            st = bnn_umma_conv(ctx, cur8, W8, B, h, w, D.C_in, D.C_out, D.pool, D.thr, D.flip, dst, nullptr, dst8, D.C_out);
+        }
+        if (st) return st;
+        if (D.pool) { h /= 2; w /= 2; }
+        if (layer_out && layer_out[k] && layer_out[k] != dst)
+            BNN_CUDA_TRY(ctx, cudaMemcpyAsync(layer_out[k], dst, (size_t)B * h * w * ((D.C_out + 31) / 32) * 4,
+                                              cudaMemcpyDeviceToDevice, ctx->stream));
+        cur8 = dst8;
+    }
+    return BNN_OK;
+}

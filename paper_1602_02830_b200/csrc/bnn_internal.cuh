@@ -30,4 +30,5 @@ static inline bool bnn_umma_shape_ok(int64_t M, int64_t N, int64_t K) {
 }
 bool bnn_umma_conv_tiling(int64_t H, int64_t W, int pool, int *TH, int *TB);
 int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B, int64_t H, int64_t W, int64_t C_in,
-                  int64_t C_out, int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, int32_t *out_sums);
+                  int64_t C_out, int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, int32_t *out_sums,
+                  int8_t *out8 = nullptr, int64_t ldo8 = 0);

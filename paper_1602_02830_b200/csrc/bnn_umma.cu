@@ -210,7 +210,7 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                     if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;      // columns beyond N stay 0
                     if (p.pool) ctl->poolw[32 * q + lane][c] = word ^ ctl->flip[buf][c];   // un-flipped (dot >= thr) bits
                     else p.out[row * p.ldo + (col0 >> 5)] = word;
-                    if (p.out8) {
+                    if (p.out8 && !p.pool) {
                         int8_t *d8 = p.out8 + row * p.ldo8 + col0;
                         uint32_t b[8];
 #pragma unroll
@@ -262,6 +262,23 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                 p.out[opix * p.ldo + (col0 >> 5)] = word;
                 if (n0 + BN >= p.N && c == nwords - 1)
                     for (int64_t w = (p.N + 31) >> 5; w < p.ldo; ++w) p.out[opix * p.ldo + w] = 0u;
+                if (p.out8) {   // the pooled pixel's signs as +-1 bytes for the next layer
+                    int8_t *d8 = p.out8 + opix * p.ldo8 + col0;
+                    if (col0 + 32 <= p.N) {
+                        uint32_t b[8];
+#pragma unroll
+                        for (int g = 0; g < 8; ++g) {
+                            const uint32_t t4 = (((word >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u;
+                            b[g] = ~(t4 * 0xfeu);
+                        }
+                        *reinterpret_cast<uint4 *>(d8) = make_uint4(b[0], b[1], b[2], b[3]);
+                        *reinterpret_cast<uint4 *>(d8 + 16) = make_uint4(b[4], b[5], b[6], b[7]);
+                    } else {
+                        for (int j = 0; j < 32; ++j)
+                            if (col0 + j < p.N) d8[j] = ((word >> j) & 1u) ? (int8_t)1 : (int8_t)-1;
+                            else if (col0 + j < p.ldo8) d8[j] = 0;
+                    }
+                }
             }
         }
     }
@@ -686,7 +703,7 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
     if (M == 0 || N == 0) return BNN_OK;
     if (pool) {   // rows are pixels of H x W images in (b, y, x) order; 128-row tiles must hold whole 2x2 windows
         int TH, TB;
-        if (!bnn_umma_conv_tiling(H, W, 1, &TH, &TB) || C || out8) return BNN_ERR_INVALID_ARG;
+        if (!bnn_umma_conv_tiling(H, W, 1, &TH, &TB) || C) return BNN_ERR_INVALID_ARG;
     }
     if ((lda8 & 15) || (ldb8 & 15) || !bnn_aligned16(A8) || !bnn_aligned16(B8)) return BNN_ERR_ALIGNMENT;
     if (M > 0x7fffffff || N > 0x7fffffff) return BNN_ERR_INVALID_ARG;
@@ -761,7 +778,8 @@ bool bnn_umma_conv_tiling(int64_t H, int64_t W, int pool, int *TH, int *TB) {
 // 3x3 / pad 1 convolution on the tensor engine.  act8: [B][H][W][C_in] +-1 bytes (C_in % 128 == 0);
 // W8: [C_out][9 * C_in] +-1 bytes.  Outputs as bnn_binary_conv2d (sums only without pooling).
 int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B, int64_t H, int64_t W, int64_t C_in,
-                  int64_t C_out, int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, int32_t *out_sums) {
+                  int64_t C_out, int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, int32_t *out_sums,
+                  int8_t *out8, int64_t ldo8) {
     int TH, TB;
     if (!bnn_umma_conv_tiling(H, W, pool, &TH, &TB) || (C_in % BK) != 0 || (pool && out_sums)) return BNN_ERR_INVALID_ARG;
     CUtensorMap mapA, mapB;
@@ -773,6 +791,7 @@ int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B,
     a.k_iters = (int)(9 * (C_in / BK));
     a.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BM >> 4) << 24);
     a.C = out_sums; a.ldc = C_out; a.out = out_bits; a.ldo = (C_out + 31) / 32; a.thr = thr; a.flip = flip;
+    a.out8 = out8; a.ldo8 = ldo8;
     a.conv = 1; a.H = (int)H; a.W = (int)W; a.TH = TH; a.TB = TB; a.c_chunks = (int)(C_in / BK); a.pool = pool;
     return umma_launch(ctx, mapA, mapB, a, bn);
 }

@@ -49,8 +49,9 @@ def prepare_mlp(ctx, weights, bns, expand_weights: bool = True):
     return {"layers": layers, "desc": desc, "_keep": keep}
 
 
-def prepare_convnet(ctx, layers):
-    """Conv layer list {wgt: Cout x 3 x 3 x Cin, bn, pool} -> packed device weights and folded thresholds."""
+def prepare_convnet(ctx, layers, expand_weights: bool = True):
+    """Conv layer list {wgt: Cout x 3 x 3 x Cin, bn, pool} -> packed device weights and folded thresholds
+    (and, with expand_weights, the weights as +-1 bytes for the tensor-core engine)."""
     out = []
     for i, L in enumerate(layers):
         wgt = L["wgt"]
@@ -63,8 +64,20 @@ def prepare_convnet(ctx, layers):
             Wp = ctx.pack_signs(_dev(ctx, flat, torch.int8), pack_along=0)[:, :9 * Cin // 32].contiguous()
             x_max = 9 * Cin
         thr, flip = fold(ctx, L["bn"], x_max)
-        out.append({"Wp": Wp, "Cin": Cin, "Cout": Cout, "pool": bool(L.get("pool")), "thr": thr, "flip": flip})
+        d = {"Wp": Wp, "Cin": Cin, "Cout": Cout, "pool": bool(L.get("pool")), "thr": thr, "flip": flip}
+        if expand_weights:
+            # the same bits viewed as Cout rows of 9*Cin: re-pack with a legal leading dimension, then expand
+            rows = ctx.pack_signs(_dev(ctx, flat, torch.int8), pack_along=0)
+            d["W8"] = ctx.expand_signs(rows, Cout, 9 * Cin)
+        out.append(d)
     return out
+
+
+def convnet_output_shape(net, B: int, H: int, W: int):
+    for L in net:
+        if L["pool"]:
+            H, W = H // 2, W // 2
+    return (B, H, W, binding.words(net[-1]["Cout"]))
 
 
 def convnet_forward(ctx, net, X_u8: torch.Tensor, keep_all: bool = False):

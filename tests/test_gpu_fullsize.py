@@ -119,6 +119,18 @@ def test_convnet_config_full_batch(ctx):
     for k, (g, w) in enumerate(zip(outs, want)):
         gh = g[torch.from_numpy(pick).cuda()].cpu().numpy()
         assert np.array_equal(np_unpack_pm1(gh, w.shape[-1]), w), f"conv layer {k}"
+    # the whole-network entry point gives the same maps as the per-layer calls
+    desc, keep = ctx.make_convnet_desc(net)
+    ws2 = torch.empty(max(ctx.convnet_workspace_bytes(desc, case["batch"], case["hw"], case["hw"]), 256), dtype=torch.uint8,
+                      device="cuda")
+    ctx.set_workspace(ws2)
+    outs2 = [torch.empty_like(o) for o in outs]
+    final = torch.empty_like(outs[-1])
+    ctx.convnet_forward(desc, Xd, case["batch"], case["hw"], case["hw"], final, layer_out=outs2)
+    ctx.device_status()
+    for k, (a1, a2) in enumerate(zip(outs, outs2)):
+        assert torch.equal(a1, a2), f"bnn_convnet_forward layer {k}"
+    assert torch.equal(final, outs[-1])
     # (b) every image, layer by layer, against torch conv2d on the GPU fed with the library's own previous layer
     B = case["batch"]
     a = Xd.float().permute(0, 3, 1, 2)

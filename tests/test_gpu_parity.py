@@ -289,6 +289,27 @@ def test_convnet_small_layer_by_layer(ctx):
         assert np.array_equal(np_unpack_pm1(host(g), w.shape[-1]), w), f"conv layer {k}"
 
 
+def test_convnet_forward_call_layer_by_layer(ctx):
+    """bnn_convnet_forward on the CUDA-core kernels (shapes too small for the tensor engine): every layer's map."""
+    case = wl.convnet_case(batch=3, hw=8, channels=(128, 96, 256, 64), seed=4)
+    want = oracle.convnet_forward(case["X"], case["layers"])
+    net = nets.prepare_convnet(ctx, case["layers"], expand_weights=False)
+    desc, keep = ctx.make_convnet_desc(net)
+    ws = torch.empty(max(ctx.convnet_workspace_bytes(desc, 3, 8, 8), 256), dtype=torch.uint8, device="cuda")
+    ctx.set_workspace(ws)
+    outs = [torch.empty(w.shape[0], w.shape[1], w.shape[2], binding.words(w.shape[3]), dtype=torch.int32, device="cuda")
+            for w in want]
+    final = torch.empty_like(outs[-1])
+    ctx.convnet_forward(desc, dev(case["X"]), 3, 8, 8, final, layer_out=outs)
+    for k, (g, w) in enumerate(zip(outs, want)):
+        assert np.array_equal(np_unpack_pm1(host(g), w.shape[-1]), w), f"conv layer {k}"
+    assert np.array_equal(host(final), host(outs[-1]))
+    ctx.set_workspace(None)
+    with pytest.raises(binding.BnnError) as e:
+        ctx.convnet_forward(desc, dev(case["X"]), 3, 8, 8, final)
+    assert e.value.status == -3
+
+
 # ------------------------------------------------------------------ bnn_mlp_forward
 def run_mlp(ctx, case, host_io=False):
     net = nets.prepare_mlp(ctx, case["weights"], case["bns"])

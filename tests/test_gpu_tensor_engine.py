@@ -221,3 +221,25 @@ def test_mlp_forward_unaligned_input_falls_back_cleanly(ctx):
     assert (np.abs(got - want_scores) <= 1e-5 * np.abs(want_scores) + 1e-6 * np.abs(want_scores).max()).all()
     ctx.set_workspace(None)
     del ws
+
+
+@pytest.mark.parametrize("pre_expanded", [True, False])
+def test_convnet_forward_chained_on_tensor_engine(ctx, pre_expanded):
+    """bnn_convnet_forward with every layer on the tensor engine: +-1 bytes handed from layer to layer (pooled and not)."""
+    B, hw = 20, 32
+    case = wl.convnet_case(batch=B, hw=hw, channels=(128, 128, 256, 128), seed=9)
+    want = oracle.convnet_forward(case["X"], case["layers"])
+    net = nets.prepare_convnet(ctx, case["layers"], expand_weights=pre_expanded)
+    desc, keep = ctx.make_convnet_desc(net)
+    need = ctx.convnet_workspace_bytes(desc, B, hw, hw)
+    ws = with_ws(ctx, need)
+    outs = [torch.empty(w.shape[0], w.shape[1], w.shape[2], binding.words(w.shape[3]), dtype=torch.int32, device="cuda")
+            for w in want]
+    final = torch.empty_like(outs[-1])
+    ctx.convnet_forward(desc, dev(case["X"]), B, hw, hw, final, layer_out=outs)
+    ctx.device_status()
+    for k, (g, w) in enumerate(zip(outs, want)):
+        assert np.array_equal(np_unpack_pm1(g.cpu().numpy(), w.shape[-1]), w), f"conv layer {k}"
+    assert torch.equal(final, outs[-1])
+    ctx.set_workspace(None)
+    del ws
