@@ -160,17 +160,22 @@ __device__ __forceinline__ void fail(Control *ctl, int code) {
 // buffer `buf`, and turn them into the requested outputs.  `ok` turns false once a wait has given up.
 template <int BN>
 __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, uint32_t tmem_base, uint32_t buf, uint32_t tc,
-                                              int64_t m0, int64_t n0, int q, int half, int lane, int et, bool &ok) {
+                                              int64_t m0, int64_t n0, int q, int half, int lane, int et, bool &ok,
+                                              int64_t (&staged_n0)[ACC_BUFS]) {
     constexpr int CHUNKS = BN / 32, CPW = CHUNKS / 2;   // 32-column chunks per tile and per warp
     const int64_t row = m0 + 32 * q + lane;
-    if (p.out) {
+    // thresholds of this column block; tiles that share it with the buffer's previous tile skip the staging
+    const bool restage = p.out && staged_n0[buf] != n0;
+    if (restage) {
         for (int e = et; e < BN; e += EPI_THREADS) ctl->thr[buf][e] = (n0 + e < p.N) ? p.thr[n0 + e] : 0x7fffffff;
         if (et < BN / 32) {
             const int64_t w = (n0 >> 5) + et;
             ctl->flip[buf][et] = (p.flip && w * 32 < p.N) ? p.flip[w] : 0u;
         }
+        staged_n0[buf] = n0;
     }
-    asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");   // the epilogue warps only
+    // the epilogue warps only: staged thresholds visible; previous tile's pooling words no longer read
+    if (restage || p.pool) asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
     if (ok && !mbar_wait(smem_u32(&ctl->acc_full[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 3); ok = false; }
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     ok = ok && (ctl->failed == 0);
@@ -378,10 +383,11 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
         const int et = threadIdx.x - 64;                 // 0 .. EPI_THREADS-1 among the epilogue threads
         uint32_t tc = 0;
         bool ok = true;
+        int64_t staged_n0[ACC_BUFS] = {-1, -1};
         for (int64_t t = blockIdx.x; t < ntiles; t += gridDim.x, ++tc) {
             const uint32_t buf = tc & 1;
             const int64_t m0 = (t % tiles_m) * BM, n0 = (t / tiles_m) * BN;
-            epilogue_tile<BN>(ctl, p, tmem_base, buf, tc, m0, n0, q, half, lane, et, ok);
+            epilogue_tile<BN>(ctl, p, tmem_base, buf, tc, m0, n0, q, half, lane, et, ok, staged_n0);
             // hand the accumulator buffer back to the MMA warp
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
@@ -523,10 +529,11 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         const int et = threadIdx.x - 64;
         uint32_t tc = 0;
         bool ok = true;
+        int64_t staged_n0[ACC_BUFS] = {-1, -1};
         for (int64_t t = pair; t < ntiles; t += npairs, ++tc) {
             const uint32_t buf = tc & 1;
             const int64_t m0 = (t % tiles_m) * (2 * BM) + rank * BM, n0 = (t / tiles_m) * BN;
-            epilogue_tile<BN>(ctl, p, tmem_base, buf, tc, m0, n0, q, half, lane, et, ok);
+            epilogue_tile<BN>(ctl, p, tmem_base, buf, tc, m0, n0, q, half, lane, et, ok, staged_n0);
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive_cta0(smem_u32(&ctl->acc_empty[buf]));
