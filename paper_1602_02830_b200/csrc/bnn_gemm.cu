@@ -197,7 +197,7 @@ template <int AKIND>
 int launch_tile(bnn_ctx *ctx, const Args &a_in, int variant) {
     Args a = a_in;
     a.one = 1u;
-    const int64_t rows = (AKIND == A_PLANES) ? 8 * a.M : a.M;     // operand rows (8 bit-plane rows per image)
+    const int64_t rows = (AKIND == A_PLANES || AKIND == A_PLANES_PRE) ? 8 * a.M : a.M;   // 8 bit-plane rows per image
     const int64_t tn = (a.N + BN - 1) / BN;
     const int64_t t128 = ((rows + 127) / 128) * tn, t64 = ((rows + 63) / 64) * tn;
     const bool csa = (variant != BNN_VARIANT_PLAIN);
@@ -223,6 +223,68 @@ int launch_tile(bnn_ctx *ctx, const Args &a_in, int variant) {
 int bnn_launch_tile_packed(bnn_ctx *ctx, const Args &a) { return launch_tile<A_PACKED>(ctx, a, ctx_variant(ctx)); }
 int bnn_launch_tile_conv(bnn_ctx *ctx, const Args &a) { return launch_tile<A_CONV>(ctx, a, ctx_variant(ctx)); }
 int bnn_launch_tile_planes(bnn_ctx *ctx, const Args &a) { return launch_tile<A_PLANES>(ctx, a, ctx_variant(ctx)); }
+
+// ------------------------------------------------------------------------------------------------
+// Bit-plane split as a pre-pass (Eq. 7): plane p of image m becomes packed row 8*m + p of `planes`, and the sum of
+// the image's bytes goes to xsum[m].  One warp per image; lane l handles 32-byte groups l, l+32, ...
+namespace {
+__global__ void __launch_bounds__(256) k_split_planes(const uint8_t *__restrict__ X, int64_t ldx, int64_t M, int64_t K,
+                                                      uint32_t *__restrict__ planes, int64_t ld_w, int32_t *__restrict__ xsum) {
+    const int lane = threadIdx.x & 31;
+    const int64_t m = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (m >= M) return;
+    const uint8_t *row = X + m * ldx;
+    int32_t sum = 0;
+    for (int64_t w = lane; w < ld_w; w += 32) {
+        uint32_t q[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+        const int64_t k0 = 32 * w;
+        if (k0 < K) {
+            if (k0 + 32 <= K && ((reinterpret_cast<uintptr_t>(row + k0) & 15u) == 0)) {
+                const uint4 a = *reinterpret_cast<const uint4 *>(row + k0), b = *reinterpret_cast<const uint4 *>(row + k0 + 16);
+                q[0] = a.x; q[1] = a.y; q[2] = a.z; q[3] = a.w; q[4] = b.x; q[5] = b.y; q[6] = b.z; q[7] = b.w;
+            } else {
+                for (int i = 0; i < 32; ++i)
+                    if (k0 + i < K) q[i >> 2] |= (uint32_t)row[k0 + i] << (8 * (i & 3));
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) sum += (int32_t)__vsadu4(q[i], 0u);
+#pragma unroll
+        for (int pl = 0; pl < 8; ++pl) {
+            uint32_t word = 0u;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) word |= plane_nibble(q[i], pl) << (4 * i);
+            planes[(8 * m + pl) * ld_w + w] = word;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (lane == 0) xsum[m] = sum;
+}
+}  // namespace
+
+size_t bnn_planes_scratch_bytes(int64_t M, int64_t K) {
+    const int64_t ld_w = ((K + 127) / 128) * 4;
+    return (((size_t)8 * M * ld_w * 4 + 255) & ~size_t(255)) + (((size_t)M * 4 + 255) & ~size_t(255));
+}
+
+// First layer on the CUDA-core kernels with the split done once into `scratch` (bnn_planes_scratch_bytes).
+int bnn_first_layer_planes_pre(bnn_ctx *ctx, const uint8_t *X, int64_t ldx, const uint32_t *Wp, int64_t ldw_w, const int32_t *thr,
+                               const uint32_t *flip, uint32_t *out_bits, int64_t ldo_w, int32_t *out_sums, int64_t lds, int64_t M,
+                               int64_t N, int64_t K, void *scratch) {
+    const int64_t ld_w = ((K + 127) / 128) * 4;
+    uint32_t *planes = static_cast<uint32_t *>(scratch);
+    int32_t *xsum = reinterpret_cast<int32_t *>(static_cast<char *>(scratch) + (((size_t)8 * M * ld_w * 4 + 255) & ~size_t(255)));
+    const int64_t blocks = (M + 7) / 8;
+    if (blocks > 0x7fffffff) return BNN_ERR_INVALID_ARG;
+    k_split_planes<<<(unsigned)blocks, 256, 0, ctx->stream>>>(X, ldx, M, K, planes, ld_w, xsum);
+    if (int st = bnn_check_launch(ctx)) return st;
+    Args a{};
+    a.A = planes; a.lda = ld_w; a.xsum = xsum; a.B = Wp; a.ldb = ldw_w;
+    a.M = M; a.N = N; a.K = K;
+    a.C = out_sums; a.ldc = lds; a.out = out_bits; a.ldo = ldo_w; a.thr = thr; a.flip = flip;
+    return launch_tile<A_PLANES_PRE>(ctx, a, ctx_variant(ctx));
+}
 
 int bnn_output_scores(bnn_ctx *ctx, const uint32_t *Ap, int64_t lda_w, const uint32_t *Wp, int64_t ldw_w,
                       const float *gamma, const float *beta, const float *mean, const float *var, double eps,
@@ -324,6 +386,10 @@ extern "C" int bnn_first_layer_bitplanes(bnn_ctx *ctx, const uint8_t *X, int64_t
         }
         if (ctx->engine == BNN_ENGINE_TENSOR) return BNN_ERR_WORKSPACE;
     }
+    // CUDA-core path.  With scratch available the bytes are split into bit-planes once (otherwise every column tile
+    // of the fused kernel splits its rows again); worth it from a few column tiles on.
+    if (N >= 512 && ctx->ws && ctx->ws_bytes >= bnn_planes_scratch_bytes(M, K))
+        return bnn_first_layer_planes_pre(ctx, X, ldx, Wp, ldw_w, thr, flip, out_bits, ldo_w, out_sums, lds, M, N, K, ctx->ws);
     Args a{};
     a.X = X; a.ldx = ldx; a.B = Wp; a.ldb = ldw_w;
     a.M = M; a.N = N; a.K = K;

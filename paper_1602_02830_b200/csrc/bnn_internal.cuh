@@ -32,3 +32,9 @@ bool bnn_umma_conv_tiling(int64_t H, int64_t W, int pool, int *TH, int *TB);
 int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B, int64_t H, int64_t W, int64_t C_in,
                   int64_t C_out, int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, int32_t *out_sums,
                   int8_t *out8 = nullptr, int64_t ldo8 = 0);
+
+// ---- bit-plane split as a pre-pass for the CUDA-core first layer (bnn_gemm.cu)
+size_t bnn_planes_scratch_bytes(int64_t M, int64_t K);
+int bnn_first_layer_planes_pre(bnn_ctx *ctx, const uint8_t *X, int64_t ldx, const uint32_t *Wp, int64_t ldw_w, const int32_t *thr,
+                               const uint32_t *flip, uint32_t *out_bits, int64_t ldo_w, int32_t *out_sums, int64_t lds, int64_t M,
+                               int64_t N, int64_t K, void *scratch);

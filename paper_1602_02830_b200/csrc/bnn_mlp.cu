@@ -40,7 +40,7 @@ struct engine_pin {
 };
 
 int forward_device(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X, int64_t ldx, int64_t batch, float *scores,
-                   int64_t lds, uint32_t *const *hidden_out, char *ws) {
+                   int64_t lds, uint32_t *const *hidden_out, char *ws, void *planes_scratch = nullptr) {
     // The layer calls below must stay on the CUDA-core kernels: the tensor engine would expand operands into the
     // context's workspace, which may be the very memory `ws` points into.
     engine_pin pin(ctx, BNN_ENGINE_POPC);
@@ -53,7 +53,10 @@ int forward_device(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X, int64_
         uint32_t *dst = bufs[k & 1];
         const int64_t ldo = act_ld(D.N);
         int st;
-        if (k == 0)
+        if (k == 0 && planes_scratch && D.N >= 512)
+            st = bnn_first_layer_planes_pre(ctx, X, ldx, D.Wp, D.ldw_w, D.thr, D.flip, dst, ldo, nullptr, 0, batch, D.N, D.K,
+                                            planes_scratch);
+        else if (k == 0)
             st = bnn_first_layer_bitplanes(ctx, X, ldx, D.Wp, D.ldw_w, D.thr, D.flip, dst, ldo, nullptr, 0, batch, D.N, D.K);
         else
             st = bnn_binary_dense(ctx, cur, act_ld(D.K), D.Wp, D.ldw_w, D.thr, D.flip, dst, ldo, batch, D.N, D.K);
@@ -136,16 +139,20 @@ size_t tensor_extra_bytes(const bnn_mlp_desc *m, int64_t batch) {
 
 }  // namespace
 
+// Offset of the bit-plane scratch of the CUDA-core first layer inside the workspace: behind the activation buffers
+// and (when the shapes qualify) the tensor engine's buffers.
+static size_t planes_offset(const bnn_mlp_desc *m, int64_t batch) {
+    size_t b = 2 * act_bytes(m, batch);
+    bool all = true;
+    for (int k = 0; k < m->n_layers - 1; ++k)
+        if (!bnn_umma_shape_ok(batch, m->layers[k].N, m->layers[k].K)) all = false;
+    if (all) b += tensor_extra_bytes(m, batch);      // room for the tensor-core engine, whatever engine is selected later
+    return b;
+}
+
 extern "C" size_t bnn_mlp_workspace_bytes(const bnn_mlp_desc *m, int64_t batch, int host_io) {
     if (check_desc(m) != BNN_OK || batch <= 0) return 0;
-    size_t b = 2 * act_bytes(m, batch);
-    // room for the tensor-core engine when the shapes qualify for it (whatever engine is selected later)
-    {
-        bool all = true;
-        for (int k = 0; k < m->n_layers - 1; ++k)
-            if (!bnn_umma_shape_ok(batch, m->layers[k].N, m->layers[k].K)) all = false;
-        if (all) b += tensor_extra_bytes(m, batch);
-    }
+    size_t b = planes_offset(m, batch) + bnn_planes_scratch_bytes(batch, m->layers[0].K);
     if (host_io) {
         b += round256((size_t)batch * m->layers[0].K);                        // staged input
         b += round256((size_t)batch * m->layers[m->n_layers - 1].N * 4);      // staged scores
@@ -164,7 +171,8 @@ extern "C" int bnn_mlp_forward(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_
     if (!guard.ok) return BNN_ERR_CUDA;
     if (tensor_applies(ctx, m, batch) && (ldx % 16) == 0 && bnn_aligned16(X))
         return forward_device_tensor(ctx, m, X, ldx, batch, scores, lds, hidden_out, static_cast<char *>(ctx->ws));
-    return forward_device(ctx, m, X, ldx, batch, scores, lds, hidden_out, static_cast<char *>(ctx->ws));
+    return forward_device(ctx, m, X, ldx, batch, scores, lds, hidden_out, static_cast<char *>(ctx->ws),
+                          static_cast<char *>(ctx->ws) + planes_offset(m, batch));
 }
 
 extern "C" int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X_host, int64_t ldx,
@@ -217,7 +225,8 @@ extern "C" int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const u
         const int64_t r0 = c * rows_per, rows = (r0 + rows_per <= batch) ? rows_per : batch - r0;
         if (nchunks > 1) BNN_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev[1 + c], 0));
         if (int st = tensor ? forward_device_tensor(ctx, m, Xd + r0 * K0, K0, rows, Sd + r0 * NL, NL, nullptr, ws)
-                            : forward_device(ctx, m, Xd + r0 * K0, K0, rows, Sd + r0 * NL, NL, nullptr, ws))
+                            : forward_device(ctx, m, Xd + r0 * K0, K0, rows, Sd + r0 * NL, NL, nullptr, ws,
+                                             ws + planes_offset(m, batch)))
             return st;
     }
     if (lds == NL)

@@ -30,7 +30,7 @@ constexpr int BN = 128;   // tile columns
 constexpr int BKW = 8;    // words of K per chunk
 constexpr int TN = 4;     // columns per lane
 
-enum { A_PACKED = 0, A_CONV = 1, A_PLANES = 2 };
+enum { A_PACKED = 0, A_CONV = 1, A_PLANES = 2, A_PLANES_PRE = 3 };   // PRE: bit-plane rows already split into `A`
 
 struct Args {
     const uint32_t *A;   // A_PACKED: packed M x K; A_CONV: packed NHWC activations
@@ -46,6 +46,7 @@ struct Args {
     int64_t ldo;
     const int32_t *thr;
     const uint32_t *flip;
+    const int32_t *xsum; // A_PLANES_PRE: sum of the 8-bit inputs of every image
     int H, W, Cw, pool;  // A_CONV geometry: image height/width, C_in/32, 2x2 pooling flag
     uint32_t one;        // always 1; a run-time value so that "popc * one + acc" stays an IMAD
 };
@@ -98,12 +99,15 @@ __global__ void __launch_bounds__(NWARPS * 32, (TM == 8) ? (512 / (NWARPS * 32))
     constexpr int NT = NWARPS * 32;
     static_assert(2 * BM <= NT && (TM == 8 || TM == 16), "at most one A load item per thread");
     constexpr int A_THREADS = 2 * BM;      // threads that load A
-    constexpr bool PLANES = (AKIND == A_PLANES);
+    constexpr bool PLANES = (AKIND == A_PLANES) || (AKIND == A_PLANES_PRE);   // 8 AND-popcount rows per image
+    constexpr bool SPLIT = (AKIND == A_PLANES);                               // ... split from bytes by this kernel
     constexpr int IMGS = BM / 8;           // A_PLANES: images per tile
 
-    __shared__ __align__(16) uint32_t As[2][BKW][BM];
+    // bit-plane mode pads the row stride: its 16-bit plane stores would otherwise hit the same bank eight times
+    constexpr int AS_LD = SPLIT ? BM + 4 : BM;
+    __shared__ __align__(16) uint32_t As[2][BKW][AS_LD];
     __shared__ __align__(16) uint32_t Bs[2][BKW][BN];
-    __shared__ int32_t aux[(AKIND == A_CONV) ? 9 * BN : (PLANES ? IMGS : 1)];
+    __shared__ int32_t aux[(AKIND == A_CONV) ? 9 * BN : (SPLIT ? IMGS : 1)];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int64_t rows_total = PLANES ? 8 * p.M : p.M;      // operand rows
@@ -118,8 +122,8 @@ __global__ void __launch_bounds__(NWARPS * 32, (TM == 8) ? (512 / (NWARPS * 32))
     const bool a_thread = tid < A_THREADS;
     const int a_row = tid % BM, a_half = (tid / BM) & 1;    // A_PACKED / A_CONV: row and which 4 of the 8 words
     const int a_img = (tid >> 4) % IMGS, a_seg = tid & 15;  // A_PLANES: image in tile and 16-byte segment of the chunk
-    const int64_t am = PLANES ? (m0 >> 3) + a_img : m0 + a_row;
-    const bool a_ok = a_thread && am < p.M;
+    const int64_t am = SPLIT ? (m0 >> 3) + a_img : m0 + a_row;
+    const bool a_ok = a_thread && am < (SPLIT ? p.M : rows_total);
     int pix_y = 0, pix_x = 0;
     int64_t pix_b = 0;
     if (AKIND == A_CONV && a_ok) {
@@ -142,7 +146,7 @@ __global__ void __launch_bounds__(NWARPS * 32, (TM == 8) ? (512 / (NWARPS * 32))
     uint4 rb[B_ITEMS];
 
     auto load_chunk = [&](int64_t c) {
-        if (AKIND == A_PACKED) {
+        if (AKIND == A_PACKED || AKIND == A_PLANES_PRE) {
             ra = load_row_words(p.A + am * p.lda, a_ok, c * BKW + 4 * a_half, Kw, tail_mask, a_vec);
         } else if (AKIND == A_CONV) {
             ra = make_uint4(0u, 0u, 0u, 0u);
@@ -193,7 +197,7 @@ __global__ void __launch_bounds__(NWARPS * 32, (TM == 8) ? (512 / (NWARPS * 32))
 
     auto store_chunk = [&](int buf) {
         if (!a_thread) {
-        } else if (PLANES) {
+        } else if (SPLIT) {
             const uint32_t w[4] = {ra.x, ra.y, ra.z, ra.w};
             x_sum += (int32_t)(__vsadu4(ra.x, 0u) + __vsadu4(ra.y, 0u) + __vsadu4(ra.z, 0u) + __vsadu4(ra.w, 0u));
 #pragma unroll
@@ -231,7 +235,7 @@ __global__ void __launch_bounds__(NWARPS * 32, (TM == 8) ? (512 / (NWARPS * 32))
             aux[e] = s;
         }
     }
-    if (PLANES) {
+    if (SPLIT) {
         if (tid < IMGS) aux[tid] = 0;
     }
 
@@ -314,7 +318,7 @@ __global__ void __launch_bounds__(NWARPS * 32, (TM == 8) ? (512 / (NWARPS * 32))
         __syncthreads();
     }
 
-    if (PLANES) {
+    if (SPLIT) {
         if (a_thread) atomicAdd(&aux[a_img], x_sum);
         __syncthreads();
     }
@@ -342,7 +346,7 @@ __global__ void __launch_bounds__(NWARPS * 32, (TM == 8) ? (512 / (NWARPS * 32))
 #pragma unroll
         for (int mi = 0; mi < IPT; ++mi) {
             const int64_t img = (m0 >> 3) + IPT * warp + mi;
-            const int32_t xs = aux[IPT * warp + mi];
+            const int32_t xs = SPLIT ? aux[IPT * warp + mi] : ((img < p.M) ? p.xsum[img] : 0);
 #pragma unroll
             for (int j = 0; j < TN; ++j) {
                 const int64_t col = n0 + lane + 32 * j;

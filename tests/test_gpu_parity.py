@@ -223,6 +223,27 @@ def test_first_layer_bitplanes(ctx, M, N, K):
     assert padding_is_zero(got, N)
 
 
+@pytest.mark.parametrize("M,N,K", [(70, 512, 784), (33, 600, 53), (260, 1024, 100), (9, 512, 1)])
+def test_first_layer_with_presplit_planes(ctx, M, N, K):
+    """With a workspace the CUDA-core first layer splits the bytes into bit-planes once, in a pre-pass."""
+    rng = np.random.default_rng(M + N + K)
+    X, W = wl.u8(rng, (M, K)), wl.pm1(rng, (K, N))
+    X[0, :] = 255
+    S = oracle.first_layer(X, W)
+    thr = rng.integers(-2000, 2000, N).astype(np.int32)
+    Wp = ctx.pack_signs(dev(W, torch.int8), pack_along=1)
+    ws = torch.empty(8 << 20, dtype=torch.uint8, device="cuda")
+    ctx.set_workspace(ws)
+    ctx.set_engine(binding.ENGINE_POPC)
+    bits, sums = ctx.first_layer_bitplanes(dev(X), Wp, M, N, K, thr=dev(thr), want_sums=True)
+    ctx.set_engine(binding.ENGINE_AUTO)
+    ctx.set_workspace(None)
+    assert np.array_equal(host(sums), S)
+    got = host(bits)
+    assert np.array_equal(np_unpack_pm1(got, N), oracle.threshold(S, thr))
+    assert padding_is_zero(got, N)
+
+
 def test_first_layer_unaligned_rows(ctx):
     M, N, K = 20, 40, 53            # row stride 53 bytes: the 16-byte fast path must not be taken blindly
     rng = np.random.default_rng(0)
