@@ -170,3 +170,60 @@ def test_dense_batch_sweep(ctx, batch):
     got = out[torch.from_numpy(rows).cuda()].cpu().numpy()
     assert np.array_equal(np_unpack_pm1(got, N), want)
     assert padding_is_zero(got, N)
+
+
+# ------------------------------------------------------------------ the paper's other network shapes (layer lists are data)
+def test_mlp_2048_unit_variant(ctx):
+    """Section 2.2: the Torch7 MNIST MLP uses 2048-unit hidden layers; same kernels, another layer list."""
+    case = wl.mlp_case(batch=4000, sizes=(784, 2048, 2048, 2048, 10), seed=6)
+    want_scores, want_hidden = oracle.mlp_forward(case["X"], case["weights"], case["bns"])
+    net = nets.prepare_mlp(ctx, case["weights"], case["bns"])
+    batch, sizes = case["batch"], case["sizes"]
+    ws = torch.empty(ctx.mlp_workspace_bytes(net["desc"], batch, False), dtype=torch.uint8, device="cuda")
+    ctx.set_workspace(ws)
+    hidden = [torch.empty(batch, binding.packed_ld(n), dtype=torch.int32, device="cuda") for n in sizes[1:-1]]
+    scores = ctx.mlp_forward(net["desc"], torch.from_numpy(case["X"]).cuda(), batch, hidden_out=hidden)
+    ctx.device_status()
+    for k, (g, w) in enumerate(zip(hidden, want_hidden)):
+        assert np.array_equal(np_unpack_pm1(g.cpu().numpy(), w.shape[1]), w), f"hidden layer {k}"
+    got = scores.cpu().numpy().astype(np.float64)
+    assert (np.abs(got - want_scores) <= 1e-5 * np.abs(want_scores) + 1e-6 * np.abs(want_scores).max()).all()
+    ctx.set_workspace(None)
+
+
+def test_convnet_half_width_variant_with_dense_tail(ctx):
+    """Section 2.4: the SVHN ConvNet has half the feature maps (64-64-128-128-256-256).  A fully-connected binary tail
+    (flattened 4 x 4 x 256 map -> 1024 -> 10-way scores) is added with the dense-layer calls: the packed NHWC map of
+    one image is already a packed row of 4096 bits."""
+    B = 40
+    case = wl.convnet_case(batch=B, channels=(64, 64, 128, 128, 256, 256), seed=11)
+    want_maps = oracle.convnet_forward(case["X"], case["layers"])
+    net = nets.prepare_convnet(ctx, case["layers"])
+    desc, keep = ctx.make_convnet_desc(net)
+    ws = torch.empty(max(ctx.convnet_workspace_bytes(desc, B, 32, 32), 256), dtype=torch.uint8, device="cuda")
+    ctx.set_workspace(ws)
+    outs = [torch.empty(w.shape[0], w.shape[1], w.shape[2], binding.words(w.shape[3]), dtype=torch.int32, device="cuda")
+            for w in want_maps]
+    final = torch.empty_like(outs[-1])
+    ctx.convnet_forward(desc, torch.from_numpy(case["X"]).cuda(), B, 32, 32, final, layer_out=outs)
+    ctx.device_status()
+    for k, (g, w) in enumerate(zip(outs, want_maps)):
+        assert np.array_equal(np_unpack_pm1(g.cpu().numpy(), w.shape[-1]), w), f"conv layer {k}"
+    # dense tail on the flattened map
+    rng = np.random.default_rng(12)
+    K = 4 * 4 * 256
+    W1, W2 = wl.pm1(rng, (K, 1024)), wl.pm1(rng, (1024, 10))
+    bn1, bn2 = wl.batchnorm_params(rng, 1024, K), wl.batchnorm_params(rng, 10, 1024)
+    flat = want_maps[-1].reshape(B, K)                                  # NHWC flattening = (y, x, c) order
+    h1 = oracle.sign_batchnorm(oracle.gemm(flat, W1), bn1)
+    want_scores = oracle.batchnorm(oracle.gemm(h1, W2), bn2)
+    thr1, flip1 = nets.fold(ctx, bn1, K)
+    W1p, W2p = nets.pack_weight(ctx, W1), nets.pack_weight(ctx, W2)
+    ctx.set_workspace(None)
+    a1 = ctx.binary_dense(final.reshape(B, K // 32), W1p, thr1, flip1, B, 1024, K)
+    S = ctx.xnor_gemm(a1, W2p, B, 10, 1024)
+    ctx.device_status()
+    assert np.array_equal(np_unpack_pm1(a1.cpu().numpy(), 1024), h1)
+    got = oracle.batchnorm(S.cpu().numpy(), bn2)                        # integer sums from the GPU, float epilogue on the host
+    assert np.array_equal(S.cpu().numpy(), oracle.gemm(h1, W2))
+    assert np.allclose(got, want_scores, rtol=0, atol=0)
