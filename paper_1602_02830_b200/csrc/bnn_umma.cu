@@ -649,8 +649,13 @@ static int umma_prepare(bnn_ctx *ctx) {
     }
     return BNN_OK;
 }
-// Tile width for N output columns: 128 when that leaves no (or less) idle MMA columns.
-static int umma_tile_n(int64_t N) { return (((N + 127) / 128) & 1) ? 128 : 256; }
+// Tile width for N output columns: 128 when that leaves no (or less) idle MMA columns, or when 256-wide tiles would
+// occupy less than half of the SMs (small batches).
+static int umma_tile_n(int64_t N, int64_t M = 0, int sm_count = 0) {
+    if (((N + 127) / 128) & 1) return 128;
+    if (M > 0 && ((M + BM - 1) / BM) * ((N + 255) / 256) * 2 <= sm_count) return 128;
+    return 256;
+}
 static size_t umma2_smem_bytes() { return (size_t)STAGES2 * STAGE2_BYTES + sizeof(Control) + 1024; }
 // Pairs of CTAs that can be resident at once for the two-SM kernel on this device (0 = cannot be used).
 static int umma2_max_pairs(bnn_ctx *ctx) {
@@ -716,7 +721,7 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
     if (M > 0x7fffffff || N > 0x7fffffff) return BNN_ERR_INVALID_ARG;
     if (K <= 0) return BNN_ERR_INVALID_ARG;      // callers route the empty product elsewhere
     CUtensorMap mapA, mapB;
-    const int bn = umma_tile_n(N);
+    const int bn = umma_tile_n(N, M, ctx->sm_count);
     const int64_t kb = ((K + 15) / 16) * 16;      // extent along K in bytes; beyond it TMA fills zeros
     // two-SM kernel: 256-wide tiles, at least two 256-row tiles, plain GEMM epilogues
     // (auto: only where it measured faster -- outputs of 2^26 elements and more, e.g. 8192 x 8192 or 65536 x 4096)
