@@ -329,7 +329,7 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
             uint32_t it = 0;
             bool ok = true;
             for (int64_t t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
-                const int m0 = (int)((t % tiles_m) * BM), n0 = (int)((t / tiles_m) * BN);
+                const int m0 = (int)((t / tiles_n) * BM), n0 = (int)((t % tiles_n) * BN);
                 for (int kit = 0; kit < p.k_iters; ++kit, ++it) {
                     const uint32_t s = it % STAGES;
                     if (it >= STAGES && !mbar_wait(smem_u32(&ctl->empty[s]), ((it / STAGES) - 1) & 1)) { fail(ctl, 1); ok = false; break; }
@@ -386,7 +386,7 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
         int64_t staged_n0[ACC_BUFS] = {-1, -1};
         for (int64_t t = blockIdx.x; t < ntiles; t += gridDim.x, ++tc) {
             const uint32_t buf = tc & 1;
-            const int64_t m0 = (t % tiles_m) * BM, n0 = (t / tiles_m) * BN;
+            const int64_t m0 = (t / tiles_n) * BM, n0 = (t % tiles_n) * BN;
             epilogue_tile<BN>(ctl, p, tmem_base, buf, tc, m0, n0, q, half, lane, et, ok, staged_n0);
             // hand the accumulator buffer back to the MMA warp
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
