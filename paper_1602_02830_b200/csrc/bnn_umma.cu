@@ -484,8 +484,8 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
             uint32_t it = 0;
             bool ok = true;
             for (int64_t t = pair; t < ntiles && ok; t += npairs) {
-                const int m0 = (int)((t % tiles_m) * (2 * BM) + rank * BM);
-                const int nb0 = (int)((t / tiles_m) * BN + rank * (BN / 2));
+                const int m0 = (int)((t / tiles_n) * (2 * BM) + rank * BM);
+                const int nb0 = (int)((t % tiles_n) * BN + rank * (BN / 2));
                 for (int kit = 0; kit < p.k_iters; ++kit, ++it) {
                     const uint32_t s = it % STAGES2;
                     if (it >= STAGES2 && !mbar_wait(smem_u32(&ctl->empty[s]), ((it / STAGES2) - 1) & 1)) { fail(ctl, 11); ok = false; break; }
@@ -532,7 +532,7 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         int64_t staged_n0[ACC_BUFS] = {-1, -1};
         for (int64_t t = pair; t < ntiles; t += npairs, ++tc) {
             const uint32_t buf = tc & 1;
-            const int64_t m0 = (t % tiles_m) * (2 * BM) + rank * BM, n0 = (t / tiles_m) * BN;
+            const int64_t m0 = (t / tiles_n) * (2 * BM) + rank * BM, n0 = (t % tiles_n) * BN;
             epilogue_tile<BN>(ctl, p, tmem_base, buf, tc, m0, n0, q, half, lane, et, ok, staged_n0);
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
