@@ -36,14 +36,6 @@ POPC_PER_CLK_PER_SM = 16
 L2_FLUSH_BYTES = 256 << 20
 
 
-def popc_words_mlp(batch, sizes):
-    """popc-words (one 32-bit XOR/AND + POPC in the plain formulation) of one forward pass."""
-    w = 8 * batch * sizes[1] * ((sizes[0] + 31) // 32)
-    for k in range(1, len(sizes) - 1):
-        w += batch * sizes[k + 1] * ((sizes[k] + 31) // 32)
-    return w
-
-
 def bit_ops_mlp(batch, sizes):
     """2 x bit-MACs of one forward pass, counting true K bits (8 planes for the first layer)."""
     ops = 2 * 8 * batch * sizes[0] * sizes[1]

@@ -1,7 +1,6 @@
 """CPU-side checks of the product's boundary: the shared library builds, loads and exports every function
 the header declares; status strings; and the host helper that folds BatchNorm + Sign into an integer
 threshold, compared with the oracle's double-precision Sign(BatchNorm(x)) over every integer x."""
-import ctypes
 import os
 import re
 
