@@ -82,6 +82,11 @@ BNN_API int bnn_set_engine(bnn_ctx *ctx, int engine);
  * cta_group::2) that share the B operand.  0 (default) = for outputs of 2^26 elements and more, where it measured
  * faster; 1 = never; 2 = wherever the kernel allows (M >= 512, 256-wide tiles).  Results are identical. */
 BNN_API int bnn_set_pair_mode(bnn_ctx *ctx, int mode);
+/* Tensor-core engine only: how +-1 x +-1 products are fed to the tensor cores.  4 (default) = each value as a 4-bit
+ * floating-point nibble (e2m1: +-1.0 is exact, block scales fixed at 1, float32 accumulators that hold these integer sums
+ * exactly for K <= 2^24): half the operand bytes and twice the instruction rate of 8 = one signed byte per value with
+ * int32 accumulators.  Layers with 8-bit inputs and the convolutions always use bytes.  Results are identical. */
+BNN_API int bnn_set_operand_bits(bnn_ctx *ctx, int bits);
 /* Workspace bytes bnn_xnor_gemm / bnn_binary_dense need to run M x N x K on the tensor-core engine
  * (0 if the shape does not qualify for it). */
 BNN_API size_t bnn_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
@@ -95,6 +100,11 @@ BNN_API size_t bnn_conv_workspace_bytes(int64_t B, int64_t H, int64_t W, int64_t
 BNN_API int64_t bnn_expanded_ld(int64_t K);
 BNN_API size_t bnn_expanded_bytes(int64_t rows, int64_t K);
 BNN_API int bnn_expand_signs(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t rows, int64_t K, int8_t *dst);
+/* The same as 4-bit floating-point nibbles (e2m1: +1 -> 0x2, -1 -> 0xa, two values per byte, value k in byte k/2 with
+ * even k in the low nibble; nibbles at positions >= K are 0).  Row pitch bnn_expanded_ld_f4(K) bytes. */
+BNN_API int64_t bnn_expanded_ld_f4(int64_t K);
+BNN_API size_t bnn_expanded_bytes_f4(int64_t rows, int64_t K);
+BNN_API int bnn_expand_signs_f4(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t rows, int64_t K, uint8_t *dst);
 /* Synchronises the context's stream and returns BNN_ERR_DEVICE_STATUS if a kernel gave up on one of its
  * bounded waits since the last call (its outputs are then undefined), BNN_OK otherwise. */
 BNN_API int bnn_device_status(bnn_ctx *ctx);
@@ -202,6 +212,8 @@ typedef struct {
     double eps;                             /* output layer only */
     const int8_t *W8; /* optional (device, may be NULL): the same weights as written by bnn_expand_signs, used by the
                          tensor-core engine; when NULL that engine expands Wp into the workspace on every call */
+    const uint8_t *W4; /* optional (device, may be NULL): the same weights as written by bnn_expand_signs_f4; what the
+                          tensor-core engine reads for layers 2.. when the operand width is 4 bits (the default) */
 } bnn_layer_desc;
 
 typedef struct {

@@ -27,14 +27,15 @@ EXPORTS = (
     "bnn_fold_batchnorm", "bnn_mlp_noalloc_max_bytes", "bnn_mlp_forward_noalloc", "bnn_set_engine",
     "bnn_gemm_workspace_bytes", "bnn_device_status", "bnn_conv_workspace_bytes", "bnn_set_tile_rows", "bnn_set_pair_mode", "bnn_expanded_ld",
     "bnn_expanded_bytes", "bnn_expand_signs", "bnn_baseline_gemm_f32", "bnn_convnet_workspace_bytes",
-    "bnn_convnet_forward",
+    "bnn_convnet_forward", "bnn_set_operand_bits", "bnn_expanded_ld_f4",
+    "bnn_expanded_bytes_f4", "bnn_expand_signs_f4",
 )
 
 
 class LayerDesc(Structure):
     _fields_ = [("Wp", c_void_p), ("ldw_w", c_int64), ("K", c_int64), ("N", c_int64), ("thr", c_void_p),
                 ("flip", c_void_p), ("gamma", c_void_p), ("beta", c_void_p), ("mean", c_void_p), ("var", c_void_p),
-                ("eps", c_double), ("W8", c_void_p)]
+                ("eps", c_double), ("W8", c_void_p), ("W4", c_void_p)]
 
 
 class MlpDesc(Structure):
@@ -82,6 +83,12 @@ def lib() -> ctypes.CDLL:
         L.bnn_set_engine.argtypes = [vp, c_int]
         L.bnn_set_tile_rows.argtypes = [vp, c_int]
         L.bnn_set_pair_mode.argtypes = [vp, c_int]
+        L.bnn_set_operand_bits.argtypes = [vp, c_int]
+        L.bnn_expanded_ld_f4.argtypes = [i64]
+        L.bnn_expanded_ld_f4.restype = i64
+        L.bnn_expanded_bytes_f4.argtypes = [i64, i64]
+        L.bnn_expanded_bytes_f4.restype = c_size_t
+        L.bnn_expand_signs_f4.argtypes = [vp, vp, i64, i64, i64, vp]
         L.bnn_expanded_ld.argtypes = [i64]
         L.bnn_expanded_ld.restype = i64
         L.bnn_expanded_bytes.argtypes = [i64, i64]
@@ -186,6 +193,16 @@ class Context:
         self._ck(lib().bnn_baseline_gemm_f32(self._h, _ptr(A), _ptr(B), _ptr(C), M, N, K), "bnn_baseline_gemm_f32")
         return C
 
+    def expand_signs_f4(self, packed, rows: int, K: int):
+        """bnn_expand_signs_f4: packed rows x K -> uint8 tensor [rows, bnn_expanded_ld_f4(K)] of e2m1 nibbles."""
+        ld = int(lib().bnn_expanded_ld_f4(K))
+        dst = self.empty(rows, ld, dtype=torch.uint8)
+        self._ck(lib().bnn_expand_signs_f4(self._h, _ptr(packed), packed.stride(0), rows, K, _ptr(dst)), "bnn_expand_signs_f4")
+        return dst
+
+    def set_operand_bits(self, bits: int):
+        self._ck(lib().bnn_set_operand_bits(self._h, bits), "bnn_set_operand_bits")
+
     def set_pair_mode(self, mode: int):
         self._ck(lib().bnn_set_pair_mode(self._h, mode), "bnn_set_pair_mode")
 
@@ -268,7 +285,7 @@ class Context:
             d.Wp = L["Wp"].data_ptr()
             d.ldw_w = L["Wp"].stride(0)
             d.K, d.N = L["K"], L["N"]
-            for name in ("thr", "flip", "gamma", "beta", "mean", "var", "W8"):
+            for name in ("thr", "flip", "gamma", "beta", "mean", "var", "W8", "W4"):
                 t = L.get(name)
                 setattr(d, name, t.data_ptr() if t is not None else None)
             d.eps = float(L.get("eps", 0.0))

@@ -20,6 +20,7 @@ extern "C" int bnn_create(bnn_ctx **out, int device, void *cuda_stream) {
     c->engine = 0;
     c->tile_rows = 8;
     c->pair_mode = 0;
+    c->operand_bits = 4;
     c->copy_stream = nullptr;
     c->copy_ready = false;
     for (int i = 0; i < 5; ++i) c->ev[i] = nullptr;
@@ -73,6 +74,12 @@ extern "C" int bnn_set_tile_rows(bnn_ctx *ctx, int rows) {
 extern "C" int bnn_set_pair_mode(bnn_ctx *ctx, int mode) {
     if (!ctx || mode < 0 || mode > 2) return BNN_ERR_INVALID_ARG;
     ctx->pair_mode = mode;
+    return BNN_OK;
+}
+
+extern "C" int bnn_set_operand_bits(bnn_ctx *ctx, int bits) {
+    if (!ctx || (bits != 4 && bits != 8)) return BNN_ERR_INVALID_ARG;
+    ctx->operand_bits = bits;
     return BNN_OK;
 }
 

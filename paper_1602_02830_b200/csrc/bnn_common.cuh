@@ -18,6 +18,7 @@ struct bnn_ctx {
     cudaStream_t copy_stream;   // internal stream for the host copies of bnn_mlp_forward_host (created on first use)
     cudaEvent_t ev[5];          // [0] work already on `stream`; [1..4] chunk copies done
     bool copy_ready;
+    int operand_bits; // tensor engine, +-1 x +-1 products: 4 = e2m1 nibbles (default), 8 = signed bytes
     int engine;    // 0 auto, 1 CUDA-core XOR-popcount kernels only, 2 tensor-core int8 engine where it applies
 };
 

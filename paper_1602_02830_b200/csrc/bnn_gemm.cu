@@ -321,6 +321,15 @@ static int gemm_like(bnn_ctx *ctx, const uint32_t *Ap, int64_t lda_w, const uint
         // tensor-core engine: both packed operands are expanded to signed bytes in the workspace first
         const size_t need = bnn_umma_operand_bytes(M, K) + bnn_umma_operand_bytes(N, K);
         if (ctx->ws && ctx->ws_bytes >= need) {
+            if (ctx->operand_bits == 4 && K <= (1 << 24)) {
+                // both operands are +-1: 4-bit (e2m1) operands, exact in the float32 accumulators
+                uint8_t *A4 = static_cast<uint8_t *>(ctx->ws);
+                uint8_t *B4 = A4 + bnn_umma_operand_bytes_f4(M, K);
+                const int64_t ld4 = bnn_umma_operand_ld_f4(K);
+                if (int st = bnn_umma_expand_f4(ctx, Ap, lda_w, M, K, A4)) return st;
+                if (int st = bnn_umma_expand_f4(ctx, Bp, ldb_w, N, K, B4)) return st;
+                return bnn_umma_gemm_f4(ctx, A4, ld4, B4, ld4, M, N, K, C, ldc, thr, flip, out, ldo_w, nullptr, 0);
+            }
             int8_t *A8 = static_cast<int8_t *>(ctx->ws);
             int8_t *B8 = A8 + bnn_umma_operand_bytes(M, K);
             const int64_t ld8 = bnn_umma_operand_ld(K);

@@ -13,7 +13,7 @@ int check_desc(const bnn_mlp_desc *m) {
     for (int k = 0; k < m->n_layers; ++k) {
         const bnn_layer_desc &L = m->layers[k];
         if (L.K <= 0 || L.N <= 0 || !L.Wp) return BNN_ERR_INVALID_ARG;
-        if (L.W8 && !bnn_aligned16(L.W8)) return BNN_ERR_ALIGNMENT;
+        if ((L.W8 && !bnn_aligned16(L.W8)) || (L.W4 && !bnn_aligned16(L.W4))) return BNN_ERR_ALIGNMENT;
         if (k > 0 && L.K != m->layers[k - 1].N) return BNN_ERR_INVALID_ARG;
         if (k < m->n_layers - 1) {
             if (!L.thr) return BNN_ERR_INVALID_ARG;
@@ -101,6 +101,8 @@ int forward_device_tensor(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X,
     int8_t *act8[2] = {reinterpret_cast<int8_t *>(ws + 2 * ab), reinterpret_cast<int8_t *>(ws + 2 * ab + a8)};
     int8_t *W8 = reinterpret_cast<int8_t *>(ws + 2 * ab + 2 * a8);
     const int L = m->n_layers;
+    // +-1 activations travel between hidden layers as e2m1 nibbles (4-bit engine) or as signed bytes
+    const bool f4 = ctx->operand_bits == 4;
     const uint32_t *cur = nullptr;
     const int8_t *cur8 = nullptr;
     for (int k = 0; k < L - 1; ++k) {
@@ -108,19 +110,28 @@ int forward_device_tensor(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X,
         uint32_t *dst = bits[k & 1];
         int8_t *dst8 = act8[k & 1];
         const int64_t ldo = act_ld(D.N);
-        const int8_t *Wk8 = D.W8;                      // expanded once by the caller, or here on every call
-        if (!Wk8) {
-            if (int st = bnn_umma_expand(ctx, D.Wp, D.ldw_w, D.N, D.K, W8)) return st;
-            Wk8 = W8;
-        }
-        const bool need8 = (k < L - 2);
+        const bool need_next = (k < L - 2);
+        const int64_t ld_next = f4 ? bnn_umma_operand_ld_f4(D.N) : bnn_umma_operand_ld(D.N);
         int st;
-        if (k == 0)
-            st = bnn_umma_gemm(ctx, X, ldx, true, Wk8, bnn_umma_operand_ld(D.K), batch, D.N, D.K, nullptr, 0, D.thr, D.flip, dst,
-                               ldo, need8 ? dst8 : nullptr, bnn_umma_operand_ld(D.N));
-        else
-            st = bnn_umma_gemm(ctx, cur8, bnn_umma_operand_ld(D.K), false, Wk8, bnn_umma_operand_ld(D.K), batch, D.N, D.K, nullptr,
-                               0, D.thr, D.flip, dst, ldo, need8 ? dst8 : nullptr, bnn_umma_operand_ld(D.N));
+        if (k == 0 || !f4) {
+            const int8_t *Wk8 = D.W8;                  // expanded once by the caller, or here on every call
+            if (!Wk8) {
+                if ((st = bnn_umma_expand(ctx, D.Wp, D.ldw_w, D.N, D.K, W8))) return st;
+                Wk8 = W8;
+            }
+            st = bnn_umma_gemm(ctx, k == 0 ? static_cast<const void *>(X) : cur8, k == 0 ? ldx : bnn_umma_operand_ld(D.K), k == 0, Wk8,
+                               bnn_umma_operand_ld(D.K), batch, D.N, D.K, nullptr, 0, D.thr, D.flip, dst, ldo,
+                               need_next ? dst8 : nullptr, ld_next, 0, 0, 0, f4 ? 1 : 0);
+        } else {
+            const uint8_t *Wk4 = D.W4;
+            if (!Wk4) {
+                if ((st = bnn_umma_expand_f4(ctx, D.Wp, D.ldw_w, D.N, D.K, reinterpret_cast<uint8_t *>(W8)))) return st;
+                Wk4 = reinterpret_cast<uint8_t *>(W8);
+            }
+            st = bnn_umma_gemm_f4(ctx, reinterpret_cast<const uint8_t *>(cur8), bnn_umma_operand_ld_f4(D.K), Wk4,
+                                  bnn_umma_operand_ld_f4(D.K), batch, D.N, D.K, nullptr, 0, D.thr, D.flip, dst, ldo,
+                                  need_next ? reinterpret_cast<uint8_t *>(dst8) : nullptr, ld_next);
+        }
         if (st) return st;
         if (hidden_out && hidden_out[k])
             BNN_CUDA_TRY(ctx, cudaMemcpyAsync(hidden_out[k], dst, (size_t)batch * ldo * 4, cudaMemcpyDeviceToDevice,

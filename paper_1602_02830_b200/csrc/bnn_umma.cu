@@ -24,7 +24,8 @@
 namespace {
 
 constexpr int BM = 128, BK = 128;               // BK in bytes = int8 elements
-constexpr int BN_MAX = 256;                     // tile width: 256, or 128 for narrow outputs (template parameter)
+constexpr int BN_MAX = 256;                     // tile width: 256, or 128 for narrow outputs; 192 = the 4-bit engine
+constexpr uint32_t SF_COL = 480;                // 4-bit engine: first of the 32 TMEM columns that hold the scale factors
 constexpr int EPI_WARPS = 8;                    // two per TMEM lane quadrant, each takes half of the tile's columns
 constexpr int EPI_THREADS = EPI_WARPS * 32;
 constexpr int NTHREADS = 64 + EPI_THREADS;
@@ -33,8 +34,9 @@ constexpr int ACC_BUFS = 2;
 template <int BN> struct Cfg {
     static constexpr uint32_t B_BYTES = BN * BK;
     static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (BN == 256) ? 4 : 6;          // 192 KB of operand stages either way
-    static constexpr uint32_t TMEM_COLS = 2 * BN;               // two accumulator buffers of BN columns
+    static constexpr int STAGES = (BN == 256) ? 4 : ((BN == 192) ? 5 : 6);   // 192-200 KB of operand stages
+    // two accumulator buffers of BN columns; the 4-bit configuration (BN = 192) also keeps 32 columns of scale factors
+    static constexpr uint32_t TMEM_COLS = (BN == 192) ? 512 : 2 * BN;
 };
 constexpr int STAGES_MAX = 6;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // a wait gives up after 2 s of wall clock
@@ -47,7 +49,8 @@ struct UmmaArgs {
     uint32_t idesc;
     int32_t *C; int64_t ldc;                     // optional int32 output
     uint32_t *out; int64_t ldo;                  // optional packed sign output
-    int8_t *out8; int64_t ldo8;                  // optional +-1 byte output (next layer's operand)
+    int8_t *out8; int64_t ldo8;                  // optional +-1 output for the next layer: bytes, or
+    int out_f4;                                  // ... e2m1 nibbles (two per byte, ldo8 in bytes) when set
     const int32_t *thr; const uint32_t *flip;
     // convolution mode (3x3, pad 1): A is a 4-D byte tensor [B][H][W][C_in]; one K step = (tap, 128-channel slice)
     int conv;               // 0 = plain GEMM
@@ -112,6 +115,15 @@ __device__ __forceinline__ void umma_i8(uint32_t tmem_d, uint64_t adesc, uint64_
         "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// 4-bit (e2m1) operands with one UE8M0 scale per 32 values; K = 64 per instruction, float32 accumulators.
+__device__ __forceinline__ void umma_mxf4(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate,
+                                          uint32_t tmem_sf) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%5], p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(tmem_sf) : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -156,6 +168,49 @@ __device__ __forceinline__ void fail(Control *ctl, int code) {
     atomicExch(&g_umma_error, code);
 }
 
+// 8 sign bits -> 8 e2m1 nibbles (+1.0 = 0x2, -1.0 = 0xa); bit i lands in nibble i.
+__device__ __forceinline__ uint32_t nibbles_of_byte(uint32_t x) {
+    uint32_t t = (x | (x << 12)) & 0x000f000fu;
+    t = (t | (t << 6)) & 0x03030303u;
+    t = (t | (t << 3)) & 0x11111111u;
+    return ((t ^ 0x11111111u) << 3) | 0x22222222u;
+}
+// The signs of 32 consecutive outputs of row `orow` (bit j of `word` = column col0 + j) in the next layer's operand
+// format: one signed byte per value, or one e2m1 nibble per value.  Positions at or beyond N are written as 0.
+__device__ __forceinline__ void store_signs(const UmmaArgs &p, uint32_t word, int64_t orow, int64_t col0) {
+    if (p.out_f4) {
+        uint8_t *d = reinterpret_cast<uint8_t *>(p.out8) + orow * p.ldo8 + (col0 >> 1);
+        if (col0 + 32 <= p.N) {
+            *reinterpret_cast<uint4 *>(d) = make_uint4(nibbles_of_byte(word & 0xffu), nibbles_of_byte((word >> 8) & 0xffu),
+                                                       nibbles_of_byte((word >> 16) & 0xffu), nibbles_of_byte(word >> 24));
+        } else {
+            for (int j = 0; j < 32; j += 2) {
+                if ((col0 + j) / 2 >= p.ldo8) break;
+                const uint32_t lo = (col0 + j < p.N) ? (((word >> j) & 1u) ? 0x2u : 0xau) : 0u;
+                const uint32_t hi = (col0 + j + 1 < p.N) ? (((word >> (j + 1)) & 1u) ? 0x2u : 0xau) : 0u;
+                d[j >> 1] = (uint8_t)(lo | (hi << 4));
+            }
+        }
+        return;
+    }
+    int8_t *d8 = p.out8 + orow * p.ldo8 + col0;
+    if (col0 + 32 <= p.N) {
+        uint32_t b[8];
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+            // 4 sign bits -> 4 bytes of +1 (0x01) / -1 (0xff)
+            const uint32_t t4 = (((word >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u;
+            b[g] = ~(t4 * 0xfeu);
+        }
+        *reinterpret_cast<uint4 *>(d8) = make_uint4(b[0], b[1], b[2], b[3]);
+        *reinterpret_cast<uint4 *>(d8 + 16) = make_uint4(b[4], b[5], b[6], b[7]);
+    } else {
+        for (int j = 0; j < 32; ++j)
+            if (col0 + j < p.N) d8[j] = ((word >> j) & 1u) ? (int8_t)1 : (int8_t)-1;
+            else if (col0 + j < p.ldo8) d8[j] = 0;
+    }
+}
+
 // One tile's epilogue for the calling epilogue warp: stage the tile's thresholds, wait for the accumulators in
 // buffer `buf`, and turn them into the requested outputs.  `ok` turns false once a wait has given up.
 template <int BN>
@@ -194,6 +249,10 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
             uint32_t (&r)[32] = (cc & 1) ? rb : ra;
             uint32_t (&rn)[32] = (cc & 1) ? ra : rb;
             if (more) tmem_ld32(tbase + (uint32_t)(32 * (c + 1)), rn);
+            if (BN == 192) {   // the 4-bit engine accumulates in float32: exact integers, converted once
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = (uint32_t)(int32_t)__uint_as_float(r[j]);
+            }
             if (row < p.M) {
                 if (p.C) {
                     int32_t *dst = p.C + row * p.ldc + col0;
@@ -215,24 +274,7 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                     if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;      // columns beyond N stay 0
                     if (p.pool) ctl->poolw[32 * q + lane][c] = word ^ ctl->flip[buf][c];   // un-flipped (dot >= thr) bits
                     else p.out[row * p.ldo + (col0 >> 5)] = word;
-                    if (p.out8 && !p.pool) {
-                        int8_t *d8 = p.out8 + row * p.ldo8 + col0;
-                        uint32_t b[8];
-#pragma unroll
-                        for (int g = 0; g < 8; ++g) {
-                            // 4 sign bits -> 4 bytes of +1 (0x01) / -1 (0xff)
-                            const uint32_t t4 = (((word >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u;
-                            b[g] = ~(t4 * 0xfeu);
-                        }
-                        if (col0 + 32 <= p.N) {
-                            *reinterpret_cast<uint4 *>(d8) = make_uint4(b[0], b[1], b[2], b[3]);
-                            *reinterpret_cast<uint4 *>(d8 + 16) = make_uint4(b[4], b[5], b[6], b[7]);
-                        } else {
-                            for (int j = 0; j < 32; ++j)
-                                if (col0 + j < p.N) d8[j] = ((word >> j) & 1u) ? (int8_t)1 : (int8_t)-1;
-                                else if (col0 + j < p.ldo8) d8[j] = 0;
-                        }
-                    }
+                    if (p.out8 && !p.pool) store_signs(p, word, row, col0);
                 }
             }
             if (more) tmem_ld_wait(rn);
@@ -267,23 +309,7 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                 p.out[opix * p.ldo + (col0 >> 5)] = word;
                 if (n0 + BN >= p.N && c == nwords - 1)
                     for (int64_t w = (p.N + 31) >> 5; w < p.ldo; ++w) p.out[opix * p.ldo + w] = 0u;
-                if (p.out8) {   // the pooled pixel's signs as +-1 bytes for the next layer
-                    int8_t *d8 = p.out8 + opix * p.ldo8 + col0;
-                    if (col0 + 32 <= p.N) {
-                        uint32_t b[8];
-#pragma unroll
-                        for (int g = 0; g < 8; ++g) {
-                            const uint32_t t4 = (((word >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u;
-                            b[g] = ~(t4 * 0xfeu);
-                        }
-                        *reinterpret_cast<uint4 *>(d8) = make_uint4(b[0], b[1], b[2], b[3]);
-                        *reinterpret_cast<uint4 *>(d8 + 16) = make_uint4(b[4], b[5], b[6], b[7]);
-                    } else {
-                        for (int j = 0; j < 32; ++j)
-                            if (col0 + j < p.N) d8[j] = ((word >> j) & 1u) ? (int8_t)1 : (int8_t)-1;
-                            else if (col0 + j < p.ldo8) d8[j] = 0;
-                    }
-                }
+                if (p.out8) store_signs(p, word, opix, col0);   // the pooled pixel's signs for the next layer
             }
         }
     }
@@ -322,6 +348,20 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = ctl->tmem_base;
+
+    if (BN == 192) {
+        // 4-bit engine: every value is exactly +-1, so every block scale is 2^0.  In UE8M0 that is the byte 0x7f, and
+        // with all 32 scale-factor columns filled with it the instruction reads 1.0 wherever it looks.
+        if (warp >= 2 && warp < 6) {
+            const uint32_t v = 0x7f7f7f7fu;
+            asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1};"
+                         ::"r"(tmem_base + SF_COL + ((uint32_t)(32 * (warp & 3)) << 16)), "r"(v) : "memory");
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    }
 
     if (warp == 0) {
         // ---------------- TMA producer
@@ -368,8 +408,14 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                     const uint64_t adesc = smem_desc_sw128(smem_u32(tiles + s * STAGE_BYTES));
                     const uint64_t bdesc = smem_desc_sw128(smem_u32(tiles + s * STAGE_BYTES + A_BYTES));
 #pragma unroll
-                    for (int k = 0; k < BK / 32; ++k)   // 32 bytes of K per instruction: start address advances by 32 B (>> 4 = 2)
-                        umma_i8(tmem_d, adesc + 2 * k, bdesc + 2 * k, p.idesc | ((uint32_t)(BN >> 3) << 17), (kit > 0 || k > 0) ? 1u : 0u);
+                    for (int k = 0; k < BK / 32; ++k) {   // 32 bytes of K per instruction: start address advances by 32 B (>> 4 = 2)
+                        if (BN == 192)   // e2m1 x e2m1 (format 1), UE8M0 scales (bit 23), N >> 3 at bit 17, M >> 4 at bit 24
+                            umma_mxf4(tmem_d, adesc + 2 * k, bdesc + 2 * k,
+                                      (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (1u << 23) | ((uint32_t)(BM >> 4) << 24),
+                                      (kit > 0 || k > 0) ? 1u : 0u, tmem_base + SF_COL);
+                        else
+                            umma_i8(tmem_d, adesc + 2 * k, bdesc + 2 * k, p.idesc | ((uint32_t)(BN >> 3) << 17), (kit > 0 || k > 0) ? 1u : 0u);
+                    }
                     umma_commit(smem_u32(&ctl->empty[s]));      // stage may be refilled once these MMAs have read it
                 }
                 umma_commit(smem_u32(&ctl->acc_full[buf]));     // accumulators of this tile complete (also after a failure)
@@ -576,6 +622,30 @@ __global__ void __launch_bounds__(256) k_expand_s8(const uint32_t *__restrict__ 
     d[1] = make_uint4(b[4], b[5], b[6], b[7]);
 }
 
+// Packed signs -> one e2m1 nibble per value (+1.0 = 0x2, -1.0 = 0xa), two per byte, value k in byte k/2 (even k in
+// the low nibble); nibbles at or beyond K are 0 (= +0.0).  One thread per 32-bit word = 16 output bytes.
+__global__ void __launch_bounds__(256) k_expand_f4(const uint32_t *__restrict__ src, int64_t ld_w, int64_t rows, int64_t K,
+                                                   uint8_t *__restrict__ dst, int64_t ld4) {
+    const int64_t wpr = ld4 >> 4;            // words per output row (ld4 is a multiple of 128 bytes)
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= rows * wpr) return;
+    const int64_t r = idx / wpr, w = idx - r * wpr;
+    const int64_t Kw = (K + 31) >> 5;
+    uint32_t bits = 0u, valid = 0u;
+    if (w < Kw) {
+        bits = src[r * ld_w + w];
+        valid = (w == Kw - 1 && (K & 31)) ? ((1u << (K & 31)) - 1u) : 0xffffffffu;
+    }
+    uint32_t q[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        const uint32_t n = nibbles_of_byte((bits >> (8 * g)) & 0xffu);
+        const uint32_t v = nibbles_of_byte((valid >> (8 * g)) & 0xffu);      // 0x2 where valid, 0xa where not
+        q[g] = n & (((~v >> 3) & 0x11111111u) * 0xfu);                         // keep the nibbles whose valid bit is set
+    }
+    *reinterpret_cast<uint4 *>(dst + r * ld4 + 16 * w) = make_uint4(q[0], q[1], q[2], q[3]);
+}
+
 // First convolution: the 3x3 neighbourhood of every pixel of an 8-bit NHWC image (9 * C_in <= 32 bytes, taps
 // outside the image as zeros) written as one 32-byte row, byte (tap * C_in + c).  One thread per pixel.
 __global__ void __launch_bounds__(256) k_im2col_u8(const uint8_t *__restrict__ act, int64_t B, int H, int W, int Cin,
@@ -645,6 +715,7 @@ static int umma_prepare(bnn_ctx *ctx) {
     if (!attr_set[ctx->device]) {
         BNN_CUDA_TRY(ctx, cudaFuncSetAttribute(k_umma_i8<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes<256>()));
         BNN_CUDA_TRY(ctx, cudaFuncSetAttribute(k_umma_i8<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes<128>()));
+        BNN_CUDA_TRY(ctx, cudaFuncSetAttribute(k_umma_i8<192>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes<192>()));
         attr_set[ctx->device] = true;
     }
     return BNN_OK;
@@ -687,7 +758,8 @@ static int umma_launch(bnn_ctx *ctx, const CUtensorMap &mapA, const CUtensorMap 
     if (int st = umma_prepare(ctx)) return st;
     const int64_t tiles = ((a.M + BM - 1) / BM) * ((a.N + bn - 1) / bn);
     const int64_t grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
-    if (bn == 256) k_umma_i8<256><<<(unsigned)grid, NTHREADS, umma_smem_bytes<256>(), ctx->stream>>>(mapA, mapB, a);
+    if (bn == 192) k_umma_i8<192><<<(unsigned)grid, NTHREADS, umma_smem_bytes<192>(), ctx->stream>>>(mapA, mapB, a);
+    else if (bn == 256) k_umma_i8<256><<<(unsigned)grid, NTHREADS, umma_smem_bytes<256>(), ctx->stream>>>(mapA, mapB, a);
     else k_umma_i8<128><<<(unsigned)grid, NTHREADS, umma_smem_bytes<128>(), ctx->stream>>>(mapA, mapB, a);
     return bnn_check_launch(ctx);
 }
@@ -708,10 +780,44 @@ int bnn_umma_expand(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t row
     return bnn_check_launch(ctx);
 }
 
+// The 4-bit operand format: pitch and size of rows x K e2m1 nibbles.
+int64_t bnn_umma_operand_ld_f4(int64_t K) { return ((K + 255) / 256) * 128; }
+size_t bnn_umma_operand_bytes_f4(int64_t rows, int64_t K) { return ((size_t)rows * bnn_umma_operand_ld_f4(K) + 255) & ~size_t(255); }
+int bnn_umma_expand_f4(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t rows, int64_t K, uint8_t *dst) {
+    const int64_t ld4 = bnn_umma_operand_ld_f4(K);
+    const int64_t total = rows * (ld4 >> 4);
+    if (total == 0) return BNN_OK;
+    const int64_t blocks = (total + 255) / 256;
+    if (blocks > 0x7fffffff) return BNN_ERR_INVALID_ARG;
+    k_expand_f4<<<(unsigned)blocks, 256, 0, ctx->stream>>>(src, ld_w, rows, K, dst, ld4);
+    return bnn_check_launch(ctx);
+}
+
+// Both operands as e2m1 nibbles (+-1 exactly; pitches in bytes): the same outputs as bnn_umma_gemm at twice the MMA
+// rate and half the operand bytes.  Accumulation is float32, exact while K <= 2^24.  out4 (optional): the signs of
+// the outputs as nibbles for a following layer, pitch ldo4 bytes.
+int bnn_umma_gemm_f4(bnn_ctx *ctx, const uint8_t *A4, int64_t lda4, const uint8_t *B4, int64_t ldb4, int64_t M, int64_t N,
+                     int64_t K, int32_t *C, int64_t ldc, const int32_t *thr, const uint32_t *flip, uint32_t *out, int64_t ldo,
+                     uint8_t *out4, int64_t ldo4) {
+    if (M == 0 || N == 0) return BNN_OK;
+    if ((lda4 & 15) || (ldb4 & 15) || !bnn_aligned16(A4) || !bnn_aligned16(B4)) return BNN_ERR_ALIGNMENT;
+    if (M > 0x7fffffff || N > 0x7fffffff || K <= 0 || K > (1 << 24)) return BNN_ERR_INVALID_ARG;
+    CUtensorMap mapA, mapB;
+    const int64_t kb = (((K + 1) / 2 + 15) / 16) * 16;      // extent along K in bytes
+    if (int st = make_map(ctx, &mapA, A4, M, kb <= lda4 ? kb : lda4, lda4, BM)) return st;
+    if (int st = make_map(ctx, &mapB, B4, N, kb <= ldb4 ? kb : ldb4, ldb4, 192)) return st;
+    UmmaArgs a{};
+    a.M = M; a.N = N;
+    a.k_iters = (int)((K + 2 * BK - 1) / (2 * BK));          // 256 values per 128-byte K step
+    a.C = C; a.ldc = ldc; a.out = out; a.ldo = ldo; a.thr = thr; a.flip = flip;
+    a.out8 = reinterpret_cast<int8_t *>(out4); a.ldo8 = ldo4; a.out_f4 = 1;
+    return umma_launch(ctx, mapA, mapB, a, 192);
+}
+
 // C / bits = A8 (M x K bytes, pitch lda8; unsigned if a_unsigned) times B8^T (N x K signed bytes, pitch ldb8).
 int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, const int8_t *B8, int64_t ldb8, int64_t M,
                   int64_t N, int64_t K, int32_t *C, int64_t ldc, const int32_t *thr, const uint32_t *flip, uint32_t *out,
-                  int64_t ldo, int8_t *out8, int64_t ldo8, int pool, int64_t H, int64_t W) {
+                  int64_t ldo, int8_t *out8, int64_t ldo8, int pool, int64_t H, int64_t W, int out_f4) {
     if (M == 0 || N == 0) return BNN_OK;
     if (pool) {   // rows are pixels of H x W images in (b, y, x) order; 128-row tiles must hold whole 2x2 windows
         int TH, TB;
@@ -735,7 +841,7 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
     a.k_iters = (int)((K + BK - 1) / BK);
     a.idesc = (2u << 4) | ((a_unsigned ? 0u : 1u) << 7) | (1u << 10) | ((uint32_t)(BM >> 4) << 24);   // N field added by the kernel
     a.C = C; a.ldc = ldc; a.out = out; a.ldo = ldo; a.out8 = out8; a.ldo8 = ldo8; a.thr = thr; a.flip = flip;
-    a.pool = pool; a.H = (int)H; a.W = (int)W;
+    a.pool = pool; a.H = (int)H; a.W = (int)W; a.out_f4 = out_f4;
     if (pairs > 0) {
         const int64_t tiles2 = ((M + 2 * BM - 1) / (2 * BM)) * ((N + 255) / 256);
         const int64_t use = tiles2 < pairs ? tiles2 : pairs;
@@ -818,6 +924,18 @@ extern "C" int bnn_expand_signs(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w,
     bnn_device_guard guard(ctx);
     if (!guard.ok) return BNN_ERR_CUDA;
     return bnn_umma_expand(ctx, src, ld_w, rows, K, dst);
+}
+
+extern "C" int64_t bnn_expanded_ld_f4(int64_t K) { return K > 0 ? bnn_umma_operand_ld_f4(K) : 0; }
+extern "C" size_t bnn_expanded_bytes_f4(int64_t rows, int64_t K) { return (rows > 0 && K > 0) ? bnn_umma_operand_bytes_f4(rows, K) : 0; }
+extern "C" int bnn_expand_signs_f4(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t rows, int64_t K, uint8_t *dst) {
+    if (!ctx || rows < 0 || K < 0) return BNN_ERR_INVALID_ARG;
+    if (rows == 0 || K == 0) return BNN_OK;
+    if (!src || !dst || ld_w < bnn_words(K)) return BNN_ERR_INVALID_ARG;
+    if (!bnn_aligned16(dst)) return BNN_ERR_ALIGNMENT;
+    bnn_device_guard guard(ctx);
+    if (!guard.ok) return BNN_ERR_CUDA;
+    return bnn_umma_expand_f4(ctx, src, ld_w, rows, K, dst);
 }
 
 // Reads (and clears) the error word the tensor-core kernel sets when one of its bounded waits gives up.

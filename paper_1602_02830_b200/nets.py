@@ -39,7 +39,10 @@ def prepare_mlp(ctx, weights, bns, expand_weights: bool = True):
         if k < L - 1:
             d["thr"], d["flip"] = fold(ctx, bn, 255 * K if k == 0 else K)
             if expand_weights:
+                # the first layer multiplies bytes by bytes; the others can run on either operand width
                 d["W8"] = ctx.expand_signs(d["Wp"], N, K)
+                if k > 0:
+                    d["W4"] = ctx.expand_signs_f4(d["Wp"], N, K)
         else:
             for name in ("gamma", "beta", "mean", "var"):
                 d[name] = _dev(ctx, bn[name], torch.float32)

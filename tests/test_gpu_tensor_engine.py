@@ -12,13 +12,15 @@ from util import np_pack_pm1, np_unpack_pm1, padding_is_zero
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module", params=[2, 1], ids=["pairs", "single"])
+@pytest.fixture(scope="module", params=[(2, 8), (1, 8), (1, 4)], ids=["pairs-bytes", "single-bytes", "nibbles"])
 def ctx(request):
-    """Tensor engine forced; with CTA pairs (cta_group::2) wherever the kernel allows, and with the single-SM kernel only."""
+    """Tensor engine forced: byte operands with CTA pairs (cta_group::2) wherever the kernel allows, byte operands on
+    the single-SM kernel, and 4-bit (e2m1) operands for the +-1 x +-1 products."""
     build.build()
     c = binding.Context(0)
     c.set_engine(binding.ENGINE_TENSOR)
-    c.set_pair_mode(request.param)
+    c.set_pair_mode(request.param[0])
+    c.set_operand_bits(request.param[1])
     yield c
     torch.cuda.synchronize()
     c.close()
@@ -107,6 +109,15 @@ def test_first_layer_tensor_engine(ctx, M, N, K):
     assert padding_is_zero(got, N)
     ctx.set_workspace(None)
     del ws
+
+
+def test_expand_signs_f4(ctx):
+    x = wl.pm1(np.random.default_rng(4), (21, 300))
+    p = ctx.pack_signs(dev(x, torch.int8))
+    e = ctx.expand_signs_f4(p, 21, 300).cpu().numpy()
+    assert e.shape == (21, 256)
+    nib = np.stack([e & 0xF, e >> 4], axis=-1).reshape(21, -1)            # value k in byte k/2, even k low
+    assert np.array_equal(nib[:, :300], np.where(x > 0, 0x2, 0xA)) and not nib[:, 300:].any()
 
 
 def test_expand_signs(ctx):
