@@ -141,6 +141,8 @@ def main():
     ap.add_argument("--engine", type=int, default=0, help="0 auto (tensor-core int8 engine for large shapes), 1 CUDA-core XOR-popcount only, 2 tensor")
     ap.add_argument("--tile-rows", type=int, default=0, help="accumulator rows per thread of the CUDA-core tile kernel (8 or 16; 0 = library default)")
     ap.add_argument("--pair-mode", type=int, default=0, help="tensor engine CTA pairs (cta_group::2): 0 = for very large outputs, 1 = never, 2 = wherever possible")
+    ap.add_argument("--operand-bits", type=int, default=4, choices=[4, 8],
+                    help="tensor engine, +-1 x +-1 products: 4 = e2m1 nibbles (kind::mxf4), 8 = signed bytes (kind::i8)")
     ap.add_argument("--no-extras", action="store_true", help="skip the GEMM / ConvNet side measurements and the CPU baseline")
     ap.add_argument("--gemm-size", type=int, default=8192)
     ap.add_argument("--section", default="all", choices=["all", "gemm", "convnet", "sweep", "fig3"],
@@ -169,6 +171,7 @@ def main():
     if args.tile_rows:
         ctx.set_tile_rows(args.tile_rows)
     ctx.set_pair_mode(args.pair_mode)
+    ctx.set_operand_bits(args.operand_bits)
 
     def sync_all():
         torch.cuda.synchronize()
@@ -224,7 +227,7 @@ def main():
     # steps run until a block is within 2 % of the one before it AND of the fastest block so far (at most 30 blocks).
     e2e_fn = lambda: ctx.mlp_forward_host(desc, Xh, BATCH, Sh)
     prev, best, e2e_warm_blocks = None, None, 0
-    for _ in range(30):
+    for _ in range(30 if args.steps >= 50 else 1):      # (short runs are profiler captures: no long warm-up there)
         blk = sum(timed_steps(e2e_fn, 100, 0)) / 100
         e2e_warm_blocks += 1
         steady = prev is not None and abs(blk - prev) <= 0.02 * prev and blk <= 1.02 * best
@@ -279,7 +282,9 @@ def main():
     popc_dense_ach = dense_ops / (popc_dense_ms / 1e3) / 1e12
     popc_mlp_ms = sum(popc_mlp_times) / len(popc_mlp_times)
     bf16_peak = float(peaks.get("bf16_tflops") or 1590.0)
-    tensor_peak = 2.0 * bf16_peak           # int8 : bf16 nominal ratio 2 (4.5 vs 2.25 PFLOP/s dense)
+    # nominal dense ratios to bf16 (2.25 PFLOP/s): int8 4.5 -> 2x, fp4 9 -> 4x
+    peak_ratio = 4.0 if args.operand_bits == 4 else 2.0
+    tensor_peak = peak_ratio * bf16_peak
     first_ms = sum(first_times) / len(first_times)
     first_ach = 2.0 * 8 * BATCH * SIZES[0] * SIZES[1] / (first_ms / 1e3) / 1e12
     mlp_ach = bit_ops_mlp(BATCH, SIZES) / (ms_per_step / 1e3) / 1e12
@@ -291,17 +296,21 @@ def main():
         "config": {"workload": "MNIST-shaped BNN MLP forward 784-4096-4096-4096-10 (8 bit-planes, 2 fused binary dense, float output), "
                                "batch 10000 per GPU, seed 1", "batch_per_gpu": BATCH, "parallelism": "replicas x%d" % world,
                    "l2": "256 MiB written between timed steps (inputs fit in L2)", "popc_variant": args.variant,
+                   "operand_bits": args.operand_bits,
                    "engine": {0: "auto (tensor-core int8 for the large layers)", 1: "CUDA-core XOR-popcount", 2: "tensor"}[args.engine]},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": BATCH * SIZES[0], "d2h_bytes_per_step": BATCH * SIZES[-1] * 4,
                 "ms_per_step": e2e_total_ms / args.steps, "ms_median": statistics.median(e2e_times), "ms_min": min(e2e_times),
                 "ms_max": max(e2e_times), "warmup_steps": 100 * e2e_warm_blocks + max(args.warmup, 3)},
         "gpu_launches": launches_per_step * args.steps,
-        "roofline": ({"bound": "tensor", "kernel": "bnn_binary_dense 10000x4096x4096 on the tensor engine (k_expand_s8 x2 + k_umma_i8, "
-                                                    "timed as one call)", "achieved": dense_ach, "peak": tensor_peak, "unit": "TFLOP/s",
-                      "frac": dense_ach / tensor_peak, "traffic": 60967424,
-                      "peak_kind": "int8 ops (2 per MAC); peak = 2 x measured bf16 burst %.1f TFLOP/s (nominal int8:bf16 ratio), "
-                                   "%s" % (bf16_peak, "of measured" if peaks else "of fallback"), "ms_per_launch": dense_ms}
+        "roofline": ({"bound": "tensor", "kernel": "bnn_binary_dense 10000x4096x4096 on the tensor engine (two operand expansion "
+                                                    "kernels + k_umma_i8<%s>, timed as one call)"
+                                                    % ("192>, tcgen05 kind::mxf4 on e2m1 nibbles" if args.operand_bits == 4 else "256>, tcgen05 kind::i8"),
+                      "achieved": dense_ach, "peak": tensor_peak, "unit": "TFLOP/s",
+                      "frac": dense_ach / tensor_peak, "traffic": 28951552 if args.operand_bits == 4 else 60967424,
+                      "peak_kind": "2 ops per MAC; peak = %.0f x measured bf16 burst %.1f TFLOP/s (nominal %s:bf16 ratio), %s"
+                                   % (peak_ratio, bf16_peak, "fp4" if args.operand_bits == 4 else "int8",
+                                      "of measured" if peaks else "of fallback"), "ms_per_launch": dense_ms}
                      if tensor_step else
                      {"bound": "alu", "kernel": "k_bit_tile (fused binary dense 10000x4096x4096)", "achieved": dense_ach,
                       "peak": popc_peak_tbitops, "unit": "Tbit-op/s", "frac": dense_ach / popc_peak_tbitops, "traffic": 7299840,
