@@ -38,7 +38,7 @@ template <int BN> struct Cfg {
     // two accumulator buffers of BN columns; the 4-bit configuration (BN = 192) also keeps 32 columns of scale factors
     static constexpr uint32_t TMEM_COLS = (BN == 192) ? 512 : 2 * BN;
 };
-constexpr int STAGES_MAX = 6;
+constexpr int STAGES_MAX = 7;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // a wait gives up after 2 s of wall clock
 
 __device__ int g_umma_error;                    // 0 = fine; otherwise a code saying which wait gave up
@@ -456,8 +456,10 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
 // both halves of B.  CTA 0 of the pair issues the MMAs; completion of every CTA's TMA loads is counted on CTA 0's
 // "full" barrier, stages and accumulators are released to both CTAs with multicast tcgen05.commit, and the
 // epilogue warps of both CTAs hand their accumulator buffer back by arriving on CTA 0's barrier.
-constexpr int STAGES2 = 6;
-constexpr uint32_t STAGE2_BYTES = 2 * A_BYTES;           // A half-tile + B half-tile, 128 rows x 128 bytes each
+template <int BN> struct Cfg2 {
+    static constexpr uint32_t STAGE_BYTES = A_BYTES + (BN / 2) * BK;    // own A rows + own half of the tile's B rows
+    static constexpr int STAGES = (BN == 256) ? 6 : 7;                  // 192 / 196 KB
+};
 constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;              // clears the CTA-rank bit of a shared::cluster address -> CTA 0 of the pair
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -494,9 +496,21 @@ __device__ __forceinline__ void mbar_arrive_cta0(uint32_t bar) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
 }
 
+// 4-bit form of the pair instruction (see umma_mxf4).
+__device__ __forceinline__ void umma_mxf4_2sm(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate,
+                                              uint32_t tmem_sf) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%5], p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(tmem_sf) : "memory");
+}
+
+template <int BN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const UmmaArgs p) {
-    constexpr int BN = 256;
+    constexpr int STAGES2 = Cfg2<BN>::STAGES;
+    constexpr uint32_t STAGE2_BYTES = Cfg2<BN>::STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     Control *ctl = reinterpret_cast<Control *>(tiles + STAGES2 * STAGE2_BYTES);
@@ -515,7 +529,7 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(2u * BN) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(Cfg<BN>::TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -523,6 +537,21 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     cluster_sync_all();                                     // both CTAs' barriers exist before anyone signals them
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = ctl->tmem_base;
+
+    if (BN == 192) {
+        // 4-bit engine: unit block scales (byte 0x7f) in this CTA's scale-factor columns; the leader's MMAs read the
+        // columns of both CTAs, so the pair synchronises once more before the first one is issued
+        if (warp >= 2 && warp < 6) {
+            const uint32_t v = 0x7f7f7f7fu;
+            asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1};"
+                         ::"r"(tmem_base + SF_COL + ((uint32_t)(32 * (warp & 3)) << 16)), "r"(v) : "memory");
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        cluster_sync_all();
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    }
 
     if (warp == 0) {
         // ---------------- TMA producer (both CTAs): own A rows, own half of the tile's B rows
@@ -548,7 +577,9 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
             uint32_t it = 0, tc = 0;
             bool ok = true;
             // the host's descriptor carries M = 128 in bits [24,29); the pair multiplies M = 256
-            const uint32_t idesc = (p.idesc & ~(0x1fu << 24)) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+            const uint32_t idesc = (BN == 192)
+                ? ((1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (1u << 23) | ((uint32_t)((2 * BM) >> 4) << 24))
+                : ((p.idesc & ~(0x1fu << 24)) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24));
             for (int64_t t = pair; t < ntiles && ok; t += npairs, ++tc) {
                 const uint32_t buf = tc & 1;
                 if (tc >= ACC_BUFS && !mbar_wait(smem_u32(&ctl->acc_empty[buf]), ((tc / ACC_BUFS) - 1) & 1)) { fail(ctl, 14); ok = false; break; }
@@ -561,8 +592,10 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                     const uint64_t adesc = smem_desc_sw128(smem_u32(tiles + s * STAGE2_BYTES));
                     const uint64_t bdesc = smem_desc_sw128(smem_u32(tiles + s * STAGE2_BYTES + A_BYTES));
 #pragma unroll
-                    for (int k = 0; k < BK / 32; ++k)
-                        umma_i8_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u);
+                    for (int k = 0; k < BK / 32; ++k) {
+                        if (BN == 192) umma_mxf4_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u, tmem_base + SF_COL);
+                        else umma_i8_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u);
+                    }
                     umma_commit_2sm(smem_u32(&ctl->empty[s]));
                 }
                 umma_commit_2sm(smem_u32(&ctl->acc_full[buf]));
@@ -591,7 +624,7 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     cluster_sync_all();                                     // nobody leaves while the peer may still read its shared memory
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2u * BN) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(Cfg<BN>::TMEM_COLS) : "memory");
     }
 }
 
@@ -727,8 +760,9 @@ static int umma_tile_n(int64_t N, int64_t M = 0, int sm_count = 0) {
     if (M > 0 && ((M + BM - 1) / BM) * ((N + 255) / 256) * 2 <= sm_count) return 128;
     return 256;
 }
-static size_t umma2_smem_bytes() { return (size_t)STAGES2 * STAGE2_BYTES + sizeof(Control) + 1024; }
+template <int BN> static size_t umma2_smem_bytes() { return (size_t)Cfg2<BN>::STAGES * Cfg2<BN>::STAGE_BYTES + sizeof(Control) + 1024; }
 // Pairs of CTAs that can be resident at once for the two-SM kernel on this device (0 = cannot be used).
+template <int BN>
 static int umma2_max_pairs(bnn_ctx *ctx) {
     static std::mutex m;
     static int cached[64];
@@ -737,16 +771,16 @@ static int umma2_max_pairs(bnn_ctx *ctx) {
     if (ctx->device < 0 || ctx->device >= 64) return 0;
     if (!have[ctx->device]) {
         int pairs = 0;
-        if (cudaFuncSetAttribute(k_umma_i8_2sm, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma2_smem_bytes()) == cudaSuccess) {
+        if (cudaFuncSetAttribute(k_umma_i8_2sm<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma2_smem_bytes<BN>()) == cudaSuccess) {
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3(2 * ctx->sm_count, 1, 1);
             cfg.blockDim = dim3(NTHREADS, 1, 1);
-            cfg.dynamicSmemBytes = umma2_smem_bytes();
+            cfg.dynamicSmemBytes = umma2_smem_bytes<BN>();
             cudaLaunchAttribute attr;
             attr.id = cudaLaunchAttributeClusterDimension;
             attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
             cfg.attrs = &attr; cfg.numAttrs = 1;
-            if (cudaOccupancyMaxActiveClusters(&pairs, k_umma_i8_2sm, &cfg) != cudaSuccess) pairs = 0;
+            if (cudaOccupancyMaxActiveClusters(&pairs, k_umma_i8_2sm<BN>, &cfg) != cudaSuccess) pairs = 0;
         }
         (void)cudaGetLastError();
         cached[ctx->device] = pairs;
@@ -804,13 +838,22 @@ int bnn_umma_gemm_f4(bnn_ctx *ctx, const uint8_t *A4, int64_t lda4, const uint8_
     if (M > 0x7fffffff || N > 0x7fffffff || K <= 0 || K > (1 << 24)) return BNN_ERR_INVALID_ARG;
     CUtensorMap mapA, mapB;
     const int64_t kb = (((K + 1) / 2 + 15) / 16) * 16;      // extent along K in bytes
+    const bool pair_want = ctx->pair_mode == 2 || (ctx->pair_mode == 0 && (double)M * (double)N >= 67108864.0);
+    const int pairs = (M >= 512 && pair_want) ? umma2_max_pairs<192>(ctx) : 0;
     if (int st = make_map(ctx, &mapA, A4, M, kb <= lda4 ? kb : lda4, lda4, BM)) return st;
-    if (int st = make_map(ctx, &mapB, B4, N, kb <= ldb4 ? kb : ldb4, ldb4, 192)) return st;
+    if (int st = make_map(ctx, &mapB, B4, N, kb <= ldb4 ? kb : ldb4, ldb4, pairs > 0 ? 96 : 192)) return st;
     UmmaArgs a{};
     a.M = M; a.N = N;
     a.k_iters = (int)((K + 2 * BK - 1) / (2 * BK));          // 256 values per 128-byte K step
     a.C = C; a.ldc = ldc; a.out = out; a.ldo = ldo; a.thr = thr; a.flip = flip;
     a.out8 = reinterpret_cast<int8_t *>(out4); a.ldo8 = ldo4; a.out_f4 = 1;
+    if (pairs > 0) {
+        if (int st = umma_prepare(ctx)) return st;
+        const int64_t tiles2 = ((M + 2 * BM - 1) / (2 * BM)) * ((N + 191) / 192);
+        const int64_t use = tiles2 < pairs ? tiles2 : pairs;
+        k_umma_i8_2sm<192><<<(unsigned)(2 * use), NTHREADS, umma2_smem_bytes<192>(), ctx->stream>>>(mapA, mapB, a);
+        return bnn_check_launch(ctx);
+    }
     return umma_launch(ctx, mapA, mapB, a, 192);
 }
 
@@ -833,7 +876,7 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
     // (auto: only where it measured faster -- outputs of 2^26 elements and more, e.g. 8192 x 8192 or 65536 x 4096)
     const bool pair_shape = bn == 256 && M >= 512 && !pool;
     const bool pair_want = ctx->pair_mode == 2 || (ctx->pair_mode == 0 && (double)M * (double)N >= 67108864.0);
-    const int pairs = (pair_shape && pair_want) ? umma2_max_pairs(ctx) : 0;
+    const int pairs = (pair_shape && pair_want) ? umma2_max_pairs<256>(ctx) : 0;
     if (int st = make_map(ctx, &mapA, A8, M, kb <= lda8 ? kb : lda8, lda8, BM)) return st;
     if (int st = make_map(ctx, &mapB, B8, N, kb <= ldb8 ? kb : ldb8, ldb8, pairs > 0 ? 128 : bn)) return st;
     UmmaArgs a{};
@@ -845,7 +888,7 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
     if (pairs > 0) {
         const int64_t tiles2 = ((M + 2 * BM - 1) / (2 * BM)) * ((N + 255) / 256);
         const int64_t use = tiles2 < pairs ? tiles2 : pairs;
-        k_umma_i8_2sm<<<(unsigned)(2 * use), NTHREADS, umma2_smem_bytes(), ctx->stream>>>(mapA, mapB, a);
+        k_umma_i8_2sm<256><<<(unsigned)(2 * use), NTHREADS, umma2_smem_bytes<256>(), ctx->stream>>>(mapA, mapB, a);
         return bnn_check_launch(ctx);
     }
     return umma_launch(ctx, mapA, mapB, a, bn);

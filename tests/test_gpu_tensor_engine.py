@@ -12,7 +12,8 @@ from util import np_pack_pm1, np_unpack_pm1, padding_is_zero
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module", params=[(2, 8), (1, 8), (1, 4)], ids=["pairs-bytes", "single-bytes", "nibbles"])
+@pytest.fixture(scope="module", params=[(2, 8), (1, 8), (1, 4), (2, 4)],
+                ids=["pairs-bytes", "single-bytes", "nibbles", "pairs-nibbles"])
 def ctx(request):
     """Tensor engine forced: byte operands with CTA pairs (cta_group::2) wherever the kernel allows, byte operands on
     the single-SM kernel, and 4-bit (e2m1) operands for the +-1 x +-1 products."""
