@@ -6,11 +6,13 @@
 //   512 bit-MACs per clock per SM), so for large shapes the packed operands are expanded to one signed byte
 //   per value (a streaming pass) and multiplied with tcgen05.mma kind::i8.  Results are the same integers.
 //
-// Kernel k_umma_i8 (persistent, one CTA per SM walking 128 x 256 output tiles, 192 threads):
+// Kernel k_umma_i8 (persistent, one CTA per SM walking 128 x 256 output tiles, 352 threads):
 //   warp 0    TMA producer: cp.async.bulk.tensor 2-D loads of 128-byte-wide K slices (128B swizzle) of both
 //             operands into a 4-stage shared-memory ring, completion on mbarriers;
 //   warp 1    allocates all 512 TMEM columns (two accumulator buffers), then one lane issues tcgen05.mma
 //             (M=128, N=256, K=32) four times per stage and releases the stage with tcgen05.commit;
+//   warp 10   second MMA issuer: takes the odd K steps of every tile (issuing a step costs one thread more clocks
+//             than the tensor core needs to run it; two issuing warps keep the tensor pipe full);
 //   warps 2-9 epilogue (two warps per TMEM lane quadrant, each half of the columns): tcgen05.ld of the int32
 //             accumulators (each thread owns one output row, 32 columns at a time, the next chunk in flight while
 //             the current one is processed), then either int32 stores, or the BatchNorm-folded threshold + Sign + repack to one
@@ -28,7 +30,8 @@ constexpr int BN_MAX = 256;                     // tile width: 256, or 128 for n
 constexpr uint32_t SF_COL = 480;                // 4-bit engine: first of the 32 TMEM columns that hold the scale factors
 constexpr int EPI_WARPS = 8;                    // two per TMEM lane quadrant, each takes half of the tile's columns
 constexpr int EPI_THREADS = EPI_WARPS * 32;
-constexpr int NTHREADS = 64 + EPI_THREADS;
+constexpr int MMA_WARP_B = 2 + EPI_WARPS;       // the second MMA-issuing warp (the first is warp 1)
+constexpr int NTHREADS = 96 + EPI_THREADS;
 constexpr uint32_t A_BYTES = BM * BK;
 constexpr int ACC_BUFS = 2;
 template <int BN> struct Cfg {
@@ -153,9 +156,10 @@ struct __align__(8) Control {
     uint64_t empty[STAGES_MAX];
     uint64_t acc_full[ACC_BUFS];
     uint64_t acc_empty[ACC_BUFS];
+    uint64_t started[ACC_BUFS];            // the tile's first (overwriting) K step has completed
     uint32_t tmem_base;
     uint32_t failed;
-    int32_t thr[ACC_BUFS][BN_MAX];
+    __align__(16) int32_t thr[ACC_BUFS][BN_MAX];   // staged thresholds: clamped int32, or float bits on the 4-bit engine
     uint32_t flip[ACC_BUFS][BN_MAX / 32];
     uint32_t poolw[BM][BN_MAX / 32 + 1];   // convolution with pooling: the sign words of every pixel of the tile
 };
@@ -170,10 +174,10 @@ __device__ __forceinline__ void fail(Control *ctl, int code) {
 
 // 8 sign bits -> 8 e2m1 nibbles (+1.0 = 0x2, -1.0 = 0xa); bit i lands in nibble i.
 __device__ __forceinline__ uint32_t nibbles_of_byte(uint32_t x) {
-    uint32_t t = (x | (x << 12)) & 0x000f000fu;
-    t = (t | (t << 6)) & 0x03030303u;
-    t = (t | (t << 3)) & 0x11111111u;
-    return ((t ^ 0x11111111u) << 3) | 0x22222222u;
+    // bit pairs -> selector nibbles 0..3, then one byte permute out of the four possible nibble pairs
+    uint32_t t = (x | (x << 4)) & 0x0f0fu;
+    t = (t | (t << 2)) & 0x3333u;
+    return __byte_perm(0x222aa2aau, 0u, t);       // pair 00 -> 0xaa, 01 -> 0xa2, 10 -> 0x2a, 11 -> 0x22
 }
 // The signs of 32 consecutive outputs of row `orow` (bit j of `word` = column col0 + j) in the next layer's operand
 // format: one signed byte per value, or one e2m1 nibble per value.  Positions at or beyond N are written as 0.
@@ -222,7 +226,13 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
     // thresholds of this column block; tiles that share it with the buffer's previous tile skip the staging
     const bool restage = p.out && staged_n0[buf] != n0;
     if (restage) {
-        for (int e = et; e < BN; e += EPI_THREADS) ctl->thr[buf][e] = (n0 + e < p.N) ? p.thr[n0 + e] : 0x7fffffff;
+        for (int e = et; e < BN; e += EPI_THREADS) {
+            const int32_t t = (n0 + e < p.N) ? p.thr[n0 + e] : 0x7fffffff;
+            // The comparison is the sign of (accumulator - threshold).  Accumulators stay below 2^30 in magnitude
+            // (2^24 on the 4-bit engine, where they are float32), so thresholds clamp to that range unchanged in meaning.
+            if (BN == 192) ctl->thr[buf][e] = __float_as_int(t > (1 << 24) ? 3.0e7f : (t < -(1 << 24) ? -3.0e7f : (float)t));
+            else ctl->thr[buf][e] = max(min(t, 1 << 30), -(1 << 30));
+        }
         if (et < BN / 32) {
             const int64_t w = (n0 >> 5) + et;
             ctl->flip[buf][et] = (p.flip && w * 32 < p.N) ? p.flip[w] : 0u;
@@ -240,8 +250,8 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
         uint32_t ra[32], rb[32];
         const int c_first = half * CPW;
         if (n0 + 32 * c_first < p.N) { tmem_ld32(tbase + (uint32_t)(32 * c_first), ra); tmem_ld_wait(ra); }
-#pragma unroll 1
-        for (int cc = 0; cc < CPW; ++cc) {
+#pragma unroll
+        for (int cc = 0; cc < CPW; ++cc) {               // unrolled: both register buffers are addressed statically
             const int c = c_first + cc;
             const int64_t col0 = n0 + 32 * c;
             if (col0 >= p.N) break;                      // uniform over the warp
@@ -249,12 +259,36 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
             uint32_t (&r)[32] = (cc & 1) ? rb : ra;
             uint32_t (&rn)[32] = (cc & 1) ? ra : rb;
             if (more) tmem_ld32(tbase + (uint32_t)(32 * (c + 1)), rn);
-            if (BN == 192) {   // the 4-bit engine accumulates in float32: exact integers, converted once
-#pragma unroll
-                for (int j = 0; j < 32; ++j) r[j] = (uint32_t)(int32_t)__uint_as_float(r[j]);
-            }
             if (row < p.M) {
+                if (p.out) {
+                    // bit j of the word = (acc[j] >= thr[j]) = NOT sign(acc[j] - thr[j]); the sign bits are shifted
+                    // into four independent 8-bit chains (funnel shift: one instruction per column after the subtract)
+                    const int4 *tp = reinterpret_cast<const int4 *>(&ctl->thr[buf][32 * c]);
+                    uint32_t w4[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+                    for (int g = 7; g >= 0; --g) {
+                        const int4 t = tp[g];
+                        const int tv[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+                        for (int i = 3; i >= 0; --i) {
+                            const int j = 4 * g + i;
+                            const uint32_t d = (BN == 192) ? __float_as_uint(__uint_as_float(r[j]) - __int_as_float(tv[i]))
+                                                           : (uint32_t)((int32_t)r[j] - tv[i]);
+                            w4[j >> 3] = __funnelshift_l(d, w4[j >> 3], 1);
+                        }
+                    }
+                    const uint32_t lt = __byte_perm(__byte_perm(w4[0], w4[1], 0x0040), __byte_perm(w4[2], w4[3], 0x0040), 0x5410);
+                    uint32_t word = ~lt ^ ctl->flip[buf][c];
+                    if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;      // columns beyond N stay 0
+                    if (p.pool) ctl->poolw[32 * q + lane][c] = word ^ ctl->flip[buf][c];   // un-flipped (dot >= thr) bits
+                    else p.out[row * p.ldo + (col0 >> 5)] = word;
+                    if (p.out8 && !p.pool) store_signs(p, word, row, col0);
+                }
                 if (p.C) {
+                    if (BN == 192) {   // the 4-bit engine accumulates in float32: exact integers
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) r[j] = (uint32_t)(int32_t)__uint_as_float(r[j]);
+                    }
                     int32_t *dst = p.C + row * p.ldc + col0;
                     if (col0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
 #pragma unroll
@@ -265,16 +299,6 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                         for (int j = 0; j < 32; ++j)
                             if (col0 + j < p.N) dst[j] = (int32_t)r[j];
                     }
-                }
-                if (p.out) {
-                    uint32_t word = 0u;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) word |= (uint32_t)((int32_t)r[j] >= ctl->thr[buf][32 * c + j]) << j;
-                    word ^= ctl->flip[buf][c];
-                    if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;      // columns beyond N stay 0
-                    if (p.pool) ctl->poolw[32 * q + lane][c] = word ^ ctl->flip[buf][c];   // un-flipped (dot >= thr) bits
-                    else p.out[row * p.ldo + (col0 >> 5)] = word;
-                    if (p.out8 && !p.pool) store_signs(p, word, row, col0);
                 }
             }
             if (more) tmem_ld_wait(rn);
@@ -336,7 +360,11 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
-        for (int b = 0; b < ACC_BUFS; ++b) { mbar_init(smem_u32(&ctl->acc_full[b]), 1); mbar_init(smem_u32(&ctl->acc_empty[b]), EPI_WARPS); }
+        for (int b = 0; b < ACC_BUFS; ++b) {
+            mbar_init(smem_u32(&ctl->acc_full[b]), 2);          // one commit from each MMA-issuing warp
+            mbar_init(smem_u32(&ctl->acc_empty[b]), EPI_WARPS);
+            mbar_init(smem_u32(&ctl->started[b]), 1);
+        }
         ctl->failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -391,9 +419,14 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                 }
             }
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer
+    } else if (warp == 1 || warp == MMA_WARP_B) {
+        // ---------------- MMA issuers.  Issuing one K step (wait, four instructions, commit) costs the issuing thread
+        // more clocks than the tensor core needs to execute it, so two warps on different schedulers share the work:
+        // warp 1 takes the even K steps of every tile, the other warp the odd ones.  All products are exact integers,
+        // so the order in which the two streams reach the accumulator does not matter, except that the overwriting
+        // first step must be there first: the second warp waits for its completion once per tile.
         if (lane == 0) {
+            const int w = (warp == 1) ? 0 : 1;
             uint32_t it = 0, tc = 0;
             bool ok = true;
             for (int64_t t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++tc) {
@@ -402,6 +435,8 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tmem_d = tmem_base + buf * BN;
                 for (int kit = 0; kit < p.k_iters; ++kit, ++it) {
+                    if ((kit & 1) != w) continue;
+                    if (kit == 1 && !mbar_wait(smem_u32(&ctl->started[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 5); ok = false; break; }
                     const uint32_t s = it % STAGES;
                     if (!mbar_wait(smem_u32(&ctl->full[s]), (it / STAGES) & 1)) { fail(ctl, 2); ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -417,11 +452,12 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                             umma_i8(tmem_d, adesc + 2 * k, bdesc + 2 * k, p.idesc | ((uint32_t)(BN >> 3) << 17), (kit > 0 || k > 0) ? 1u : 0u);
                     }
                     umma_commit(smem_u32(&ctl->empty[s]));      // stage may be refilled once these MMAs have read it
+                    if (kit == 0) umma_commit(smem_u32(&ctl->started[buf]));
                 }
-                umma_commit(smem_u32(&ctl->acc_full[buf]));     // accumulators of this tile complete (also after a failure)
+                umma_commit(smem_u32(&ctl->acc_full[buf]));     // this warp's share of the tile complete (also after a failure)
             }
         }
-    } else {
+    } else if (warp < 2 + EPI_WARPS) {
         // ---------------- epilogue: warps 2..9; warp w may only touch TMEM lanes 32*(w%4) .. +31, so two warps share
         // each lane quadrant and split the tile's columns between them
         const int q = warp & 3;
@@ -489,6 +525,10 @@ __device__ __forceinline__ void umma_commit_2sm(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                  ::"r"(bar), "h"(mask) : "memory");
 }
+// The same for a barrier of the issuing CTA alone.
+__device__ __forceinline__ void umma_commit_2sm_local(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
 // Arrive on the barrier at the same offset in CTA 0 of the cluster.
 __device__ __forceinline__ void mbar_arrive_cta0(uint32_t bar) {
     uint32_t remote;
@@ -524,7 +564,11 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES2; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
-        for (int b = 0; b < ACC_BUFS; ++b) { mbar_init(smem_u32(&ctl->acc_full[b]), 1); mbar_init(smem_u32(&ctl->acc_empty[b]), 2 * EPI_WARPS); }
+        for (int b = 0; b < ACC_BUFS; ++b) {
+            mbar_init(smem_u32(&ctl->acc_full[b]), 2);          // one multicast commit from each of the leader's MMA warps
+            mbar_init(smem_u32(&ctl->acc_empty[b]), 2 * EPI_WARPS);
+            mbar_init(smem_u32(&ctl->started[b]), 1);
+        }
         ctl->failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -571,9 +615,10 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                 }
             }
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer: the leader CTA only, for both tensor cores
+    } else if (warp == 1 || warp == MMA_WARP_B) {
+        // ---------------- MMA issuers: two warps of the leader CTA only (even / odd K steps), for both tensor cores
         if (lane == 0 && rank == 0) {
+            const int w = (warp == 1) ? 0 : 1;
             uint32_t it = 0, tc = 0;
             bool ok = true;
             // the host's descriptor carries M = 128 in bits [24,29); the pair multiplies M = 256
@@ -586,6 +631,8 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tmem_d = tmem_base + buf * BN;
                 for (int kit = 0; kit < p.k_iters; ++kit, ++it) {
+                    if ((kit & 1) != w) continue;
+                    if (kit == 1 && !mbar_wait(smem_u32(&ctl->started[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 15); ok = false; break; }
                     const uint32_t s = it % STAGES2;
                     if (!mbar_wait(smem_u32(&ctl->full[s]), (it / STAGES2) & 1)) { fail(ctl, 12); ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -597,11 +644,12 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                         else umma_i8_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u);
                     }
                     umma_commit_2sm(smem_u32(&ctl->empty[s]));
+                    if (kit == 0) umma_commit_2sm_local(smem_u32(&ctl->started[buf]));
                 }
                 umma_commit_2sm(smem_u32(&ctl->acc_full[buf]));
             }
         }
-    } else {
+    } else if (warp < 2 + EPI_WARPS) {
         // ---------------- epilogue (both CTAs): this CTA's 128 rows of the pair's tile
         const int q = warp & 3;
         const int half = (warp - 2) >> 2;
@@ -869,6 +917,7 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
     if ((lda8 & 15) || (ldb8 & 15) || !bnn_aligned16(A8) || !bnn_aligned16(B8)) return BNN_ERR_ALIGNMENT;
     if (M > 0x7fffffff || N > 0x7fffffff) return BNN_ERR_INVALID_ARG;
     if (K <= 0) return BNN_ERR_INVALID_ARG;      // callers route the empty product elsewhere
+    if (K > (a_unsigned ? (1 << 22) : (1 << 30)) - 1) return BNN_ERR_INVALID_ARG;   // |accumulator| < 2^30 (thresholding subtracts)
     CUtensorMap mapA, mapB;
     const int bn = umma_tile_n(N, M, ctx->sm_count);
     const int64_t kb = ((K + 15) / 16) * 16;      // extent along K in bytes; beyond it TMA fills zeros
