@@ -30,8 +30,9 @@ constexpr int BN_MAX = 256;                     // tile width: 256, or 128 for n
 constexpr uint32_t SF_COL = 480;                // 4-bit engine: first of the 32 TMEM columns that hold the scale factors
 constexpr int EPI_WARPS = 8;                    // two per TMEM lane quadrant, each takes half of the tile's columns
 constexpr int EPI_THREADS = EPI_WARPS * 32;
-constexpr int MMA_WARP_B = 2 + EPI_WARPS;       // the second MMA-issuing warp (the first is warp 1)
-constexpr int NTHREADS = 96 + EPI_THREADS;
+constexpr int N_ISSUE = 2;                      // MMA-issuing warps: warp 1 and the warps from MMA_WARP_B on
+constexpr int MMA_WARP_B = 2 + EPI_WARPS;
+constexpr int NTHREADS = 64 + EPI_THREADS + 32 * (N_ISSUE - 1);
 constexpr uint32_t A_BYTES = BM * BK;
 constexpr int ACC_BUFS = 2;
 template <int BN> struct Cfg {
@@ -151,7 +152,7 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
         :: "memory");
 }
 
-struct __align__(8) Control {
+struct __align__(16) Control {
     uint64_t full[STAGES_MAX];
     uint64_t empty[STAGES_MAX];
     uint64_t acc_full[ACC_BUFS];
@@ -361,7 +362,7 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
         for (int b = 0; b < ACC_BUFS; ++b) {
-            mbar_init(smem_u32(&ctl->acc_full[b]), 2);          // one commit from each MMA-issuing warp
+            mbar_init(smem_u32(&ctl->acc_full[b]), N_ISSUE);    // one commit from each MMA-issuing warp
             mbar_init(smem_u32(&ctl->acc_empty[b]), EPI_WARPS);
             mbar_init(smem_u32(&ctl->started[b]), 1);
         }
@@ -419,40 +420,43 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                 }
             }
         }
-    } else if (warp == 1 || warp == MMA_WARP_B) {
+    } else if (warp == 1 || warp >= MMA_WARP_B) {
         // ---------------- MMA issuers.  Issuing one K step (wait, four instructions, commit) costs the issuing thread
-        // more clocks than the tensor core needs to execute it, so two warps on different schedulers share the work:
-        // warp 1 takes the even K steps of every tile, the other warp the odd ones.  All products are exact integers,
-        // so the order in which the two streams reach the accumulator does not matter, except that the overwriting
-        // first step must be there first: the second warp waits for its completion once per tile.
+        // more clocks than the tensor core needs to execute it, so N_ISSUE warps on different schedulers share the work
+        // round-robin over the K steps of every tile.  All products are exact integers, so the order in which the
+        // streams reach the accumulator does not matter, except that the overwriting first step must be there
+        // first: the other warps wait for its completion once per tile.
         if (lane == 0) {
-            const int w = (warp == 1) ? 0 : 1;
-            uint32_t it = 0, tc = 0;
+            const int w = (warp == 1) ? 0 : warp - MMA_WARP_B + 1;   // this warp takes K steps w, w + N_ISSUE, ...
+            // e2m1 x e2m1 (format 1), UE8M0 scales (bit 23) on the 4-bit engine; N >> 3 at bit 17, M >> 4 at bit 24
+            const uint32_t idesc = (BN == 192)
+                ? ((1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (1u << 23) | ((uint32_t)(BM >> 4) << 24))
+                : (p.idesc | ((uint32_t)(BN >> 3) << 17));
+            const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+            const uint64_t adesc0 = smem_desc_sw128(smem_u32(tiles)), bdesc0 = smem_desc_sw128(smem_u32(tiles + A_BYTES));
+            uint32_t it0 = 0, tc = 0;                    // it0: K steps of this CTA before the current tile
             bool ok = true;
-            for (int64_t t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++tc) {
+            for (int64_t t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++tc, it0 += (uint32_t)p.k_iters) {
                 const uint32_t buf = tc & 1;
                 if (tc >= ACC_BUFS && !mbar_wait(smem_u32(&ctl->acc_empty[buf]), ((tc / ACC_BUFS) - 1) & 1)) { fail(ctl, 4); ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tmem_d = tmem_base + buf * BN;
-                for (int kit = 0; kit < p.k_iters; ++kit, ++it) {
-                    if ((kit & 1) != w) continue;
-                    if (kit == 1 && !mbar_wait(smem_u32(&ctl->started[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 5); ok = false; break; }
-                    const uint32_t s = it % STAGES;
-                    if (!mbar_wait(smem_u32(&ctl->full[s]), (it / STAGES) & 1)) { fail(ctl, 2); ok = false; break; }
+                uint32_t s = (it0 + w) % STAGES, par = ((it0 + w) / STAGES) & 1;   // ring slot and phase of this warp's next step
+                for (int kit = w; kit < p.k_iters; kit += N_ISSUE) {
+                    if (w > 0 && kit == w && !mbar_wait(smem_u32(&ctl->started[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 5); ok = false; break; }
+                    if (!mbar_wait(full0 + 8 * s, par)) { fail(ctl, 2); ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint64_t adesc = smem_desc_sw128(smem_u32(tiles + s * STAGE_BYTES));
-                    const uint64_t bdesc = smem_desc_sw128(smem_u32(tiles + s * STAGE_BYTES + A_BYTES));
+                    const uint64_t adesc = adesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
+                    const uint64_t bdesc = bdesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k) {   // 32 bytes of K per instruction: start address advances by 32 B (>> 4 = 2)
-                        if (BN == 192)   // e2m1 x e2m1 (format 1), UE8M0 scales (bit 23), N >> 3 at bit 17, M >> 4 at bit 24
-                            umma_mxf4(tmem_d, adesc + 2 * k, bdesc + 2 * k,
-                                      (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (1u << 23) | ((uint32_t)(BM >> 4) << 24),
-                                      (kit > 0 || k > 0) ? 1u : 0u, tmem_base + SF_COL);
-                        else
-                            umma_i8(tmem_d, adesc + 2 * k, bdesc + 2 * k, p.idesc | ((uint32_t)(BN >> 3) << 17), (kit > 0 || k > 0) ? 1u : 0u);
+                        if (BN == 192) umma_mxf4(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u, tmem_base + SF_COL);
+                        else umma_i8(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u);
                     }
-                    umma_commit(smem_u32(&ctl->empty[s]));      // stage may be refilled once these MMAs have read it
+                    umma_commit(empty0 + 8 * s);                // stage may be refilled once these MMAs have read it
                     if (kit == 0) umma_commit(smem_u32(&ctl->started[buf]));
+                    s += N_ISSUE;
+                    if (s >= (uint32_t)STAGES) { s -= STAGES; par ^= 1u; }
                 }
                 umma_commit(smem_u32(&ctl->acc_full[buf]));     // this warp's share of the tile complete (also after a failure)
             }
@@ -565,7 +569,7 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES2; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
         for (int b = 0; b < ACC_BUFS; ++b) {
-            mbar_init(smem_u32(&ctl->acc_full[b]), 2);          // one multicast commit from each of the leader's MMA warps
+            mbar_init(smem_u32(&ctl->acc_full[b]), N_ISSUE);    // one multicast commit from each of the leader's MMA warps
             mbar_init(smem_u32(&ctl->acc_empty[b]), 2 * EPI_WARPS);
             mbar_init(smem_u32(&ctl->started[b]), 1);
         }
@@ -615,36 +619,39 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                 }
             }
         }
-    } else if (warp == 1 || warp == MMA_WARP_B) {
+    } else if (warp == 1 || warp >= MMA_WARP_B) {
         // ---------------- MMA issuers: two warps of the leader CTA only (even / odd K steps), for both tensor cores
         if (lane == 0 && rank == 0) {
-            const int w = (warp == 1) ? 0 : 1;
-            uint32_t it = 0, tc = 0;
-            bool ok = true;
+            const int w = (warp == 1) ? 0 : warp - MMA_WARP_B + 1;
             // the host's descriptor carries M = 128 in bits [24,29); the pair multiplies M = 256
             const uint32_t idesc = (BN == 192)
                 ? ((1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (1u << 23) | ((uint32_t)((2 * BM) >> 4) << 24))
                 : ((p.idesc & ~(0x1fu << 24)) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24));
-            for (int64_t t = pair; t < ntiles && ok; t += npairs, ++tc) {
+            const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+            const uint64_t adesc0 = smem_desc_sw128(smem_u32(tiles)), bdesc0 = smem_desc_sw128(smem_u32(tiles + A_BYTES));
+            uint32_t it0 = 0, tc = 0;
+            bool ok = true;
+            for (int64_t t = pair; t < ntiles && ok; t += npairs, ++tc, it0 += (uint32_t)p.k_iters) {
                 const uint32_t buf = tc & 1;
                 if (tc >= ACC_BUFS && !mbar_wait(smem_u32(&ctl->acc_empty[buf]), ((tc / ACC_BUFS) - 1) & 1)) { fail(ctl, 14); ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tmem_d = tmem_base + buf * BN;
-                for (int kit = 0; kit < p.k_iters; ++kit, ++it) {
-                    if ((kit & 1) != w) continue;
-                    if (kit == 1 && !mbar_wait(smem_u32(&ctl->started[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 15); ok = false; break; }
-                    const uint32_t s = it % STAGES2;
-                    if (!mbar_wait(smem_u32(&ctl->full[s]), (it / STAGES2) & 1)) { fail(ctl, 12); ok = false; break; }
+                uint32_t s = (it0 + w) % STAGES2, par = ((it0 + w) / STAGES2) & 1;
+                for (int kit = w; kit < p.k_iters; kit += N_ISSUE) {
+                    if (w > 0 && kit == w && !mbar_wait(smem_u32(&ctl->started[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 15); ok = false; break; }
+                    if (!mbar_wait(full0 + 8 * s, par)) { fail(ctl, 12); ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint64_t adesc = smem_desc_sw128(smem_u32(tiles + s * STAGE2_BYTES));
-                    const uint64_t bdesc = smem_desc_sw128(smem_u32(tiles + s * STAGE2_BYTES + A_BYTES));
+                    const uint64_t adesc = adesc0 + (uint64_t)(s * (STAGE2_BYTES >> 4));
+                    const uint64_t bdesc = bdesc0 + (uint64_t)(s * (STAGE2_BYTES >> 4));
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k) {
                         if (BN == 192) umma_mxf4_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u, tmem_base + SF_COL);
                         else umma_i8_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u);
                     }
-                    umma_commit_2sm(smem_u32(&ctl->empty[s]));
+                    umma_commit_2sm(empty0 + 8 * s);
                     if (kit == 0) umma_commit_2sm_local(smem_u32(&ctl->started[buf]));
+                    s += N_ISSUE;
+                    if (s >= (uint32_t)STAGES2) { s -= STAGES2; par ^= 1u; }
                 }
                 umma_commit_2sm(smem_u32(&ctl->acc_full[buf]));
             }
