@@ -893,7 +893,7 @@ int bnn_umma_gemm_f4(bnn_ctx *ctx, const uint8_t *A4, int64_t lda4, const uint8_
     if (M > 0x7fffffff || N > 0x7fffffff || K <= 0 || K > (1 << 24)) return BNN_ERR_INVALID_ARG;
     CUtensorMap mapA, mapB;
     const int64_t kb = (((K + 1) / 2 + 15) / 16) * 16;      // extent along K in bytes
-    const bool pair_want = ctx->pair_mode == 2 || (ctx->pair_mode == 0 && (double)M * (double)N >= 67108864.0);
+    const bool pair_want = ctx->pair_mode == 2 || (ctx->pair_mode == 0 && (double)M * (double)N >= 33554432.0);
     const int pairs = (M >= 512 && pair_want) ? umma2_max_pairs<192>(ctx) : 0;
     if (int st = make_map(ctx, &mapA, A4, M, kb <= lda4 ? kb : lda4, lda4, BM)) return st;
     if (int st = make_map(ctx, &mapB, B4, N, kb <= ldb4 ? kb : ldb4, ldb4, pairs > 0 ? 96 : 192)) return st;
