@@ -297,17 +297,18 @@ def main():
                                "batch 10000 per GPU, seed 1", "batch_per_gpu": BATCH, "parallelism": "replicas x%d" % world,
                    "l2": "256 MiB written between timed steps (inputs fit in L2)", "popc_variant": args.variant,
                    "operand_bits": args.operand_bits,
-                   "engine": {0: "auto (tensor-core int8 for the large layers)", 1: "CUDA-core XOR-popcount", 2: "tensor"}[args.engine]},
+                   "engine": {0: "auto (tensor-core engine for the large layers)", 1: "CUDA-core XOR-popcount", 2: "tensor"}[args.engine]},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": BATCH * SIZES[0], "d2h_bytes_per_step": BATCH * SIZES[-1] * 4,
                 "ms_per_step": e2e_total_ms / args.steps, "ms_median": statistics.median(e2e_times), "ms_min": min(e2e_times),
                 "ms_max": max(e2e_times), "warmup_steps": 100 * e2e_warm_blocks + max(args.warmup, 3)},
         "gpu_launches": launches_per_step * args.steps,
         "roofline": ({"bound": "tensor", "kernel": "bnn_binary_dense 10000x4096x4096 on the tensor engine (two operand expansion "
-                                                    "kernels + k_umma_i8<%s>, timed as one call)"
-                                                    % ("192>, tcgen05 kind::mxf4 on e2m1 nibbles" if args.operand_bits == 4 else "256>, tcgen05 kind::i8"),
+                                                    "kernels + %s, timed as one call)"
+                                                    % ("k_umma_i8_2sm<192>, CTA pairs, tcgen05 kind::mxf4 on e2m1 nibbles" if args.operand_bits == 4
+                                                       else "k_umma_i8<256>, tcgen05 kind::i8"),
                       "achieved": dense_ach, "peak": tensor_peak, "unit": "TFLOP/s",
-                      "frac": dense_ach / tensor_peak, "traffic": 28951552 if args.operand_bits == 4 else 60967424,
+                      "frac": dense_ach / tensor_peak, "traffic": 28962048 if args.operand_bits == 4 else 60967424,
                       "peak_kind": "2 ops per MAC; peak = %.0f x measured bf16 burst %.1f TFLOP/s (nominal %s:bf16 ratio), %s"
                                    % (peak_ratio, bf16_peak, "fp4" if args.operand_bits == 4 else "int8",
                                       "of measured" if peaks else "of fallback"), "ms_per_launch": dense_ms}
