@@ -111,6 +111,9 @@ int forward_device_tensor(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X,
         int8_t *dst8 = act8[k & 1];
         const int64_t ldo = act_ld(D.N);
         const bool need_next = (k < L - 2);
+        // packed sign words are only needed by the output layer and by callers who asked for the hidden activations;
+        // the next hidden layer reads the expanded operand
+        uint32_t *dst_bits = (!need_next || (hidden_out && hidden_out[k])) ? dst : nullptr;
         const int64_t ld_next = f4 ? bnn_umma_operand_ld_f4(D.N) : bnn_umma_operand_ld(D.N);
         int st;
         if (k == 0 || !f4) {
@@ -120,7 +123,7 @@ int forward_device_tensor(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X,
                 Wk8 = W8;
             }
             st = bnn_umma_gemm(ctx, k == 0 ? static_cast<const void *>(X) : cur8, k == 0 ? ldx : bnn_umma_operand_ld(D.K), k == 0, Wk8,
-                               bnn_umma_operand_ld(D.K), batch, D.N, D.K, nullptr, 0, D.thr, D.flip, dst, ldo,
+                               bnn_umma_operand_ld(D.K), batch, D.N, D.K, nullptr, 0, D.thr, D.flip, dst_bits, ldo,
                                need_next ? dst8 : nullptr, ld_next, 0, 0, 0, f4 ? 1 : 0);
         } else {
             const uint8_t *Wk4 = D.W4;
@@ -129,7 +132,7 @@ int forward_device_tensor(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X,
                 Wk4 = reinterpret_cast<uint8_t *>(W8);
             }
             st = bnn_umma_gemm_f4(ctx, reinterpret_cast<const uint8_t *>(cur8), bnn_umma_operand_ld_f4(D.K), Wk4,
-                                  bnn_umma_operand_ld_f4(D.K), batch, D.N, D.K, nullptr, 0, D.thr, D.flip, dst, ldo,
+                                  bnn_umma_operand_ld_f4(D.K), batch, D.N, D.K, nullptr, 0, D.thr, D.flip, dst_bits, ldo,
                                   need_next ? reinterpret_cast<uint8_t *>(dst8) : nullptr, ld_next);
         }
         if (st) return st;

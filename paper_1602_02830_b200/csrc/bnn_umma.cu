@@ -28,7 +28,11 @@ namespace {
 constexpr int BM = 128, BK = 128;               // BK in bytes = int8 elements
 constexpr int BN_MAX = 256;                     // tile width: 256, or 128 for narrow outputs; 192 = the 4-bit engine
 constexpr uint32_t SF_COL = 480;                // 4-bit engine: first of the 32 TMEM columns that hold the scale factors
-constexpr int EPI_WARPS = 8;                    // two per TMEM lane quadrant, each takes half of the tile's columns
+#ifndef BNN_EPI_WARPS
+#define BNN_EPI_WARPS 8
+#endif
+constexpr int EPI_WARPS = BNN_EPI_WARPS;        // EPW per TMEM lane quadrant; the tile's 32-column chunks go round-robin over them
+constexpr int EPW = EPI_WARPS / 4;
 constexpr int EPI_THREADS = EPI_WARPS * 32;
 constexpr int N_ISSUE = 2;                      // MMA-issuing warps: warp 1 and the warps from MMA_WARP_B on
 constexpr int MMA_WARP_B = 2 + EPI_WARPS;
@@ -216,93 +220,125 @@ __device__ __forceinline__ void store_signs(const UmmaArgs &p, uint32_t word, in
     }
 }
 
+// One 32-column chunk of accumulators (r, one output row per thread) -> the requested outputs.
+template <int BN>
+__device__ __forceinline__ void epilogue_chunk(Control *ctl, const UmmaArgs &p, uint32_t (&r)[32], uint32_t buf, int c, int64_t col0,
+                                               int64_t row, int q, int lane) {
+    if (row >= p.M) return;
+    if (p.thr) {                                         // thresholded signs: packed words and/or the next layer's operand
+        // bit j of the word = (acc[j] >= thr[j]) = NOT sign(acc[j] - thr[j]); the sign bits are shifted
+        // into four independent 8-bit chains (funnel shift: one instruction per column after the subtract)
+        const int4 *tp = reinterpret_cast<const int4 *>(&ctl->thr[buf][32 * c]);
+        uint32_t w4[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int g = 7; g >= 0; --g) {
+            const int4 t = tp[g];
+            const int tv[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+            for (int i = 3; i >= 0; --i) {
+                const int j = 4 * g + i;
+                const uint32_t d = (BN == 192) ? __float_as_uint(__uint_as_float(r[j]) - __int_as_float(tv[i]))
+                                               : (uint32_t)((int32_t)r[j] - tv[i]);
+                w4[j >> 3] = __funnelshift_l(d, w4[j >> 3], 1);
+            }
+        }
+        const uint32_t lt = __byte_perm(__byte_perm(w4[0], w4[1], 0x0040), __byte_perm(w4[2], w4[3], 0x0040), 0x5410);
+        uint32_t word = ~lt ^ ctl->flip[buf][c];
+        if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;      // columns beyond N stay 0
+        if (p.pool) ctl->poolw[32 * q + lane][c] = word ^ ctl->flip[buf][c];   // un-flipped (dot >= thr) bits
+        else if (p.out) p.out[row * p.ldo + (col0 >> 5)] = word;
+        if (p.out8 && !p.pool) store_signs(p, word, row, col0);
+    }
+    if (p.C) {
+        if (BN == 192) {   // the 4-bit engine accumulates in float32: exact integers
+#pragma unroll
+            for (int j = 0; j < 32; ++j) r[j] = (uint32_t)(int32_t)__uint_as_float(r[j]);
+        }
+        int32_t *dst = p.C + row * p.ldc + col0;
+        if (col0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<int4 *>(dst + j) = make_int4((int)r[j], (int)r[j + 1], (int)r[j + 2], (int)r[j + 3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (col0 + j < p.N) dst[j] = (int32_t)r[j];
+        }
+    }
+}
+
 // One tile's epilogue for the calling epilogue warp: stage the tile's thresholds, wait for the accumulators in
 // buffer `buf`, and turn them into the requested outputs.  `ok` turns false once a wait has given up.
+// The staged form of a threshold.  The comparison is the sign of (accumulator - threshold); accumulators stay below 2^30
+// in magnitude (2^24 on the 4-bit engine, where they are float32), so thresholds clamp to that range unchanged in meaning.
+template <int BN>
+__device__ __forceinline__ int32_t staged_threshold(int32_t t) {
+    if (BN == 192) return __float_as_int(t > (1 << 24) ? 3.0e7f : (t < -(1 << 24) ? -3.0e7f : (float)t));
+    return max(min(t, 1 << 30), -(1 << 30));
+}
+
+// n0_next: first column of the tile this CTA handles next (-1: none).  Its thresholds are fetched from global memory
+// while this tile is processed and staged for the other buffer at the end, so no tile but the first waits for them.
 template <int BN>
 __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, uint32_t tmem_base, uint32_t buf, uint32_t tc,
-                                              int64_t m0, int64_t n0, int q, int half, int lane, int et, bool &ok,
-                                              int64_t (&staged_n0)[ACC_BUFS]) {
-    constexpr int CHUNKS = BN / 32, CPW = CHUNKS / 2;   // 32-column chunks per tile and per warp
+                                              int64_t m0, int64_t n0, int64_t n0_next, int q, int half, int lane, int et, bool &ok) {
+    static_assert(BN <= EPI_THREADS, "one staged threshold per epilogue thread");
+    constexpr int CHUNKS = BN / 32, CPW = CHUNKS / 2;   // 32-column chunks per tile and per warp (two warps per quadrant)
     const int64_t row = m0 + 32 * q + lane;
-    // thresholds of this column block; tiles that share it with the buffer's previous tile skip the staging
-    const bool restage = p.out && staged_n0[buf] != n0;
-    if (restage) {
-        for (int e = et; e < BN; e += EPI_THREADS) {
-            const int32_t t = (n0 + e < p.N) ? p.thr[n0 + e] : 0x7fffffff;
-            // The comparison is the sign of (accumulator - threshold).  Accumulators stay below 2^30 in magnitude
-            // (2^24 on the 4-bit engine, where they are float32), so thresholds clamp to that range unchanged in meaning.
-            if (BN == 192) ctl->thr[buf][e] = __float_as_int(t > (1 << 24) ? 3.0e7f : (t < -(1 << 24) ? -3.0e7f : (float)t));
-            else ctl->thr[buf][e] = max(min(t, 1 << 30), -(1 << 30));
-        }
+    if (p.thr && tc == 0) {                              // the first tile stages its own thresholds
+        if (et < BN) ctl->thr[buf][et] = staged_threshold<BN>((n0 + et < p.N) ? p.thr[n0 + et] : 0x7fffffff);
         if (et < BN / 32) {
             const int64_t w = (n0 >> 5) + et;
             ctl->flip[buf][et] = (p.flip && w * 32 < p.N) ? p.flip[w] : 0u;
         }
-        staged_n0[buf] = n0;
     }
     // the epilogue warps only: staged thresholds visible; previous tile's pooling words no longer read
-    if (restage || p.pool) asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
+    if (p.thr) asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
+    const bool have_next = p.thr && n0_next >= 0;
+    int32_t next_thr = 0x7fffffff;
+    uint32_t next_flip = 0u;
+    if (have_next) {
+        if (et < BN && n0_next + et < p.N) next_thr = p.thr[n0_next + et];
+        if (et < BN / 32) {
+            const int64_t w = (n0_next >> 5) + et;
+            if (p.flip && w * 32 < p.N) next_flip = p.flip[w];
+        }
+    }
     if (ok && !mbar_wait(smem_u32(&ctl->acc_full[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 3); ok = false; }
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     ok = ok && (ctl->failed == 0);
     if (ok) {
-        // chunk c+1 is fetched from tensor memory while chunk c is processed
         const uint32_t tbase = tmem_base + ((uint32_t)(32 * q) << 16) + buf * BN;
-        uint32_t ra[32], rb[32];
-        const int c_first = half * CPW;
-        if (n0 + 32 * c_first < p.N) { tmem_ld32(tbase + (uint32_t)(32 * c_first), ra); tmem_ld_wait(ra); }
+        if constexpr (EPW == 2 && (CHUNKS % 2) == 0) {
+            // two warps per quadrant, each a contiguous half of the columns: chunk c+1 is fetched from tensor memory
+            // while chunk c is processed (unrolled, so both register buffers are addressed statically)
+            uint32_t ra[32], rb[32];
+            const int c_first = half * CPW;
+            if (n0 + 32 * c_first < p.N) { tmem_ld32(tbase + (uint32_t)(32 * c_first), ra); tmem_ld_wait(ra); }
 #pragma unroll
-        for (int cc = 0; cc < CPW; ++cc) {               // unrolled: both register buffers are addressed statically
-            const int c = c_first + cc;
-            const int64_t col0 = n0 + 32 * c;
-            if (col0 >= p.N) break;                      // uniform over the warp
-            const bool more = (cc + 1 < CPW) && (col0 + 32 < p.N);
-            uint32_t (&r)[32] = (cc & 1) ? rb : ra;
-            uint32_t (&rn)[32] = (cc & 1) ? ra : rb;
-            if (more) tmem_ld32(tbase + (uint32_t)(32 * (c + 1)), rn);
-            if (row < p.M) {
-                if (p.out) {
-                    // bit j of the word = (acc[j] >= thr[j]) = NOT sign(acc[j] - thr[j]); the sign bits are shifted
-                    // into four independent 8-bit chains (funnel shift: one instruction per column after the subtract)
-                    const int4 *tp = reinterpret_cast<const int4 *>(&ctl->thr[buf][32 * c]);
-                    uint32_t w4[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-                    for (int g = 7; g >= 0; --g) {
-                        const int4 t = tp[g];
-                        const int tv[4] = {t.x, t.y, t.z, t.w};
-#pragma unroll
-                        for (int i = 3; i >= 0; --i) {
-                            const int j = 4 * g + i;
-                            const uint32_t d = (BN == 192) ? __float_as_uint(__uint_as_float(r[j]) - __int_as_float(tv[i]))
-                                                           : (uint32_t)((int32_t)r[j] - tv[i]);
-                            w4[j >> 3] = __funnelshift_l(d, w4[j >> 3], 1);
-                        }
-                    }
-                    const uint32_t lt = __byte_perm(__byte_perm(w4[0], w4[1], 0x0040), __byte_perm(w4[2], w4[3], 0x0040), 0x5410);
-                    uint32_t word = ~lt ^ ctl->flip[buf][c];
-                    if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;      // columns beyond N stay 0
-                    if (p.pool) ctl->poolw[32 * q + lane][c] = word ^ ctl->flip[buf][c];   // un-flipped (dot >= thr) bits
-                    else p.out[row * p.ldo + (col0 >> 5)] = word;
-                    if (p.out8 && !p.pool) store_signs(p, word, row, col0);
-                }
-                if (p.C) {
-                    if (BN == 192) {   // the 4-bit engine accumulates in float32: exact integers
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) r[j] = (uint32_t)(int32_t)__uint_as_float(r[j]);
-                    }
-                    int32_t *dst = p.C + row * p.ldc + col0;
-                    if (col0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4)
-                            *reinterpret_cast<int4 *>(dst + j) = make_int4((int)r[j], (int)r[j + 1], (int)r[j + 2], (int)r[j + 3]);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (col0 + j < p.N) dst[j] = (int32_t)r[j];
-                    }
-                }
+            for (int cc = 0; cc < CPW; ++cc) {
+                const int c = c_first + cc;
+                const int64_t col0 = n0 + 32 * c;
+                if (col0 >= p.N) break;                      // uniform over the warp
+                const bool more = (cc + 1 < CPW) && (col0 + 32 < p.N);
+                uint32_t (&r)[32] = (cc & 1) ? rb : ra;
+                uint32_t (&rn)[32] = (cc & 1) ? ra : rb;
+                if (more) tmem_ld32(tbase + (uint32_t)(32 * (c + 1)), rn);
+                epilogue_chunk<BN>(ctl, p, r, buf, c, col0, row, q, lane);
+                if (more) tmem_ld_wait(rn);
             }
-            if (more) tmem_ld_wait(rn);
+        } else {
+            // more warps per quadrant: chunks go round-robin over them, one register buffer, and the other warps of
+            // the scheduler cover the load latency
+            uint32_t r[32];
+#pragma unroll 1
+            for (int c = half; c < CHUNKS; c += EPW) {
+                const int64_t col0 = n0 + 32 * c;
+                if (col0 >= p.N) break;                      // uniform over the warp
+                tmem_ld32(tbase + (uint32_t)(32 * c), r);
+                tmem_ld_wait(r);
+                epilogue_chunk<BN>(ctl, p, r, buf, c, col0, row, q, lane);
+            }
         }
         // padding words of the packed output
         if (half == 0 && p.out && !p.pool && row < p.M && n0 + BN >= p.N) {
@@ -337,6 +373,12 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                 if (p.out8) store_signs(p, word, opix, col0);   // the pooled pixel's signs for the next layer
             }
         }
+    }
+    if (have_next) {
+        // Every epilogue thread has passed this tile's barrier, so none still reads the other buffer's thresholds (they
+        // belonged to the previous tile); the next tile's barrier makes these visible.
+        if (et < BN) ctl->thr[buf ^ 1u][et] = staged_threshold<BN>(next_thr);
+        if (et < BN / 32) ctl->flip[buf ^ 1u][et] = next_flip;
     }
 }
 
@@ -469,11 +511,15 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
         const int et = threadIdx.x - 64;                 // 0 .. EPI_THREADS-1 among the epilogue threads
         uint32_t tc = 0;
         bool ok = true;
-        int64_t staged_n0[ACC_BUFS] = {-1, -1};
-        for (int64_t t = blockIdx.x; t < ntiles; t += gridDim.x, ++tc) {
+        // 32-bit tile arithmetic (the host checks the tile count)
+        const uint32_t tn = (uint32_t)tiles_n, nt = (uint32_t)ntiles;
+        for (uint32_t t = blockIdx.x; t < nt; t += gridDim.x, ++tc) {
             const uint32_t buf = tc & 1;
-            const int64_t m0 = (t / tiles_n) * BM, n0 = (t % tiles_n) * BN;
-            epilogue_tile<BN>(ctl, p, tmem_base, buf, tc, m0, n0, q, half, lane, et, ok, staged_n0);
+            const uint32_t tm_i = t / tn;
+            const int64_t m0 = (int64_t)tm_i * BM, n0 = (int64_t)(t - tm_i * tn) * BN;
+            const uint32_t t2 = t + gridDim.x;
+            const int64_t n0_next = (t2 < nt) ? (int64_t)(t2 % tn) * BN : -1;
+            epilogue_tile<BN>(ctl, p, tmem_base, buf, tc, m0, n0, n0_next, q, half, lane, et, ok);
             // hand the accumulator buffer back to the MMA warp
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
@@ -663,11 +709,14 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         const int et = threadIdx.x - 64;
         uint32_t tc = 0;
         bool ok = true;
-        int64_t staged_n0[ACC_BUFS] = {-1, -1};
-        for (int64_t t = pair; t < ntiles; t += npairs, ++tc) {
+        const uint32_t tn = (uint32_t)tiles_n, nt = (uint32_t)ntiles, np = (uint32_t)npairs;
+        for (uint32_t t = (uint32_t)pair; t < nt; t += np, ++tc) {
             const uint32_t buf = tc & 1;
-            const int64_t m0 = (t / tiles_n) * (2 * BM) + rank * BM, n0 = (t % tiles_n) * BN;
-            epilogue_tile<BN>(ctl, p, tmem_base, buf, tc, m0, n0, q, half, lane, et, ok, staged_n0);
+            const uint32_t tm_i = t / tn;
+            const int64_t m0 = (int64_t)tm_i * (2 * BM) + rank * BM, n0 = (int64_t)(t - tm_i * tn) * BN;
+            const uint32_t t2 = t + np;
+            const int64_t n0_next = (t2 < nt) ? (int64_t)(t2 % tn) * BN : -1;
+            epilogue_tile<BN>(ctl, p, tmem_base, buf, tc, m0, n0, n0_next, q, half, lane, et, ok);
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive_cta0(smem_u32(&ctl->acc_empty[buf]));
@@ -846,6 +895,7 @@ static int umma2_max_pairs(bnn_ctx *ctx) {
 static int umma_launch(bnn_ctx *ctx, const CUtensorMap &mapA, const CUtensorMap &mapB, const UmmaArgs &a, int bn) {
     if (int st = umma_prepare(ctx)) return st;
     const int64_t tiles = ((a.M + BM - 1) / BM) * ((a.N + bn - 1) / bn);
+    if (tiles >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;      // the kernels count tiles in 32 bits
     const int64_t grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
     if (bn == 192) k_umma_i8<192><<<(unsigned)grid, NTHREADS, umma_smem_bytes<192>(), ctx->stream>>>(mapA, mapB, a);
     else if (bn == 256) k_umma_i8<256><<<(unsigned)grid, NTHREADS, umma_smem_bytes<256>(), ctx->stream>>>(mapA, mapB, a);
@@ -905,6 +955,7 @@ int bnn_umma_gemm_f4(bnn_ctx *ctx, const uint8_t *A4, int64_t lda4, const uint8_
     if (pairs > 0) {
         if (int st = umma_prepare(ctx)) return st;
         const int64_t tiles2 = ((M + 2 * BM - 1) / (2 * BM)) * ((N + 191) / 192);
+        if (tiles2 >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;
         const int64_t use = tiles2 < pairs ? tiles2 : pairs;
         k_umma_i8_2sm<192><<<(unsigned)(2 * use), NTHREADS, umma2_smem_bytes<192>(), ctx->stream>>>(mapA, mapB, a);
         return bnn_check_launch(ctx);
@@ -919,7 +970,7 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
     if (M == 0 || N == 0) return BNN_OK;
     if (pool) {   // rows are pixels of H x W images in (b, y, x) order; 128-row tiles must hold whole 2x2 windows
         int TH, TB;
-        if (!bnn_umma_conv_tiling(H, W, 1, &TH, &TB) || C) return BNN_ERR_INVALID_ARG;
+        if (!bnn_umma_conv_tiling(H, W, 1, &TH, &TB) || C || !out) return BNN_ERR_INVALID_ARG;
     }
     if ((lda8 & 15) || (ldb8 & 15) || !bnn_aligned16(A8) || !bnn_aligned16(B8)) return BNN_ERR_ALIGNMENT;
     if (M > 0x7fffffff || N > 0x7fffffff) return BNN_ERR_INVALID_ARG;
@@ -943,6 +994,7 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
     a.pool = pool; a.H = (int)H; a.W = (int)W; a.out_f4 = out_f4;
     if (pairs > 0) {
         const int64_t tiles2 = ((M + 2 * BM - 1) / (2 * BM)) * ((N + 255) / 256);
+        if (tiles2 >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;
         const int64_t use = tiles2 < pairs ? tiles2 : pairs;
         k_umma_i8_2sm<256><<<(unsigned)(2 * use), NTHREADS, umma2_smem_bytes<256>(), ctx->stream>>>(mapA, mapB, a);
         return bnn_check_launch(ctx);
@@ -998,7 +1050,7 @@ int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B,
                   int64_t C_out, int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, int32_t *out_sums,
                   int8_t *out8, int64_t ldo8) {
     int TH, TB;
-    if (!bnn_umma_conv_tiling(H, W, pool, &TH, &TB) || (C_in % BK) != 0 || (pool && out_sums)) return BNN_ERR_INVALID_ARG;
+    if (!bnn_umma_conv_tiling(H, W, pool, &TH, &TB) || (C_in % BK) != 0 || (pool && (out_sums || !out_bits))) return BNN_ERR_INVALID_ARG;
     CUtensorMap mapA, mapB;
     const int bn = umma_tile_n(C_out);
     if (int st = make_map_nhwc(ctx, &mapA, act8, B, H, W, C_in, (int)W, TH, TB)) return st;
