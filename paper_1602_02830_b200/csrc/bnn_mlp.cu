@@ -207,14 +207,20 @@ extern "C" int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const u
     float *Sd = reinterpret_cast<float *>(ws + fwd + round256((size_t)batch * K0));
 
     // Row chunks are independent through every layer, so for a large batch on the tensor engine the input is copied
-    // in up to three chunks on an internal stream while the previous chunk is already running through the layers.
-    // Chunk sizes are multiples of 128 rows (whole tiles).
+    // in chunks on an internal stream while the previous chunk is already running through the layers.  Every chunk
+    // pays the fixed cost of its four kernels, so there are only two, the first the smaller one (its copy is not
+    // overlapped with anything): boundaries at multiples of 128 rows (whole tiles).
+#ifndef BNN_E2E_SPLIT_PCT
+#define BNN_E2E_SPLIT_PCT 40
+#endif
     int nchunks = 1;
-    int64_t rows_per = batch;
+    int64_t bounds[3] = {0, batch, batch};
     if (tensor && batch >= 6144) {
-        nchunks = 3;
-        rows_per = (((batch + nchunks - 1) / nchunks + 127) / 128) * 128;
-        if (!tensor_applies(ctx, m, batch - 2 * rows_per > 0 ? batch - 2 * rows_per : 1)) nchunks = 1, rows_per = batch;
+        const int64_t first = ((batch * BNN_E2E_SPLIT_PCT / 100 + 127) / 128) * 128;
+        if (first > 0 && first < batch && tensor_applies(ctx, m, first) && tensor_applies(ctx, m, batch - first)) {
+            nchunks = 2;
+            bounds[1] = first;
+        }
     }
     if (nchunks > 1 && !ctx->copy_ready) {
         BNN_CUDA_TRY(ctx, cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
@@ -227,7 +233,7 @@ extern "C" int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const u
         BNN_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->ev[0], 0));
     }
     for (int c = 0; c < nchunks; ++c) {
-        const int64_t r0 = c * rows_per, rows = (r0 + rows_per <= batch) ? rows_per : batch - r0;
+        const int64_t r0 = bounds[c], rows = bounds[c + 1] - r0;
         if (ldx == K0)   // contiguous: one linear copy
             BNN_CUDA_TRY(ctx, cudaMemcpyAsync(Xd + r0 * K0, X_host + r0 * ldx, (size_t)K0 * rows, cudaMemcpyHostToDevice, cs));
         else
@@ -236,7 +242,7 @@ extern "C" int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const u
         if (nchunks > 1) BNN_CUDA_TRY(ctx, cudaEventRecord(ctx->ev[1 + c], cs));
     }
     for (int c = 0; c < nchunks; ++c) {
-        const int64_t r0 = c * rows_per, rows = (r0 + rows_per <= batch) ? rows_per : batch - r0;
+        const int64_t r0 = bounds[c], rows = bounds[c + 1] - r0;
         if (nchunks > 1) BNN_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev[1 + c], 0));
         if (int st = tensor ? forward_device_tensor(ctx, m, Xd + r0 * K0, K0, rows, Sd + r0 * NL, NL, nullptr, ws)
                             : forward_device(ctx, m, Xd + r0 * K0, K0, rows, Sd + r0 * NL, NL, nullptr, ws,
