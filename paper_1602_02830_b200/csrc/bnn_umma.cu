@@ -54,6 +54,7 @@ __device__ int g_umma_error;                    // 0 = fine; otherwise a code sa
 struct UmmaArgs {
     int64_t M, N;
     int k_iters;            // ceil(K_bytes / BK)
+    int k_last;             // MMAs (32 bytes of K each) that the last K step still needs: 1..4
     uint32_t idesc;
     int32_t *C; int64_t ldc;                     // optional int32 output
     uint32_t *out; int64_t ldo;                  // optional packed sign output
@@ -490,8 +491,10 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint64_t adesc = adesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
                     const uint64_t bdesc = bdesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
+                    const int nk = (kit == p.k_iters - 1) ? p.k_last : BK / 32;   // the last step may end early (K not a multiple of BK)
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k) {   // 32 bytes of K per instruction: start address advances by 32 B (>> 4 = 2)
+                        if (k >= nk) break;
                         if (BN == 192) umma_mxf4(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u, tmem_base + SF_COL);
                         else umma_i8(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u);
                     }
@@ -689,8 +692,10 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint64_t adesc = adesc0 + (uint64_t)(s * (STAGE2_BYTES >> 4));
                     const uint64_t bdesc = bdesc0 + (uint64_t)(s * (STAGE2_BYTES >> 4));
+                    const int nk = (kit == p.k_iters - 1) ? p.k_last : BK / 32;
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k) {
+                        if (k >= nk) break;
                         if (BN == 192) umma_mxf4_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u, tmem_base + SF_COL);
                         else umma_i8_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u);
                     }
@@ -950,6 +955,7 @@ int bnn_umma_gemm_f4(bnn_ctx *ctx, const uint8_t *A4, int64_t lda4, const uint8_
     UmmaArgs a{};
     a.M = M; a.N = N;
     a.k_iters = (int)((K + 2 * BK - 1) / (2 * BK));          // 256 values per 128-byte K step
+    a.k_last = (int)((K - 2 * BK * (int64_t)(a.k_iters - 1) + 63) / 64);
     a.C = C; a.ldc = ldc; a.out = out; a.ldo = ldo; a.thr = thr; a.flip = flip;
     a.out8 = reinterpret_cast<int8_t *>(out4); a.ldo8 = ldo4; a.out_f4 = 1;
     if (pairs > 0) {
@@ -989,6 +995,7 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
     UmmaArgs a{};
     a.M = M; a.N = N;
     a.k_iters = (int)((K + BK - 1) / BK);
+    a.k_last = (int)((K - BK * (int64_t)(a.k_iters - 1) + 31) / 32);
     a.idesc = (2u << 4) | ((a_unsigned ? 0u : 1u) << 7) | (1u << 10) | ((uint32_t)(BM >> 4) << 24);   // N field added by the kernel
     a.C = C; a.ldc = ldc; a.out = out; a.ldo = ldo; a.out8 = out8; a.ldo8 = ldo8; a.thr = thr; a.flip = flip;
     a.pool = pool; a.H = (int)H; a.W = (int)W; a.out_f4 = out_f4;
@@ -1058,6 +1065,7 @@ int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B,
     UmmaArgs a{};
     a.M = B * H * W; a.N = C_out;
     a.k_iters = (int)(9 * (C_in / BK));
+    a.k_last = BK / 32;
     a.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BM >> 4) << 24);
     a.C = out_sums; a.ldc = C_out; a.out = out_bits; a.ldo = (C_out + 31) / 32; a.thr = thr; a.flip = flip;
     a.out8 = out8; a.ldo8 = ldo8;
