@@ -69,7 +69,7 @@ __device__ __forceinline__ void warp_sum_many(int32_t (&v)[V], int lane) {
 }
 
 template <int RSMAX, int MODE>
-__global__ void __launch_bounds__(256) k_skinny(const SkinnyArgs p) {
+__global__ void __launch_bounds__(256, (RSMAX <= 16) ? 3 : 1) k_skinny(const SkinnyArgs p) {
     extern __shared__ __align__(16) uint32_t smem[];
     const int64_t Kw = (p.K + 31) >> 5;
     const int64_t Kw4 = (Kw + 3) & ~int64_t(3);
@@ -86,10 +86,21 @@ __global__ void __launch_bounds__(256) k_skinny(const SkinnyArgs p) {
     for (int cc = 0; cc < 4; ++cc)
         b[cc] = load_row_words(p.L + (lrow0 + cc) * p.ldl_w, lrow0 + cc < p.RL, 4 * lane, Kw, tail_mask, true);
 
-    for (int64_t e = tid; e < p.RS * (Kw4 >> 2); e += 256) {
-        const int64_t r = e / (Kw4 >> 2), q = e % (Kw4 >> 2);
-        const uint4 v = load_row_words(p.S + r * p.lds_w, true, 4 * q, Kw, tail_mask, true);
-        *reinterpret_cast<uint4 *>(Ss + r * Kw4 + 4 * q) = v;
+    {   // 32-bit index arithmetic: RS <= 32 rows of at most 2^24 128-bit groups
+        const uint32_t gpr = (uint32_t)(Kw4 >> 2), total = (uint32_t)p.RS * gpr;
+        for (uint32_t e = tid; e < total; e += 256) {
+            const uint32_t r = e / gpr, q = e - r * gpr;
+            const uint4 v = load_row_words(p.S + (int64_t)r * p.lds_w, true, 4 * (int64_t)q, Kw, tail_mask, true);
+            *reinterpret_cast<uint4 *>(Ss + (int64_t)r * Kw4 + 4 * q) = v;
+        }
+    }
+    // output scores: per output s the affine form of BatchNorm, a = gamma / sqrt(var + eps), b = beta - mean * a, once
+    // per CTA in double (the square root and the division are the expensive part)
+    __shared__ double bn_a[32], bn_b[32];
+    if (MODE == 1 && tid < p.RS) {
+        const double a = (double)p.gamma[tid] / sqrt((double)p.var[tid] + p.eps);
+        bn_a[tid] = a;
+        bn_b[tid] = (double)p.beta[tid] - (double)p.mean[tid] * a;
     }
     __syncthreads();
 
@@ -157,9 +168,7 @@ __global__ void __launch_bounds__(256) k_skinny(const SkinnyArgs p) {
         for (int e = tid; e < 32 * (int)p.RS; e += 256) {
             const int lc = e / (int)p.RS, s = e % (int)p.RS;
             if (l0 + lc < p.RL) {
-                const double x = (double)res[lc * RSMAX + s];
-                const double xhat = (x - (double)p.mean[s]) / sqrt((double)p.var[s] + p.eps);
-                p.scores[(l0 + lc) * p.ld_scores + s] = (float)((double)p.gamma[s] * xhat + (double)p.beta[s]);
+                p.scores[(l0 + lc) * p.ld_scores + s] = (float)fma((double)res[lc * RSMAX + s], bn_a[s], bn_b[s]);
             }
         }
     }
