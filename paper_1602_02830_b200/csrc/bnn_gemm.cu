@@ -19,6 +19,7 @@ struct SkinnyArgs {
     const uint32_t *L; int64_t ldl_w; int64_t RL;
     int64_t K;
     int32_t *C; int64_t ldc;
+    int c_rows_are_large;   // C[l * ldc + s] (the small operand supplies the columns) instead of C[s * ldc + l]
     uint32_t *out; int64_t ldo;
     const int32_t *thr; const uint32_t *flip;
     float *scores; int64_t ld_scores;
@@ -141,7 +142,12 @@ __global__ void __launch_bounds__(256, (RSMAX <= 16) ? 3 : 1) k_skinny(const Ski
     __syncthreads();
 
     if (MODE == 0) {
-        if (p.C) {
+        if (p.C && p.c_rows_are_large) {
+            for (int e = tid; e < 32 * (int)p.RS; e += 256) {
+                const int lc = e / (int)p.RS, s = e - lc * (int)p.RS;
+                if (l0 + lc < p.RL) p.C[(l0 + lc) * p.ldc + s] = res[lc * RSMAX + s];
+            }
+        } else if (p.C) {
             for (int e = tid; e < 32 * (int)p.RS; e += 256) {
                 const int s = e >> 5, lc = e & 31;
                 if (l0 + lc < p.RL) p.C[(int64_t)s * p.ldc + l0 + lc] = res[lc * RSMAX + s];
@@ -354,6 +360,14 @@ static int gemm_like(bnn_ctx *ctx, const uint32_t *Ap, int64_t lda_w, const uint
         s.L = Bp; s.ldl_w = ldb_w; s.RL = N;
         s.K = K;
         s.C = C; s.ldc = ldc; s.out = out; s.ldo = ldo_w; s.thr = thr; s.flip = flip;
+        return launch_skinny<0>(ctx, s);
+    }
+    if (N <= 32 && C && !out && skinny_fits(N, K)) {   // few columns (e.g. a 10-way output layer as a plain product): roles swapped
+        SkinnyArgs s{};
+        s.S = Bp; s.lds_w = ldb_w; s.RS = N;
+        s.L = Ap; s.ldl_w = lda_w; s.RL = M;
+        s.K = K;
+        s.C = C; s.ldc = ldc; s.c_rows_are_large = 1;
         return launch_skinny<0>(ctx, s);
     }
     Args a{};

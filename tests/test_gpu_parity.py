@@ -84,7 +84,9 @@ def gemm_gpu(ctx, A, B):
 
 
 SMALL = [(1, 1, 1), (2, 3, 31), (3, 2, 32), (33, 1, 33), (1, 33, 63), (5, 7, 64), (4, 4, 65), (3, 5, 100),
-         (33, 33, 100), (40, 130, 257), (64, 256, 512), (129, 127, 300), (200, 260, 1000), (257, 129, 4100)]
+         (33, 33, 100), (40, 130, 257), (64, 256, 512), (129, 127, 300), (200, 260, 1000), (257, 129, 4100),
+         # many rows times few columns (the output layer as a plain product): small-operand kernel with the roles swapped
+         (300, 10, 4096), (1000, 32, 100), (77, 17, 33)]
 
 
 @pytest.mark.parametrize("variant", VARIANTS)
