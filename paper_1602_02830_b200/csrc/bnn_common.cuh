@@ -31,6 +31,27 @@ struct bnn_ctx {
         }                                                    \
     } while (0)
 
+// Programmatic dependent launch: the kernel may be set up on the GPU while its predecessor in the stream still runs.
+// Kernels launched this way call bnn_pdl_wait() before their first access to global memory; it returns once the
+// predecessor has completed and its writes are visible (immediately for an ordinary launch).
+template <typename... KArgs, typename... Args>
+static inline cudaError_t bnn_launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                               Args &&...args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#ifdef __CUDACC__
+__device__ __forceinline__ void bnn_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel of the stream be set up as soon as every CTA of this one has got here (it still waits in
+// bnn_pdl_wait for this kernel to finish before it touches memory).
+__device__ __forceinline__ void bnn_pdl_launch_next() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+
 static inline int bnn_check_launch(bnn_ctx *ctx) {
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {

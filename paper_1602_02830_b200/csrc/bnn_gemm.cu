@@ -79,6 +79,8 @@ __global__ void __launch_bounds__(256, (RSMAX <= 16) ? 3 : 1) k_skinny(const Ski
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t tail_mask = (p.K & 31) ? ((1u << (p.K & 31)) - 1u) : 0xffffffffu;
     const int64_t l0 = (int64_t)blockIdx.x * 32;
+    bnn_pdl_launch_next();
+    bnn_pdl_wait();
 
     // the warp's four rows of the large operand: their first 128-bit chunks are requested before anything else
     const int64_t lrow0 = l0 + warp * 4;
@@ -191,7 +193,7 @@ int launch_skinny(bnn_ctx *ctx, const SkinnyArgs &a) {
         if (smem > 48 * 1024)                                                                                  \
             BNN_CUDA_TRY(ctx, cudaFuncSetAttribute(k_skinny<R, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                                    (int)smem));                                                \
-        k_skinny<R, MODE><<<grid, 256, smem, ctx->stream>>>(a);                                                \
+        BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_skinny<R, MODE>, dim3(grid), dim3(256), smem, ctx->stream, a)); \
     } while (0)
     switch (rsmax) {
         case 1: BNN_SK(1); break;

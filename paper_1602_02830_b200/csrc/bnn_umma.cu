@@ -420,6 +420,8 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = ctl->tmem_base;
+    bnn_pdl_launch_next();
+    bnn_pdl_wait();                                      // barriers and tensor memory were set up while the predecessor drained
 
     if (BN == 192) {
         // 4-bit engine: every value is exactly +-1, so every block scale is 2^0.  In UE8M0 that is the byte 0x7f, and
@@ -634,6 +636,8 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     cluster_sync_all();                                     // both CTAs' barriers exist before anyone signals them
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = ctl->tmem_base;
+    bnn_pdl_launch_next();
+    bnn_pdl_wait();
 
     if (BN == 192) {
         // 4-bit engine: unit block scales (byte 0x7f) in this CTA's scale-factor columns; the leader's MMAs read the
@@ -742,6 +746,8 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
 // One thread per 32-bit word = 32 output bytes (two 128-bit stores).
 __global__ void __launch_bounds__(256) k_expand_s8(const uint32_t *__restrict__ src, int64_t ld_w, int64_t rows, int64_t K,
                                                    int8_t *__restrict__ dst, int64_t ld8) {
+    bnn_pdl_launch_next();
+    bnn_pdl_wait();
     const int64_t wpr = ld8 >> 5;            // words per output row (ld8 is a multiple of 32)
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= rows * wpr) return;
@@ -768,6 +774,8 @@ __global__ void __launch_bounds__(256) k_expand_s8(const uint32_t *__restrict__ 
 // the low nibble); nibbles at or beyond K are 0 (= +0.0).  One thread per 32-bit word = 16 output bytes.
 __global__ void __launch_bounds__(256) k_expand_f4(const uint32_t *__restrict__ src, int64_t ld_w, int64_t rows, int64_t K,
                                                    uint8_t *__restrict__ dst, int64_t ld4) {
+    bnn_pdl_launch_next();
+    bnn_pdl_wait();
     const int64_t wpr = ld4 >> 4;            // words per output row (ld4 is a multiple of 128 bytes)
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= rows * wpr) return;
@@ -792,6 +800,8 @@ __global__ void __launch_bounds__(256) k_expand_f4(const uint32_t *__restrict__ 
 // outside the image as zeros) written as one 32-byte row, byte (tap * C_in + c).  One thread per pixel.
 __global__ void __launch_bounds__(256) k_im2col_u8(const uint8_t *__restrict__ act, int64_t B, int H, int W, int Cin,
                                                    uint8_t *__restrict__ dst) {
+    bnn_pdl_launch_next();
+    bnn_pdl_wait();
     const int64_t pix = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (pix >= B * H * W) return;
     const int x = (int)(pix % W), y = (int)((pix / W) % H);
@@ -902,9 +912,10 @@ static int umma_launch(bnn_ctx *ctx, const CUtensorMap &mapA, const CUtensorMap 
     const int64_t tiles = ((a.M + BM - 1) / BM) * ((a.N + bn - 1) / bn);
     if (tiles >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;      // the kernels count tiles in 32 bits
     const int64_t grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
-    if (bn == 192) k_umma_i8<192><<<(unsigned)grid, NTHREADS, umma_smem_bytes<192>(), ctx->stream>>>(mapA, mapB, a);
-    else if (bn == 256) k_umma_i8<256><<<(unsigned)grid, NTHREADS, umma_smem_bytes<256>(), ctx->stream>>>(mapA, mapB, a);
-    else k_umma_i8<128><<<(unsigned)grid, NTHREADS, umma_smem_bytes<128>(), ctx->stream>>>(mapA, mapB, a);
+    const dim3 g((unsigned)grid), b(NTHREADS);
+    if (bn == 192) BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8<192>, g, b, umma_smem_bytes<192>(), ctx->stream, mapA, mapB, a));
+    else if (bn == 256) BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8<256>, g, b, umma_smem_bytes<256>(), ctx->stream, mapA, mapB, a));
+    else BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8<128>, g, b, umma_smem_bytes<128>(), ctx->stream, mapA, mapB, a));
     return bnn_check_launch(ctx);
 }
 
@@ -920,7 +931,7 @@ int bnn_umma_expand(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t row
     if (total == 0) return BNN_OK;
     const int64_t blocks = (total + 255) / 256;
     if (blocks > 0x7fffffff) return BNN_ERR_INVALID_ARG;
-    k_expand_s8<<<(unsigned)blocks, 256, 0, ctx->stream>>>(src, ld_w, rows, K, dst, ld8);
+    BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_expand_s8, dim3((unsigned)blocks), dim3(256), 0, ctx->stream, src, ld_w, rows, K, dst, ld8));
     return bnn_check_launch(ctx);
 }
 
@@ -933,7 +944,7 @@ int bnn_umma_expand_f4(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t 
     if (total == 0) return BNN_OK;
     const int64_t blocks = (total + 255) / 256;
     if (blocks > 0x7fffffff) return BNN_ERR_INVALID_ARG;
-    k_expand_f4<<<(unsigned)blocks, 256, 0, ctx->stream>>>(src, ld_w, rows, K, dst, ld4);
+    BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_expand_f4, dim3((unsigned)blocks), dim3(256), 0, ctx->stream, src, ld_w, rows, K, dst, ld4));
     return bnn_check_launch(ctx);
 }
 
@@ -963,7 +974,8 @@ int bnn_umma_gemm_f4(bnn_ctx *ctx, const uint8_t *A4, int64_t lda4, const uint8_
         const int64_t tiles2 = ((M + 2 * BM - 1) / (2 * BM)) * ((N + 191) / 192);
         if (tiles2 >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;
         const int64_t use = tiles2 < pairs ? tiles2 : pairs;
-        k_umma_i8_2sm<192><<<(unsigned)(2 * use), NTHREADS, umma2_smem_bytes<192>(), ctx->stream>>>(mapA, mapB, a);
+        BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8_2sm<192>, dim3((unsigned)(2 * use)), dim3(NTHREADS), umma2_smem_bytes<192>(),
+                                               ctx->stream, mapA, mapB, a));
         return bnn_check_launch(ctx);
     }
     return umma_launch(ctx, mapA, mapB, a, 192);
@@ -1003,7 +1015,8 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
         const int64_t tiles2 = ((M + 2 * BM - 1) / (2 * BM)) * ((N + 255) / 256);
         if (tiles2 >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;
         const int64_t use = tiles2 < pairs ? tiles2 : pairs;
-        k_umma_i8_2sm<256><<<(unsigned)(2 * use), NTHREADS, umma2_smem_bytes<256>(), ctx->stream>>>(mapA, mapB, a);
+        BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8_2sm<256>, dim3((unsigned)(2 * use)), dim3(NTHREADS), umma2_smem_bytes<256>(),
+                                               ctx->stream, mapA, mapB, a));
         return bnn_check_launch(ctx);
     }
     return umma_launch(ctx, mapA, mapB, a, bn);
@@ -1031,7 +1044,7 @@ int bnn_umma_im2col_u8(bnn_ctx *ctx, const uint8_t *act, int64_t B, int64_t H, i
     if (total == 0) return BNN_OK;
     const int64_t blocks = (total + 255) / 256;
     if (blocks > 0x7fffffff || 9 * C_in > 32) return BNN_ERR_INVALID_ARG;
-    k_im2col_u8<<<(unsigned)blocks, 256, 0, ctx->stream>>>(act, B, (int)H, (int)W, (int)C_in, dst);
+    BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_im2col_u8, dim3((unsigned)blocks), dim3(256), 0, ctx->stream, act, B, (int)H, (int)W, (int)C_in, dst));
     return bnn_check_launch(ctx);
 }
 
