@@ -199,8 +199,8 @@ BNN_API int bnn_convnet_forward(bnn_ctx *ctx, const bnn_convnet_desc *net, const
 
 /* ---------------------------------------------------------------------------------------------
  * Whole MLP forward (Algorithm 4): first layer on 8-bit inputs, hidden binary layers, real-valued
- * output layer  score = gamma * ((dot - mean) / sqrt(var + eps)) + beta  (evaluated in double,
- * stored as float32).
+ * output layer  score = gamma * ((dot - mean) / sqrt(var + eps)) + beta  (evaluated in double as
+ * dot * a + b with a = gamma / sqrt(var + eps), b = beta - mean * a, rounded once to float32).
  */
 typedef struct {
     const uint32_t *Wp;  /* packed N x K weights (device) */

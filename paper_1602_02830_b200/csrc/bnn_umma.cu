@@ -1,22 +1,27 @@
 // Tensor-core engine for the large products: the +-1 (or 8-bit x +-1) product evaluated EXACTLY by the
-// 5th-generation tensor cores as an int8 GEMM with int32 accumulation in tensor memory.
+// 5th-generation tensor cores, accumulators in tensor memory.
 //
 //   Section 4 states that the binary kernel and an ordinary matrix product return identical outputs on +-1
-//   inputs.  On sm_100a the ordinary product has a far higher ceiling than the POPC pipe (8192 int8 MACs vs
-//   512 bit-MACs per clock per SM), so for large shapes the packed operands are expanded to one signed byte
-//   per value (a streaming pass) and multiplied with tcgen05.mma kind::i8.  Results are the same integers.
+//   inputs.  On sm_100a the ordinary product has a far higher ceiling than the POPC pipe (8192 int8 or 16384
+//   4-bit MACs against 512 bit-MACs per clock per SM), so for large shapes the packed operands are expanded
+//   (a streaming pass) and multiplied on the tensor cores.  Results are the same integers.
+//     bytes   (+1 = 0x01, -1 = 0xff; the 8-bit first layer's pixels as they are): tcgen05.mma kind::i8, int32
+//             accumulators, 128 x 256 tiles (128 x 128 for narrow outputs);
+//     nibbles (e2m1: +1 = 0x2, -1 = 0xa): tcgen05.mma kind::mxf4.block_scale with every block scale 2^0 (32 TMEM
+//             columns filled once with the UE8M0 byte 0x7f), float32 accumulators (exact while K <= 2^24),
+//             128 x 192 tiles, twice the MMA rate and half the operand bytes.
 //
-// Kernel k_umma_i8 (persistent, one CTA per SM walking 128 x 256 output tiles, 352 threads):
-//   warp 0    TMA producer: cp.async.bulk.tensor 2-D loads of 128-byte-wide K slices (128B swizzle) of both
-//             operands into a 4-stage shared-memory ring, completion on mbarriers;
-//   warp 1    allocates all 512 TMEM columns (two accumulator buffers), then one lane issues tcgen05.mma
-//             (M=128, N=256, K=32) four times per stage and releases the stage with tcgen05.commit;
-//   warp 10   second MMA issuer: takes the odd K steps of every tile (issuing a step costs one thread more clocks
-//             than the tensor core needs to run it; two issuing warps keep the tensor pipe full);
-//   warps 2-9 epilogue (two warps per TMEM lane quadrant, each half of the columns): tcgen05.ld of the int32
-//             accumulators (each thread owns one output row, 32 columns at a time, the next chunk in flight while
-//             the current one is processed), then either int32 stores, or the BatchNorm-folded threshold + Sign + repack to one
-//             32-bit word per 32 columns (and, for the next layer, the same signs as bytes).
+// Kernel k_umma_i8<BN> (persistent, one CTA per SM walking 128 x BN output tiles, column blocks fastest):
+//   warp 0       TMA producer: cp.async.bulk.tensor loads of 128-byte-wide K slices (128B swizzle) of both
+//                operands into a ring of 4-6 shared-memory stages, completion on mbarriers;
+//   warps 1, 10  MMA issuers: one lane each, alternate K steps of every tile (issuing a step costs one thread more
+//                clocks than the tensor core needs to run it); four MMAs per step, tcgen05.commit releases the
+//                stage; warp 1 also allocates the 512 TMEM columns (two accumulator buffers);
+//   warps 2-9    epilogue (two warps per TMEM lane quadrant, each half of the columns): tcgen05.ld of the
+//                accumulators (one output row per thread, 32 columns at a time, the next chunk in flight while the
+//                current one is processed), then int32 stores, or the BatchNorm-folded threshold + Sign as one
+//                32-bit word per 32 columns and/or the same signs in the next layer's operand format.
+// Kernel k_umma_i8_2sm<BN>: the same with a cluster of two CTAs on one 256 x BN tile (cta_group::2).
 // Every wait is bounded: after the limit the kernel records an error code and runs to its end without
 // touching the accumulators, so a failure surfaces as BNN_ERR_DEVICE_STATUS instead of a hang.
 #include "bnn_internal.cuh"
