@@ -105,6 +105,18 @@ BNN_API int bnn_expand_signs(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, in
 BNN_API int64_t bnn_expanded_ld_f4(int64_t K);
 BNN_API size_t bnn_expanded_bytes_f4(int64_t rows, int64_t K);
 BNN_API int bnn_expand_signs_f4(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t rows, int64_t K, uint8_t *dst);
+/* Hidden layer (Algorithm 4: product, BatchNorm folded to thr / flip, Sign) on operands that are already in an
+ * expanded format, i.e. the tensor-core kernel of bnn_binary_dense without its two expansion passes: for callers that
+ * keep weights and activations expanded, as bnn_mlp_forward does between its layers.
+ *   operand_bits 8: A_exp M x K and W_exp N x K as written by bnn_expand_signs (pitches in bytes, multiples of 16);
+ *   operand_bits 4: as written by bnn_expand_signs_f4 (K <= 2^24).
+ *   out_bits (optional): packed M x N signs, pitch ldo_w words, like bnn_binary_dense.
+ *   out_exp  (optional): the same signs in the operand format of the next layer (same operand_bits), pitch
+ *                        ldo_exp bytes >= bnn_expanded_ld(N) or bnn_expanded_ld_f4(N); at least one output is required.
+ * Runs on the context's stream; BNN_ERR_ALIGNMENT for pointers or pitches that are not multiples of 16 bytes. */
+BNN_API int bnn_binary_dense_expanded(bnn_ctx *ctx, const void *A_exp, int64_t lda_bytes, const void *W_exp, int64_t ldw_bytes,
+                                      int operand_bits, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits,
+                                      int64_t ldo_w, void *out_exp, int64_t ldo_exp, int64_t M, int64_t N, int64_t K);
 /* Synchronises the context's stream and returns BNN_ERR_DEVICE_STATUS if a kernel gave up on one of its
  * bounded waits since the last call (its outputs are then undefined), BNN_OK otherwise. */
 BNN_API int bnn_device_status(bnn_ctx *ctx);

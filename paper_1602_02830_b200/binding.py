@@ -28,7 +28,7 @@ EXPORTS = (
     "bnn_gemm_workspace_bytes", "bnn_device_status", "bnn_conv_workspace_bytes", "bnn_set_tile_rows", "bnn_set_pair_mode", "bnn_expanded_ld",
     "bnn_expanded_bytes", "bnn_expand_signs", "bnn_baseline_gemm_f32", "bnn_convnet_workspace_bytes",
     "bnn_convnet_forward", "bnn_set_operand_bits", "bnn_expanded_ld_f4",
-    "bnn_expanded_bytes_f4", "bnn_expand_signs_f4",
+    "bnn_expanded_bytes_f4", "bnn_expand_signs_f4", "bnn_binary_dense_expanded",
 )
 
 
@@ -89,6 +89,7 @@ def lib() -> ctypes.CDLL:
         L.bnn_expanded_bytes_f4.argtypes = [i64, i64]
         L.bnn_expanded_bytes_f4.restype = c_size_t
         L.bnn_expand_signs_f4.argtypes = [vp, vp, i64, i64, i64, vp]
+        L.bnn_binary_dense_expanded.argtypes = [vp, vp, i64, vp, i64, ctypes.c_int, vp, vp, vp, i64, vp, i64, i64, i64, i64]
         L.bnn_expanded_ld.argtypes = [i64]
         L.bnn_expanded_ld.restype = i64
         L.bnn_expanded_bytes.argtypes = [i64, i64]
@@ -199,6 +200,20 @@ class Context:
         dst = self.empty(rows, ld, dtype=torch.uint8)
         self._ck(lib().bnn_expand_signs_f4(self._h, _ptr(packed), packed.stride(0), rows, K, _ptr(dst)), "bnn_expand_signs_f4")
         return dst
+
+    def binary_dense_expanded(self, A_exp, W_exp, bits: int, thr, flip, M, N, K, want_bits=True, want_exp=False):
+        """bnn_binary_dense_expanded: operands as written by expand_signs (bits 8) or expand_signs_f4 (bits 4).
+        Returns (packed signs or None, signs in the next layer's operand format or None)."""
+        out = self.empty(M, packed_ld(N)) if want_bits else None
+        out_exp = None
+        if want_exp:
+            ld = int(lib().bnn_expanded_ld_f4(N) if bits == 4 else lib().bnn_expanded_ld(N))
+            out_exp = self.empty(M, ld, dtype=torch.uint8 if bits == 4 else torch.int8)
+        self._ck(lib().bnn_binary_dense_expanded(self._h, _ptr(A_exp), A_exp.stride(0) * A_exp.element_size(), _ptr(W_exp),
+                                                 W_exp.stride(0) * W_exp.element_size(), bits, _ptr(thr), _ptr(flip), _ptr(out),
+                                                 packed_ld(N), _ptr(out_exp), out_exp.stride(0) if out_exp is not None else 0,
+                                                 M, N, K), "bnn_binary_dense_expanded")
+        return out, out_exp
 
     def set_operand_bits(self, bits: int):
         self._ck(lib().bnn_set_operand_bits(self._h, bits), "bnn_set_operand_bits")

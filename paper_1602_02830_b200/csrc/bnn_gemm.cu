@@ -392,6 +392,30 @@ extern "C" int bnn_binary_dense(bnn_ctx *ctx, const uint32_t *Ap, int64_t lda_w,
     return gemm_like(ctx, Ap, lda_w, Wp, ldw_w, nullptr, 0, thr, flip, out, ldo_w, M, N, K);
 }
 
+extern "C" int bnn_binary_dense_expanded(bnn_ctx *ctx, const void *A_exp, int64_t lda_bytes, const void *W_exp, int64_t ldw_bytes,
+                                         int operand_bits, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits,
+                                         int64_t ldo_w, void *out_exp, int64_t ldo_exp, int64_t M, int64_t N, int64_t K) {
+    if (!ctx || M < 0 || N < 0 || K <= 0 || (operand_bits != 4 && operand_bits != 8)) return BNN_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return BNN_OK;
+    if (!A_exp || !W_exp || !thr || (!out_bits && !out_exp)) return BNN_ERR_INVALID_ARG;
+    const int64_t ld_min = operand_bits == 4 ? bnn_umma_operand_ld_f4(K) : bnn_umma_operand_ld(K);
+    if (lda_bytes < ld_min || ldw_bytes < ld_min) return BNN_ERR_INVALID_ARG;
+    if (out_bits)
+        if (int st = bnn_check_packed(out_bits, ldo_w, N, M)) return st;
+    if (out_exp) {
+        const int64_t lo_min = operand_bits == 4 ? bnn_umma_operand_ld_f4(N) : bnn_umma_operand_ld(N);
+        if (ldo_exp < lo_min) return BNN_ERR_INVALID_ARG;
+        if ((ldo_exp & 15) || !bnn_aligned16(out_exp)) return BNN_ERR_ALIGNMENT;
+    }
+    bnn_device_guard guard(ctx);
+    if (!guard.ok) return BNN_ERR_CUDA;
+    if (operand_bits == 4)
+        return bnn_umma_gemm_f4(ctx, static_cast<const uint8_t *>(A_exp), lda_bytes, static_cast<const uint8_t *>(W_exp), ldw_bytes,
+                                M, N, K, nullptr, 0, thr, flip, out_bits, ldo_w, static_cast<uint8_t *>(out_exp), ldo_exp);
+    return bnn_umma_gemm(ctx, A_exp, lda_bytes, false, static_cast<const int8_t *>(W_exp), ldw_bytes, M, N, K, nullptr, 0, thr,
+                         flip, out_bits, ldo_w, static_cast<int8_t *>(out_exp), ldo_exp);
+}
+
 extern "C" int bnn_first_layer_bitplanes(bnn_ctx *ctx, const uint8_t *X, int64_t ldx, const uint32_t *Wp,
                                          int64_t ldw_w, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits,
                                          int64_t ldo_w, int32_t *out_sums, int64_t lds, int64_t M, int64_t N,

@@ -128,6 +128,31 @@ def test_expand_signs(ctx):
     assert e.shape == (37, 384) and np.array_equal(e[:, :300], x) and not e[:, 300:].any()
 
 
+@pytest.mark.parametrize("bits", [4, 8])
+@pytest.mark.parametrize("M,N,K", [(700, 520, 1000), (1030, 200, 4100), (300, 130, 64)])
+def test_binary_dense_expanded(ctx, M, N, K, bits):
+    """The tensor kernel on operands the caller keeps expanded: packed signs and the next layer's operand, chained
+    through a second layer, against the oracle."""
+    rng = np.random.default_rng(M + N + K + bits)
+    A, W1, W2 = wl.pm1(rng, (M, K)), wl.pm1(rng, (N, K)), wl.pm1(rng, (96, N))
+    thr1 = rng.integers(-30, 31, N).astype(np.int32)
+    thr2 = rng.integers(-10, 11, 96).astype(np.int32)
+    flip1 = rng.integers(0, 2, N).astype(np.uint8)
+    h = oracle.threshold(oracle.gemm(A, W1.T.copy()), thr1, flip1)
+    want2 = oracle.threshold(oracle.gemm(h, W2.T.copy()), thr2, np.zeros(96, np.uint8))
+    expand = ctx.expand_signs_f4 if bits == 4 else ctx.expand_signs
+    Ae = expand(ctx.pack_signs(dev(A, torch.int8)), M, K)
+    W1e = expand(ctx.pack_signs(dev(W1, torch.int8)), N, K)
+    W2e = expand(ctx.pack_signs(dev(W2, torch.int8)), 96, N)
+    flip_p = dev(np_pack_pm1(2 * flip1.astype(np.int8)[None, :] - 1)[0].view(np.int32))
+    out, out_exp = ctx.binary_dense_expanded(Ae, W1e, bits, dev(thr1), flip_p, M, N, K, want_bits=True, want_exp=True)
+    out2, _ = ctx.binary_dense_expanded(out_exp, W2e, bits, dev(thr2), None, M, 96, N)
+    ctx.device_status()
+    got = out.cpu().numpy()
+    assert np.array_equal(np_unpack_pm1(got, N), h) and padding_is_zero(got, N)
+    assert np.array_equal(np_unpack_pm1(out2.cpu().numpy(), 96), want2)
+
+
 @pytest.mark.parametrize("pre_expanded", [True, False])
 @pytest.mark.parametrize("host_io", [False, True])
 def test_mlp_forward_tensor_engine(ctx, host_io, pre_expanded):
