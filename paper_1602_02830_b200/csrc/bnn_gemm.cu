@@ -80,14 +80,18 @@ __global__ void __launch_bounds__(256, (RSMAX <= 16) ? 3 : 1) k_skinny(const Ski
     const uint32_t tail_mask = (p.K & 31) ? ((1u << (p.K & 31)) - 1u) : 0xffffffffu;
     const int64_t l0 = (int64_t)blockIdx.x * 32;
     bnn_pdl_launch_next();
-    bnn_pdl_wait();
+    // Output-layer mode: the small operand and the BatchNorm parameters are weights, not products of the preceding
+    // kernel, so they are staged while that kernel still drains; only the activations wait for it.
+    if (MODE != 1) bnn_pdl_wait();
 
     // the warp's four rows of the large operand: their first 128-bit chunks are requested before anything else
     const int64_t lrow0 = l0 + warp * 4;
     uint4 b[4];
+    if (MODE != 1) {
 #pragma unroll
-    for (int cc = 0; cc < 4; ++cc)
-        b[cc] = load_row_words(p.L + (lrow0 + cc) * p.ldl_w, lrow0 + cc < p.RL, 4 * lane, Kw, tail_mask, true);
+        for (int cc = 0; cc < 4; ++cc)
+            b[cc] = load_row_words(p.L + (lrow0 + cc) * p.ldl_w, lrow0 + cc < p.RL, 4 * lane, Kw, tail_mask, true);
+    }
 
     {   // 32-bit index arithmetic: RS <= 32 rows of at most 2^24 128-bit groups
         const uint32_t gpr = (uint32_t)(Kw4 >> 2), total = (uint32_t)p.RS * gpr;
@@ -104,6 +108,12 @@ __global__ void __launch_bounds__(256, (RSMAX <= 16) ? 3 : 1) k_skinny(const Ski
         const double a = (double)p.gamma[tid] / sqrt((double)p.var[tid] + p.eps);
         bn_a[tid] = a;
         bn_b[tid] = (double)p.beta[tid] - (double)p.mean[tid] * a;
+    }
+    if (MODE == 1) {
+        bnn_pdl_wait();
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc)
+            b[cc] = load_row_words(p.L + (lrow0 + cc) * p.ldl_w, lrow0 + cc < p.RL, 4 * lane, Kw, tail_mask, true);
     }
     __syncthreads();
 
