@@ -33,7 +33,10 @@ struct bnn_ctx {
 
 // Programmatic dependent launch: the kernel may be set up on the GPU while its predecessor in the stream still runs.
 // Kernels launched this way call bnn_pdl_wait() before their first access to global memory; it returns once the
-// predecessor has completed and its writes are visible (immediately for an ordinary launch).
+// predecessor has completed and its writes are visible (immediately for an ordinary launch).  They release their own
+// successor (bnn_pdl_launch_next) only after that wait, so by the time a kernel runs at all, everything older than its
+// immediate predecessor is complete: the only data a kernel may touch before its wait is data that the immediately
+// preceding kernel does not write (weights and parameters prepared earlier).
 template <typename... KArgs, typename... Args>
 static inline cudaError_t bnn_launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
                                                Args &&...args) {

@@ -79,10 +79,9 @@ __global__ void __launch_bounds__(256, (RSMAX <= 16) ? 3 : 1) k_skinny(const Ski
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t tail_mask = (p.K & 31) ? ((1u << (p.K & 31)) - 1u) : 0xffffffffu;
     const int64_t l0 = (int64_t)blockIdx.x * 32;
-    bnn_pdl_launch_next();
     // Output-layer mode: the small operand and the BatchNorm parameters are weights, not products of the preceding
     // kernel, so they are staged while that kernel still drains; only the activations wait for it.
-    if (MODE != 1) bnn_pdl_wait();
+    if (MODE != 1) { bnn_pdl_wait(); bnn_pdl_launch_next(); }
 
     // the warp's four rows of the large operand: their first 128-bit chunks are requested before anything else
     const int64_t lrow0 = l0 + warp * 4;
@@ -111,6 +110,7 @@ __global__ void __launch_bounds__(256, (RSMAX <= 16) ? 3 : 1) k_skinny(const Ski
     }
     if (MODE == 1) {
         bnn_pdl_wait();
+        bnn_pdl_launch_next();
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc)
             b[cc] = load_row_words(p.L + (lrow0 + cc) * p.ldl_w, lrow0 + cc < p.RL, 4 * lane, Kw, tail_mask, true);

@@ -20,14 +20,15 @@ int64_t bnn_umma_operand_ld(int64_t K);                   // its row pitch in by
 int bnn_umma_expand(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t rows, int64_t K, int8_t *dst);
 int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, const int8_t *B8, int64_t ldb8, int64_t M,
                   int64_t N, int64_t K, int32_t *C, int64_t ldc, const int32_t *thr, const uint32_t *flip, uint32_t *out,
-                  int64_t ldo, int8_t *out8, int64_t ldo8, int pool = 0, int64_t H = 0, int64_t W = 0, int out_f4 = 0);
+                  int64_t ldo, int8_t *out8, int64_t ldo8, int pool = 0, int64_t H = 0, int64_t W = 0, int out_f4 = 0,
+                  int b_static = 0);   // b_static: B8 is not written by the kernel launched just before (it may be read early)
 // 4-bit (e2m1) operands: +-1 exactly, twice the MMA rate of the byte format (plain products only)
 int64_t bnn_umma_operand_ld_f4(int64_t K);
 size_t bnn_umma_operand_bytes_f4(int64_t rows, int64_t K);
 int bnn_umma_expand_f4(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t rows, int64_t K, uint8_t *dst);
 int bnn_umma_gemm_f4(bnn_ctx *ctx, const uint8_t *A4, int64_t lda4, const uint8_t *B4, int64_t ldb4, int64_t M, int64_t N,
                      int64_t K, int32_t *C, int64_t ldc, const int32_t *thr, const uint32_t *flip, uint32_t *out, int64_t ldo,
-                     uint8_t *out4, int64_t ldo4);
+                     uint8_t *out4, int64_t ldo4, int b_static = 0);
 int bnn_umma_im2col_u8(bnn_ctx *ctx, const uint8_t *act, int64_t B, int64_t H, int64_t W, int64_t C_in, uint8_t *dst);
 // First convolution on the tensor engine: worth it from this many pixels / filters on.
 static inline bool bnn_umma_first_conv_ok(int64_t pixels, int64_t C_out) { return pixels >= 16384 && C_out >= 64; }

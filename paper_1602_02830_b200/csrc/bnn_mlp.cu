@@ -124,7 +124,8 @@ int forward_device_tensor(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X,
             }
             st = bnn_umma_gemm(ctx, k == 0 ? static_cast<const void *>(X) : cur8, k == 0 ? ldx : bnn_umma_operand_ld(D.K), k == 0, Wk8,
                                bnn_umma_operand_ld(D.K), batch, D.N, D.K, nullptr, 0, D.thr, D.flip, dst_bits, ldo,
-                               need_next ? dst8 : nullptr, ld_next, 0, 0, 0, f4 ? 1 : 0);
+                               need_next ? dst8 : nullptr, ld_next, 0, 0, 0, f4 ? 1 : 0,
+                               (k > 0 && D.W8) ? 1 : 0);   // from layer 2 on the kernel before wrote activations, not these weights
         } else {
             const uint8_t *Wk4 = D.W4;
             if (!Wk4) {
@@ -133,7 +134,7 @@ int forward_device_tensor(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X,
             }
             st = bnn_umma_gemm_f4(ctx, reinterpret_cast<const uint8_t *>(cur8), bnn_umma_operand_ld_f4(D.K), Wk4,
                                   bnn_umma_operand_ld_f4(D.K), batch, D.N, D.K, nullptr, 0, D.thr, D.flip, dst_bits, ldo,
-                                  need_next ? reinterpret_cast<uint8_t *>(dst8) : nullptr, ld_next);
+                                  need_next ? reinterpret_cast<uint8_t *>(dst8) : nullptr, ld_next, D.W4 ? 1 : 0);
         }
         if (st) return st;
         if (hidden_out && hidden_out[k])

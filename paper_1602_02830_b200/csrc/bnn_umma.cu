@@ -71,6 +71,7 @@ struct UmmaArgs {
     int H, W, TH, TB;       // image size; a 128-pixel tile = TB images x TH rows x W columns
     int c_chunks;           // C_in / 128
     int pool;               // 2x2 max-pool (as OR of the sign bits) before the packed store
+    int b_static;           // B (weights) is not written by the kernel launched just before this one
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -425,8 +426,9 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = ctl->tmem_base;
-    bnn_pdl_launch_next();
-    bnn_pdl_wait();                                      // barriers and tensor memory were set up while the predecessor drained
+    // Barriers and tensor memory were set up while the preceding kernel drained; what reads or writes global memory
+    // waits for it below (bnn_pdl_wait): the producer (after requesting weights that kernel does not write), the
+    // epilogue warps at once; they also release this kernel's own successor.
 
     if (BN == 192) {
         // 4-bit engine: every value is exactly +-1, so every block scale is 2^0.  In UE8M0 that is the byte 0x7f, and
@@ -451,7 +453,20 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
             // with them a 3x3 convolution's producer could not keep up: 128 -> 128 channels at 32 x 32, 88 -> 57 us).
             uint32_t s = 0, ph = 0;                      // ring slot, and the number of times the ring has wrapped
             const uint32_t tn32 = (uint32_t)tiles_n;
+            // B is weights, not a product of the preceding kernel: its share of the first ring fill is requested before
+            // the wait for that kernel, A's after it
+            const int npre = !p.b_static ? 0 : (p.k_iters < STAGES ? p.k_iters : STAGES);
+            {
+                const int n0f = (int)((blockIdx.x % tn32) * BN);
+                for (int kit = 0; kit < npre; ++kit) {
+                    const uint32_t bar = smem_u32(&ctl->full[kit]);
+                    mbar_expect_tx(bar, STAGE_BYTES);
+                    tma_load_2d(smem_u32(tiles + kit * STAGE_BYTES + A_BYTES), &mapB, kit * BK, n0f, bar);
+                }
+            }
+            bnn_pdl_wait();
             for (uint32_t t = blockIdx.x; t < (uint32_t)ntiles && ok; t += gridDim.x) {
+                const bool first_tile = (t == blockIdx.x);
                 const uint32_t tm = t / tn32;
                 const int m0 = (int)(tm * BM), n0 = (int)((t - tm * tn32) * BN);
                 int b0 = 0, y0 = 0;
@@ -464,9 +479,10 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                 }
                 int cc = 0, tx = -1, ty = -1;            // channel slice and tap offsets of the current K step
                 for (int kit = 0; kit < p.k_iters; ++kit) {
+                    const bool pre = first_tile && kit < npre;      // B already requested, bytes already expected
                     if (ph > 0 && !mbar_wait(smem_u32(&ctl->empty[s]), (ph - 1) & 1)) { fail(ctl, 1); ok = false; break; }
                     const uint32_t bar = smem_u32(&ctl->full[s]);
-                    mbar_expect_tx(bar, STAGE_BYTES);
+                    if (!pre) mbar_expect_tx(bar, STAGE_BYTES);
                     const uint32_t dst = smem_u32(tiles + s * STAGE_BYTES);
                     if (p.conv) {
                         tma_load_4d(dst, &mapA, cc * BK, tx, y0 + ty, b0, bar);
@@ -474,7 +490,7 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                     } else {
                         tma_load_2d(dst, &mapA, kit * BK, m0, bar);
                     }
-                    tma_load_2d(dst + A_BYTES, &mapB, kit * BK, n0, bar);
+                    if (!pre) tma_load_2d(dst + A_BYTES, &mapB, kit * BK, n0, bar);
                     if (++s == (uint32_t)STAGES) { s = 0; ++ph; }
                 }
             }
@@ -525,6 +541,8 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
     } else if (warp < 2 + EPI_WARPS) {
         // ---------------- epilogue: warps 2..9; warp w may only touch TMEM lanes 32*(w%4) .. +31, so two warps share
         // each lane quadrant and split the tile's columns between them
+        bnn_pdl_wait();
+        bnn_pdl_launch_next();
         const int q = warp & 3;
         const int half = (warp - 2) >> 2;
         const int et = threadIdx.x - 64;                 // 0 .. EPI_THREADS-1 among the epilogue threads
@@ -650,8 +668,6 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     cluster_sync_all();                                     // both CTAs' barriers exist before anyone signals them
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = ctl->tmem_base;
-    bnn_pdl_launch_next();
-    bnn_pdl_wait();
 
     if (BN == 192) {
         // 4-bit engine: unit block scales (byte 0x7f) in this CTA's scale-factor columns; the leader's MMAs read the
@@ -674,16 +690,28 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
             bool ok = true;
             uint32_t s = 0, ph = 0;                      // ring slot, and the number of times the ring has wrapped
             const uint32_t tn32 = (uint32_t)tiles_n;
+            // the weights of the first ring fill are requested before the wait for the preceding kernel (see k_umma_i8)
+            const int npre = !p.b_static ? 0 : (p.k_iters < STAGES2 ? p.k_iters : STAGES2);
+            {
+                const int nb0f = (int)(((uint32_t)pair % tn32) * BN + rank * (BN / 2));
+                for (int kit = 0; kit < npre; ++kit) {
+                    if (rank == 0) mbar_expect_tx(smem_u32(&ctl->full[kit]), 2 * STAGE2_BYTES);
+                    tma_load_2d_2sm(smem_u32(tiles + kit * STAGE2_BYTES + A_BYTES), &mapB, kit * BK, nb0f, smem_u32(&ctl->full[kit]) & PEER_MASK);
+                }
+            }
+            bnn_pdl_wait();
             for (uint32_t t = (uint32_t)pair; t < (uint32_t)ntiles && ok; t += (uint32_t)npairs) {
+                const bool first_tile = (t == (uint32_t)pair);
                 const uint32_t tm = t / tn32;
                 const int m0 = (int)(tm * (2 * BM) + rank * BM);
                 const int nb0 = (int)((t - tm * tn32) * BN + rank * (BN / 2));
                 for (int kit = 0; kit < p.k_iters; ++kit) {
+                    const bool pre = first_tile && kit < npre;
                     if (ph > 0 && !mbar_wait(smem_u32(&ctl->empty[s]), (ph - 1) & 1)) { fail(ctl, 11); ok = false; break; }
-                    if (rank == 0) mbar_expect_tx(smem_u32(&ctl->full[s]), 2 * STAGE2_BYTES);   // the bytes of both CTAs
+                    if (rank == 0 && !pre) mbar_expect_tx(smem_u32(&ctl->full[s]), 2 * STAGE2_BYTES);   // the bytes of both CTAs
                     const uint32_t bar0 = smem_u32(&ctl->full[s]) & PEER_MASK;
                     tma_load_2d_2sm(smem_u32(tiles + s * STAGE2_BYTES), &mapA, kit * BK, m0, bar0);
-                    tma_load_2d_2sm(smem_u32(tiles + s * STAGE2_BYTES + A_BYTES), &mapB, kit * BK, nb0, bar0);
+                    if (!pre) tma_load_2d_2sm(smem_u32(tiles + s * STAGE2_BYTES + A_BYTES), &mapB, kit * BK, nb0, bar0);
                     if (++s == (uint32_t)STAGES2) { s = 0; ++ph; }
                 }
             }
@@ -729,6 +757,8 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         }
     } else if (warp < 2 + EPI_WARPS) {
         // ---------------- epilogue (both CTAs): this CTA's 128 rows of the pair's tile
+        bnn_pdl_wait();
+        bnn_pdl_launch_next();
         const int q = warp & 3;
         const int half = (warp - 2) >> 2;
         const int et = threadIdx.x - 64;
@@ -762,8 +792,8 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
 // One thread per 32-bit word = 32 output bytes (two 128-bit stores).
 __global__ void __launch_bounds__(256) k_expand_s8(const uint32_t *__restrict__ src, int64_t ld_w, int64_t rows, int64_t K,
                                                    int8_t *__restrict__ dst, int64_t ld8) {
-    bnn_pdl_launch_next();
     bnn_pdl_wait();
+    bnn_pdl_launch_next();
     const int64_t wpr = ld8 >> 5;            // words per output row (ld8 is a multiple of 32)
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= rows * wpr) return;
@@ -790,8 +820,8 @@ __global__ void __launch_bounds__(256) k_expand_s8(const uint32_t *__restrict__ 
 // the low nibble); nibbles at or beyond K are 0 (= +0.0).  One thread per 32-bit word = 16 output bytes.
 __global__ void __launch_bounds__(256) k_expand_f4(const uint32_t *__restrict__ src, int64_t ld_w, int64_t rows, int64_t K,
                                                    uint8_t *__restrict__ dst, int64_t ld4) {
-    bnn_pdl_launch_next();
     bnn_pdl_wait();
+    bnn_pdl_launch_next();
     const int64_t wpr = ld4 >> 4;            // words per output row (ld4 is a multiple of 128 bytes)
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= rows * wpr) return;
@@ -816,8 +846,8 @@ __global__ void __launch_bounds__(256) k_expand_f4(const uint32_t *__restrict__ 
 // outside the image as zeros) written as one 32-byte row, byte (tap * C_in + c).  One thread per pixel.
 __global__ void __launch_bounds__(256) k_im2col_u8(const uint8_t *__restrict__ act, int64_t B, int H, int W, int Cin,
                                                    uint8_t *__restrict__ dst) {
-    bnn_pdl_launch_next();
     bnn_pdl_wait();
+    bnn_pdl_launch_next();
     const int64_t pix = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (pix >= B * H * W) return;
     const int x = (int)(pix % W), y = (int)((pix / W) % H);
@@ -969,7 +999,7 @@ int bnn_umma_expand_f4(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t 
 // the outputs as nibbles for a following layer, pitch ldo4 bytes.
 int bnn_umma_gemm_f4(bnn_ctx *ctx, const uint8_t *A4, int64_t lda4, const uint8_t *B4, int64_t ldb4, int64_t M, int64_t N,
                      int64_t K, int32_t *C, int64_t ldc, const int32_t *thr, const uint32_t *flip, uint32_t *out, int64_t ldo,
-                     uint8_t *out4, int64_t ldo4) {
+                     uint8_t *out4, int64_t ldo4, int b_static) {
     if (M == 0 || N == 0) return BNN_OK;
     if ((lda4 & 15) || (ldb4 & 15) || !bnn_aligned16(A4) || !bnn_aligned16(B4)) return BNN_ERR_ALIGNMENT;
     if (M > 0x7fffffff || N > 0x7fffffff || K <= 0 || K > (1 << 24)) return BNN_ERR_INVALID_ARG;
@@ -984,7 +1014,7 @@ int bnn_umma_gemm_f4(bnn_ctx *ctx, const uint8_t *A4, int64_t lda4, const uint8_
     a.k_iters = (int)((K + 2 * BK - 1) / (2 * BK));          // 256 values per 128-byte K step
     a.k_last = (int)((K - 2 * BK * (int64_t)(a.k_iters - 1) + 63) / 64);
     a.C = C; a.ldc = ldc; a.out = out; a.ldo = ldo; a.thr = thr; a.flip = flip;
-    a.out8 = reinterpret_cast<int8_t *>(out4); a.ldo8 = ldo4; a.out_f4 = 1;
+    a.out8 = reinterpret_cast<int8_t *>(out4); a.ldo8 = ldo4; a.out_f4 = 1; a.b_static = b_static;
     if (pairs > 0) {
         if (int st = umma_prepare(ctx)) return st;
         const int64_t tiles2 = ((M + 2 * BM - 1) / (2 * BM)) * ((N + 191) / 192);
@@ -1000,7 +1030,7 @@ int bnn_umma_gemm_f4(bnn_ctx *ctx, const uint8_t *A4, int64_t lda4, const uint8_
 // C / bits = A8 (M x K bytes, pitch lda8; unsigned if a_unsigned) times B8^T (N x K signed bytes, pitch ldb8).
 int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, const int8_t *B8, int64_t ldb8, int64_t M,
                   int64_t N, int64_t K, int32_t *C, int64_t ldc, const int32_t *thr, const uint32_t *flip, uint32_t *out,
-                  int64_t ldo, int8_t *out8, int64_t ldo8, int pool, int64_t H, int64_t W, int out_f4) {
+                  int64_t ldo, int8_t *out8, int64_t ldo8, int pool, int64_t H, int64_t W, int out_f4, int b_static) {
     if (M == 0 || N == 0) return BNN_OK;
     if (pool) {   // rows are pixels of H x W images in (b, y, x) order; 128-row tiles must hold whole 2x2 windows
         int TH, TB;
@@ -1026,7 +1056,7 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
     a.k_last = (int)((K - BK * (int64_t)(a.k_iters - 1) + 31) / 32);
     a.idesc = (2u << 4) | ((a_unsigned ? 0u : 1u) << 7) | (1u << 10) | ((uint32_t)(BM >> 4) << 24);   // N field added by the kernel
     a.C = C; a.ldc = ldc; a.out = out; a.ldo = ldo; a.out8 = out8; a.ldo8 = ldo8; a.thr = thr; a.flip = flip;
-    a.pool = pool; a.H = (int)H; a.W = (int)W; a.out_f4 = out_f4;
+    a.pool = pool; a.H = (int)H; a.W = (int)W; a.out_f4 = out_f4; a.b_static = b_static;
     if (pairs > 0) {
         const int64_t tiles2 = ((M + 2 * BM - 1) / (2 * BM)) * ((N + 255) / 256);
         if (tiles2 >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;
