@@ -33,15 +33,22 @@ namespace {
 constexpr int BM = 128, BK = 128;               // BK in bytes = int8 elements
 constexpr int BN_MAX = 256;                     // tile width: 256, or 128 for narrow outputs; 192 = the 4-bit engine
 constexpr uint32_t SF_COL = 480;                // 4-bit engine: first of the 32 TMEM columns that hold the scale factors
-#ifndef BNN_EPI_WARPS
-#define BNN_EPI_WARPS 8
+constexpr int N_ISSUE = 2;                      // MMA-issuing warps: warp 1 and the warps behind the epilogue warps
+// Epilogue warps per tile width: EPW per TMEM lane quadrant.  With two, each takes a contiguous half of the columns and
+// prefetches its next chunk; with four, chunks go round-robin and the other warps of the scheduler cover the load
+// latency (one register buffer, so the kernel fits 608 threads).  Four measured faster where signs are the output of
+// 256-wide tiles (first layer of the MLP, convolutions), two where int32 sums are stored (the 192-wide GEMM).
+template <int BN> struct Warps {
+#ifdef BNN_EPI_WARPS
+    static constexpr int EPI_WARPS = BNN_EPI_WARPS;
+#else
+    static constexpr int EPI_WARPS = (BN == 256) ? 16 : 8;
 #endif
-constexpr int EPI_WARPS = BNN_EPI_WARPS;        // EPW per TMEM lane quadrant; the tile's 32-column chunks go round-robin over them
-constexpr int EPW = EPI_WARPS / 4;
-constexpr int EPI_THREADS = EPI_WARPS * 32;
-constexpr int N_ISSUE = 2;                      // MMA-issuing warps: warp 1 and the warps from MMA_WARP_B on
-constexpr int MMA_WARP_B = 2 + EPI_WARPS;
-constexpr int NTHREADS = 64 + EPI_THREADS + 32 * (N_ISSUE - 1);
+    static constexpr int EPW = EPI_WARPS / 4;
+    static constexpr int EPI_THREADS = EPI_WARPS * 32;
+    static constexpr int MMA_WARP_B = 2 + EPI_WARPS;                 // the second MMA-issuing warp (the first is warp 1)
+    static constexpr int NTHREADS = 64 + EPI_THREADS + 32 * (N_ISSUE - 1);
+};
 constexpr uint32_t A_BYTES = BM * BK;
 constexpr int ACC_BUFS = 2;
 template <int BN> struct Cfg {
@@ -289,6 +296,7 @@ __device__ __forceinline__ int32_t staged_threshold(int32_t t) {
 template <int BN>
 __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, uint32_t tmem_base, uint32_t buf, uint32_t tc,
                                               int64_t m0, int64_t n0, int64_t n0_next, int q, int half, int lane, int et, bool &ok) {
+    constexpr int EPW = Warps<BN>::EPW, EPI_THREADS = Warps<BN>::EPI_THREADS;
     static_assert(BN <= EPI_THREADS, "one staged threshold per epilogue thread");
     constexpr int CHUNKS = BN / 32, CPW = CHUNKS / 2;   // 32-column chunks per tile and per warp (two warps per quadrant)
     const int64_t row = m0 + 32 * q + lane;
@@ -393,10 +401,11 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
 // runs on across tiles; the accumulator is double-buffered in tensor memory (2 x 256 columns), so the
 // epilogue of tile i overlaps the main loop of tile i+1.
 template <int BN>
-__global__ void __launch_bounds__(NTHREADS, 1)
+__global__ void __launch_bounds__(Warps<BN>::NTHREADS, 1)
 k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const UmmaArgs p) {
     constexpr int STAGES = Cfg<BN>::STAGES;
     constexpr uint32_t STAGE_BYTES = Cfg<BN>::STAGE_BYTES;
+    constexpr int EPI_WARPS = Warps<BN>::EPI_WARPS, MMA_WARP_B = Warps<BN>::MMA_WARP_B;
     constexpr uint32_t TMEM_COLS = Cfg<BN>::TMEM_COLS;
     extern __shared__ uint8_t smem_raw[];
     // operand tiles need 1024-byte alignment for the 128-byte swizzle pattern
@@ -634,10 +643,11 @@ __device__ __forceinline__ void umma_mxf4_2sm(uint32_t tmem_d, uint64_t adesc, u
 }
 
 template <int BN>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(Warps<BN>::NTHREADS, 1)
 k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const UmmaArgs p) {
     constexpr int STAGES2 = Cfg2<BN>::STAGES;
     constexpr uint32_t STAGE2_BYTES = Cfg2<BN>::STAGE_BYTES;
+    constexpr int EPI_WARPS = Warps<BN>::EPI_WARPS, MMA_WARP_B = Warps<BN>::MMA_WARP_B;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     Control *ctl = reinterpret_cast<Control *>(tiles + STAGES2 * STAGE2_BYTES);
@@ -939,7 +949,7 @@ static int umma2_max_pairs(bnn_ctx *ctx) {
         if (cudaFuncSetAttribute(k_umma_i8_2sm<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma2_smem_bytes<BN>()) == cudaSuccess) {
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3(2 * ctx->sm_count, 1, 1);
-            cfg.blockDim = dim3(NTHREADS, 1, 1);
+            cfg.blockDim = dim3(Warps<BN>::NTHREADS, 1, 1);
             cfg.dynamicSmemBytes = umma2_smem_bytes<BN>();
             cudaLaunchAttribute attr;
             attr.id = cudaLaunchAttributeClusterDimension;
@@ -958,10 +968,10 @@ static int umma_launch(bnn_ctx *ctx, const CUtensorMap &mapA, const CUtensorMap 
     const int64_t tiles = ((a.M + BM - 1) / BM) * ((a.N + bn - 1) / bn);
     if (tiles >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;      // the kernels count tiles in 32 bits
     const int64_t grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
-    const dim3 g((unsigned)grid), b(NTHREADS);
-    if (bn == 192) BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8<192>, g, b, umma_smem_bytes<192>(), ctx->stream, mapA, mapB, a));
-    else if (bn == 256) BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8<256>, g, b, umma_smem_bytes<256>(), ctx->stream, mapA, mapB, a));
-    else BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8<128>, g, b, umma_smem_bytes<128>(), ctx->stream, mapA, mapB, a));
+    const dim3 g((unsigned)grid);
+    if (bn == 192) BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8<192>, g, dim3(Warps<192>::NTHREADS), umma_smem_bytes<192>(), ctx->stream, mapA, mapB, a));
+    else if (bn == 256) BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8<256>, g, dim3(Warps<256>::NTHREADS), umma_smem_bytes<256>(), ctx->stream, mapA, mapB, a));
+    else BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8<128>, g, dim3(Warps<128>::NTHREADS), umma_smem_bytes<128>(), ctx->stream, mapA, mapB, a));
     return bnn_check_launch(ctx);
 }
 
@@ -1020,7 +1030,7 @@ int bnn_umma_gemm_f4(bnn_ctx *ctx, const uint8_t *A4, int64_t lda4, const uint8_
         const int64_t tiles2 = ((M + 2 * BM - 1) / (2 * BM)) * ((N + 191) / 192);
         if (tiles2 >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;
         const int64_t use = tiles2 < pairs ? tiles2 : pairs;
-        BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8_2sm<192>, dim3((unsigned)(2 * use)), dim3(NTHREADS), umma2_smem_bytes<192>(),
+        BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8_2sm<192>, dim3((unsigned)(2 * use)), dim3(Warps<192>::NTHREADS), umma2_smem_bytes<192>(),
                                                ctx->stream, mapA, mapB, a));
         return bnn_check_launch(ctx);
     }
@@ -1061,7 +1071,7 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
         const int64_t tiles2 = ((M + 2 * BM - 1) / (2 * BM)) * ((N + 255) / 256);
         if (tiles2 >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;
         const int64_t use = tiles2 < pairs ? tiles2 : pairs;
-        BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8_2sm<256>, dim3((unsigned)(2 * use)), dim3(NTHREADS), umma2_smem_bytes<256>(),
+        BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8_2sm<256>, dim3((unsigned)(2 * use)), dim3(Warps<256>::NTHREADS), umma2_smem_bytes<256>(),
                                                ctx->stream, mapA, mapB, a));
         return bnn_check_launch(ctx);
     }
