@@ -37,12 +37,12 @@ constexpr int N_ISSUE = 2;                      // MMA-issuing warps: warp 1 and
 // Epilogue warps per tile width: EPW per TMEM lane quadrant.  With two, each takes a contiguous half of the columns and
 // prefetches its next chunk; with four, chunks go round-robin and the other warps of the scheduler cover the load
 // latency (one register buffer, so the kernel fits 608 threads).  Four measured faster where signs are the output of
-// 256-wide tiles (first layer of the MLP, convolutions), two where int32 sums are stored (the 192-wide GEMM).
+// 256- and 128-wide tiles (first layer of the MLP, convolutions), two where int32 sums are stored (the 192-wide GEMM).
 template <int BN> struct Warps {
 #ifdef BNN_EPI_WARPS
     static constexpr int EPI_WARPS = BNN_EPI_WARPS;
 #else
-    static constexpr int EPI_WARPS = (BN == 256) ? 16 : 8;
+    static constexpr int EPI_WARPS = (BN == 192) ? 8 : 16;
 #endif
     static constexpr int EPW = EPI_WARPS / 4;
     static constexpr int EPI_THREADS = EPI_WARPS * 32;
