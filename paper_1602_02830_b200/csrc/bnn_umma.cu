@@ -854,6 +854,8 @@ __global__ void __launch_bounds__(256) k_expand_f4(const uint32_t *__restrict__ 
 
 // First convolution: the 3x3 neighbourhood of every pixel of an 8-bit NHWC image (9 * C_in <= 32 bytes, taps
 // outside the image as zeros) written as one 32-byte row, byte (tap * C_in + c).  One thread per pixel.
+// CIN > 0: the channel count as a compile-time constant (the packing below then stays in registers); 0: run-time Cin.
+template <int CIN>
 __global__ void __launch_bounds__(256) k_im2col_u8(const uint8_t *__restrict__ act, int64_t B, int H, int W, int Cin,
                                                    uint8_t *__restrict__ dst) {
     bnn_pdl_wait();
@@ -863,13 +865,27 @@ __global__ void __launch_bounds__(256) k_im2col_u8(const uint8_t *__restrict__ a
     const int x = (int)(pix % W), y = (int)((pix / W) % H);
     const int64_t b = pix / ((int64_t)W * H);
     uint32_t w[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
-    for (int tap = 0; tap < 9; ++tap) {
-        const int yy = y + tap / 3 - 1, xx = x + tap % 3 - 1;
-        if (yy < 0 || yy >= H || xx < 0 || xx >= W) continue;
-        const uint8_t *px = act + ((b * H + yy) * W + xx) * Cin;
-        for (int c = 0; c < Cin; ++c) {
-            const int k = tap * Cin + c;
-            w[k >> 2] |= (uint32_t)px[c] << (8 * (k & 3));
+    if (CIN > 0) {
+#pragma unroll
+        for (int tap = 0; tap < 9; ++tap) {
+            const int yy = y + tap / 3 - 1, xx = x + tap % 3 - 1;
+            if (yy < 0 || yy >= H || xx < 0 || xx >= W) continue;
+            const uint8_t *px = act + ((b * H + yy) * W + xx) * CIN;
+#pragma unroll
+            for (int c = 0; c < CIN; ++c) {
+                const int k = tap * CIN + c;
+                w[k >> 2] |= (uint32_t)px[c] << (8 * (k & 3));
+            }
+        }
+    } else {
+        for (int tap = 0; tap < 9; ++tap) {
+            const int yy = y + tap / 3 - 1, xx = x + tap % 3 - 1;
+            if (yy < 0 || yy >= H || xx < 0 || xx >= W) continue;
+            const uint8_t *px = act + ((b * H + yy) * W + xx) * Cin;
+            for (int c = 0; c < Cin; ++c) {
+                const int k = tap * Cin + c;
+                w[k >> 2] |= (uint32_t)px[c] << (8 * (k & 3));
+            }
         }
     }
     uint4 *d = reinterpret_cast<uint4 *>(dst + pix * 32);
@@ -1100,7 +1116,12 @@ int bnn_umma_im2col_u8(bnn_ctx *ctx, const uint8_t *act, int64_t B, int64_t H, i
     if (total == 0) return BNN_OK;
     const int64_t blocks = (total + 255) / 256;
     if (blocks > 0x7fffffff || 9 * C_in > 32) return BNN_ERR_INVALID_ARG;
-    BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_im2col_u8, dim3((unsigned)blocks), dim3(256), 0, ctx->stream, act, B, (int)H, (int)W, (int)C_in, dst));
+    if (C_in == 3)
+        BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_im2col_u8<3>, dim3((unsigned)blocks), dim3(256), 0, ctx->stream, act, B, (int)H, (int)W, (int)C_in, dst));
+    else if (C_in == 1)
+        BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_im2col_u8<1>, dim3((unsigned)blocks), dim3(256), 0, ctx->stream, act, B, (int)H, (int)W, (int)C_in, dst));
+    else
+        BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_im2col_u8<0>, dim3((unsigned)blocks), dim3(256), 0, ctx->stream, act, B, (int)H, (int)W, (int)C_in, dst));
     return bnn_check_launch(ctx);
 }
 
