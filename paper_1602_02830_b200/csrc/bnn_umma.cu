@@ -800,6 +800,11 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
 // ---------------------------------------------------------------------------------------------------------
 // Packed signs -> one signed byte per value (+1 = 0x01, -1 = 0xff); bytes at or beyond K are 0.
 // One thread per 32-bit word = 32 output bytes (two 128-bit stores).
+// Thread index -> (row, word of the row): 32-bit division whenever the launch has fewer than 2^32 threads' worth of words.
+__device__ __forceinline__ void row_and_word(int64_t idx, int64_t wpr, int64_t total, int64_t &r, int64_t &w) {
+    if (total <= 0xffffffffll) { const uint32_t rr = (uint32_t)idx / (uint32_t)wpr; r = rr; w = (uint32_t)idx - rr * (uint32_t)wpr; }
+    else { r = idx / wpr; w = idx - r * wpr; }
+}
 __global__ void __launch_bounds__(256) k_expand_s8(const uint32_t *__restrict__ src, int64_t ld_w, int64_t rows, int64_t K,
                                                    int8_t *__restrict__ dst, int64_t ld8) {
     bnn_pdl_wait();
@@ -807,7 +812,8 @@ __global__ void __launch_bounds__(256) k_expand_s8(const uint32_t *__restrict__ 
     const int64_t wpr = ld8 >> 5;            // words per output row (ld8 is a multiple of 32)
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= rows * wpr) return;
-    const int64_t r = idx / wpr, w = idx - r * wpr;
+    int64_t r, w;
+    row_and_word(idx, wpr, rows * wpr, r, w);
     const int64_t Kw = (K + 31) >> 5;
     uint32_t bits = 0u, valid = 0u;
     if (w < Kw) {
@@ -815,11 +821,19 @@ __global__ void __launch_bounds__(256) k_expand_s8(const uint32_t *__restrict__ 
         valid = (w == Kw - 1 && (K & 31)) ? ((1u << (K & 31)) - 1u) : 0xffffffffu;
     }
     uint32_t b[8];
+    if (valid == 0xffffffffu) {              // every word but a row's last one
 #pragma unroll
-    for (int g = 0; g < 8; ++g) {
-        const uint32_t t = (((bits >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u;      // 0/1 bytes
-        const uint32_t v = (((valid >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u;
-        b[g] = (~(t * 0xfeu)) & (v * 0xffu);
+        for (int g = 0; g < 8; ++g) {
+            const uint32_t t = (((bits >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u;      // 0/1 bytes
+            b[g] = ~(t * 0xfeu);
+        }
+    } else {
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+            const uint32_t t = (((bits >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u;
+            const uint32_t v = (((valid >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u;
+            b[g] = (~(t * 0xfeu)) & (v * 0xffu);
+        }
     }
     uint4 *d = reinterpret_cast<uint4 *>(dst + r * ld8 + 32 * w);
     d[0] = make_uint4(b[0], b[1], b[2], b[3]);
@@ -835,7 +849,8 @@ __global__ void __launch_bounds__(256) k_expand_f4(const uint32_t *__restrict__ 
     const int64_t wpr = ld4 >> 4;            // words per output row (ld4 is a multiple of 128 bytes)
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= rows * wpr) return;
-    const int64_t r = idx / wpr, w = idx - r * wpr;
+    int64_t r, w;
+    row_and_word(idx, wpr, rows * wpr, r, w);
     const int64_t Kw = (K + 31) >> 5;
     uint32_t bits = 0u, valid = 0u;
     if (w < Kw) {
@@ -843,11 +858,16 @@ __global__ void __launch_bounds__(256) k_expand_f4(const uint32_t *__restrict__ 
         valid = (w == Kw - 1 && (K & 31)) ? ((1u << (K & 31)) - 1u) : 0xffffffffu;
     }
     uint32_t q[4];
+    if (valid == 0xffffffffu) {              // every word but a row's last one
 #pragma unroll
-    for (int g = 0; g < 4; ++g) {
-        const uint32_t n = nibbles_of_byte((bits >> (8 * g)) & 0xffu);
-        const uint32_t v = nibbles_of_byte((valid >> (8 * g)) & 0xffu);      // 0x2 where valid, 0xa where not
-        q[g] = n & (((~v >> 3) & 0x11111111u) * 0xfu);                         // keep the nibbles whose valid bit is set
+        for (int g = 0; g < 4; ++g) q[g] = nibbles_of_byte((bits >> (8 * g)) & 0xffu);
+    } else {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const uint32_t n = nibbles_of_byte((bits >> (8 * g)) & 0xffu);
+            const uint32_t v = nibbles_of_byte((valid >> (8 * g)) & 0xffu);      // 0x2 where valid, 0xa where not
+            q[g] = n & (((~v >> 3) & 0x11111111u) * 0xfu);                         // keep the nibbles whose valid bit is set
+        }
     }
     *reinterpret_cast<uint4 *>(dst + r * ld4 + 16 * w) = make_uint4(q[0], q[1], q[2], q[3]);
 }
