@@ -265,14 +265,21 @@ __device__ __forceinline__ void epilogue_chunk(Control *ctl, const UmmaArgs &p, 
     }
     if (p.C) {
         if (BN == 192) {   // the 4-bit engine accumulates in float32: exact integers
+            if (p.k_iters <= (1 << 14)) {
+                // |sum| <= K <= 2^22: adding 1.5 * 2^23 leaves the integer in the low mantissa bits (an add and a
+                // subtract on the full-rate pipes instead of a quarter-rate conversion)
 #pragma unroll
-            for (int j = 0; j < 32; ++j) r[j] = (uint32_t)(int32_t)__uint_as_float(r[j]);
+                for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + 12582912.0f) - 0x4b400000u;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = (uint32_t)(int32_t)__uint_as_float(r[j]);
+            }
         }
         int32_t *dst = p.C + row * p.ldc + col0;
         if (col0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
 #pragma unroll
             for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<int4 *>(dst + j) = make_int4((int)r[j], (int)r[j + 1], (int)r[j + 2], (int)r[j + 3]);
+                __stcs(reinterpret_cast<int4 *>(dst + j), make_int4((int)r[j], (int)r[j + 1], (int)r[j + 2], (int)r[j + 3]));   // streamed: the sums are not re-read, the operands are
         } else {
 #pragma unroll
             for (int j = 0; j < 32; ++j)
