@@ -225,8 +225,13 @@ __device__ __forceinline__ void store_signs(const UmmaArgs &p, uint32_t word, in
             const uint32_t t4 = (((word >> (4 * g)) & 0xfu) * 0x00204081u) & 0x01010101u;
             b[g] = ~(t4 * 0xfeu);
         }
-        *reinterpret_cast<uint4 *>(d8) = make_uint4(b[0], b[1], b[2], b[3]);
-        *reinterpret_cast<uint4 *>(d8 + 16) = make_uint4(b[4], b[5], b[6], b[7]);
+        if ((reinterpret_cast<uintptr_t>(d8) & 31u) == 0) {   // one 256-bit store: a whole 32-byte sector per thread
+            asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                         ::"l"(d8), "r"(b[0]), "r"(b[1]), "r"(b[2]), "r"(b[3]), "r"(b[4]), "r"(b[5]), "r"(b[6]), "r"(b[7]) : "memory");
+        } else {
+            *reinterpret_cast<uint4 *>(d8) = make_uint4(b[0], b[1], b[2], b[3]);
+            *reinterpret_cast<uint4 *>(d8 + 16) = make_uint4(b[4], b[5], b[6], b[7]);
+        }
     } else {
         for (int j = 0; j < 32; ++j)
             if (col0 + j < p.N) d8[j] = ((word >> j) & 1u) ? (int8_t)1 : (int8_t)-1;
@@ -276,7 +281,15 @@ __device__ __forceinline__ void epilogue_chunk(Control *ctl, const UmmaArgs &p, 
             }
         }
         int32_t *dst = p.C + row * p.ldc + col0;
-        if (col0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
+        if (col0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 31u) == 0)) {
+            // 256-bit stores: whole 32-byte sectors, four instructions for the thread's 128 bytes; streamed, because the
+            // sums are not re-read while the operands are
+#pragma unroll
+            for (int j = 0; j < 32; j += 8)
+                asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                             ::"l"(dst + j), "r"(r[j]), "r"(r[j + 1]), "r"(r[j + 2]), "r"(r[j + 3]), "r"(r[j + 4]), "r"(r[j + 5]),
+                               "r"(r[j + 6]), "r"(r[j + 7]) : "memory");
+        } else if (col0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
 #pragma unroll
             for (int j = 0; j < 32; j += 4)
                 __stcs(reinterpret_cast<int4 *>(dst + j), make_int4((int)r[j], (int)r[j + 1], (int)r[j + 2], (int)r[j + 3]));   // streamed: the sums are not re-read, the operands are
