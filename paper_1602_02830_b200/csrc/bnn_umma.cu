@@ -820,6 +820,11 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
 // ---------------------------------------------------------------------------------------------------------
 // Packed signs -> one signed byte per value (+1 = 0x01, -1 = 0xff); bytes at or beyond K are 0.
 // One thread per 32-bit word = 32 output bytes (two 128-bit stores).
+// 32 bytes to a 32-byte aligned global address in one instruction (a whole sector per thread).
+__device__ __forceinline__ void store_256(void *dst, const uint32_t (&v)[8]) {
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"l"(dst), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
+}
 // Thread index -> (row, word of the row): 32-bit division whenever the launch has fewer than 2^32 threads' worth of words.
 __device__ __forceinline__ void row_and_word(int64_t idx, int64_t wpr, int64_t total, int64_t &r, int64_t &w) {
     if (total <= 0xffffffffll) { const uint32_t rr = (uint32_t)idx / (uint32_t)wpr; r = rr; w = (uint32_t)idx - rr * (uint32_t)wpr; }
@@ -855,29 +860,18 @@ __global__ void __launch_bounds__(256) k_expand_s8(const uint32_t *__restrict__ 
             b[g] = (~(t * 0xfeu)) & (v * 0xffu);
         }
     }
-    uint4 *d = reinterpret_cast<uint4 *>(dst + r * ld8 + 32 * w);
-    d[0] = make_uint4(b[0], b[1], b[2], b[3]);
-    d[1] = make_uint4(b[4], b[5], b[6], b[7]);
+    int8_t *d = dst + r * ld8 + 32 * w;
+    if ((reinterpret_cast<uintptr_t>(d) & 31u) == 0) {
+        store_256(d, b);
+    } else {
+        reinterpret_cast<uint4 *>(d)[0] = make_uint4(b[0], b[1], b[2], b[3]);
+        reinterpret_cast<uint4 *>(d)[1] = make_uint4(b[4], b[5], b[6], b[7]);
+    }
 }
 
 // Packed signs -> one e2m1 nibble per value (+1.0 = 0x2, -1.0 = 0xa), two per byte, value k in byte k/2 (even k in
-// the low nibble); nibbles at or beyond K are 0 (= +0.0).  One thread per 32-bit word = 16 output bytes.
-__global__ void __launch_bounds__(256) k_expand_f4(const uint32_t *__restrict__ src, int64_t ld_w, int64_t rows, int64_t K,
-                                                   uint8_t *__restrict__ dst, int64_t ld4) {
-    bnn_pdl_wait();
-    bnn_pdl_launch_next();
-    const int64_t wpr = ld4 >> 4;            // words per output row (ld4 is a multiple of 128 bytes)
-    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= rows * wpr) return;
-    int64_t r, w;
-    row_and_word(idx, wpr, rows * wpr, r, w);
-    const int64_t Kw = (K + 31) >> 5;
-    uint32_t bits = 0u, valid = 0u;
-    if (w < Kw) {
-        bits = src[r * ld_w + w];
-        valid = (w == Kw - 1 && (K & 31)) ? ((1u << (K & 31)) - 1u) : 0xffffffffu;
-    }
-    uint32_t q[4];
+// the low nibble); nibbles at or beyond K are 0 (= +0.0).  One thread per two 32-bit words = 32 output bytes.
+__device__ __forceinline__ void expand_word_f4(uint32_t bits, uint32_t valid, uint32_t *q) {
     if (valid == 0xffffffffu) {              // every word but a row's last one
 #pragma unroll
         for (int g = 0; g < 4; ++g) q[g] = nibbles_of_byte((bits >> (8 * g)) & 0xffu);
@@ -889,7 +883,37 @@ __global__ void __launch_bounds__(256) k_expand_f4(const uint32_t *__restrict__ 
             q[g] = n & (((~v >> 3) & 0x11111111u) * 0xfu);                         // keep the nibbles whose valid bit is set
         }
     }
-    *reinterpret_cast<uint4 *>(dst + r * ld4 + 16 * w) = make_uint4(q[0], q[1], q[2], q[3]);
+}
+__global__ void __launch_bounds__(256) k_expand_f4(const uint32_t *__restrict__ src, int64_t ld_w, int64_t rows, int64_t K,
+                                                   uint8_t *__restrict__ dst, int64_t ld4) {
+    bnn_pdl_wait();
+    bnn_pdl_launch_next();
+    const int64_t ppr = ld4 >> 5;            // word pairs per output row (ld4 is a multiple of 128 bytes)
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= rows * ppr) return;
+    int64_t r, pw;
+    row_and_word(idx, ppr, rows * ppr, r, pw);
+    const int64_t Kw = (K + 31) >> 5, w = 2 * pw;
+    const uint32_t last = (K & 31) ? ((1u << (K & 31)) - 1u) : 0xffffffffu;
+    uint32_t bits[2] = {0u, 0u}, valid[2] = {0u, 0u};
+    if (w + 1 < Kw) {                        // both words inside the row: one 64-bit load (rows are 16-byte aligned)
+        const uint2 v = *reinterpret_cast<const uint2 *>(src + r * ld_w + w);
+        bits[0] = v.x; bits[1] = v.y;
+        valid[0] = 0xffffffffu; valid[1] = (w + 1 == Kw - 1) ? last : 0xffffffffu;
+    } else if (w < Kw) {
+        bits[0] = src[r * ld_w + w];
+        valid[0] = (w == Kw - 1) ? last : 0xffffffffu;
+    }
+    uint32_t q[8];
+    expand_word_f4(bits[0], valid[0], q);
+    expand_word_f4(bits[1], valid[1], q + 4);
+    uint8_t *d = dst + r * ld4 + 32 * pw;
+    if ((reinterpret_cast<uintptr_t>(d) & 31u) == 0) {
+        store_256(d, q);
+    } else {
+        reinterpret_cast<uint4 *>(d)[0] = make_uint4(q[0], q[1], q[2], q[3]);
+        reinterpret_cast<uint4 *>(d)[1] = make_uint4(q[4], q[5], q[6], q[7]);
+    }
 }
 
 // First convolution: the 3x3 neighbourhood of every pixel of an 8-bit NHWC image (9 * C_in <= 32 bytes, taps
@@ -928,9 +952,13 @@ __global__ void __launch_bounds__(256) k_im2col_u8(const uint8_t *__restrict__ a
             }
         }
     }
-    uint4 *d = reinterpret_cast<uint4 *>(dst + pix * 32);
-    d[0] = make_uint4(w[0], w[1], w[2], w[3]);
-    d[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    uint8_t *d = dst + pix * 32;
+    if ((reinterpret_cast<uintptr_t>(d) & 31u) == 0) {
+        store_256(d, w);
+    } else {
+        reinterpret_cast<uint4 *>(d)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+        reinterpret_cast<uint4 *>(d)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    }
 }
 
 typedef CUresult (*encode_fn_t)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
@@ -1052,7 +1080,7 @@ int64_t bnn_umma_operand_ld_f4(int64_t K) { return ((K + 255) / 256) * 128; }
 size_t bnn_umma_operand_bytes_f4(int64_t rows, int64_t K) { return ((size_t)rows * bnn_umma_operand_ld_f4(K) + 255) & ~size_t(255); }
 int bnn_umma_expand_f4(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t rows, int64_t K, uint8_t *dst) {
     const int64_t ld4 = bnn_umma_operand_ld_f4(K);
-    const int64_t total = rows * (ld4 >> 4);
+    const int64_t total = rows * (ld4 >> 5);      // one thread per two words
     if (total == 0) return BNN_OK;
     const int64_t blocks = (total + 255) / 256;
     if (blocks > 0x7fffffff) return BNN_ERR_INVALID_ARG;
