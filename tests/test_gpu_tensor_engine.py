@@ -280,3 +280,40 @@ def test_convnet_forward_chained_on_tensor_engine(ctx, pre_expanded):
     assert torch.equal(final, outs[-1])
     ctx.set_workspace(None)
     del ws
+
+
+def test_back_to_back_calls_without_synchronisation(ctx):
+    """Dependent launches let a kernel be set up while its predecessor still runs.  Many calls queued without a host
+    synchronisation, alternating inputs and sharing one workspace (every call's expansion pass overwrites what the
+    previous call's kernel read), must still give each call its own result."""
+    M, N, K = 1500, 640, 2048
+    rng = np.random.default_rng(123)
+    As = [wl.pm1(rng, (M, K)) for _ in range(3)]
+    W = wl.pm1(rng, (N, K))
+    thr = rng.integers(-20, 21, N).astype(np.int32)
+    wants = [oracle.threshold(oracle.gemm(A, W.T.copy()), thr) for A in As]
+    Aps = [ctx.pack_signs(dev(A, torch.int8)) for A in As]
+    Wp = ctx.pack_signs(dev(W, torch.int8))
+    thr_d = dev(thr)
+    ws = with_ws(ctx, ctx.gemm_workspace_bytes(M, N, K))
+    outs = []
+    for i in range(24):
+        outs.append((i % 3, ctx.binary_dense(Aps[i % 3], Wp, thr_d, None, M, N, K)))
+    # the whole MLP, alternating two batches, into separate score buffers
+    batch, sizes = 2000, (784, 1024, 1100, 1024, 10)     # every hidden layer large enough for the tensor engine
+    case = wl.mlp_case(batch=batch, sizes=sizes, seed=5)
+    X2 = wl.u8(np.random.default_rng(6), (batch, sizes[0]))
+    want_s = [oracle.mlp_forward(X, case["weights"], case["bns"])[0] for X in (case["X"], X2)]
+    net = nets.prepare_mlp(ctx, case["weights"], case["bns"])
+    ws2 = with_ws(ctx, ctx.mlp_workspace_bytes(net["desc"], batch, False))
+    Xd = [dev(case["X"]), dev(X2)]
+    scores = [(i % 2, ctx.mlp_forward(net["desc"], Xd[i % 2], batch)) for i in range(16)]
+    ctx.device_status()
+    for k, o in outs:
+        assert np.array_equal(np_unpack_pm1(o.cpu().numpy(), N), wants[k])
+    for k, sc in scores:
+        got = sc.cpu().numpy().astype(np.float64)
+        tol = 1e-5 * np.abs(want_s[k]) + 1e-6 * np.abs(want_s[k]).max()
+        assert (np.abs(got - want_s[k]) <= tol).all()
+    ctx.set_workspace(None)
+    del ws, ws2
