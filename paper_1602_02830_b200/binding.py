@@ -155,11 +155,13 @@ class Context:
             raise BnnError(st, "bnn_create")
         self._h = h
         self._ws = None
+        self._destroy = lib().bnn_destroy      # kept here: module globals may be gone when __del__ runs at interpreter exit
 
     def close(self):
-        if getattr(self, "_h", None):
-            lib().bnn_destroy(self._h)
-            self._h = None
+        h, destroy = getattr(self, "_h", None), getattr(self, "_destroy", None)
+        if h and destroy is not None:
+            destroy(h)
+        self._h = None
 
     __del__ = close
 
