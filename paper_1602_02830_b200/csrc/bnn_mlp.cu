@@ -249,12 +249,29 @@ extern "C" int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const u
                             : forward_device(ctx, m, Xd + r0 * K0, K0, rows, Sd + r0 * NL, NL, nullptr, ws,
                                              ws + planes_offset(m, batch)))
             return st;
+        if (nchunks > 1 && c + 1 < nchunks) {
+            // this chunk's scores travel back on the copy stream while the next chunk runs through the layers
+            BNN_CUDA_TRY(ctx, cudaEventRecord(ctx->ev[3], ctx->stream));
+            BNN_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->ev[3], 0));
+            if (lds == NL)
+                BNN_CUDA_TRY(ctx, cudaMemcpyAsync(scores_host + r0 * lds, Sd + r0 * NL, (size_t)NL * 4 * rows, cudaMemcpyDeviceToHost, cs));
+            else
+                BNN_CUDA_TRY(ctx, cudaMemcpy2DAsync(scores_host + r0 * lds, (size_t)lds * 4, Sd + r0 * NL, (size_t)NL * 4,
+                                                    (size_t)NL * 4, (size_t)rows, cudaMemcpyDeviceToHost, cs));
+            BNN_CUDA_TRY(ctx, cudaEventRecord(ctx->ev[4], cs));
+        }
     }
-    if (lds == NL)
-        BNN_CUDA_TRY(ctx, cudaMemcpyAsync(scores_host, Sd, (size_t)NL * 4 * batch, cudaMemcpyDeviceToHost, ctx->stream));
-    else
-        BNN_CUDA_TRY(ctx, cudaMemcpy2DAsync(scores_host, (size_t)lds * 4, Sd, (size_t)NL * 4, (size_t)NL * 4, (size_t)batch,
-                                            cudaMemcpyDeviceToHost, ctx->stream));
+    {
+        // the last chunk's (or all) scores on the context's stream, which also waits for the earlier chunks' copies
+        const int64_t r0 = bounds[nchunks - 1], rows = batch - r0;
+        if (lds == NL)
+            BNN_CUDA_TRY(ctx, cudaMemcpyAsync(scores_host + r0 * lds, Sd + r0 * NL, (size_t)NL * 4 * rows, cudaMemcpyDeviceToHost,
+                                              ctx->stream));
+        else
+            BNN_CUDA_TRY(ctx, cudaMemcpy2DAsync(scores_host + r0 * lds, (size_t)lds * 4, Sd + r0 * NL, (size_t)NL * 4, (size_t)NL * 4,
+                                                (size_t)rows, cudaMemcpyDeviceToHost, ctx->stream));
+        if (nchunks > 1) BNN_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev[4], 0));
+    }
     return BNN_OK;
 }
 
