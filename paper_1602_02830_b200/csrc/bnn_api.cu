@@ -23,7 +23,7 @@ extern "C" int bnn_create(bnn_ctx **out, int device, void *cuda_stream) {
     c->operand_bits = 4;
     c->copy_stream = nullptr;
     c->copy_ready = false;
-    for (int i = 0; i < 5; ++i) c->ev[i] = nullptr;
+    for (int i = 0; i < 8; ++i) c->ev[i] = nullptr;
     if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
         delete c;
         return BNN_ERR_CUDA;
@@ -38,7 +38,7 @@ extern "C" int bnn_destroy(bnn_ctx *ctx) {
         bnn_device_guard guard(ctx);
         if (guard.ok) {
             cudaStreamSynchronize(ctx->copy_stream);
-            for (int i = 0; i < 5; ++i) cudaEventDestroy(ctx->ev[i]);
+            for (int i = 0; i < 8; ++i) cudaEventDestroy(ctx->ev[i]);
             cudaStreamDestroy(ctx->copy_stream);
         }
     }

@@ -16,7 +16,7 @@ struct bnn_ctx {
     int tile_rows; // accumulator rows per thread of the tiled popc kernel: 16 or 8
     int pair_mode; // tensor engine: 0 = CTA pairs (cta_group::2) for very large outputs, 1 = never, 2 = wherever the kernel allows
     cudaStream_t copy_stream;   // internal stream for the host copies of bnn_mlp_forward_host (created on first use)
-    cudaEvent_t ev[5];          // [0] work already on `stream`; [1..4] chunk copies done
+    cudaEvent_t ev[8];          // [0] work already on `stream`; [1..4] chunk copies done; [5] chunk computed; [6] scores copied
     bool copy_ready;
     int operand_bits; // tensor engine, +-1 x +-1 products: 4 = e2m1 nibbles (default), 8 = signed bytes
     int engine;    // 0 auto, 1 CUDA-core XOR-popcount kernels only, 2 tensor-core int8 engine where it applies

@@ -214,18 +214,27 @@ extern "C" int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const u
 #ifndef BNN_E2E_SPLIT_PCT
 #define BNN_E2E_SPLIT_PCT 40
 #endif
+#ifndef BNN_E2E_SPLIT2_PCT
+#define BNN_E2E_SPLIT2_PCT 0          // second boundary (0: two chunks)
+#endif
     int nchunks = 1;
-    int64_t bounds[3] = {0, batch, batch};
+    int64_t bounds[5] = {0, batch, batch, batch, batch};
     if (tensor && batch >= 6144) {
         const int64_t first = ((batch * BNN_E2E_SPLIT_PCT / 100 + 127) / 128) * 128;
+        const int64_t second = ((batch * BNN_E2E_SPLIT2_PCT / 100 + 127) / 128) * 128;
         if (first > 0 && first < batch && tensor_applies(ctx, m, first) && tensor_applies(ctx, m, batch - first)) {
             nchunks = 2;
             bounds[1] = first;
+            if (BNN_E2E_SPLIT2_PCT > 0 && second > first && second < batch && tensor_applies(ctx, m, second - first) &&
+                tensor_applies(ctx, m, batch - second)) {
+                nchunks = 3;
+                bounds[2] = second;
+            }
         }
     }
     if (nchunks > 1 && !ctx->copy_ready) {
         BNN_CUDA_TRY(ctx, cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
-        for (int i = 0; i < 5; ++i) BNN_CUDA_TRY(ctx, cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming));
+        for (int i = 0; i < 8; ++i) BNN_CUDA_TRY(ctx, cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming));
         ctx->copy_ready = true;
     }
     cudaStream_t cs = nchunks > 1 ? ctx->copy_stream : ctx->stream;
@@ -251,14 +260,14 @@ extern "C" int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const u
             return st;
         if (nchunks > 1 && c + 1 < nchunks) {
             // this chunk's scores travel back on the copy stream while the next chunk runs through the layers
-            BNN_CUDA_TRY(ctx, cudaEventRecord(ctx->ev[3], ctx->stream));
-            BNN_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->ev[3], 0));
+            BNN_CUDA_TRY(ctx, cudaEventRecord(ctx->ev[5], ctx->stream));
+            BNN_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->ev[5], 0));
             if (lds == NL)
                 BNN_CUDA_TRY(ctx, cudaMemcpyAsync(scores_host + r0 * lds, Sd + r0 * NL, (size_t)NL * 4 * rows, cudaMemcpyDeviceToHost, cs));
             else
                 BNN_CUDA_TRY(ctx, cudaMemcpy2DAsync(scores_host + r0 * lds, (size_t)lds * 4, Sd + r0 * NL, (size_t)NL * 4,
                                                     (size_t)NL * 4, (size_t)rows, cudaMemcpyDeviceToHost, cs));
-            BNN_CUDA_TRY(ctx, cudaEventRecord(ctx->ev[4], cs));
+            BNN_CUDA_TRY(ctx, cudaEventRecord(ctx->ev[6], cs));
         }
     }
     {
@@ -270,7 +279,7 @@ extern "C" int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const u
         else
             BNN_CUDA_TRY(ctx, cudaMemcpy2DAsync(scores_host + r0 * lds, (size_t)lds * 4, Sd + r0 * NL, (size_t)NL * 4, (size_t)NL * 4,
                                                 (size_t)rows, cudaMemcpyDeviceToHost, ctx->stream));
-        if (nchunks > 1) BNN_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev[4], 0));
+        if (nchunks > 1) BNN_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev[6], 0));
     }
     return BNN_OK;
 }
