@@ -277,6 +277,9 @@ extern "C" int bnn_convnet_forward(bnn_ctx *ctx, const bnn_convnet_desc *net, co
         const bnn_conv_layer_desc &D = net->layers[k];
         uint32_t *dst = (k == L - 1) ? out_bits : bits[k & 1];
         int8_t *dst8 = (k < L - 1) ? act8[k & 1] : nullptr;
+        // an inner layer's packed map is only written when the caller asked for it (the next layer reads the bytes);
+        // the pooling epilogue always goes through it
+        if (k < L - 1 && !D.pool && !(layer_out && layer_out[k])) dst = nullptr;
         const int8_t *W8 = D.W8;
         if (!W8) {
             // first layer: one word per filter; others: C_out rows of 9 * C_in bits
@@ -293,7 +296,7 @@ extern "C" int bnn_convnet_forward(bnn_ctx *ctx, const bnn_convnet_desc *net, co
         }
         if (st) return st;
         if (D.pool) { h /= 2; w /= 2; }
-        if (layer_out && layer_out[k] && layer_out[k] != dst)
+        if (dst && layer_out && layer_out[k] && layer_out[k] != dst)
             BNN_CUDA_TRY(ctx, cudaMemcpyAsync(layer_out[k], dst, (size_t)B * h * w * ((D.C_out + 31) / 32) * 4,
                                               cudaMemcpyDeviceToDevice, ctx->stream));
         cur8 = dst8;
