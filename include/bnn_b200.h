@@ -113,6 +113,8 @@ BNN_API int bnn_expand_signs_f4(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w,
  *   out_bits (optional): packed M x N signs, pitch ldo_w words, like bnn_binary_dense.
  *   out_exp  (optional): the same signs in the operand format of the next layer (same operand_bits), pitch
  *                        ldo_exp bytes >= bnn_expanded_ld(N) or bnn_expanded_ld_f4(N); at least one output is required.
+ *                        Values N .. roundup(N, 32) - 1 of a row are written as 0 (all that a following layer with
+ *                        K = N reads); the rest of the pitch is left untouched.
  * Runs on the context's stream; BNN_ERR_ALIGNMENT for pointers or pitches that are not multiples of 16 bytes. */
 BNN_API int bnn_binary_dense_expanded(bnn_ctx *ctx, const void *A_exp, int64_t lda_bytes, const void *W_exp, int64_t ldw_bytes,
                                       int operand_bits, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits,

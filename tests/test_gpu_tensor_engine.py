@@ -129,7 +129,8 @@ def test_expand_signs(ctx):
 
 
 @pytest.mark.parametrize("bits", [4, 8])
-@pytest.mark.parametrize("M,N,K", [(700, 520, 1000), (1030, 200, 4100), (300, 130, 64)])
+@pytest.mark.parametrize("M,N,K", [(700, 520, 1000), (1030, 200, 4100), (300, 130, 64), (1, 1, 1), (1, 33, 31),
+                                   (2, 1, 257), (129, 193, 300), (5, 400, 2), (257, 31, 513)])
 def test_binary_dense_expanded(ctx, M, N, K, bits):
     """The tensor kernel on operands the caller keeps expanded: packed signs and the next layer's operand, chained
     through a second layer, against the oracle."""
@@ -150,6 +151,9 @@ def test_binary_dense_expanded(ctx, M, N, K, bits):
     ctx.device_status()
     got = out.cpu().numpy()
     assert np.array_equal(np_unpack_pm1(got, N), h) and padding_is_zero(got, N)
+    # the expanded output equals the expansion of the packed one up to the end of the last 32-value group
+    nb = (N + 31) // 32 * 32 // (2 if bits == 4 else 1)
+    assert torch.equal(expand(out, M, N)[:, :nb].cpu().view(torch.uint8), out_exp[:, :nb].cpu().view(torch.uint8))
     assert np.array_equal(np_unpack_pm1(out2.cpu().numpy(), 96), want2)
 
 
