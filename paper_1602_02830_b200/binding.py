@@ -44,7 +44,7 @@ class MlpDesc(Structure):
 
 class ConvLayerDesc(Structure):
     _fields_ = [("Wp", c_void_p), ("C_in", c_int64), ("C_out", c_int64), ("pool", c_int32), ("thr", c_void_p),
-                ("flip", c_void_p), ("W8", c_void_p)]
+                ("flip", c_void_p), ("W8", c_void_p), ("W4", c_void_p)]
 
 
 class ConvNetDesc(Structure):
@@ -310,7 +310,7 @@ class Context:
         return desc, (arr, layers)
 
     def make_convnet_desc(self, layers):
-        """layers: list of dicts with Wp, Cin, Cout, pool, thr, flip and optionally W8.  Returns (ConvNetDesc, keep-alive)."""
+        """layers: list of dicts with Wp, Cin, Cout, pool, thr, flip and optionally W8, W4.  Returns (ConvNetDesc, keep-alive)."""
         arr = (ConvLayerDesc * len(layers))()
         for d, L in zip(arr, layers):
             d.Wp = L["Wp"].data_ptr()
@@ -318,6 +318,7 @@ class Context:
             d.thr = L["thr"].data_ptr()
             d.flip = L["flip"].data_ptr() if L.get("flip") is not None else None
             d.W8 = L["W8"].data_ptr() if L.get("W8") is not None else None
+            d.W4 = L["W4"].data_ptr() if L.get("W4") is not None else None
         return ConvNetDesc(len(layers), arr), (arr, layers)
 
     def convnet_workspace_bytes(self, desc, B: int, H: int, W: int) -> int:

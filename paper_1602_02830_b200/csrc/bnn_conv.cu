@@ -272,27 +272,43 @@ extern "C" int bnn_convnet_forward(bnn_ctx *ctx, const bnn_convnet_desc *net, co
         return st;
     }
 
+    // A layer with a multiple of 256 input channels runs on 4-bit operands (e2m1 nibbles, twice the MMA rate and half
+    // the operand bytes); the layer before it then writes nibbles instead of bytes.
+    auto on_nibbles = [&](int k) { return k > 0 && k < L && ctx->operand_bits != 8 && (net->layers[k].C_in % 256) == 0; };
     const int8_t *cur8 = nullptr;
     for (int k = 0; k < L; ++k) {
         const bnn_conv_layer_desc &D = net->layers[k];
         uint32_t *dst = (k == L - 1) ? out_bits : bits[k & 1];
         int8_t *dst8 = (k < L - 1) ? act8[k & 1] : nullptr;
+        const int next_f4 = on_nibbles(k + 1) ? 1 : 0;
+        const int64_t ldo8 = next_f4 ? D.C_out / 2 : D.C_out;
         // an inner layer's packed map is only written when the caller asked for it (the next layer reads the bytes);
         // the pooling epilogue always goes through it
         if (k < L - 1 && !D.pool && !(layer_out && layer_out[k])) dst = nullptr;
-        const int8_t *W8 = D.W8;
-        if (!W8) {
-            // first layer: one word per filter; others: C_out rows of 9 * C_in bits
-            if (int st = bnn_umma_expand(ctx, D.Wp, k == 0 ? 1 : 9 * (D.C_in / 32), D.C_out, 9 * D.C_in, w8_scratch)) return st;
-            W8 = w8_scratch;
-        }
         int st;
-        if (k == 0) {
-            if ((st = bnn_umma_im2col_u8(ctx, X, B, h, w, D.C_in, im2col))) return st;
-            st = bnn_umma_gemm(ctx, im2col, 32, true, W8, bnn_umma_operand_ld(9 * D.C_in), B * h * w, D.C_out, 9 * D.C_in, nullptr, 0,
-                               D.thr, D.flip, dst, (D.C_out + 31) / 32, dst8, D.C_out, D.pool, h, w);
+        if (on_nibbles(k)) {
+            const uint8_t *W4 = D.W4;
+            if (!W4) {
+                uint8_t *w4_scratch = reinterpret_cast<uint8_t *>(w8_scratch);      // half the size of the byte form
+                if ((st = bnn_umma_expand_f4(ctx, D.Wp, 9 * (D.C_in / 32), D.C_out, 9 * D.C_in, w4_scratch))) return st;
+                W4 = w4_scratch;
+            }
+            st = bnn_umma_conv_f4(ctx, reinterpret_cast<const uint8_t *>(cur8), W4, B, h, w, D.C_in, D.C_out, D.pool, D.thr, D.flip, dst,
+                                  reinterpret_cast<uint8_t *>(dst8), ldo8);
         } else {
-            st = bnn_umma_conv(ctx, cur8, W8, B, h, w, D.C_in, D.C_out, D.pool, D.thr, D.flip, dst, nullptr, dst8, D.C_out);
+            const int8_t *W8 = D.W8;
+            if (!W8) {
+                // first layer: one word per filter; others: C_out rows of 9 * C_in bits
+                if ((st = bnn_umma_expand(ctx, D.Wp, k == 0 ? 1 : 9 * (D.C_in / 32), D.C_out, 9 * D.C_in, w8_scratch))) return st;
+                W8 = w8_scratch;
+            }
+            if (k == 0) {
+                if ((st = bnn_umma_im2col_u8(ctx, X, B, h, w, D.C_in, im2col))) return st;
+                st = bnn_umma_gemm(ctx, im2col, 32, true, W8, bnn_umma_operand_ld(9 * D.C_in), B * h * w, D.C_out, 9 * D.C_in, nullptr, 0,
+                                   D.thr, D.flip, dst, (D.C_out + 31) / 32, dst8, ldo8, D.pool, h, w, next_f4);
+            } else {
+                st = bnn_umma_conv(ctx, cur8, W8, B, h, w, D.C_in, D.C_out, D.pool, D.thr, D.flip, dst, nullptr, dst8, ldo8, next_f4);
+            }
         }
         if (st) return st;
         if (D.pool) { h /= 2; w /= 2; }

@@ -1213,7 +1213,7 @@ bool bnn_umma_conv_tiling(int64_t H, int64_t W, int pool, int *TH, int *TB) {
 // W8: [C_out][9 * C_in] +-1 bytes.  Outputs as bnn_binary_conv2d (sums only without pooling).
 int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B, int64_t H, int64_t W, int64_t C_in,
                   int64_t C_out, int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, int32_t *out_sums,
-                  int8_t *out8, int64_t ldo8) {
+                  int8_t *out8, int64_t ldo8, int out_f4) {
     int TH, TB;
     if (!bnn_umma_conv_tiling(H, W, pool, &TH, &TB) || (C_in % BK) != 0 || (pool && (out_sums || !out_bits))) return BNN_ERR_INVALID_ARG;
     CUtensorMap mapA, mapB;
@@ -1226,9 +1226,33 @@ int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B,
     a.k_last = BK / 32;
     a.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BM >> 4) << 24);
     a.C = out_sums; a.ldc = C_out; a.out = out_bits; a.ldo = (C_out + 31) / 32; a.thr = thr; a.flip = flip;
-    a.out8 = out8; a.ldo8 = ldo8;
+    a.out8 = out8; a.ldo8 = ldo8; a.out_f4 = out_f4;
     a.conv = 1; a.H = (int)H; a.W = (int)W; a.TH = TH; a.TB = TB; a.c_chunks = (int)(C_in / BK); a.pool = pool;
     return umma_launch(ctx, mapA, mapB, a, bn);
+}
+
+// The same convolution on 4-bit operands: act4 [B][H][W][C_in / 2] and W4 [C_out][9 * C_in / 2] bytes of e2m1 nibbles
+// (C_in % 256 == 0, so that a K step is one tap and 256 channels = 128 bytes per pixel); pixels outside the image arrive
+// as zero nibbles (+0.0).  Outputs: packed signs and / or nibbles for the next layer (out4, pitch ldo4 bytes per pixel).
+int bnn_umma_conv_f4(bnn_ctx *ctx, const uint8_t *act4, const uint8_t *W4, int64_t B, int64_t H, int64_t W, int64_t C_in,
+                     int64_t C_out, int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, uint8_t *out4,
+                     int64_t ldo4) {
+    int TH, TB;
+    if (!bnn_umma_conv_tiling(H, W, pool, &TH, &TB) || (C_in % (2 * BK)) != 0 || !thr || (pool && !out_bits) || (!out_bits && !out4))
+        return BNN_ERR_INVALID_ARG;
+    if (!bnn_aligned16(act4) || !bnn_aligned16(W4)) return BNN_ERR_ALIGNMENT;
+    CUtensorMap mapA, mapB;
+    if (int st = make_map_nhwc(ctx, &mapA, act4, B, H, W, C_in / 2, (int)W, TH, TB)) return st;
+    if (int st = make_map(ctx, &mapB, W4, C_out, 9 * C_in / 2, 9 * C_in / 2, 192)) return st;
+    UmmaArgs a{};
+    a.M = B * H * W; a.N = C_out;
+    a.c_chunks = (int)(C_in / (2 * BK));
+    a.k_iters = 9 * a.c_chunks;
+    a.k_last = BK / 32;
+    a.out = out_bits; a.ldo = (C_out + 31) / 32; a.thr = thr; a.flip = flip;
+    a.out8 = reinterpret_cast<int8_t *>(out4); a.ldo8 = ldo4; a.out_f4 = 1;
+    a.conv = 1; a.H = (int)H; a.W = (int)W; a.TH = TH; a.TB = TB; a.pool = pool;
+    return umma_launch(ctx, mapA, mapB, a, 192);
 }
 
 extern "C" int64_t bnn_expanded_ld(int64_t K) { return K > 0 ? bnn_umma_operand_ld(K) : 0; }

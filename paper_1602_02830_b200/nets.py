@@ -54,7 +54,7 @@ def prepare_mlp(ctx, weights, bns, expand_weights: bool = True):
 
 def prepare_convnet(ctx, layers, expand_weights: bool = True):
     """Conv layer list {wgt: Cout x 3 x 3 x Cin, bn, pool} -> packed device weights and folded thresholds
-    (and, with expand_weights, the weights as +-1 bytes for the tensor-core engine)."""
+    (and, with expand_weights, the weights as +-1 bytes and, where used, 4-bit nibbles for the tensor-core engine)."""
     out = []
     for i, L in enumerate(layers):
         wgt = L["wgt"]
@@ -72,6 +72,8 @@ def prepare_convnet(ctx, layers, expand_weights: bool = True):
             # the same bits viewed as Cout rows of 9*Cin: re-pack with a legal leading dimension, then expand
             rows = ctx.pack_signs(_dev(ctx, flat, torch.int8), pack_along=0)
             d["W8"] = ctx.expand_signs(rows, Cout, 9 * Cin)
+            if i > 0 and Cin % 256 == 0:                       # layers the library runs on 4-bit operands
+                d["W4"] = ctx.expand_signs_f4(rows, Cout, 9 * Cin)
         out.append(d)
     return out
 
