@@ -273,7 +273,7 @@ extern "C" int bnn_convnet_forward(bnn_ctx *ctx, const bnn_convnet_desc *net, co
     }
 
     // A layer with a multiple of 256 input channels runs on 4-bit operands (e2m1 nibbles, twice the MMA rate and half
-    // the operand bytes); the layer before it then writes nibbles instead of bytes.
+    // the operand bytes; a K step is one tap and 256 channels); the layer before it then writes nibbles instead of bytes.
     auto on_nibbles = [&](int k) { return k > 0 && k < L && ctx->operand_bits != 8 && (net->layers[k].C_in % 256) == 0; };
     const int8_t *cur8 = nullptr;
     for (int k = 0; k < L; ++k) {

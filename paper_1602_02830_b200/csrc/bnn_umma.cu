@@ -628,6 +628,11 @@ __device__ __forceinline__ void tma_load_2d_2sm(uint32_t dst, const CUtensorMap 
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
+__device__ __forceinline__ void tma_load_4d_2sm(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, int c3, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void umma_i8_2sm(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -735,11 +740,23 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                 const uint32_t tm = t / tn32;
                 const int m0 = (int)(tm * (2 * BM) + rank * BM);
                 const int nb0 = (int)((t - tm * tn32) * BN + rank * (BN / 2));
+                int b0 = 0, y0 = 0;
+                if (p.conv) {
+                    // this CTA's 128 pixels of the pair's 256 (see k_umma_i8): first image and row, taps per K step
+                    const int tm128 = 2 * (int)tm + (int)rank, tiles_per_img = p.H / p.TH;
+                    b0 = (p.TB > 1) ? tm128 * p.TB : tm128 / tiles_per_img;
+                    y0 = (p.TB > 1) ? 0 : (tm128 % tiles_per_img) * p.TH;
+                }
+                int cc = 0, tx = -1, ty = -1;
                 for (int kit = 0; kit < p.k_iters; ++kit) {
                     const bool pre = first_tile && kit < npre;
                     if (ph > 0 && !mbar_wait(smem_u32(&ctl->empty[s]), (ph - 1) & 1)) { fail(ctl, 11); ok = false; break; }
                     if (rank == 0 && !pre) mbar_expect_tx(smem_u32(&ctl->full[s]), 2 * STAGE2_BYTES);   // the bytes of both CTAs
                     const uint32_t bar0 = smem_u32(&ctl->full[s]) & PEER_MASK;
+                    if (p.conv) {
+                        tma_load_4d_2sm(smem_u32(tiles + s * STAGE2_BYTES), &mapA, cc * BK, tx, y0 + ty, b0, bar0);
+                        if (++cc == p.c_chunks) { cc = 0; if (++tx == 2) { tx = -1; ++ty; } }
+                    } else
                     tma_load_2d_2sm(smem_u32(tiles + s * STAGE2_BYTES), &mapA, kit * BK, m0, bar0);
                     if (!pre) tma_load_2d_2sm(smem_u32(tiles + s * STAGE2_BYTES + A_BYTES), &mapB, kit * BK, nb0, bar0);
                     if (++s == (uint32_t)STAGES2) { s = 0; ++ph; }
@@ -1242,8 +1259,12 @@ int bnn_umma_conv_f4(bnn_ctx *ctx, const uint8_t *act4, const uint8_t *W4, int64
         return BNN_ERR_INVALID_ARG;
     if (!bnn_aligned16(act4) || !bnn_aligned16(W4)) return BNN_ERR_ALIGNMENT;
     CUtensorMap mapA, mapB;
+    // CTA pairs (each CTA its own 128 pixels and half of the tile's filters) cut the operand bytes per CTA by 30 %, but
+    // measured slower on the ConvNet's layers (0.162 against 0.158 ms per batch of 256): on request only
+    const int pairs = (ctx->pair_mode == 2 && B * H * W >= 512) ? umma2_max_pairs<192>(ctx) : 0;
+    if (pairs > 0) { if (int st = umma_prepare(ctx)) return st; }
     if (int st = make_map_nhwc(ctx, &mapA, act4, B, H, W, C_in / 2, (int)W, TH, TB)) return st;
-    if (int st = make_map(ctx, &mapB, W4, C_out, 9 * C_in / 2, 9 * C_in / 2, 192)) return st;
+    if (int st = make_map(ctx, &mapB, W4, C_out, 9 * C_in / 2, 9 * C_in / 2, pairs > 0 ? 96 : 192)) return st;
     UmmaArgs a{};
     a.M = B * H * W; a.N = C_out;
     a.c_chunks = (int)(C_in / (2 * BK));
@@ -1252,6 +1273,14 @@ int bnn_umma_conv_f4(bnn_ctx *ctx, const uint8_t *act4, const uint8_t *W4, int64
     a.out = out_bits; a.ldo = (C_out + 31) / 32; a.thr = thr; a.flip = flip;
     a.out8 = reinterpret_cast<int8_t *>(out4); a.ldo8 = ldo4; a.out_f4 = 1;
     a.conv = 1; a.H = (int)H; a.W = (int)W; a.TH = TH; a.TB = TB; a.pool = pool;
+    if (pairs > 0) {
+        const int64_t tiles2 = ((a.M + 2 * BM - 1) / (2 * BM)) * ((C_out + 191) / 192);
+        if (tiles2 >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;
+        const int64_t use = tiles2 < pairs ? tiles2 : pairs;
+        BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8_2sm<192>, dim3((unsigned)(2 * use)), dim3(Warps<192>::NTHREADS), umma2_smem_bytes<192>(),
+                                               ctx->stream, mapA, mapB, a));
+        return bnn_check_launch(ctx);
+    }
     return umma_launch(ctx, mapA, mapB, a, 192);
 }
 
