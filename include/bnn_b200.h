@@ -85,9 +85,8 @@ BNN_API int bnn_set_pair_mode(bnn_ctx *ctx, int mode);
 /* Tensor-core engine only: how +-1 x +-1 products are fed to the tensor cores.  4 (default) = each value as a 4-bit
  * floating-point nibble (e2m1: +-1.0 is exact, block scales fixed at 1, float32 accumulators that hold these integer sums
  * exactly for K <= 2^24): half the operand bytes and twice the instruction rate of 8 = one signed byte per value with
- * int32 accumulators.  Layers with 8-bit inputs always use bytes, and so do a single bnn_binary_conv2d call and the
- * layers of bnn_convnet_forward whose C_in is not a multiple of 256 (a K step of the 4-bit kernel is 256 channels of
- * one tap).  Results are identical. */
+ * int32 accumulators.  Layers with 8-bit inputs always use bytes, and so do convolutions whose C_in is not a multiple
+ * of 256 (a K step of the 4-bit kernel is 256 channels of one tap).  Results are identical. */
 BNN_API int bnn_set_operand_bits(bnn_ctx *ctx, int bits);
 /* Workspace bytes bnn_xnor_gemm / bnn_binary_dense need to run M x N x K on the tensor-core engine
  * (0 if the shape does not qualify for it). */

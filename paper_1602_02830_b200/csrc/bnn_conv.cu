@@ -134,6 +134,14 @@ extern "C" int bnn_binary_conv2d(bnn_ctx *ctx, const uint32_t *act, const uint8_
         if (ctx->engine != BNN_ENGINE_POPC && shape_ok) {
             const size_t a_bytes = bnn_umma_operand_bytes(B * H * W, C_in), w_bytes = bnn_umma_operand_bytes(C_out, 9 * C_in);
             if (ctx->ws && ctx->ws_bytes >= a_bytes + w_bytes) {
+                if (ctx->operand_bits != 8 && (C_in % 256) == 0) {
+                    // 4-bit operands (one tap and 256 channels per K step): half the bytes, twice the MMA rate
+                    uint8_t *act4 = static_cast<uint8_t *>(ctx->ws);
+                    uint8_t *W4 = act4 + bnn_umma_operand_bytes_f4(B * H * W, C_in);
+                    if (int st = bnn_umma_expand_f4(ctx, act, Cw, B * H * W, C_in, act4)) return st;
+                    if (int st = bnn_umma_expand_f4(ctx, Wp, 9 * Cw, C_out, 9 * C_in, W4)) return st;
+                    return bnn_umma_conv_f4(ctx, act4, W4, B, H, W, C_in, C_out, pool, thr, flip, out_bits, nullptr, 0, out_sums);
+                }
                 int8_t *act8 = static_cast<int8_t *>(ctx->ws);
                 int8_t *W8 = act8 + a_bytes;
                 if (int st = bnn_umma_expand(ctx, act, Cw, B * H * W, C_in, act8)) return st;

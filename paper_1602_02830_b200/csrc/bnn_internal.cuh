@@ -42,7 +42,7 @@ int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B,
                   int8_t *out8 = nullptr, int64_t ldo8 = 0, int out_f4 = 0);   // out_f4: out8 receives e2m1 nibbles (ldo8 bytes per pixel)
 int bnn_umma_conv_f4(bnn_ctx *ctx, const uint8_t *act4, const uint8_t *W4, int64_t B, int64_t H, int64_t W, int64_t C_in,
                      int64_t C_out, int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, uint8_t *out4,
-                     int64_t ldo4);
+                     int64_t ldo4, int32_t *out_sums = nullptr);
 
 // ---- bit-plane split as a pre-pass for the CUDA-core first layer (bnn_gemm.cu)
 size_t bnn_planes_scratch_bytes(int64_t M, int64_t K);

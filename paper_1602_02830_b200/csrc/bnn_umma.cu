@@ -1250,12 +1250,14 @@ int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B,
 
 // The same convolution on 4-bit operands: act4 [B][H][W][C_in / 2] and W4 [C_out][9 * C_in / 2] bytes of e2m1 nibbles
 // (C_in % 256 == 0, so that a K step is one tap and 256 channels = 128 bytes per pixel); pixels outside the image arrive
-// as zero nibbles (+0.0).  Outputs: packed signs and / or nibbles for the next layer (out4, pitch ldo4 bytes per pixel).
+// as zero nibbles (+0.0).  Outputs: packed signs and / or nibbles for the next layer (out4, pitch ldo4 bytes per pixel),
+// or the int32 sums (not with pooling).
 int bnn_umma_conv_f4(bnn_ctx *ctx, const uint8_t *act4, const uint8_t *W4, int64_t B, int64_t H, int64_t W, int64_t C_in,
                      int64_t C_out, int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, uint8_t *out4,
-                     int64_t ldo4) {
+                     int64_t ldo4, int32_t *out_sums) {
     int TH, TB;
-    if (!bnn_umma_conv_tiling(H, W, pool, &TH, &TB) || (C_in % (2 * BK)) != 0 || !thr || (pool && !out_bits) || (!out_bits && !out4))
+    if (!bnn_umma_conv_tiling(H, W, pool, &TH, &TB) || (C_in % (2 * BK)) != 0 || (pool && (out_sums || !out_bits)) ||
+        (!out_bits && !out4 && !out_sums) || ((out_bits || out4) && !thr))
         return BNN_ERR_INVALID_ARG;
     if (!bnn_aligned16(act4) || !bnn_aligned16(W4)) return BNN_ERR_ALIGNMENT;
     CUtensorMap mapA, mapB;
@@ -1270,7 +1272,7 @@ int bnn_umma_conv_f4(bnn_ctx *ctx, const uint8_t *act4, const uint8_t *W4, int64
     a.c_chunks = (int)(C_in / (2 * BK));
     a.k_iters = 9 * a.c_chunks;
     a.k_last = BK / 32;
-    a.out = out_bits; a.ldo = (C_out + 31) / 32; a.thr = thr; a.flip = flip;
+    a.C = out_sums; a.ldc = C_out; a.out = out_bits; a.ldo = (C_out + 31) / 32; a.thr = thr; a.flip = flip;
     a.out8 = reinterpret_cast<int8_t *>(out4); a.ldo8 = ldo4; a.out_f4 = 1;
     a.conv = 1; a.H = (int)H; a.W = (int)W; a.TH = TH; a.TB = TB; a.pool = pool;
     if (pairs > 0) {
