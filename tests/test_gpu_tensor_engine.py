@@ -289,6 +289,32 @@ def test_convnet_forward_chained_on_tensor_engine(ctx, pre_expanded, channels):
     del ws
 
 
+def test_mlp_forward_host_on_a_side_stream_in_chunks():
+    """Host-buffer forward large enough to be copied in two chunks (internal copy stream, events), on a context bound to
+    a stream of its own, called twice back to back with different inputs and no synchronisation in between."""
+    batch, sizes = 6400, (784, 1024, 1024, 10)
+    cases = [wl.mlp_case(batch=batch, sizes=sizes, seed=s) for s in (31, 32)]
+    cases[1]["weights"], cases[1]["bns"] = cases[0]["weights"], cases[0]["bns"]      # same network, other inputs
+    wants = [oracle.mlp_forward(c["X"], c["weights"], c["bns"])[0] for c in cases]
+    build.build()
+    s = torch.cuda.Stream()
+    c2 = binding.Context(0, stream=s)
+    with torch.cuda.stream(s):
+        net = nets.prepare_mlp(c2, cases[0]["weights"], cases[0]["bns"])
+        ws = with_ws(c2, c2.mlp_workspace_bytes(net["desc"], batch, True))
+        Xh = [torch.from_numpy(c["X"]).pin_memory() for c in cases]
+        Sh = [torch.empty(batch, sizes[-1], dtype=torch.float32).pin_memory() for _ in cases]
+        for x, o in zip(Xh, Sh):
+            c2.mlp_forward_host(net["desc"], x, batch, o)
+        c2.device_status()
+    for o, want in zip(Sh, wants):
+        got = o.numpy().astype(np.float64)
+        assert (np.abs(got - want) <= 1e-5 * np.abs(want) + 1e-6 * np.abs(want).max()).all()
+    c2.set_workspace(None)
+    c2.close()
+    del ws
+
+
 def test_back_to_back_calls_without_synchronisation(ctx):
     """Dependent launches let a kernel be set up while its predecessor still runs.  Many calls queued without a host
     synchronisation, alternating inputs and sharing one workspace (every call's expansion pass overwrites what the
