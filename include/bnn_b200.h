@@ -79,8 +79,8 @@ BNN_API int bnn_set_tile_rows(bnn_ctx *ctx, int rows);
  * matrix product return identical outputs). */
 BNN_API int bnn_set_engine(bnn_ctx *ctx, int engine);
 /* Tensor-core engine only: plain products can run on pairs of SMs (thread-block clusters of two, tcgen05
- * cta_group::2) that share the B operand.  0 (default) = for outputs of 2^26 elements and more, where it measured
- * faster; 1 = never; 2 = wherever the kernel allows (M >= 512, 256-wide tiles).  Results are identical. */
+ * cta_group::2) that share the B operand.  0 (default) = for outputs of 6 million elements and more, where it measured
+ * faster; 1 = never; 2 = wherever the kernel allows (M >= 512; also the 4-bit convolutions).  Results are identical. */
 BNN_API int bnn_set_pair_mode(bnn_ctx *ctx, int mode);
 /* Tensor-core engine only: how +-1 x +-1 products are fed to the tensor cores.  4 (default) = each value as a 4-bit
  * floating-point nibble (e2m1: +-1.0 is exact, block scales fixed at 1, float32 accumulators that hold these integer sums

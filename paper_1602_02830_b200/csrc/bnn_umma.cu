@@ -183,8 +183,9 @@ struct __align__(16) Control {
     uint32_t poolw[BM][BN_MAX / 32 + 1];   // convolution with pooling: the sign words of every pixel of the tile
 };
 
+// Relaxed for the same reason as mbar_arrive_cta0 below: the barrier hands back tensor memory only.
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+    asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void fail(Control *ctl, int code) {
     ctl->failed = (uint32_t)code;
@@ -650,11 +651,14 @@ __device__ __forceinline__ void umma_commit_2sm(uint32_t bar) {
 __device__ __forceinline__ void umma_commit_2sm_local(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// Arrive on the barrier at the same offset in CTA 0 of the cluster.
+// Arrive on the barrier at the same offset in CTA 0 of the cluster.  Relaxed: the barrier hands back tensor memory, whose
+// reads are ordered by tcgen05.wait::ld and the tcgen05 fence before the arrival; nothing written to memory is passed
+// on through it.  (With release semantics at cluster scope the arrival waited for the epilogue's global stores to
+// complete: ~3800 clocks per tile, during which the issuing warps could not reuse the accumulator buffer.)
 __device__ __forceinline__ void mbar_arrive_cta0(uint32_t bar) {
     uint32_t remote;
     asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(remote) : "r"(bar));
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
 }
 
 // 4-bit form of the pair instruction (see umma_mxf4).
@@ -1116,7 +1120,7 @@ int bnn_umma_gemm_f4(bnn_ctx *ctx, const uint8_t *A4, int64_t lda4, const uint8_
     if (M > 0x7fffffff || N > 0x7fffffff || K <= 0 || K > (1 << 24)) return BNN_ERR_INVALID_ARG;
     CUtensorMap mapA, mapB;
     const int64_t kb = (((K + 1) / 2 + 15) / 16) * 16;      // extent along K in bytes
-    const bool pair_want = ctx->pair_mode == 2 || (ctx->pair_mode == 0 && (double)M * (double)N >= 33554432.0);
+    const bool pair_want = ctx->pair_mode == 2 || (ctx->pair_mode == 0 && (double)M * (double)N >= 6.0e6);
     const int pairs = (M >= 512 && pair_want) ? umma2_max_pairs<192>(ctx) : 0;
     if (int st = make_map(ctx, &mapA, A4, M, kb <= lda4 ? kb : lda4, lda4, BM)) return st;
     if (int st = make_map(ctx, &mapB, B4, N, kb <= ldb4 ? kb : ldb4, ldb4, pairs > 0 ? 96 : 192)) return st;
@@ -1155,9 +1159,9 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
     const int bn = umma_tile_n(N, M, ctx->sm_count);
     const int64_t kb = ((K + 15) / 16) * 16;      // extent along K in bytes; beyond it TMA fills zeros
     // two-SM kernel: 256-wide tiles, at least two 256-row tiles, plain GEMM epilogues
-    // (auto: only where it measured faster -- outputs of 2^26 elements and more, e.g. 8192 x 8192 or 65536 x 4096)
+    // (auto: where it measured faster -- from about 1500 x 4096 outputs on; below that the larger tiles leave SMs idle)
     const bool pair_shape = bn == 256 && M >= 512 && !pool;
-    const bool pair_want = ctx->pair_mode == 2 || (ctx->pair_mode == 0 && (double)M * (double)N >= 67108864.0);
+    const bool pair_want = ctx->pair_mode == 2 || (ctx->pair_mode == 0 && (double)M * (double)N >= 6.0e6);
     const int pairs = (pair_shape && pair_want) ? umma2_max_pairs<256>(ctx) : 0;
     if (int st = make_map(ctx, &mapA, A8, M, kb <= lda8 ? kb : lda8, lda8, BM)) return st;
     if (int st = make_map(ctx, &mapB, B8, N, kb <= ldb8 ? kb : ldb8, ldb8, pairs > 0 ? 128 : bn)) return st;
