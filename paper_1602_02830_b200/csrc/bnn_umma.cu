@@ -201,9 +201,25 @@ __device__ __forceinline__ uint32_t nibbles_of_byte(uint32_t x) {
 }
 // The signs of 32 consecutive outputs of row `orow` (bit j of `word` = column col0 + j) in the next layer's operand
 // format: one signed byte per value, or one e2m1 nibble per value.  Positions at or beyond N are written as 0.
-__device__ __forceinline__ void store_signs(const UmmaArgs &p, uint32_t word, int64_t orow, int64_t col0) {
+// role / hold (nibble output): a warp that takes two adjacent 32-column chunks keeps the first chunk's 16 bytes (role 1)
+// and writes both with one 32-byte store when it has the second (role 2): whole sectors instead of half ones.
+__device__ __forceinline__ void store_signs(const UmmaArgs &p, uint32_t word, int64_t orow, int64_t col0, int role = 0,
+                                            uint4 *hold = nullptr) {
     if (p.out_f4) {
         uint8_t *d = reinterpret_cast<uint8_t *>(p.out8) + orow * p.ldo8 + (col0 >> 1);
+        if (role != 0) {
+            // both chunks whole, and the pair's 32 bytes on a 32-byte boundary (the same answer in both roles)
+            const int64_t first = (role == 1) ? col0 : col0 - 32;
+            uint8_t *d0 = reinterpret_cast<uint8_t *>(p.out8) + orow * p.ldo8 + (first >> 1);
+            if (first + 64 <= p.N && (reinterpret_cast<uintptr_t>(d0) & 31u) == 0) {
+                const uint4 v = make_uint4(nibbles_of_byte(word & 0xffu), nibbles_of_byte((word >> 8) & 0xffu),
+                                           nibbles_of_byte((word >> 16) & 0xffu), nibbles_of_byte(word >> 24));
+                if (role == 1) { *hold = v; return; }
+                asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                             ::"l"(d0), "r"(hold->x), "r"(hold->y), "r"(hold->z), "r"(hold->w), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+                return;
+            }
+        }
         if (col0 + 32 <= p.N) {
             *reinterpret_cast<uint4 *>(d) = make_uint4(nibbles_of_byte(word & 0xffu), nibbles_of_byte((word >> 8) & 0xffu),
                                                        nibbles_of_byte((word >> 16) & 0xffu), nibbles_of_byte(word >> 24));
@@ -243,7 +259,7 @@ __device__ __forceinline__ void store_signs(const UmmaArgs &p, uint32_t word, in
 // One 32-column chunk of accumulators (r, one output row per thread) -> the requested outputs.
 template <int BN>
 __device__ __forceinline__ void epilogue_chunk(Control *ctl, const UmmaArgs &p, uint32_t (&r)[32], uint32_t buf, int c, int64_t col0,
-                                               int64_t row, int q, int lane) {
+                                               int64_t row, int q, int lane, int role = 0, uint4 *hold = nullptr) {
     if (row >= p.M) return;
     if (p.thr) {                                         // thresholded signs: packed words and/or the next layer's operand
         // bit j of the word = (acc[j] >= thr[j]) = NOT sign(acc[j] - thr[j]); the sign bits are shifted
@@ -267,7 +283,7 @@ __device__ __forceinline__ void epilogue_chunk(Control *ctl, const UmmaArgs &p, 
         if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;      // columns beyond N stay 0
         if (p.pool) ctl->poolw[32 * q + lane][c] = word ^ ctl->flip[buf][c];   // un-flipped (dot >= thr) bits
         else if (p.out) p.out[row * p.ldo + (col0 >> 5)] = word;
-        if (p.out8 && !p.pool) store_signs(p, word, row, col0);
+        if (p.out8 && !p.pool) store_signs(p, word, row, col0, role, hold);
     }
     if (p.C) {
         if (BN == 192) {   // the 4-bit engine accumulates in float32: exact integers
@@ -367,13 +383,27 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
             // more warps per quadrant: chunks go round-robin over them, one register buffer, and the other warps of
             // the scheduler cover the load latency
             uint32_t r[32];
+            if constexpr (CHUNKS == 2 * EPW) {
+                // two adjacent chunks per warp, so that nibble outputs leave as whole 32-byte sectors
+                uint4 hold = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll 1
-            for (int c = half; c < CHUNKS; c += EPW) {
-                const int64_t col0 = n0 + 32 * c;
-                if (col0 >= p.N) break;                      // uniform over the warp
-                tmem_ld32(tbase + (uint32_t)(32 * c), r);
-                tmem_ld_wait(r);
-                epilogue_chunk<BN>(ctl, p, r, buf, c, col0, row, q, lane);
+                for (int i = 0; i < 2; ++i) {
+                    const int c = 2 * half + i;
+                    const int64_t col0 = n0 + 32 * c;
+                    if (col0 >= p.N) break;                  // uniform over the warp
+                    tmem_ld32(tbase + (uint32_t)(32 * c), r);
+                    tmem_ld_wait(r);
+                    epilogue_chunk<BN>(ctl, p, r, buf, c, col0, row, q, lane, 1 + i, &hold);
+                }
+            } else {
+#pragma unroll 1
+                for (int c = half; c < CHUNKS; c += EPW) {
+                    const int64_t col0 = n0 + 32 * c;
+                    if (col0 >= p.N) break;                  // uniform over the warp
+                    tmem_ld32(tbase + (uint32_t)(32 * c), r);
+                    tmem_ld_wait(r);
+                    epilogue_chunk<BN>(ctl, p, r, buf, c, col0, row, q, lane);
+                }
             }
         }
         // padding words of the packed output
