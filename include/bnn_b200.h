@@ -159,7 +159,9 @@ BNN_API int bnn_binary_dense(bnn_ctx *ctx, const uint32_t *Ap, int64_t lda_w, co
 /* ---------------------------------------------------------------------------------------------
  * First layer on 8-bit inputs (Section 1.6, Eq. 6-7; Algorithm 4, step 1):
  *   s[m][n] = sum_i X[m][i] * w[i][n] = sum_{p=1..8} 2^(p-1) * (x^p[m] . w[:,n]),  x^p in {0,1}.
- *   X  M x K uint8 row-major (ldx elements), Wp packed N x K.
+ *   X  M x K uint8 row-major (ldx elements), Wp packed N x K.  The tensor-core engine needs X 16-byte aligned and
+ *      ldx a multiple of 16 (otherwise the CUDA-core kernels run); rows that start on 32-byte boundaries (ldx a
+ *      multiple of 32, e.g. 800 for K = 784) are fetched in whole sectors and make the layer about 15 % faster.
  *   out_sums (or NULL): M x N int32, leading dimension lds.
  *   out_bits (or NULL): packed M x N, bit = (s >= thr[n]) XOR flip_bit[n]; thr is required then.
  * At least one output must be given.
@@ -241,7 +243,8 @@ typedef struct {
 
 /* Scratch bytes bnn_mlp_forward (host_io = 0) or bnn_mlp_forward_host (host_io = 1) need for `batch`. */
 BNN_API size_t bnn_mlp_workspace_bytes(const bnn_mlp_desc *m, int64_t batch, int host_io);
-/* X batch x K0 uint8 (device, ldx), scores batch x N_last float32 (device, lds).
+/* X batch x K0 uint8 (device, ldx; see bnn_first_layer_bitplanes for what ldx means to the tensor-core engine),
+ * scores batch x N_last float32 (device, lds).
  * If `hidden_out` is not NULL it is a host array of n_layers-1 device pointers (entries may be NULL);
  * hidden layer k's packed activations (batch x N_k, leading dimension ceil(N_k/128)*4 words)
  * are also copied there.  Needs a workspace (BNN_ERR_WORKSPACE otherwise). */
