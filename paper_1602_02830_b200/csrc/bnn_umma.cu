@@ -1269,8 +1269,12 @@ int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B,
     if (!bnn_umma_conv_tiling(H, W, pool, &TH, &TB) || (C_in % BK) != 0 || (pool && (out_sums || !out_bits))) return BNN_ERR_INVALID_ARG;
     CUtensorMap mapA, mapB;
     const int bn = umma_tile_n(C_out);
+    // CTA pairs (each CTA its own 128 pixels and half of the tile's filters) from 6 M outputs on, as for plain products
+    const bool pair_want = ctx->pair_mode == 2 || (ctx->pair_mode == 0 && (double)(B * H * W) * (double)C_out >= 6.0e6);
+    const int pairs = !(B * H * W >= 512 && pair_want) ? 0 : (bn == 256 ? umma2_max_pairs<256>(ctx) : umma2_max_pairs<128>(ctx));
+    if (pairs > 0) { if (int st = umma_prepare(ctx)) return st; }
     if (int st = make_map_nhwc(ctx, &mapA, act8, B, H, W, C_in, (int)W, TH, TB)) return st;
-    if (int st = make_map(ctx, &mapB, W8, C_out, 9 * C_in, 9 * C_in, bn)) return st;
+    if (int st = make_map(ctx, &mapB, W8, C_out, 9 * C_in, 9 * C_in, pairs > 0 ? bn / 2 : bn)) return st;
     UmmaArgs a{};
     a.M = B * H * W; a.N = C_out;
     a.k_iters = (int)(9 * (C_in / BK));
@@ -1279,6 +1283,14 @@ int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B,
     a.C = out_sums; a.ldc = C_out; a.out = out_bits; a.ldo = (C_out + 31) / 32; a.thr = thr; a.flip = flip;
     a.out8 = out8; a.ldo8 = ldo8; a.out_f4 = out_f4;
     a.conv = 1; a.H = (int)H; a.W = (int)W; a.TH = TH; a.TB = TB; a.c_chunks = (int)(C_in / BK); a.pool = pool;
+    if (pairs > 0) {
+        const int64_t tiles2 = ((a.M + 2 * BM - 1) / (2 * BM)) * ((C_out + bn - 1) / bn);
+        if (tiles2 >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;
+        const dim3 grid((unsigned)(2 * (tiles2 < pairs ? tiles2 : pairs)));
+        if (bn == 256) BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8_2sm<256>, grid, dim3(Warps<256>::NTHREADS), umma2_smem_bytes<256>(), ctx->stream, mapA, mapB, a));
+        else BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8_2sm<128>, grid, dim3(Warps<128>::NTHREADS), umma2_smem_bytes<128>(), ctx->stream, mapA, mapB, a));
+        return bnn_check_launch(ctx);
+    }
     return umma_launch(ctx, mapA, mapB, a, bn);
 }
 
