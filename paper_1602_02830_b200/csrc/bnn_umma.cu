@@ -428,11 +428,9 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                 word ^= ctl->flip[buf][c];
                 const int64_t col0 = n0 + 32 * c;
                 if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;
-                // output pixel: same image, (y/2, x/2)
-                const int64_t img = pix / ((int64_t)p.H * p.W);
-                const int64_t rem = pix - img * (int64_t)p.H * p.W;
-                const int64_t oy = (rem / p.W) >> 1, ox = (rem % p.W) >> 1;
-                const int64_t opix = (img * (p.H >> 1) + oy) * Wo + ox;
+                // output pixel: same image, (y/2, x/2).  The tile starts at x = 0 of an even row and holds whole rows (of
+                // one image or of TB whole images), so its 32 windows are 32 consecutive output pixels from m0 / 4 on.
+                const int64_t opix = (m0 >> 2) + win;
                 p.out[opix * p.ldo + (col0 >> 5)] = word;
                 if (n0 + BN >= p.N && c == nwords - 1)
                     for (int64_t w = (p.N + 31) >> 5; w < p.ldo; ++w) p.out[opix * p.ldo + w] = 0u;
