@@ -33,6 +33,8 @@ namespace {
 constexpr int BM = 128, BK = 128;               // BK in bytes = int8 elements
 constexpr int BN_MAX = 256;                     // tile width: 256, or 128 for narrow outputs; 192 = the 4-bit engine
 constexpr uint32_t SF_COL = 480;                // 4-bit engine: first of the 32 TMEM columns that hold the scale factors
+// Tile widths of the 4-bit engine: 192, and 224 for the pair kernel (two accumulator buffers + 32 scale columns <= 512)
+constexpr bool is_f4(int bn) { return bn == 192 || bn == 224; }
 constexpr int N_ISSUE = 2;                      // MMA-issuing warps: warp 1 and the warps behind the epilogue warps
 // Epilogue warps per tile width: EPW per TMEM lane quadrant.  With two, each takes a contiguous half of the columns and
 // prefetches its next chunk; with four, chunks go round-robin and the other warps of the scheduler cover the load
@@ -42,7 +44,7 @@ template <int BN> struct Warps {
 #ifdef BNN_EPI_WARPS
     static constexpr int EPI_WARPS = BNN_EPI_WARPS;
 #else
-    static constexpr int EPI_WARPS = (BN == 192) ? 8 : 16;
+    static constexpr int EPI_WARPS = is_f4(BN) ? 8 : 16;
 #endif
     static constexpr int EPW = EPI_WARPS / 4;
     static constexpr int EPI_THREADS = EPI_WARPS * 32;
@@ -54,9 +56,9 @@ constexpr int ACC_BUFS = 2;
 template <int BN> struct Cfg {
     static constexpr uint32_t B_BYTES = BN * BK;
     static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (BN == 256) ? 4 : ((BN == 192) ? 5 : 6);   // 192-200 KB of operand stages
+    static constexpr int STAGES = (BN == 256) ? 4 : (is_f4(BN) ? 5 : 6);   // 192-200 KB of operand stages
     // two accumulator buffers of BN columns; the 4-bit configuration (BN = 192) also keeps 32 columns of scale factors
-    static constexpr uint32_t TMEM_COLS = (BN == 192) ? 512 : 2 * BN;
+    static constexpr uint32_t TMEM_COLS = is_f4(BN) ? 512 : 2 * BN;
 };
 constexpr int STAGES_MAX = 7;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // a wait gives up after 2 s of wall clock
@@ -273,7 +275,7 @@ __device__ __forceinline__ void epilogue_chunk(Control *ctl, const UmmaArgs &p, 
 #pragma unroll
             for (int i = 3; i >= 0; --i) {
                 const int j = 4 * g + i;
-                const uint32_t d = (BN == 192) ? __float_as_uint(__uint_as_float(r[j]) - __int_as_float(tv[i]))
+                const uint32_t d = is_f4(BN) ? __float_as_uint(__uint_as_float(r[j]) - __int_as_float(tv[i]))
                                                : (uint32_t)((int32_t)r[j] - tv[i]);
                 w4[j >> 3] = __funnelshift_l(d, w4[j >> 3], 1);
             }
@@ -286,7 +288,7 @@ __device__ __forceinline__ void epilogue_chunk(Control *ctl, const UmmaArgs &p, 
         if (p.out8 && !p.pool) store_signs(p, word, row, col0, role, hold);
     }
     if (p.C) {
-        if (BN == 192) {   // the 4-bit engine accumulates in float32: exact integers
+        if (is_f4(BN)) {   // the 4-bit engine accumulates in float32: exact integers
             if (p.k_iters <= (1 << 14)) {
                 // |sum| <= K <= 2^22: adding 1.5 * 2^23 leaves the integer in the low mantissa bits (an add and a
                 // subtract on the full-rate pipes instead of a quarter-rate conversion)
@@ -324,7 +326,7 @@ __device__ __forceinline__ void epilogue_chunk(Control *ctl, const UmmaArgs &p, 
 // in magnitude (2^24 on the 4-bit engine, where they are float32), so thresholds clamp to that range unchanged in meaning.
 template <int BN>
 __device__ __forceinline__ int32_t staged_threshold(int32_t t) {
-    if (BN == 192) return __float_as_int(t > (1 << 24) ? 3.0e7f : (t < -(1 << 24) ? -3.0e7f : (float)t));
+    if (is_f4(BN)) return __float_as_int(t > (1 << 24) ? 3.0e7f : (t < -(1 << 24) ? -3.0e7f : (float)t));
     return max(min(t, 1 << 30), -(1 << 30));
 }
 
@@ -335,7 +337,7 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                                               int64_t m0, int64_t n0, int64_t n0_next, int q, int half, int lane, int et, bool &ok) {
     constexpr int EPW = Warps<BN>::EPW, EPI_THREADS = Warps<BN>::EPI_THREADS;
     static_assert(BN <= EPI_THREADS, "one staged threshold per epilogue thread");
-    constexpr int CHUNKS = BN / 32, CPW = CHUNKS / 2;   // 32-column chunks per tile and per warp (two warps per quadrant)
+    constexpr int CHUNKS = BN / 32, CPW = (CHUNKS + 1) / 2;   // 32-column chunks per tile and (at most) per warp with two warps per quadrant
     const int64_t row = m0 + 32 * q + lane;
     if (p.thr && tc == 0) {                              // the first tile stages its own thresholds
         if (et < BN) ctl->thr[buf][et] = staged_threshold<BN>((n0 + et < p.N) ? p.thr[n0 + et] : 0x7fffffff);
@@ -361,18 +363,19 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
     ok = ok && (ctl->failed == 0);
     if (ok) {
         const uint32_t tbase = tmem_base + ((uint32_t)(32 * q) << 16) + buf * BN;
-        if constexpr (EPW == 2 && (CHUNKS % 2) == 0) {
-            // two warps per quadrant, each a contiguous half of the columns: chunk c+1 is fetched from tensor memory
-            // while chunk c is processed (unrolled, so both register buffers are addressed statically)
+        if constexpr (EPW == 2) {
+            // two warps per quadrant, each a contiguous half of the columns (the first one chunk more when their number
+            // is odd): chunk c+1 is fetched from tensor memory while chunk c is processed (unrolled, so both register
+            // buffers are addressed statically)
             uint32_t ra[32], rb[32];
-            const int c_first = half * CPW;
+            const int c_first = half * CPW, c_end = half ? CHUNKS : CPW;
             if (n0 + 32 * c_first < p.N) { tmem_ld32(tbase + (uint32_t)(32 * c_first), ra); tmem_ld_wait(ra); }
 #pragma unroll
             for (int cc = 0; cc < CPW; ++cc) {
                 const int c = c_first + cc;
                 const int64_t col0 = n0 + 32 * c;
-                if (col0 >= p.N) break;                      // uniform over the warp
-                const bool more = (cc + 1 < CPW) && (col0 + 32 < p.N);
+                if (c >= c_end || col0 >= p.N) break;        // uniform over the warp
+                const bool more = (c + 1 < c_end) && (col0 + 32 < p.N);
                 uint32_t (&r)[32] = (cc & 1) ? rb : ra;
                 uint32_t (&rn)[32] = (cc & 1) ? ra : rb;
                 if (more) tmem_ld32(tbase + (uint32_t)(32 * (c + 1)), rn);
@@ -488,7 +491,7 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
     // waits for it below (bnn_pdl_wait): the producer (after requesting weights that kernel does not write), the
     // epilogue warps at once; they also release this kernel's own successor.
 
-    if (BN == 192) {
+    if (is_f4(BN)) {
         // 4-bit engine: every value is exactly +-1, so every block scale is 2^0.  In UE8M0 that is the byte 0x7f, and
         // with all 32 scale-factor columns filled with it the instruction reads 1.0 wherever it looks.
         if (warp >= 2 && warp < 6) {
@@ -562,7 +565,7 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
         if (lane == 0) {
             const int w = (warp == 1) ? 0 : warp - MMA_WARP_B + 1;   // this warp takes K steps w, w + N_ISSUE, ...
             // e2m1 x e2m1 (format 1), UE8M0 scales (bit 23) on the 4-bit engine; N >> 3 at bit 17, M >> 4 at bit 24
-            const uint32_t idesc = (BN == 192)
+            const uint32_t idesc = is_f4(BN)
                 ? ((1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (1u << 23) | ((uint32_t)(BM >> 4) << 24))
                 : (p.idesc | ((uint32_t)(BN >> 3) << 17));
             const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
@@ -585,7 +588,7 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k) {   // 32 bytes of K per instruction: start address advances by 32 B (>> 4 = 2)
                         if (k >= nk) break;
-                        if (BN == 192) umma_mxf4(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u, tmem_base + SF_COL);
+                        if (is_f4(BN)) umma_mxf4(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u, tmem_base + SF_COL);
                         else umma_i8(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u);
                     }
                     umma_commit(empty0 + 8 * s);                // stage may be refilled once these MMAs have read it
@@ -736,7 +739,7 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = ctl->tmem_base;
 
-    if (BN == 192) {
+    if (is_f4(BN)) {
         // 4-bit engine: unit block scales (byte 0x7f) in this CTA's scale-factor columns; the leader's MMAs read the
         // columns of both CTAs, so the pair synchronises once more before the first one is issued
         if (warp >= 2 && warp < 6) {
@@ -800,7 +803,7 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         if (lane == 0 && rank == 0) {
             const int w = (warp == 1) ? 0 : warp - MMA_WARP_B + 1;
             // the host's descriptor carries M = 128 in bits [24,29); the pair multiplies M = 256
-            const uint32_t idesc = (BN == 192)
+            const uint32_t idesc = is_f4(BN)
                 ? ((1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (1u << 23) | ((uint32_t)((2 * BM) >> 4) << 24))
                 : ((p.idesc & ~(0x1fu << 24)) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24));
             const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
@@ -823,7 +826,7 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k) {
                         if (k >= nk) break;
-                        if (BN == 192) umma_mxf4_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u, tmem_base + SF_COL);
+                        if (is_f4(BN)) umma_mxf4_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u, tmem_base + SF_COL);
                         else umma_i8_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u);
                     }
                     umma_commit_2sm(empty0 + 8 * s);
@@ -1149,9 +1152,27 @@ int bnn_umma_gemm_f4(bnn_ctx *ctx, const uint8_t *A4, int64_t lda4, const uint8_
     CUtensorMap mapA, mapB;
     const int64_t kb = (((K + 1) / 2 + 15) / 16) * 16;      // extent along K in bytes
     const bool pair_want = ctx->pair_mode == 2 || (ctx->pair_mode == 0 && (double)M * (double)N >= 6.0e6);
-    const int pairs = (M >= 512 && pair_want) ? umma2_max_pairs<192>(ctx) : 0;
+    // Pair kernel: 224- or 192-wide tiles.  A K step brings 128 + bn / 2 box rows into every CTA and the chip delivers
+    // ~0.54 rows per clock and SM: 415 clocks for a 192-wide step whose MMAs take 384, but 444 clocks for a 224-wide one
+    // whose MMAs take 448, so the wider tile is not held up by L2 and costs ~1.09 x the narrower one for 1.17 x the
+    // columns (measured).  The kernel's time is the largest number of tiles one pair gets, times that cost.
+    int bn2 = 192;
+    {
+        const int p224 = umma2_max_pairs<224>(ctx), p192 = umma2_max_pairs<192>(ctx);
+        if (p224 > 0 && p192 > 0) {
+            const int64_t tm2 = (M + 2 * BM - 1) / (2 * BM);
+            const int64_t r224 = (tm2 * ((N + 223) / 224) + p224 - 1) / p224, r192 = (tm2 * ((N + 191) / 192) + p192 - 1) / p192;
+            if (1.09 * (double)r224 <= (double)r192) bn2 = 224;
+        } else if (p224 > 0) {
+            bn2 = 224;
+        }
+    }
+#ifdef BNN_F4_PAIR_TILE
+    bn2 = BNN_F4_PAIR_TILE;
+#endif
+    const int pairs = !(M >= 512 && pair_want) ? 0 : (bn2 == 224 ? umma2_max_pairs<224>(ctx) : umma2_max_pairs<192>(ctx));
     if (int st = make_map(ctx, &mapA, A4, M, kb <= lda4 ? kb : lda4, lda4, BM)) return st;
-    if (int st = make_map(ctx, &mapB, B4, N, kb <= ldb4 ? kb : ldb4, ldb4, pairs > 0 ? 96 : 192)) return st;
+    if (int st = make_map(ctx, &mapB, B4, N, kb <= ldb4 ? kb : ldb4, ldb4, pairs > 0 ? bn2 / 2 : 192)) return st;
     UmmaArgs a{};
     a.M = M; a.N = N;
     a.k_iters = (int)((K + 2 * BK - 1) / (2 * BK));          // 256 values per 128-byte K step
@@ -1160,11 +1181,15 @@ int bnn_umma_gemm_f4(bnn_ctx *ctx, const uint8_t *A4, int64_t lda4, const uint8_
     a.out8 = reinterpret_cast<int8_t *>(out4); a.ldo8 = ldo4; a.out_f4 = 1; a.b_static = b_static;
     if (pairs > 0) {
         if (int st = umma_prepare(ctx)) return st;
-        const int64_t tiles2 = ((M + 2 * BM - 1) / (2 * BM)) * ((N + 191) / 192);
+        const int64_t tiles2 = ((M + 2 * BM - 1) / (2 * BM)) * ((N + bn2 - 1) / bn2);
         if (tiles2 >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;
         const int64_t use = tiles2 < pairs ? tiles2 : pairs;
-        BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8_2sm<192>, dim3((unsigned)(2 * use)), dim3(Warps<192>::NTHREADS), umma2_smem_bytes<192>(),
-                                               ctx->stream, mapA, mapB, a));
+        if (bn2 == 224)
+            BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8_2sm<224>, dim3((unsigned)(2 * use)), dim3(Warps<224>::NTHREADS), umma2_smem_bytes<224>(),
+                                                   ctx->stream, mapA, mapB, a));
+        else
+            BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8_2sm<192>, dim3((unsigned)(2 * use)), dim3(Warps<192>::NTHREADS), umma2_smem_bytes<192>(),
+                                                   ctx->stream, mapA, mapB, a));
         return bnn_check_launch(ctx);
     }
     return umma_launch(ctx, mapA, mapB, a, 192);
