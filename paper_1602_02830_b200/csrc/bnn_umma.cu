@@ -9,19 +9,22 @@
 //             accumulators, 128 x 256 tiles (128 x 128 for narrow outputs);
 //     nibbles (e2m1: +1 = 0x2, -1 = 0xa): tcgen05.mma kind::mxf4.block_scale with every block scale 2^0 (32 TMEM
 //             columns filled once with the UE8M0 byte 0x7f), float32 accumulators (exact while K <= 2^24),
-//             128 x 192 tiles, twice the MMA rate and half the operand bytes.
+//             128 x 192 tiles (CTA pairs: 256 x 192 or 256 x 224), twice the MMA rate and half the operand bytes.
 //
 // Kernel k_umma_i8<BN> (persistent, one CTA per SM walking 128 x BN output tiles, column blocks fastest):
 //   warp 0       TMA producer: cp.async.bulk.tensor loads of 128-byte-wide K slices (128B swizzle) of both
 //                operands into a ring of 4-6 shared-memory stages, completion on mbarriers;
-//   warps 1, 10  MMA issuers: one lane each, alternate K steps of every tile (issuing a step costs one thread more
-//                clocks than the tensor core needs to run it); four MMAs per step, tcgen05.commit releases the
-//                stage; warp 1 also allocates the 512 TMEM columns (two accumulator buffers);
-//   warps 2-9    epilogue (two warps per TMEM lane quadrant, each half of the columns): tcgen05.ld of the
-//                accumulators (one output row per thread, 32 columns at a time, the next chunk in flight while the
-//                current one is processed), then int32 stores, or the BatchNorm-folded threshold + Sign as one
-//                32-bit word per 32 columns and/or the same signs in the next layer's operand format.
-// Kernel k_umma_i8_2sm<BN>: the same with a cluster of two CTAs on one 256 x BN tile (cta_group::2).
+//   warp 1 and the last warp  MMA issuers: one lane each, alternate K steps of every tile (issuing a step costs one
+//                thread more clocks than the tensor core needs to run it); four MMAs per step, tcgen05.commit
+//                releases the stage; warp 1 also allocates the TMEM columns (two accumulator buffers);
+//   warps 2 ..   epilogue, 8 warps on the 4-bit tiles (two per TMEM lane quadrant, each a contiguous half of the
+//                columns, the next 32-column chunk in flight while the current one is processed), 16 on the byte
+//                tiles (four per quadrant): tcgen05.ld of the accumulators (one output row per thread), then int32
+//                stores, or the BatchNorm-folded threshold + Sign as one 32-bit word per 32 columns and/or the same
+//                signs in the next layer's operand format.
+// Kernel k_umma_i8_2sm<BN>: the same with a cluster of two CTAs on one 256 x BN tile (cta_group::2); BN = 256 or 128
+// for bytes, 192 or 224 for nibbles (224: the widest tile whose two accumulator buffers and scale columns fit tensor
+// memory; its K step brings 240 operand rows for 448 clocks of MMAs, which L2 can deliver, see bnn_umma_gemm_f4).
 // Every wait is bounded: after the limit the kernel records an error code and runs to its end without
 // touching the accumulators, so a failure surfaces as BNN_ERR_DEVICE_STATUS instead of a hang.
 #include "bnn_internal.cuh"
