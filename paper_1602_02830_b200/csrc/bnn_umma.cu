@@ -1165,9 +1165,9 @@ int bnn_umma_gemm_f4(bnn_ctx *ctx, const uint8_t *A4, int64_t lda4, const uint8_
         if (p224 > 0 && p192 > 0) {
             const int64_t tm2 = (M + 2 * BM - 1) / (2 * BM);
             const int64_t r224 = (tm2 * ((N + 223) / 224) + p224 - 1) / p224, r192 = (tm2 * ((N + 191) / 192) + p192 - 1) / p192;
-            // (operands that do not stay in L2 make the product wait for HBM instead; 16384^3 measured 1.62 ms on 224-wide
-            // and 1.54 ms on 192-wide tiles)
-            if (1.09 * (double)r224 <= (double)r192 && (double)(M + N) * (double)kb <= 1.0e8) bn2 = 224;
+            // (a B operand that does not stay in L2 between the row blocks makes the product wait for HBM instead:
+            // 16384^3, 134 MB of B, measured 1.62 ms on 224-wide and 1.55 ms on 192-wide tiles)
+            if (1.09 * (double)r224 <= (double)r192 && (double)N * (double)kb <= 6.4e7) bn2 = 224;
         } else if (p224 > 0) {
             bn2 = 224;
         }
