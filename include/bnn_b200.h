@@ -74,9 +74,10 @@ BNN_API int bnn_set_tile_rows(bnn_ctx *ctx, int rows);
  *       (bnn_gemm_workspace_bytes / bnn_mlp_workspace_bytes), otherwise the CUDA-core kernels;
  *   1 = CUDA-core XOR-popcount kernels only (Eq. 8 as the paper computes it);
  *   2 = tensor-core engine wherever the shape qualifies; BNN_ERR_WORKSPACE if the workspace is too small.
- * The tensor-core engine expands the packed operands to one signed byte per value in the workspace and
- * multiplies them with int8 tensor-core instructions (Section 4: on +-1 inputs the binary kernel and an ordinary
- * matrix product return identical outputs). */
+ * The tensor-core engine expands the packed operands in the workspace to the format bnn_set_operand_bits selects
+ * (4-bit e2m1 nibbles by default, signed bytes for layers with 8-bit inputs) and multiplies them exactly with
+ * tcgen05 tensor-core instructions (Section 4: on +-1 inputs the binary kernel and an ordinary matrix product
+ * return identical outputs).  Engine 1 is the XOR-popcount form the popc roofline applies to. */
 BNN_API int bnn_set_engine(bnn_ctx *ctx, int engine);
 /* Tensor-core engine only: plain products can run on pairs of SMs (thread-block clusters of two, tcgen05
  * cta_group::2) that share the B operand.  0 (default) = for outputs of 6 million elements and more, where it measured
@@ -120,6 +121,16 @@ BNN_API int bnn_expand_signs_f4(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w,
 BNN_API int bnn_binary_dense_expanded(bnn_ctx *ctx, const void *A_exp, int64_t lda_bytes, const void *W_exp, int64_t ldw_bytes,
                                       int operand_bits, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits,
                                       int64_t ldo_w, void *out_exp, int64_t ldo_exp, int64_t M, int64_t N, int64_t K);
+/* Tensor-core engine only: every wait of its kernels on a barrier (operands arrived, stage free, accumulator ready) is
+ * bounded.  A wait that lasts longer than `ns` nanoseconds of wall clock (default 2 s; 1 .. 60 s) gives up: the kernel
+ * records a code, skips the rest of its work, frees its tensor memory and ends normally, and the other waiters of the
+ * same CTA (and of its partner in a CTA pair) stop at their next look, so one failure costs about one limit.
+ * bnn_device_status then reports BNN_ERR_DEVICE_STATUS and the context stays usable. */
+BNN_API int bnn_set_wait_limit_ns(bnn_ctx *ctx, uint64_t ns);
+/* Test hook for the failure path above (host-side injection, nothing faults): while on = 1 the tensor-core kernels
+ * launched through this context run in their single-SM form with a producer that requests no operands, so their
+ * consumers' waits run into the limit.  Outputs of such calls are undefined.  on = 0 restores normal operation. */
+BNN_API int bnn_debug_drop_loads(bnn_ctx *ctx, int on);
 /* Synchronises the context's stream and returns BNN_ERR_DEVICE_STATUS if a kernel gave up on one of its
  * bounded waits since the last call (its outputs are then undefined), BNN_OK otherwise. */
 BNN_API int bnn_device_status(bnn_ctx *ctx);
@@ -277,7 +288,8 @@ BNN_API int bnn_baseline_gemm_f32(bnn_ctx *ctx, const float *A, const float *B, 
  * is supplied by the library, from an array that is part of the library image.
  *
  * Same arguments and results as bnn_mlp_forward (device X and scores; no hidden_out), no workspace needed
- * and none used.  Limits and rules:
+ * and none used: a workspace that was lent to the context for other calls is neither read nor written.
+ * Limits and rules:
  *  - batch * ceil(widest hidden layer / 128) * 16 bytes must not exceed bnn_mlp_noalloc_max_bytes()
  *    (512 KiB: e.g. batch 1024 at 4096 units); beyond that the call returns BNN_ERR_TOO_LARGE and does nothing.
  *    Every GPU that loads the library holds 1 MiB for this array until the process exits.

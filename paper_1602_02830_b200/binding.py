@@ -28,7 +28,8 @@ EXPORTS = (
     "bnn_gemm_workspace_bytes", "bnn_device_status", "bnn_conv_workspace_bytes", "bnn_set_tile_rows", "bnn_set_pair_mode", "bnn_expanded_ld",
     "bnn_expanded_bytes", "bnn_expand_signs", "bnn_baseline_gemm_f32", "bnn_convnet_workspace_bytes",
     "bnn_convnet_forward", "bnn_set_operand_bits", "bnn_expanded_ld_f4",
-    "bnn_expanded_bytes_f4", "bnn_expand_signs_f4", "bnn_binary_dense_expanded",
+    "bnn_expanded_bytes_f4", "bnn_expand_signs_f4", "bnn_binary_dense_expanded", "bnn_set_wait_limit_ns",
+    "bnn_debug_drop_loads",
 )
 
 
@@ -84,6 +85,8 @@ def lib() -> ctypes.CDLL:
         L.bnn_set_tile_rows.argtypes = [vp, c_int]
         L.bnn_set_pair_mode.argtypes = [vp, c_int]
         L.bnn_set_operand_bits.argtypes = [vp, c_int]
+        L.bnn_set_wait_limit_ns.argtypes = [vp, ctypes.c_uint64]
+        L.bnn_debug_drop_loads.argtypes = [vp, c_int]
         L.bnn_expanded_ld_f4.argtypes = [i64]
         L.bnn_expanded_ld_f4.restype = i64
         L.bnn_expanded_bytes_f4.argtypes = [i64, i64]
@@ -219,6 +222,12 @@ class Context:
 
     def set_operand_bits(self, bits: int):
         self._ck(lib().bnn_set_operand_bits(self._h, bits), "bnn_set_operand_bits")
+
+    def set_wait_limit_ns(self, ns: int):
+        self._ck(lib().bnn_set_wait_limit_ns(self._h, ns), "bnn_set_wait_limit_ns")
+
+    def debug_drop_loads(self, on: bool):
+        self._ck(lib().bnn_debug_drop_loads(self._h, int(on)), "bnn_debug_drop_loads")
 
     def set_pair_mode(self, mode: int):
         self._ck(lib().bnn_set_pair_mode(self._h, mode), "bnn_set_pair_mode")

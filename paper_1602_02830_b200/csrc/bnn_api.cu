@@ -21,6 +21,8 @@ extern "C" int bnn_create(bnn_ctx **out, int device, void *cuda_stream) {
     c->tile_rows = 8;
     c->pair_mode = 0;
     c->operand_bits = 4;
+    c->wait_limit_ns = 2000000000ull;
+    c->drop_loads = 0;
     c->copy_stream = nullptr;
     c->copy_ready = false;
     for (int i = 0; i < 8; ++i) c->ev[i] = nullptr;
@@ -80,6 +82,18 @@ extern "C" int bnn_set_pair_mode(bnn_ctx *ctx, int mode) {
 extern "C" int bnn_set_operand_bits(bnn_ctx *ctx, int bits) {
     if (!ctx || (bits != 4 && bits != 8)) return BNN_ERR_INVALID_ARG;
     ctx->operand_bits = bits;
+    return BNN_OK;
+}
+
+extern "C" int bnn_set_wait_limit_ns(bnn_ctx *ctx, uint64_t ns) {
+    if (!ctx || ns == 0 || ns > 60000000000ull) return BNN_ERR_INVALID_ARG;
+    ctx->wait_limit_ns = ns;
+    return BNN_OK;
+}
+
+extern "C" int bnn_debug_drop_loads(bnn_ctx *ctx, int on) {
+    if (!ctx || (on != 0 && on != 1)) return BNN_ERR_INVALID_ARG;
+    ctx->drop_loads = on;
     return BNN_OK;
 }
 

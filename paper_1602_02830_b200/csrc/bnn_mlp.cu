@@ -13,6 +13,7 @@ int check_desc(const bnn_mlp_desc *m) {
     for (int k = 0; k < m->n_layers; ++k) {
         const bnn_layer_desc &L = m->layers[k];
         if (L.K <= 0 || L.N <= 0 || !L.Wp) return BNN_ERR_INVALID_ARG;
+        if (int st = bnn_check_packed(L.Wp, L.ldw_w, L.K, L.N)) return st;   // every kernel reads the rows with 128-bit loads
         if ((L.W8 && !bnn_aligned16(L.W8)) || (L.W4 && !bnn_aligned16(L.W4))) return BNN_ERR_ALIGNMENT;
         if (k > 0 && L.K != m->layers[k - 1].N) return BNN_ERR_INVALID_ARG;
         if (k < m->n_layers - 1) {
@@ -30,6 +31,15 @@ size_t act_bytes(const bnn_mlp_desc *m, int64_t batch) {
     for (int k = 0; k < m->n_layers - 1; ++k) widest = m->layers[k].N > widest ? m->layers[k].N : widest;
     return round256((size_t)batch * act_ld(widest) * 4);
 }
+
+// Hides the context's workspace for the duration of a call and puts it back on scope exit.
+struct workspace_hide {
+    bnn_ctx *ctx;
+    void *ws;
+    size_t bytes;
+    explicit workspace_hide(bnn_ctx *c) : ctx(c), ws(c->ws), bytes(c->ws_bytes) { c->ws = nullptr; c->ws_bytes = 0; }
+    ~workspace_hide() { ctx->ws = ws; ctx->ws_bytes = bytes; }
+};
 
 // Restores the context's engine choice on scope exit.
 struct engine_pin {
@@ -177,8 +187,8 @@ extern "C" size_t bnn_mlp_workspace_bytes(const bnn_mlp_desc *m, int64_t batch, 
 
 extern "C" int bnn_mlp_forward(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X, int64_t ldx, int64_t batch,
                                float *scores, int64_t lds, uint32_t *const *hidden_out) {
+    if (int st = check_desc(m)) return st;      // the descriptor first: its errors need no context to be found
     if (!ctx || batch < 0) return BNN_ERR_INVALID_ARG;
-    if (int st = check_desc(m)) return st;
     if (batch == 0) return BNN_OK;
     if (!X || !scores || ldx < m->layers[0].K || lds < m->layers[m->n_layers - 1].N) return BNN_ERR_INVALID_ARG;
     if (!ctx->ws || ctx->ws_bytes < bnn_mlp_workspace_bytes(m, batch, 0)) return BNN_ERR_WORKSPACE;
@@ -192,8 +202,8 @@ extern "C" int bnn_mlp_forward(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_
 
 extern "C" int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X_host, int64_t ldx,
                                     int64_t batch, float *scores_host, int64_t lds) {
+    if (int st = check_desc(m)) return st;      // the descriptor first: its errors need no context to be found
     if (!ctx || batch < 0) return BNN_ERR_INVALID_ARG;
-    if (int st = check_desc(m)) return st;
     if (batch == 0) return BNN_OK;
     const int64_t K0 = m->layers[0].K, NL = m->layers[m->n_layers - 1].N;
     if (!X_host || !scores_host || ldx < K0 || lds < NL) return BNN_ERR_INVALID_ARG;
@@ -324,8 +334,8 @@ extern "C" size_t bnn_mlp_noalloc_max_bytes(void) { return kNoAllocBufferBytes; 
 
 extern "C" int bnn_mlp_forward_noalloc(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint8_t *X, int64_t ldx,
                                        int64_t batch, float *scores, int64_t lds) {
+    if (int st = check_desc(m)) return st;      // the descriptor first: its errors need no context to be found
     if (!ctx || batch < 0) return BNN_ERR_INVALID_ARG;
-    if (int st = check_desc(m)) return st;
     if (batch == 0) return BNN_OK;
     if (!X || !scores || ldx < m->layers[0].K || lds < m->layers[m->n_layers - 1].N) return BNN_ERR_INVALID_ARG;
     // one activation buffer = batch rows of the widest hidden layer, packed; it must fit the built-in array
@@ -336,5 +346,8 @@ extern "C" int bnn_mlp_forward_noalloc(bnn_ctx *ctx, const bnn_mlp_desc *m, cons
     if (int st = noalloc_scratch(ctx, &scratch)) return st;
     // Nothing in the scratch has to start at zero: every layer writes all words of its output rows, padding
     // included, before the next layer reads them; what an earlier call left behind is never read.
+    // A workspace that the caller lent to the context for other calls stays untouched: with it hidden, the first layer
+    // takes its fused form, which needs no bit-plane scratch, and no layer can pick the tensor engine.
+    workspace_hide hide(ctx);
     return forward_device(ctx, m, X, ldx, batch, scores, lds, nullptr, scratch);
 }

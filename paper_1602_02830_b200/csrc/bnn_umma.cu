@@ -64,7 +64,6 @@ template <int BN> struct Cfg {
     static constexpr uint32_t TMEM_COLS = is_f4(BN) ? 512 : 2 * BN;
 };
 constexpr int STAGES_MAX = 7;
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // a wait gives up after 2 s of wall clock
 
 __device__ int g_umma_error;                    // 0 = fine; otherwise a code saying which wait gave up
 
@@ -84,6 +83,8 @@ struct UmmaArgs {
     int c_chunks;           // C_in / 128
     int pool;               // 2x2 max-pool (as OR of the sign bits) before the packed store
     int b_static;           // B (weights) is not written by the kernel launched just before this one
+    unsigned long long wait_ns;   // how long a wait on a barrier may last before the kernel gives up
+    int drop_loads;         // test hook (single-SM kernel): the producer issues no loads, every consumer's wait runs out
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -99,23 +100,6 @@ __device__ __forceinline__ unsigned long long global_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    unsigned long long t0 = 0;
-    for (uint32_t i = 0;; ++i) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-        if (done) return true;
-        if ((i & 63u) == 63u) {
-            const unsigned long long now = global_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) return false;
-        }
-    }
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
     asm volatile(
@@ -192,9 +176,31 @@ struct __align__(16) Control {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// Records that a wait gave up (the first code wins): in this CTA's control block, where every other waiter of the CTA
+// looks, and in the device word that bnn_device_status reads.
 __device__ __forceinline__ void fail(Control *ctl, int code) {
-    ctl->failed = (uint32_t)code;
-    atomicExch(&g_umma_error, code);
+    if (*reinterpret_cast<volatile uint32_t *>(&ctl->failed) == 0u) *reinterpret_cast<volatile uint32_t *>(&ctl->failed) = (uint32_t)code;
+    atomicCAS(&g_umma_error, 0, code);
+}
+// Bounded wait on a phase parity: false once `limit_ns` of wall clock have passed, or as soon as another wait of this
+// CTA (or of its partner in a pair) has given up, so that one failure costs one limit and not one per waiter.
+__device__ __forceinline__ bool mbar_wait(const Control *ctl, unsigned long long limit_ns, uint32_t bar, uint32_t parity) {
+    unsigned long long t0 = 0;
+    for (uint32_t i = 0;; ++i) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+        if ((i & 63u) == 63u) {
+            if (*reinterpret_cast<const volatile uint32_t *>(&ctl->failed) != 0u) return false;
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > limit_ns) return false;
+        }
+    }
 }
 
 // 8 sign bits -> 8 e2m1 nibbles (+1.0 = 0x2, -1.0 = 0xa); bit i lands in nibble i.
@@ -361,7 +367,7 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
             if (p.flip && w * 32 < p.N) next_flip = p.flip[w];
         }
     }
-    if (ok && !mbar_wait(smem_u32(&ctl->acc_full[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 3); ok = false; }
+    if (ok && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->acc_full[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 3); ok = false; }
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     ok = ok && (ctl->failed == 0);
     if (ok) {
@@ -509,8 +515,8 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
     }
 
     if (warp == 0) {
-        // ---------------- TMA producer
-        if (lane == 0) {
+        // ---------------- TMA producer (with the test hook set it requests nothing: every consumer's wait runs out)
+        if (lane == 0 && !p.drop_loads) {
             bool ok = true;
             // The loop below runs once per K step in a single thread that shares its scheduler with epilogue warps:
             // everything per tile is computed once, ring slot / phase / tap advance incrementally (no divisions inside;
@@ -544,7 +550,7 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                 int cc = 0, tx = -1, ty = -1;            // channel slice and tap offsets of the current K step
                 for (int kit = 0; kit < p.k_iters; ++kit) {
                     const bool pre = first_tile && kit < npre;      // B already requested, bytes already expected
-                    if (ph > 0 && !mbar_wait(smem_u32(&ctl->empty[s]), (ph - 1) & 1)) { fail(ctl, 1); ok = false; break; }
+                    if (ph > 0 && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->empty[s]), (ph - 1) & 1)) { fail(ctl, 1); ok = false; break; }
                     const uint32_t bar = smem_u32(&ctl->full[s]);
                     if (!pre) mbar_expect_tx(bar, STAGE_BYTES);
                     const uint32_t dst = smem_u32(tiles + s * STAGE_BYTES);
@@ -577,13 +583,13 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
             bool ok = true;
             for (int64_t t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++tc, it0 += (uint32_t)p.k_iters) {
                 const uint32_t buf = tc & 1;
-                if (tc >= ACC_BUFS && !mbar_wait(smem_u32(&ctl->acc_empty[buf]), ((tc / ACC_BUFS) - 1) & 1)) { fail(ctl, 4); ok = false; break; }
+                if (tc >= ACC_BUFS && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->acc_empty[buf]), ((tc / ACC_BUFS) - 1) & 1)) { fail(ctl, 4); ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tmem_d = tmem_base + buf * BN;
                 uint32_t s = (it0 + w) % STAGES, par = ((it0 + w) / STAGES) & 1;   // ring slot and phase of this warp's next step
                 for (int kit = w; kit < p.k_iters; kit += N_ISSUE) {
-                    if (w > 0 && kit == w && !mbar_wait(smem_u32(&ctl->started[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 5); ok = false; break; }
-                    if (!mbar_wait(full0 + 8 * s, par)) { fail(ctl, 2); ok = false; break; }
+                    if (w > 0 && kit == w && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->started[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 5); ok = false; break; }
+                    if (!mbar_wait(ctl, p.wait_ns, full0 + 8 * s, par)) { fail(ctl, 2); ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint64_t adesc = adesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
                     const uint64_t bdesc = bdesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
@@ -695,6 +701,16 @@ __device__ __forceinline__ void mbar_arrive_cta0(uint32_t bar) {
     asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
 }
 
+// A failed wait in one CTA of a pair: recorded locally (fail) and in the partner's control block, so that the partner's
+// waiters stop at their next look instead of each running into the limit.  Both CTAs stay resident until the
+// cluster-wide barrier at the end of the kernel, so the partner's shared memory is there to be written.
+__device__ __forceinline__ void fail_pair(Control *ctl, int code) {
+    fail(ctl, code);
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(&ctl->failed)), "r"(cluster_ctarank() ^ 1u));
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(remote), "r"((uint32_t)code) : "memory");
+}
+
 // 4-bit form of the pair instruction (see umma_mxf4).
 __device__ __forceinline__ void umma_mxf4_2sm(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate,
                                               uint32_t tmem_sf) {
@@ -788,7 +804,7 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                 int cc = 0, tx = -1, ty = -1;
                 for (int kit = 0; kit < p.k_iters; ++kit) {
                     const bool pre = first_tile && kit < npre;
-                    if (ph > 0 && !mbar_wait(smem_u32(&ctl->empty[s]), (ph - 1) & 1)) { fail(ctl, 11); ok = false; break; }
+                    if (ph > 0 && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->empty[s]), (ph - 1) & 1)) { fail_pair(ctl, 11); ok = false; break; }
                     if (rank == 0 && !pre) mbar_expect_tx(smem_u32(&ctl->full[s]), 2 * STAGE2_BYTES);   // the bytes of both CTAs
                     const uint32_t bar0 = smem_u32(&ctl->full[s]) & PEER_MASK;
                     if (p.conv) {
@@ -815,13 +831,13 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
             bool ok = true;
             for (int64_t t = pair; t < ntiles && ok; t += npairs, ++tc, it0 += (uint32_t)p.k_iters) {
                 const uint32_t buf = tc & 1;
-                if (tc >= ACC_BUFS && !mbar_wait(smem_u32(&ctl->acc_empty[buf]), ((tc / ACC_BUFS) - 1) & 1)) { fail(ctl, 14); ok = false; break; }
+                if (tc >= ACC_BUFS && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->acc_empty[buf]), ((tc / ACC_BUFS) - 1) & 1)) { fail_pair(ctl, 14); ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tmem_d = tmem_base + buf * BN;
                 uint32_t s = (it0 + w) % STAGES2, par = ((it0 + w) / STAGES2) & 1;
                 for (int kit = w; kit < p.k_iters; kit += N_ISSUE) {
-                    if (w > 0 && kit == w && !mbar_wait(smem_u32(&ctl->started[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 15); ok = false; break; }
-                    if (!mbar_wait(full0 + 8 * s, par)) { fail(ctl, 12); ok = false; break; }
+                    if (w > 0 && kit == w && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->started[buf]), (tc / ACC_BUFS) & 1)) { fail_pair(ctl, 15); ok = false; break; }
+                    if (!mbar_wait(ctl, p.wait_ns, full0 + 8 * s, par)) { fail_pair(ctl, 12); ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint64_t adesc = adesc0 + (uint64_t)(s * (STAGE2_BYTES >> 4));
                     const uint64_t bdesc = bdesc0 + (uint64_t)(s * (STAGE2_BYTES >> 4));
@@ -1175,10 +1191,11 @@ int bnn_umma_gemm_f4(bnn_ctx *ctx, const uint8_t *A4, int64_t lda4, const uint8_
 #ifdef BNN_F4_PAIR_TILE
     bn2 = BNN_F4_PAIR_TILE;
 #endif
-    const int pairs = !(M >= 512 && pair_want) ? 0 : (bn2 == 224 ? umma2_max_pairs<224>(ctx) : umma2_max_pairs<192>(ctx));
+    const int pairs = (!(M >= 512 && pair_want) || ctx->drop_loads) ? 0 : (bn2 == 224 ? umma2_max_pairs<224>(ctx) : umma2_max_pairs<192>(ctx));
     if (int st = make_map(ctx, &mapA, A4, M, kb <= lda4 ? kb : lda4, lda4, BM)) return st;
     if (int st = make_map(ctx, &mapB, B4, N, kb <= ldb4 ? kb : ldb4, ldb4, pairs > 0 ? bn2 / 2 : 192)) return st;
     UmmaArgs a{};
+    a.wait_ns = ctx->wait_limit_ns; a.drop_loads = ctx->drop_loads;
     a.M = M; a.N = N;
     a.k_iters = (int)((K + 2 * BK - 1) / (2 * BK));          // 256 values per 128-byte K step
     a.k_last = (int)((K - 2 * BK * (int64_t)(a.k_iters - 1) + 63) / 64);
@@ -1220,10 +1237,11 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
     // (auto: where it measured faster -- from about 1500 x 4096 outputs on; below that the larger tiles leave SMs idle)
     const bool pair_shape = bn == 256 && M >= 512 && !pool;
     const bool pair_want = ctx->pair_mode == 2 || (ctx->pair_mode == 0 && (double)M * (double)N >= 6.0e6);
-    const int pairs = (pair_shape && pair_want) ? umma2_max_pairs<256>(ctx) : 0;
+    const int pairs = (pair_shape && pair_want && !ctx->drop_loads) ? umma2_max_pairs<256>(ctx) : 0;
     if (int st = make_map(ctx, &mapA, A8, M, kb <= lda8 ? kb : lda8, lda8, BM)) return st;
     if (int st = make_map(ctx, &mapB, B8, N, kb <= ldb8 ? kb : ldb8, ldb8, pairs > 0 ? 128 : bn)) return st;
     UmmaArgs a{};
+    a.wait_ns = ctx->wait_limit_ns; a.drop_loads = ctx->drop_loads;
     a.M = M; a.N = N;
     a.k_iters = (int)((K + BK - 1) / BK);
     a.k_last = (int)((K - BK * (int64_t)(a.k_iters - 1) + 31) / 32);
@@ -1299,11 +1317,12 @@ int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B,
     const int bn = umma_tile_n(C_out);
     // CTA pairs (each CTA its own 128 pixels and half of the tile's filters) from 6 M outputs on, as for plain products
     const bool pair_want = ctx->pair_mode == 2 || (ctx->pair_mode == 0 && (double)(B * H * W) * (double)C_out >= 6.0e6);
-    const int pairs = !(B * H * W >= 512 && pair_want) ? 0 : (bn == 256 ? umma2_max_pairs<256>(ctx) : umma2_max_pairs<128>(ctx));
+    const int pairs = (!(B * H * W >= 512 && pair_want) || ctx->drop_loads) ? 0 : (bn == 256 ? umma2_max_pairs<256>(ctx) : umma2_max_pairs<128>(ctx));
     if (pairs > 0) { if (int st = umma_prepare(ctx)) return st; }
     if (int st = make_map_nhwc(ctx, &mapA, act8, B, H, W, C_in, (int)W, TH, TB)) return st;
     if (int st = make_map(ctx, &mapB, W8, C_out, 9 * C_in, 9 * C_in, pairs > 0 ? bn / 2 : bn)) return st;
     UmmaArgs a{};
+    a.wait_ns = ctx->wait_limit_ns; a.drop_loads = ctx->drop_loads;
     a.M = B * H * W; a.N = C_out;
     a.k_iters = (int)(9 * (C_in / BK));
     a.k_last = BK / 32;
@@ -1337,11 +1356,12 @@ int bnn_umma_conv_f4(bnn_ctx *ctx, const uint8_t *act4, const uint8_t *W4, int64
     CUtensorMap mapA, mapB;
     // CTA pairs (each CTA its own 128 pixels and half of the tile's filters) cut the operand bytes per CTA by 30 %, but
     // measured slower on the ConvNet's layers (0.162 against 0.158 ms per batch of 256): on request only
-    const int pairs = (ctx->pair_mode == 2 && B * H * W >= 512) ? umma2_max_pairs<192>(ctx) : 0;
+    const int pairs = (ctx->pair_mode == 2 && B * H * W >= 512 && !ctx->drop_loads) ? umma2_max_pairs<192>(ctx) : 0;
     if (pairs > 0) { if (int st = umma_prepare(ctx)) return st; }
     if (int st = make_map_nhwc(ctx, &mapA, act4, B, H, W, C_in / 2, (int)W, TH, TB)) return st;
     if (int st = make_map(ctx, &mapB, W4, C_out, 9 * C_in / 2, 9 * C_in / 2, pairs > 0 ? 96 : 192)) return st;
     UmmaArgs a{};
+    a.wait_ns = ctx->wait_limit_ns; a.drop_loads = ctx->drop_loads;
     a.M = B * H * W; a.N = C_out;
     a.c_chunks = (int)(C_in / (2 * BK));
     a.k_iters = 9 * a.c_chunks;
@@ -1363,10 +1383,14 @@ int bnn_umma_conv_f4(bnn_ctx *ctx, const uint8_t *act4, const uint8_t *W4, int64
 extern "C" int64_t bnn_expanded_ld(int64_t K) { return K > 0 ? bnn_umma_operand_ld(K) : 0; }
 extern "C" size_t bnn_expanded_bytes(int64_t rows, int64_t K) { return (rows > 0 && K > 0) ? bnn_umma_operand_bytes(rows, K) : 0; }
 extern "C" int bnn_expand_signs(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t rows, int64_t K, int8_t *dst) {
-    if (!ctx || rows < 0 || K < 0) return BNN_ERR_INVALID_ARG;
+    if (rows < 0 || K < 0) return BNN_ERR_INVALID_ARG;
+    if (rows > 0 && K > 0) {   // the layout first: its errors need no context to be found
+        if (!src || !dst) return BNN_ERR_INVALID_ARG;
+        if (int st = bnn_check_packed(src, ld_w, K, rows)) return st;      // the kernels read the rows with 64- and 128-bit loads
+        if (!bnn_aligned16(dst)) return BNN_ERR_ALIGNMENT;
+    }
+    if (!ctx) return BNN_ERR_INVALID_ARG;
     if (rows == 0 || K == 0) return BNN_OK;
-    if (!src || !dst || ld_w < bnn_words(K)) return BNN_ERR_INVALID_ARG;
-    if (!bnn_aligned16(dst)) return BNN_ERR_ALIGNMENT;
     bnn_device_guard guard(ctx);
     if (!guard.ok) return BNN_ERR_CUDA;
     return bnn_umma_expand(ctx, src, ld_w, rows, K, dst);
@@ -1375,10 +1399,14 @@ extern "C" int bnn_expand_signs(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w,
 extern "C" int64_t bnn_expanded_ld_f4(int64_t K) { return K > 0 ? bnn_umma_operand_ld_f4(K) : 0; }
 extern "C" size_t bnn_expanded_bytes_f4(int64_t rows, int64_t K) { return (rows > 0 && K > 0) ? bnn_umma_operand_bytes_f4(rows, K) : 0; }
 extern "C" int bnn_expand_signs_f4(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w, int64_t rows, int64_t K, uint8_t *dst) {
-    if (!ctx || rows < 0 || K < 0) return BNN_ERR_INVALID_ARG;
+    if (rows < 0 || K < 0) return BNN_ERR_INVALID_ARG;
+    if (rows > 0 && K > 0) {
+        if (!src || !dst) return BNN_ERR_INVALID_ARG;
+        if (int st = bnn_check_packed(src, ld_w, K, rows)) return st;
+        if (!bnn_aligned16(dst)) return BNN_ERR_ALIGNMENT;
+    }
+    if (!ctx) return BNN_ERR_INVALID_ARG;
     if (rows == 0 || K == 0) return BNN_OK;
-    if (!src || !dst || ld_w < bnn_words(K)) return BNN_ERR_INVALID_ARG;
-    if (!bnn_aligned16(dst)) return BNN_ERR_ALIGNMENT;
     bnn_device_guard guard(ctx);
     if (!guard.ok) return BNN_ERR_CUDA;
     return bnn_umma_expand_f4(ctx, src, ld_w, rows, K, dst);

@@ -36,8 +36,8 @@ def test_library_exports_every_declared_function(lib):
 
 def test_status_strings(lib):
     assert lib.bnn_status_string(0) == b"ok"
-    seen = {lib.bnn_status_string(s) for s in range(-5, 1)}
-    assert len(seen) == 6
+    seen = {lib.bnn_status_string(s) for s in range(-6, 1)}
+    assert len(seen) == 7
 
 
 def test_host_argument_errors_need_no_gpu(lib):
@@ -47,6 +47,46 @@ def test_host_argument_errors_need_no_gpu(lib):
     assert lib.bnn_xnor_gemm(None, None, 0, None, 0, None, 0, 1, 1, 1) == -1
     assert lib.bnn_fold_batchnorm(None, None, None, None, 0.0, 4, 10, None, None) == -1
     assert lib.bnn_fold_batchnorm(None, None, None, None, 0.0, 0, 10, None, None) == 0
+
+
+def _fake_mlp_desc(ldw_first=28, ptr=0x1000, wp_first=None):
+    """A two-layer descriptor whose pointers are never dereferenced (every call below fails, or only sizes things)."""
+    arr = (binding.LayerDesc * 2)()
+    arr[0].Wp, arr[0].ldw_w, arr[0].K, arr[0].N, arr[0].thr = (wp_first or ptr), ldw_first, 784, 256, ptr
+    arr[1].Wp, arr[1].ldw_w, arr[1].K, arr[1].N = ptr, 8, 256, 10
+    arr[1].gamma = arr[1].beta = arr[1].mean = arr[1].var = ptr
+    return binding.MlpDesc(2, arr), arr
+
+
+def test_mlp_descriptor_layout_errors_need_no_gpu(lib):
+    """A packed weight matrix with an odd or too small leading dimension, or a misaligned base, is refused by every MLP
+    entry point before anything could be launched (the kernels read the rows with 128-bit loads)."""
+    import ctypes
+    good, keep = _fake_mlp_desc()
+    assert lib.bnn_mlp_workspace_bytes(ctypes.byref(good), 100, 0) > 0
+    calls = (lambda d: lib.bnn_mlp_forward(None, ctypes.byref(d), None, 784, 100, None, 10, None),
+             lambda d: lib.bnn_mlp_forward_host(None, ctypes.byref(d), None, 784, 100, None, 10),
+             lambda d: lib.bnn_mlp_forward_noalloc(None, ctypes.byref(d), None, 784, 100, None, 10))
+    for bad_kwargs, status in (({"ldw_first": 25}, -2), ({"ldw_first": 27}, -2), ({"ldw_first": 24}, -1),
+                               ({"wp_first": 0x1004}, -2)):
+        bad, keep2 = _fake_mlp_desc(**bad_kwargs)
+        assert lib.bnn_mlp_workspace_bytes(ctypes.byref(bad), 100, 0) == 0
+        for call in calls:
+            assert call(bad) == status
+    for call in calls:
+        assert call(good) == -1              # a sound descriptor gets as far as the missing context
+
+
+def test_expand_layout_errors_need_no_gpu(lib):
+    """bnn_expand_signs / _f4 read the packed source with 64- and 128-bit loads: the packed-matrix rule is enforced."""
+    for fn in (lib.bnn_expand_signs, lib.bnn_expand_signs_f4):
+        assert fn(None, 0x1000, 5, 8, 130, 0x2000) == -2      # odd leading dimension
+        assert fn(None, 0x1000, 6, 8, 130, 0x2000) == -2      # not a multiple of 4 words
+        assert fn(None, 0x1004, 8, 8, 130, 0x2000) == -2      # source only 4-byte aligned
+        assert fn(None, 0x1000, 4, 8, 130, 0x2000) == -1      # leading dimension below ceil(K / 32)
+        assert fn(None, 0x1000, 8, 8, 130, 0x2008) == -2      # destination not 16-byte aligned
+        assert fn(None, 0x1000, 8, 8, 130, 0x2000) == -1      # sound layout: stops at the missing context
+        assert fn(None, None, 0, 0, 130, None) == -1          # empty problem, still no context
 
 
 def _fold_matches_oracle(bn, x_max):

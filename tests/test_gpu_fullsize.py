@@ -227,3 +227,94 @@ def test_convnet_half_width_variant_with_dense_tail(ctx):
     got = oracle.batchnorm(S.cpu().numpy(), bn2)                        # integer sums from the GPU, float epilogue on the host
     assert np.array_equal(S.cpu().numpy(), oracle.gemm(h1, W2))
     assert np.allclose(got, want_scores, rtol=0, atol=0)
+
+
+# ------------------------------------------------------------------ the other literal readings of the two network configurations
+def test_mlp_other_reading_four_wide_layers(ctx):
+    """The MLP configuration can also be read as "a first layer, THEN three more binary layers of 4096 units": weights
+    784x4096, three times 4096x4096, 4096x10 (one 4096x4096 layer more than the paper's topology, Section 2.1).  The layer
+    list is data: same calls, every hidden layer against the oracle."""
+    case = wl.mlp_case(batch=2500, sizes=(784, 4096, 4096, 4096, 4096, 10), seed=21)
+    want_scores, want_hidden = oracle.mlp_forward(case["X"], case["weights"], case["bns"])
+    net = nets.prepare_mlp(ctx, case["weights"], case["bns"])
+    batch, sizes = case["batch"], case["sizes"]
+    ws = torch.empty(ctx.mlp_workspace_bytes(net["desc"], batch, False), dtype=torch.uint8, device="cuda")
+    ctx.set_workspace(ws)
+    hidden = [torch.empty(batch, binding.packed_ld(n), dtype=torch.int32, device="cuda") for n in sizes[1:-1]]
+    scores = ctx.mlp_forward(net["desc"], torch.from_numpy(case["X"]).cuda(), batch, hidden_out=hidden)
+    ctx.device_status()
+    assert len(hidden) == 4
+    for k, (g, w) in enumerate(zip(hidden, want_hidden)):
+        assert np.array_equal(np_unpack_pm1(g.cpu().numpy(), w.shape[1]), w), f"hidden layer {k}"
+    got = scores.cpu().numpy().astype(np.float64)
+    assert (np.abs(got - want_scores) <= 1e-5 * np.abs(want_scores) + 1e-6 * np.abs(want_scores).max()).all()
+    assert np.array_equal(got.argmax(1), want_scores.argmax(1))
+    ctx.set_workspace(None)
+
+
+def other_reading_convnet(batch, seed=22):
+    """The ConvNet configuration read as "a first layer, THEN binary convolutions of widths 128-128-256-256-512-512":
+    seven convolutions, the 8-bit one followed by six binary ones (one 128 -> 128 convolution more than the paper's
+    topology), a 2x2 max-pool after every second binary one."""
+    case = wl.convnet_case(batch=batch, channels=(128, 128, 128, 256, 256, 512, 512), seed=seed)
+    for i, L in enumerate(case["layers"]):
+        L["pool"] = i in (2, 4, 6)
+    return case
+
+
+def test_convnet_other_reading_seven_convolutions(ctx):
+    B = 16
+    case = other_reading_convnet(B)
+    want_maps = oracle.convnet_forward(case["X"], case["layers"])
+    assert want_maps[-1].shape == (B, 4, 4, 512)
+    net = nets.prepare_convnet(ctx, case["layers"])
+    desc, keep = ctx.make_convnet_desc(net)
+    ws = torch.empty(max(ctx.convnet_workspace_bytes(desc, B, 32, 32), 256), dtype=torch.uint8, device="cuda")
+    ctx.set_workspace(ws)
+    outs = [torch.empty(w.shape[0], w.shape[1], w.shape[2], binding.words(w.shape[3]), dtype=torch.int32, device="cuda")
+            for w in want_maps]
+    final = torch.empty_like(outs[-1])
+    ctx.convnet_forward(desc, torch.from_numpy(case["X"]).cuda(), B, 32, 32, final, layer_out=outs)
+    ctx.device_status()
+    for k, (g, w) in enumerate(zip(outs, want_maps)):
+        assert np.array_equal(np_unpack_pm1(g.cpu().numpy(), w.shape[-1]), w), f"conv layer {k}"
+    assert torch.equal(final, outs[-1])
+    ctx.set_workspace(None)
+
+
+def test_full_width_convnet_with_dense_tail(ctx):
+    """Sections 2.3-2.4: the CIFAR-10 ConvNet ends in fully-connected binary layers.  The full-width convolution stack
+    (128-128-256-256-512-512) followed by 8192 -> 1024 -> 1024 -> 10 on the flattened 4 x 4 x 512 map: the packed NHWC map
+    of one image is already a packed row of 8192 bits, so the tail is two fused dense calls and one plain product."""
+    B = 24
+    case = wl.convnet_case(batch=B, seed=23)
+    want_maps = oracle.convnet_forward(case["X"], case["layers"])
+    net = nets.prepare_convnet(ctx, case["layers"])
+    desc, keep = ctx.make_convnet_desc(net)
+    ws = torch.empty(max(ctx.convnet_workspace_bytes(desc, B, 32, 32), 256), dtype=torch.uint8, device="cuda")
+    ctx.set_workspace(ws)
+    final = torch.empty(B, 4, 4, 16, dtype=torch.int32, device="cuda")
+    ctx.convnet_forward(desc, torch.from_numpy(case["X"]).cuda(), B, 32, 32, final)
+    ctx.device_status()
+    assert np.array_equal(np_unpack_pm1(final.cpu().numpy(), 512), want_maps[-1])
+    rng = np.random.default_rng(24)
+    K = 4 * 4 * 512
+    W1, W2, W3 = wl.pm1(rng, (K, 1024)), wl.pm1(rng, (1024, 1024)), wl.pm1(rng, (1024, 10))
+    bn1, bn2, bn3 = wl.batchnorm_params(rng, 1024, K), wl.batchnorm_params(rng, 1024, 1024), wl.batchnorm_params(rng, 10, 1024)
+    flat = want_maps[-1].reshape(B, K)                                  # NHWC flattening = (y, x, c) order
+    h1 = oracle.sign_batchnorm(oracle.gemm(flat, W1), bn1)
+    h2 = oracle.sign_batchnorm(oracle.gemm(h1, W2), bn2)
+    want_sums = oracle.gemm(h2, W3)
+    thr1, flip1 = nets.fold(ctx, bn1, K)
+    thr2, flip2 = nets.fold(ctx, bn2, 1024)
+    W1p, W2p, W3p = (nets.pack_weight(ctx, W) for W in (W1, W2, W3))
+    ctx.set_workspace(None)
+    a1 = ctx.binary_dense(final.reshape(B, K // 32), W1p, thr1, flip1, B, 1024, K)
+    a2 = ctx.binary_dense(a1, W2p, thr2, flip2, B, 1024, 1024)
+    S = ctx.xnor_gemm(a2, W3p, B, 10, 1024)
+    ctx.device_status()
+    assert np.array_equal(np_unpack_pm1(a1.cpu().numpy(), 1024), h1)
+    assert np.array_equal(np_unpack_pm1(a2.cpu().numpy(), 1024), h2)
+    assert np.array_equal(S.cpu().numpy(), want_sums)
+    got = oracle.batchnorm(S.cpu().numpy(), bn3)                        # integer sums from the GPU; the affine is the oracle's
+    assert np.array_equal(got.argmax(1), oracle.batchnorm(want_sums, bn3).argmax(1))
