@@ -121,6 +121,12 @@ BNN_API int bnn_expand_signs_f4(bnn_ctx *ctx, const uint32_t *src, int64_t ld_w,
 BNN_API int bnn_binary_dense_expanded(bnn_ctx *ctx, const void *A_exp, int64_t lda_bytes, const void *W_exp, int64_t ldw_bytes,
                                       int operand_bits, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits,
                                       int64_t ldo_w, void *out_exp, int64_t ldo_exp, int64_t M, int64_t N, int64_t K);
+/* Tensor-core engine only: how a 3x3 convolution brings its input into shared memory.  0 (default) = halo tiles: per
+ * tile and horizontal tap one slab of TH + 2 image rows, read at three row offsets for the three vertical taps (a
+ * third of the input traffic; the tile's weights stay resident where they fit); 1 = one 128-pixel operand box per tap.
+ * Geometries the halo form does not cover (tile rows that are not whole 1024-byte groups) use form 1 either way.
+ * Results are identical. */
+BNN_API int bnn_set_conv_form(bnn_ctx *ctx, int form);
 /* Tensor-core engine only: every wait of its kernels on a barrier (operands arrived, stage free, accumulator ready) is
  * bounded.  A wait that lasts longer than `ns` nanoseconds of wall clock (default 2 s; 1 .. 60 s) gives up: the kernel
  * records a code, skips the rest of its work, frees its tensor memory and ends normally, and the other waiters of the

@@ -29,7 +29,7 @@ EXPORTS = (
     "bnn_expanded_bytes", "bnn_expand_signs", "bnn_baseline_gemm_f32", "bnn_convnet_workspace_bytes",
     "bnn_convnet_forward", "bnn_set_operand_bits", "bnn_expanded_ld_f4",
     "bnn_expanded_bytes_f4", "bnn_expand_signs_f4", "bnn_binary_dense_expanded", "bnn_set_wait_limit_ns",
-    "bnn_debug_drop_loads",
+    "bnn_debug_drop_loads", "bnn_set_conv_form",
 )
 
 
@@ -87,6 +87,7 @@ def lib() -> ctypes.CDLL:
         L.bnn_set_operand_bits.argtypes = [vp, c_int]
         L.bnn_set_wait_limit_ns.argtypes = [vp, ctypes.c_uint64]
         L.bnn_debug_drop_loads.argtypes = [vp, c_int]
+        L.bnn_set_conv_form.argtypes = [vp, c_int]
         L.bnn_expanded_ld_f4.argtypes = [i64]
         L.bnn_expanded_ld_f4.restype = i64
         L.bnn_expanded_bytes_f4.argtypes = [i64, i64]
@@ -228,6 +229,9 @@ class Context:
 
     def debug_drop_loads(self, on: bool):
         self._ck(lib().bnn_debug_drop_loads(self._h, int(on)), "bnn_debug_drop_loads")
+
+    def set_conv_form(self, form: int):
+        self._ck(lib().bnn_set_conv_form(self._h, form), "bnn_set_conv_form")
 
     def set_pair_mode(self, mode: int):
         self._ck(lib().bnn_set_pair_mode(self._h, mode), "bnn_set_pair_mode")

@@ -23,6 +23,7 @@ extern "C" int bnn_create(bnn_ctx **out, int device, void *cuda_stream) {
     c->operand_bits = 4;
     c->wait_limit_ns = 2000000000ull;
     c->drop_loads = 0;
+    c->conv_form = 0;
     c->copy_stream = nullptr;
     c->copy_ready = false;
     for (int i = 0; i < 8; ++i) c->ev[i] = nullptr;
@@ -88,6 +89,12 @@ extern "C" int bnn_set_operand_bits(bnn_ctx *ctx, int bits) {
 extern "C" int bnn_set_wait_limit_ns(bnn_ctx *ctx, uint64_t ns) {
     if (!ctx || ns == 0 || ns > 60000000000ull) return BNN_ERR_INVALID_ARG;
     ctx->wait_limit_ns = ns;
+    return BNN_OK;
+}
+
+extern "C" int bnn_set_conv_form(bnn_ctx *ctx, int form) {
+    if (!ctx || (form != 0 && form != 1)) return BNN_ERR_INVALID_ARG;
+    ctx->conv_form = form;
     return BNN_OK;
 }
 

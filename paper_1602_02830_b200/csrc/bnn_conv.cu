@@ -302,7 +302,7 @@ extern "C" int bnn_convnet_forward(bnn_ctx *ctx, const bnn_convnet_desc *net, co
                 W4 = w4_scratch;
             }
             st = bnn_umma_conv_f4(ctx, reinterpret_cast<const uint8_t *>(cur8), W4, B, h, w, D.C_in, D.C_out, D.pool, D.thr, D.flip, dst,
-                                  reinterpret_cast<uint8_t *>(dst8), ldo8);
+                                  reinterpret_cast<uint8_t *>(dst8), ldo8, nullptr, D.W4 ? 1 : 0);
         } else {
             const int8_t *W8 = D.W8;
             if (!W8) {
@@ -315,7 +315,7 @@ extern "C" int bnn_convnet_forward(bnn_ctx *ctx, const bnn_convnet_desc *net, co
                 st = bnn_umma_gemm(ctx, im2col, 32, true, W8, bnn_umma_operand_ld(9 * D.C_in), B * h * w, D.C_out, 9 * D.C_in, nullptr, 0,
                                    D.thr, D.flip, dst, (D.C_out + 31) / 32, dst8, ldo8, D.pool, h, w, next_f4);
             } else {
-                st = bnn_umma_conv(ctx, cur8, W8, B, h, w, D.C_in, D.C_out, D.pool, D.thr, D.flip, dst, nullptr, dst8, ldo8, next_f4);
+                st = bnn_umma_conv(ctx, cur8, W8, B, h, w, D.C_in, D.C_out, D.pool, D.thr, D.flip, dst, nullptr, dst8, ldo8, next_f4, D.W8 ? 1 : 0);
             }
         }
         if (st) return st;

@@ -64,8 +64,16 @@ template <int BN> struct Cfg {
     static constexpr uint32_t TMEM_COLS = is_f4(BN) ? 512 : 2 * BN;
 };
 constexpr int STAGES_MAX = 7;
+constexpr int B_STAGES_MAX = 18;                // weight stages of the halo-tile convolution kernel (9 taps x 2 channel slices resident)
 
 __device__ int g_umma_error;                    // 0 = fine; otherwise a code saying which wait gave up
+#ifdef BNN_TRACE
+// Instrumented builds only: clock stamps of CTA 0, [role][tile][slot].
+__device__ long long g_trace[8 * 16 * 16];
+#define BNN_TR(role, tile, slot) do { if (blockIdx.x == 0 && (tile) < 16) g_trace[((role) * 16 + (tile)) * 16 + (slot)] = clock64(); } while (0)
+#else
+#define BNN_TR(role, tile, slot) do { } while (0)
+#endif
 
 struct UmmaArgs {
     int64_t M, N;
@@ -83,6 +91,13 @@ struct UmmaArgs {
     int c_chunks;           // C_in / 128
     int pool;               // 2x2 max-pool (as OR of the sign bits) before the packed store
     int b_static;           // B (weights) is not written by the kernel launched just before this one
+    // halo-tile convolution kernel (k_umma_conv): A stages hold a (TH + 2)-row slab of the input per horizontal tap
+    int a_stage_bytes, n_a_stages;   // bytes of one slab = (TH + 2) * TB * W * 128; slabs in the ring
+    int n_b_stages;         // weight stages of BN x 128 bytes
+    int b_resident;         // all k_iters weight stages stay in shared memory (this CTA's tiles share their filters)
+    int dy_bytes;           // one image row of the slab: TB * W * 128 bytes
+    int tap_bytes;          // bytes of one tap in a filter row of the weight matrix (C_in bytes, or C_in / 2 for nibbles)
+    int perm;               // rows of a tile are ordered (y, image, x) instead of (image, y, x)  (TB > 1)
     unsigned long long wait_ns;   // how long a wait on a barrier may last before the kernel gives up
     int drop_loads;         // test hook (single-SM kernel): the producer issues no loads, every consumer's wait runs out
 };
@@ -165,6 +180,8 @@ struct __align__(16) Control {
     uint64_t acc_full[ACC_BUFS];
     uint64_t acc_empty[ACC_BUFS];
     uint64_t started[ACC_BUFS];            // the tile's first (overwriting) K step has completed
+    uint64_t full_b[B_STAGES_MAX];         // k_umma_conv: its weight ring (full / empty above are its slab ring)
+    uint64_t empty_b[B_STAGES_MAX];
     uint32_t tmem_base;
     uint32_t failed;
     __align__(16) int32_t thr[ACC_BUFS][BN_MAX];   // staged thresholds: clamped int32, or float bits on the 4-bit engine
@@ -268,9 +285,9 @@ __device__ __forceinline__ void store_signs(const UmmaArgs &p, uint32_t word, in
 }
 
 // One 32-column chunk of accumulators (r, one output row per thread) -> the requested outputs.
-template <int BN>
+template <int BN, bool F4 = is_f4(BN)>
 __device__ __forceinline__ void epilogue_chunk(Control *ctl, const UmmaArgs &p, uint32_t (&r)[32], uint32_t buf, int c, int64_t col0,
-                                               int64_t row, int q, int lane, int role = 0, uint4 *hold = nullptr) {
+                                               int64_t row, int lin, int role = 0, uint4 *hold = nullptr) {
     if (row >= p.M) return;
     if (p.thr) {                                         // thresholded signs: packed words and/or the next layer's operand
         // bit j of the word = (acc[j] >= thr[j]) = NOT sign(acc[j] - thr[j]); the sign bits are shifted
@@ -284,7 +301,7 @@ __device__ __forceinline__ void epilogue_chunk(Control *ctl, const UmmaArgs &p, 
 #pragma unroll
             for (int i = 3; i >= 0; --i) {
                 const int j = 4 * g + i;
-                const uint32_t d = is_f4(BN) ? __float_as_uint(__uint_as_float(r[j]) - __int_as_float(tv[i]))
+                const uint32_t d = F4 ? __float_as_uint(__uint_as_float(r[j]) - __int_as_float(tv[i]))
                                                : (uint32_t)((int32_t)r[j] - tv[i]);
                 w4[j >> 3] = __funnelshift_l(d, w4[j >> 3], 1);
             }
@@ -292,12 +309,12 @@ __device__ __forceinline__ void epilogue_chunk(Control *ctl, const UmmaArgs &p, 
         const uint32_t lt = __byte_perm(__byte_perm(w4[0], w4[1], 0x0040), __byte_perm(w4[2], w4[3], 0x0040), 0x5410);
         uint32_t word = ~lt ^ ctl->flip[buf][c];
         if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;      // columns beyond N stay 0
-        if (p.pool) ctl->poolw[32 * q + lane][c] = word ^ ctl->flip[buf][c];   // un-flipped (dot >= thr) bits
+        if (p.pool) ctl->poolw[lin][c] = word ^ ctl->flip[buf][c];   // un-flipped (dot >= thr) bits
         else if (p.out) p.out[row * p.ldo + (col0 >> 5)] = word;
         if (p.out8 && !p.pool) store_signs(p, word, row, col0, role, hold);
     }
     if (p.C) {
-        if (is_f4(BN)) {   // the 4-bit engine accumulates in float32: exact integers
+        if (F4) {   // the 4-bit engine accumulates in float32: exact integers
             if (p.k_iters <= (1 << 14)) {
                 // |sum| <= K <= 2^22: adding 1.5 * 2^23 leaves the integer in the low mantissa bits (an add and a
                 // subtract on the full-rate pipes instead of a quarter-rate conversion)
@@ -333,30 +350,42 @@ __device__ __forceinline__ void epilogue_chunk(Control *ctl, const UmmaArgs &p, 
 // buffer `buf`, and turn them into the requested outputs.  `ok` turns false once a wait has given up.
 // The staged form of a threshold.  The comparison is the sign of (accumulator - threshold); accumulators stay below 2^30
 // in magnitude (2^24 on the 4-bit engine, where they are float32), so thresholds clamp to that range unchanged in meaning.
-template <int BN>
+template <bool F4>
 __device__ __forceinline__ int32_t staged_threshold(int32_t t) {
-    if (is_f4(BN)) return __float_as_int(t > (1 << 24) ? 3.0e7f : (t < -(1 << 24) ? -3.0e7f : (float)t));
+    if (F4) return __float_as_int(t > (1 << 24) ? 3.0e7f : (t < -(1 << 24) ? -3.0e7f : (float)t));
     return max(min(t, 1 << 30), -(1 << 30));
 }
 
 // n0_next: first column of the tile this CTA handles next (-1: none).  Its thresholds are fetched from global memory
 // while this tile is processed and staged for the other buffer at the end, so no tile but the first waits for them.
-template <int BN>
+// Row i of a convolution tile -> the pixel's position in (image, y, x) order inside the tile.  The halo-tile kernel keeps
+// tiles of several small images in (y, image, x) order, so that one tap's rows are evenly spaced in shared memory.
+__device__ __forceinline__ int tile_lin(const UmmaArgs &p, int i) {
+    if (!p.perm) return i;
+    const int x = i % p.W, b = (i / p.W) % p.TB, y = i / (p.W * p.TB);
+    return (b * p.TH + y) * p.W + x;
+}
+
+template <int BN, bool F4 = is_f4(BN), int EPI_WARPS = Warps<BN>::EPI_WARPS>
 __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, uint32_t tmem_base, uint32_t buf, uint32_t tc,
                                               int64_t m0, int64_t n0, int64_t n0_next, int q, int half, int lane, int et, bool &ok) {
-    constexpr int EPW = Warps<BN>::EPW, EPI_THREADS = Warps<BN>::EPI_THREADS;
+    constexpr int EPW = EPI_WARPS / 4, EPI_THREADS = EPI_WARPS * 32;
     static_assert(BN <= EPI_THREADS, "one staged threshold per epilogue thread");
     constexpr int CHUNKS = BN / 32, CPW = (CHUNKS + 1) / 2;   // 32-column chunks per tile and (at most) per warp with two warps per quadrant
-    const int64_t row = m0 + 32 * q + lane;
+    const int lin = tile_lin(p, 32 * q + lane);
+    const int64_t row = m0 + lin;
     if (p.thr && tc == 0) {                              // the first tile stages its own thresholds
-        if (et < BN) ctl->thr[buf][et] = staged_threshold<BN>((n0 + et < p.N) ? p.thr[n0 + et] : 0x7fffffff);
+        if (et < BN) ctl->thr[buf][et] = staged_threshold<F4>((n0 + et < p.N) ? p.thr[n0 + et] : 0x7fffffff);
         if (et < BN / 32) {
             const int64_t w = (n0 >> 5) + et;
             ctl->flip[buf][et] = (p.flip && w * 32 < p.N) ? p.flip[w] : 0u;
         }
     }
+    const int tr_role = (et == 0) ? 3 : ((et == EPI_THREADS - 32) ? 4 : -1);
+    if (tr_role >= 0) BNN_TR(tr_role, tc, 0);
     // the epilogue warps only: staged thresholds visible; previous tile's pooling words no longer read
     if (p.thr) asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
+    if (tr_role >= 0) BNN_TR(tr_role, tc, 1);
     const bool have_next = p.thr && n0_next >= 0;
     int32_t next_thr = 0x7fffffff;
     uint32_t next_flip = 0u;
@@ -367,10 +396,20 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
             if (p.flip && w * 32 < p.N) next_flip = p.flip[w];
         }
     }
-    if (ok && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->acc_full[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 3); ok = false; }
+    // One warp polls the "accumulator full" barrier; the others park on a hardware barrier until it has seen it.  A
+    // polling warp takes an issue slot on every turn of its loop, and with four of them on each scheduler the two
+    // MMA-issuing threads, which share those schedulers, needed three times as long per instruction: a tile of nine
+    // short K steps then ran at 40 % of the tensor pipe's rate.
+    if (et < 32 && ok && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->acc_full[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 3); ok = false; }
+    asm volatile("bar.sync 2, %0;" ::"n"(EPI_THREADS) : "memory");
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (tr_role >= 0) BNN_TR(tr_role, tc, 2);
     ok = ok && (ctl->failed == 0);
+#ifdef EXP_NO_EPI
+    if (false) {                                         // experiment: the accumulators are never read
+#else
     if (ok) {
+#endif
         const uint32_t tbase = tmem_base + ((uint32_t)(32 * q) << 16) + buf * BN;
         if constexpr (EPW == 2) {
             // two warps per quadrant, each a contiguous half of the columns (the first one chunk more when their number
@@ -388,7 +427,7 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                 uint32_t (&r)[32] = (cc & 1) ? rb : ra;
                 uint32_t (&rn)[32] = (cc & 1) ? ra : rb;
                 if (more) tmem_ld32(tbase + (uint32_t)(32 * (c + 1)), rn);
-                epilogue_chunk<BN>(ctl, p, r, buf, c, col0, row, q, lane);
+                epilogue_chunk<BN, F4>(ctl, p, r, buf, c, col0, row, lin);
                 if (more) tmem_ld_wait(rn);
             }
         } else {
@@ -405,7 +444,7 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                     if (col0 >= p.N) break;                  // uniform over the warp
                     tmem_ld32(tbase + (uint32_t)(32 * c), r);
                     tmem_ld_wait(r);
-                    epilogue_chunk<BN>(ctl, p, r, buf, c, col0, row, q, lane, 1 + i, &hold);
+                    epilogue_chunk<BN, F4>(ctl, p, r, buf, c, col0, row, lin, 1 + i, &hold);
                 }
             } else {
 #pragma unroll 1
@@ -414,7 +453,7 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                     if (col0 >= p.N) break;                  // uniform over the warp
                     tmem_ld32(tbase + (uint32_t)(32 * c), r);
                     tmem_ld_wait(r);
-                    epilogue_chunk<BN>(ctl, p, r, buf, c, col0, row, q, lane);
+                    epilogue_chunk<BN, F4>(ctl, p, r, buf, c, col0, row, lin);
                 }
             }
         }
@@ -423,6 +462,7 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
             for (int64_t w = (p.N + 31) >> 5; w < p.ldo; ++w) p.out[row * p.ldo + w] = 0u;
         }
     }
+    if (tr_role >= 0) BNN_TR(tr_role, tc, 3);
     if (p.pool) {
         // 2x2 max-pool then threshold == OR of the four thresholded bits, then flip.  The tile holds TB images
         // x TH rows x W columns (TH, W even), i.e. 32 whole windows; 256 (window, word) items for 128 threads.
@@ -450,12 +490,14 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
             }
         }
     }
+    if (tr_role >= 0) BNN_TR(tr_role, tc, 4);
     if (have_next) {
         // Every epilogue thread has passed this tile's barrier, so none still reads the other buffer's thresholds (they
         // belonged to the previous tile); the next tile's barrier makes these visible.
-        if (et < BN) ctl->thr[buf ^ 1u][et] = staged_threshold<BN>(next_thr);
+        if (et < BN) ctl->thr[buf ^ 1u][et] = staged_threshold<F4>(next_thr);
         if (et < BN / 32) ctl->flip[buf ^ 1u][et] = next_flip;
     }
+    if (tr_role >= 0) BNN_TR(tr_role, tc, 5);
 }
 
 // Persistent: gridDim.x CTAs (one per SM) walk the tile list with stride gridDim.x.  The shared-memory ring
@@ -888,6 +930,8 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     }
 }
 
+#include "bnn_umma_conv.cuh"
+
 // ---------------------------------------------------------------------------------------------------------
 // Packed signs -> one signed byte per value (+1 = 0x01, -1 = 0xff); bytes at or beyond K are 0.
 // One thread per 32-bit word = 32 output bytes (two 128-bit stores).
@@ -1306,13 +1350,159 @@ bool bnn_umma_conv_tiling(int64_t H, int64_t W, int pool, int *TH, int *TB) {
     return true;
 }
 
+// ---- halo-tile convolution kernel (bnn_umma_conv.cuh): geometry, shared-memory plan and launch
+namespace {
+constexpr size_t SMEM_OPT_IN = 227 * 1024;      // dynamic shared memory a CTA can opt in to on sm_100
+// Activation map with the dimensions ordered (channel byte, column, image, row): a box of {128, W, TB, TH + 2} lands in
+// shared memory as [row][image][column] rows of 128 bytes.  cb = bytes of channels per pixel.
+int make_map_slab(bnn_ctx *ctx, CUtensorMap *map, const void *base, int64_t B, int64_t H, int64_t W, int64_t cb, int TH, int TB) {
+    encode_fn_t enc;
+    if (int st = get_encode(ctx, &enc)) return st;
+    cuuint64_t dims[4] = {(cuuint64_t)cb, (cuuint64_t)W, (cuuint64_t)B, (cuuint64_t)H};
+    cuuint64_t strides[3] = {(cuuint64_t)cb, (cuuint64_t)(H * W * cb), (cuuint64_t)(W * cb)};
+    cuuint32_t box[4] = {(cuuint32_t)BK, (cuuint32_t)W, (cuuint32_t)TB, (cuuint32_t)(TH + 2)};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { ctx->last_cuda_error = (int)r; return BNN_ERR_CUDA; }
+    return BNN_OK;
+}
+// Launch with programmatic stream serialization and, for the pair form, clusters of two CTAs.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_conv_kernel(void (*kernel)(KArgs...), bool pair, dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args &&...args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = pair ? 2 : 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+// Per instantiation and device: opt in to the large shared memory once; for the pair form also ask how many clusters of
+// two can be resident at once (0 = the pair form cannot be used).
+template <int BN, bool F4, bool PAIR>
+int conv_kernel_prepare(bnn_ctx *ctx, int *max_pairs) {
+    static std::mutex m;
+    static bool done[64] = {};
+    static int pairs[64] = {};
+    std::lock_guard<std::mutex> lock(m);
+    if (ctx->device < 0 || ctx->device >= 64) return BNN_ERR_INVALID_ARG;
+    if (!done[ctx->device]) {
+        BNN_CUDA_TRY(ctx, cudaFuncSetAttribute(k_umma_conv<BN, F4, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_OPT_IN));
+        if (PAIR) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(2 * ctx->sm_count, 1, 1);
+            cfg.blockDim = dim3(ConvCfg<BN, F4, PAIR>::NTHREADS, 1, 1);
+            cfg.dynamicSmemBytes = SMEM_OPT_IN;
+            cudaLaunchAttribute attr;
+            attr.id = cudaLaunchAttributeClusterDimension;
+            attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+            cfg.attrs = &attr; cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, k_umma_conv<BN, F4, PAIR>, &cfg) != cudaSuccess) n = 0;
+            (void)cudaGetLastError();
+            pairs[ctx->device] = n;
+        }
+        done[ctx->device] = true;
+    }
+    if (max_pairs) *max_pairs = pairs[ctx->device];
+    return BNN_OK;
+}
+template <int BN, bool F4, bool PAIR>
+int conv_halo_launch_t(bnn_ctx *ctx, const CUtensorMap &mapA, const CUtensorMap &mapB, const UmmaArgs &a, unsigned grid, size_t smem) {
+    BNN_CUDA_TRY(ctx, launch_conv_kernel(k_umma_conv<BN, F4, PAIR>, PAIR, dim3(grid), dim3(ConvCfg<BN, F4, PAIR>::NTHREADS), smem, ctx->stream, mapA, mapB, a));
+    return bnn_check_launch(ctx);
+}
+}  // namespace
+
+// Whether the halo-tile kernel takes this layer: slabs of whole 1024-byte swizzle periods per image row of the tile.
+static bool conv_halo_ok(const bnn_ctx *ctx, int64_t W, int TH, int TB) {
+    if (ctx->conv_form == 1 || ctx->drop_loads) return false;
+    return ((TB * W) % 8) == 0 && W <= 256 && TB <= 256 && TH + 2 <= 256 && (size_t)(TH + 2) * TB * W * BK <= 48 * 1024;
+}
+
+// act: [B][H][W][cb] bytes (cb = C_in bytes, or C_in / 2 for nibbles; a multiple of 128), Wt: [C_out][9 * cb].  `a` arrives
+// with the outputs, thresholds, pooling and tile geometry filled in.
+static int conv_halo_launch(bnn_ctx *ctx, bool f4, const void *act, const void *Wt, int64_t B, int64_t H, int64_t W, int64_t cb,
+                            int64_t C_out, int TH, int TB, UmmaArgs a, int b_static) {
+    const int c_chunks = (int)(cb / BK);
+    const size_t a_stage = (size_t)(TH + 2) * TB * W * BK;
+    const size_t avail = SMEM_OPT_IN - 1024 - sizeof(Control);
+    // 1. CTA pairs with the tile's filters resident, half of them in each CTA: 256 filters per tile on bytes, 128 on nibbles
+    //    (two accumulator buffers and the scale columns must fit the 512 columns of tensor memory).
+    bool pair = false, resident = false;
+    int bn = 128, nb = 0, max_pairs = 0;
+    if (ctx->pair_mode != 1 && a.M > BM) {
+        bn = f4 ? 128 : (C_out > 128 ? 256 : 128);
+        nb = 9 * c_chunks;
+        int st = BNN_OK;
+        if (f4) st = conv_kernel_prepare<128, true, true>(ctx, &max_pairs);
+        else if (bn == 256) st = conv_kernel_prepare<256, false, true>(ctx, &max_pairs);
+        else st = conv_kernel_prepare<128, false, true>(ctx, &max_pairs);
+        if (st) return st;
+        const int64_t tn = (C_out + bn - 1) / bn;
+        pair = resident = max_pairs > 0 && nb <= B_STAGES_MAX && (size_t)nb * (bn / 2) * BK + 2 * a_stage <= avail && tn <= max_pairs;
+    }
+    // 2. otherwise one CTA per tile: resident weights where 128 filters fit, else streamed through a ring
+    if (!pair) {
+        bn = 128;
+        resident = c_chunks == 1 && 9 * (size_t)128 * BK + 2 * a_stage <= avail && (C_out + 127) / 128 <= ctx->sm_count;
+        if (!resident && C_out > 128) bn = f4 ? 192 : 256;
+        nb = resident ? 9 : 4;
+        int st = BNN_OK;
+        if (f4) st = bn == 128 ? conv_kernel_prepare<128, true, false>(ctx, nullptr) : conv_kernel_prepare<192, true, false>(ctx, nullptr);
+        else st = bn == 128 ? conv_kernel_prepare<128, false, false>(ctx, nullptr) : conv_kernel_prepare<256, false, false>(ctx, nullptr);
+        if (st) return st;
+    }
+    const size_t b_stage = (size_t)(pair ? bn / 2 : bn) * BK, b_bytes = (size_t)nb * b_stage;
+    int na = (int)((avail - b_bytes) / a_stage);
+    na = na > 4 ? 4 : na;
+    if (na < 2) return BNN_ERR_INVALID_ARG;
+    CUtensorMap mapA, mapB;
+    if (int st = make_map_slab(ctx, &mapA, act, B, H, W, cb, TH, TB)) return st;
+    if (int st = make_map(ctx, &mapB, Wt, C_out, 9 * cb, 9 * cb, (int)(b_stage / BK))) return st;
+    a.conv = 1; a.H = (int)H; a.W = (int)W; a.TH = TH; a.TB = TB; a.c_chunks = c_chunks;
+    a.k_iters = 9 * c_chunks; a.k_last = BK / 32;
+    a.a_stage_bytes = (int)a_stage; a.n_a_stages = na; a.n_b_stages = nb; a.b_resident = resident ? 1 : 0;
+    a.dy_bytes = (int)(TB * W * BK); a.tap_bytes = (int)cb; a.perm = TB > 1 ? 1 : 0; a.b_static = b_static;
+    const int64_t tn = (C_out + bn - 1) / bn;
+    const int64_t tile_m = pair ? 2 * BM : BM, tiles = ((a.M + tile_m - 1) / tile_m) * tn;
+    if (tiles >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;
+    const int64_t units_max = pair ? max_pairs : ctx->sm_count;
+    int64_t units = tiles < units_max ? tiles : units_max;
+    if (resident && tiles > units) units = (units_max / tn) * tn;       // a multiple of the filter blocks: one block per CTA (pair)
+    const unsigned grid = (unsigned)(pair ? 2 * units : units);
+    const size_t smem = (size_t)na * a_stage + b_bytes + sizeof(Control) + 1024;
+    if (pair) {
+        if (f4) return conv_halo_launch_t<128, true, true>(ctx, mapA, mapB, a, grid, smem);
+        return bn == 256 ? conv_halo_launch_t<256, false, true>(ctx, mapA, mapB, a, grid, smem)
+                         : conv_halo_launch_t<128, false, true>(ctx, mapA, mapB, a, grid, smem);
+    }
+    if (f4) return bn == 128 ? conv_halo_launch_t<128, true, false>(ctx, mapA, mapB, a, grid, smem)
+                             : conv_halo_launch_t<192, true, false>(ctx, mapA, mapB, a, grid, smem);
+    return bn == 128 ? conv_halo_launch_t<128, false, false>(ctx, mapA, mapB, a, grid, smem)
+                     : conv_halo_launch_t<256, false, false>(ctx, mapA, mapB, a, grid, smem);
+}
+
 // 3x3 / pad 1 convolution on the tensor engine.  act8: [B][H][W][C_in] +-1 bytes (C_in % 128 == 0);
 // W8: [C_out][9 * C_in] +-1 bytes.  Outputs as bnn_binary_conv2d (sums only without pooling).
 int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B, int64_t H, int64_t W, int64_t C_in,
                   int64_t C_out, int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, int32_t *out_sums,
-                  int8_t *out8, int64_t ldo8, int out_f4) {
+                  int8_t *out8, int64_t ldo8, int out_f4, int b_static) {
     int TH, TB;
     if (!bnn_umma_conv_tiling(H, W, pool, &TH, &TB) || (C_in % BK) != 0 || (pool && (out_sums || !out_bits))) return BNN_ERR_INVALID_ARG;
+    if (conv_halo_ok(ctx, W, TH, TB)) {
+        UmmaArgs h{};
+        h.wait_ns = ctx->wait_limit_ns;
+        h.M = B * H * W; h.N = C_out;
+        h.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BM >> 4) << 24);
+        h.C = out_sums; h.ldc = C_out; h.out = out_bits; h.ldo = (C_out + 31) / 32; h.thr = thr; h.flip = flip;
+        h.out8 = out8; h.ldo8 = ldo8; h.out_f4 = out_f4; h.pool = pool;
+        return conv_halo_launch(ctx, false, act8, W8, B, H, W, C_in, C_out, TH, TB, h, b_static);
+    }
     CUtensorMap mapA, mapB;
     const int bn = umma_tile_n(C_out);
     // CTA pairs (each CTA its own 128 pixels and half of the tile's filters) from 6 M outputs on, as for plain products
@@ -1347,12 +1537,20 @@ int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B,
 // or the int32 sums (not with pooling).
 int bnn_umma_conv_f4(bnn_ctx *ctx, const uint8_t *act4, const uint8_t *W4, int64_t B, int64_t H, int64_t W, int64_t C_in,
                      int64_t C_out, int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, uint8_t *out4,
-                     int64_t ldo4, int32_t *out_sums) {
+                     int64_t ldo4, int32_t *out_sums, int b_static) {
     int TH, TB;
     if (!bnn_umma_conv_tiling(H, W, pool, &TH, &TB) || (C_in % (2 * BK)) != 0 || (pool && (out_sums || !out_bits)) ||
         (!out_bits && !out4 && !out_sums) || ((out_bits || out4) && !thr))
         return BNN_ERR_INVALID_ARG;
     if (!bnn_aligned16(act4) || !bnn_aligned16(W4)) return BNN_ERR_ALIGNMENT;
+    if (conv_halo_ok(ctx, W, TH, TB)) {
+        UmmaArgs h{};
+        h.wait_ns = ctx->wait_limit_ns;
+        h.M = B * H * W; h.N = C_out;
+        h.C = out_sums; h.ldc = C_out; h.out = out_bits; h.ldo = (C_out + 31) / 32; h.thr = thr; h.flip = flip;
+        h.out8 = reinterpret_cast<int8_t *>(out4); h.ldo8 = ldo4; h.out_f4 = 1; h.pool = pool;
+        return conv_halo_launch(ctx, true, act4, W4, B, H, W, C_in / 2, C_out, TH, TB, h, b_static);
+    }
     CUtensorMap mapA, mapB;
     // CTA pairs (each CTA its own 128 pixels and half of the tile's filters) cut the operand bytes per CTA by 30 %, but
     // measured slower on the ConvNet's layers (0.162 against 0.158 ms per batch of 256): on request only
@@ -1414,6 +1612,14 @@ extern "C" int bnn_expand_signs_f4(bnn_ctx *ctx, const uint32_t *src, int64_t ld
 
 // Reads (and clears) the error word the tensor-core kernel sets when one of its bounded waits gives up.
 // Synchronises the context's stream.
+#ifdef BNN_TRACE
+extern "C" BNN_API int bnn_trace_read(long long *host, int clear) {
+    if (cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * 8 * 16 * 16) != cudaSuccess) return BNN_ERR_CUDA;
+    if (clear) { static long long z[8 * 16 * 16]; if (cudaMemcpyToSymbol(g_trace, z, sizeof(z)) != cudaSuccess) return BNN_ERR_CUDA; }
+    return BNN_OK;
+}
+#endif
+
 extern "C" int bnn_device_status(bnn_ctx *ctx) {
     if (!ctx) return BNN_ERR_INVALID_ARG;
     bnn_device_guard guard(ctx);

@@ -188,8 +188,15 @@ def test_mlp_forward_tensor_engine(ctx, host_io, pre_expanded):
 
 @pytest.mark.parametrize("B,H,W,Cin,Cout,pool", [(8, 32, 32, 128, 128, False), (8, 32, 32, 128, 200, True),
                                                  (16, 16, 16, 256, 256, True), (33, 8, 8, 512, 512, True),
-                                                 (35, 8, 8, 256, 300, False), (3, 64, 64, 128, 128, True)])
-def test_binary_conv2d_tensor_engine(ctx, B, H, W, Cin, Cout, pool):
+                                                 (35, 8, 8, 256, 300, False), (3, 64, 64, 128, 128, True),
+                                                 (300, 4, 4, 256, 128, True), (260, 4, 4, 128, 256, False),
+                                                 (5, 16, 16, 512, 200, False), (9, 32, 32, 128, 384, False)])
+@pytest.mark.parametrize("form", [0, 1], ids=["halo-tiles", "box-per-tap"])
+def test_binary_conv2d_tensor_engine(ctx, B, H, W, Cin, Cout, pool, form):
+    """Both ways the tensor engine brings a convolution's input into shared memory (bnn_set_conv_form): halo tiles (one slab
+    per horizontal tap, read at three row offsets; several small images per tile are kept in (row, image, column) order)
+    and one operand box per tap.  Image sizes 64, 32, 16, 8 and 4: one, one, one, two and eight images per 128-pixel tile."""
+    ctx.set_conv_form(form)
     rng = np.random.default_rng(B + H + Cin + Cout)
     act = wl.pm1(rng, (B, H, W, Cin))
     wgt = wl.pm1(rng, (Cout, 3, 3, Cin))
@@ -213,6 +220,7 @@ def test_binary_conv2d_tensor_engine(ctx, B, H, W, Cin, Cout, pool):
     assert np.array_equal(np_unpack_pm1(got, Cout), want)
     assert padding_is_zero(got, Cout)
     ctx.set_workspace(None)
+    ctx.set_conv_form(0)
     del ws
 
 
