@@ -276,6 +276,19 @@ BNN_API int bnn_mlp_forward_host(bnn_ctx *ctx, const bnn_mlp_desc *m, const uint
                          int64_t batch, float *scores_host, int64_t lds);
 
 /* ---------------------------------------------------------------------------------------------
+ * Measurement helper (Section 4 counts the XNOR-popcount step as "1 + 4 + 1" cycles on the GPUs of 2016): the issue rates
+ * of this GPU's integer pipes, in thread-level results per clock and SM, timed in register-only loops on every SM:
+ * POPC alone, LOP3 alone, and the xor / popc / add sequence of Eq. 8 (counted per popcount word).  The popcount roofline
+ * of a benchmark is  SMs x popc rate x 32 bit-MACs x 2 x SM clock.
+ *   scratch: device memory, at least sm_count * 4104 bytes, 8-byte aligned (BNN_ERR_WORKSPACE / BNN_ERR_ALIGNMENT).
+ * Runs on the context's stream and synchronises it; the three results are host doubles. */
+BNN_API int bnn_measure_pipe_rates(bnn_ctx *ctx, void *scratch, size_t scratch_bytes, double *popc_per_clk_per_sm,
+                                   double *lop3_per_clk_per_sm, double *xor_popc_add_per_clk_per_sm);
+/* Name and tile shape of the tensor-core kernel this context launched last ("" if none yet): lets a benchmark label its
+ * numbers with what actually ran.  The string is owned by the context and valid until its next call. */
+BNN_API const char *bnn_last_tensor_kernel(const bnn_ctx *ctx);
+
+/* ---------------------------------------------------------------------------------------------
  * Context only (Section 4, Fig. 3): the paper's comparison point, a deliberately unoptimized matrix product of the
  * +-1 values held as float32 (one thread per output).  A is M x K, B is K x N, C is M x N, all row-major device
  * float32.  Not used by any other call. */

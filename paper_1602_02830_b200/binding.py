@@ -29,7 +29,7 @@ EXPORTS = (
     "bnn_expanded_bytes", "bnn_expand_signs", "bnn_baseline_gemm_f32", "bnn_convnet_workspace_bytes",
     "bnn_convnet_forward", "bnn_set_operand_bits", "bnn_expanded_ld_f4",
     "bnn_expanded_bytes_f4", "bnn_expand_signs_f4", "bnn_binary_dense_expanded", "bnn_set_wait_limit_ns",
-    "bnn_debug_drop_loads", "bnn_set_conv_form",
+    "bnn_debug_drop_loads", "bnn_set_conv_form", "bnn_measure_pipe_rates", "bnn_last_tensor_kernel",
 )
 
 
@@ -88,6 +88,9 @@ def lib() -> ctypes.CDLL:
         L.bnn_set_wait_limit_ns.argtypes = [vp, ctypes.c_uint64]
         L.bnn_debug_drop_loads.argtypes = [vp, c_int]
         L.bnn_set_conv_form.argtypes = [vp, c_int]
+        L.bnn_measure_pipe_rates.argtypes = [vp, vp, c_size_t, POINTER(c_double), POINTER(c_double), POINTER(c_double)]
+        L.bnn_last_tensor_kernel.argtypes = [vp]
+        L.bnn_last_tensor_kernel.restype = ctypes.c_char_p
         L.bnn_expanded_ld_f4.argtypes = [i64]
         L.bnn_expanded_ld_f4.restype = i64
         L.bnn_expanded_bytes_f4.argtypes = [i64, i64]
@@ -229,6 +232,18 @@ class Context:
 
     def debug_drop_loads(self, on: bool):
         self._ck(lib().bnn_debug_drop_loads(self._h, int(on)), "bnn_debug_drop_loads")
+
+    def measure_pipe_rates(self):
+        """bnn_measure_pipe_rates -> dict of thread-level results per clock and SM (popc, lop3, xor+popc+add)."""
+        sms = torch.cuda.get_device_properties(self.device).multi_processor_count
+        scratch = self.empty(sms * 4104, dtype=torch.uint8)
+        a, b, c = c_double(), c_double(), c_double()
+        self._ck(lib().bnn_measure_pipe_rates(self._h, _ptr(scratch), scratch.numel(), ctypes.byref(a), ctypes.byref(b),
+                                              ctypes.byref(c)), "bnn_measure_pipe_rates")
+        return {"popc": a.value, "lop3": b.value, "xor_popc_add": c.value}
+
+    def last_tensor_kernel(self) -> str:
+        return lib().bnn_last_tensor_kernel(self._h).decode()
 
     def set_conv_form(self, form: int):
         self._ck(lib().bnn_set_conv_form(self._h, form), "bnn_set_conv_form")

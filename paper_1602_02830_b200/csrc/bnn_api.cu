@@ -24,6 +24,7 @@ extern "C" int bnn_create(bnn_ctx **out, int device, void *cuda_stream) {
     c->wait_limit_ns = 2000000000ull;
     c->drop_loads = 0;
     c->conv_form = 0;
+    c->last_kernel[0] = 0;
     c->copy_stream = nullptr;
     c->copy_ready = false;
     for (int i = 0; i < 8; ++i) c->ev[i] = nullptr;
@@ -109,6 +110,8 @@ extern "C" int bnn_set_engine(bnn_ctx *ctx, int engine) {
     ctx->engine = engine;
     return BNN_OK;
 }
+
+extern "C" const char *bnn_last_tensor_kernel(const bnn_ctx *ctx) { return ctx ? ctx->last_kernel : ""; }
 
 extern "C" int bnn_last_cuda_error(const bnn_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
 

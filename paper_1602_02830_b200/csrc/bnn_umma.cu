@@ -1162,8 +1162,12 @@ static int umma2_max_pairs(bnn_ctx *ctx) {
     }
     return cached[ctx->device];
 }
+static void note_kernel(bnn_ctx *ctx, const char *name, int bn, const char *operands, const char *extra = "") {
+    snprintf(ctx->last_kernel, sizeof(ctx->last_kernel), "%s<%d> %s%s", name, bn, operands, extra);
+}
 static int umma_launch(bnn_ctx *ctx, const CUtensorMap &mapA, const CUtensorMap &mapB, const UmmaArgs &a, int bn) {
     if (int st = umma_prepare(ctx)) return st;
+    note_kernel(ctx, "k_umma_i8", bn, is_f4(bn) ? "128 x bn tiles, tcgen05 kind::mxf4 on e2m1 nibbles" : "128 x bn tiles, tcgen05 kind::i8 on bytes");
     const int64_t tiles = ((a.M + BM - 1) / BM) * ((a.N + bn - 1) / bn);
     if (tiles >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;      // the kernels count tiles in 32 bits
     const int64_t grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
@@ -1250,6 +1254,7 @@ int bnn_umma_gemm_f4(bnn_ctx *ctx, const uint8_t *A4, int64_t lda4, const uint8_
         const int64_t tiles2 = ((M + 2 * BM - 1) / (2 * BM)) * ((N + bn2 - 1) / bn2);
         if (tiles2 >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;
         const int64_t use = tiles2 < pairs ? tiles2 : pairs;
+        note_kernel(ctx, "k_umma_i8_2sm", bn2, "CTA pairs, 256 x bn tiles, tcgen05 cta_group::2 kind::mxf4 on e2m1 nibbles");
         if (bn2 == 224)
             BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8_2sm<224>, dim3((unsigned)(2 * use)), dim3(Warps<224>::NTHREADS), umma2_smem_bytes<224>(),
                                                    ctx->stream, mapA, mapB, a));
@@ -1296,6 +1301,7 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
         const int64_t tiles2 = ((M + 2 * BM - 1) / (2 * BM)) * ((N + 255) / 256);
         if (tiles2 >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;
         const int64_t use = tiles2 < pairs ? tiles2 : pairs;
+        note_kernel(ctx, "k_umma_i8_2sm", 256, "CTA pairs, 256 x bn tiles, tcgen05 cta_group::2 kind::i8 on bytes");
         BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8_2sm<256>, dim3((unsigned)(2 * use)), dim3(Warps<256>::NTHREADS), umma2_smem_bytes<256>(),
                                                ctx->stream, mapA, mapB, a));
         return bnn_check_launch(ctx);
@@ -1476,6 +1482,8 @@ static int conv_halo_launch(bnn_ctx *ctx, bool f4, const void *act, const void *
     if (resident && tiles > units) units = (units_max / tn) * tn;       // a multiple of the filter blocks: one block per CTA (pair)
     const unsigned grid = (unsigned)(pair ? 2 * units : units);
     const size_t smem = (size_t)na * a_stage + b_bytes + sizeof(Control) + 1024;
+    note_kernel(ctx, "k_umma_conv", bn, f4 ? "halo tiles, kind::mxf4 on e2m1 nibbles" : "halo tiles, kind::i8 on bytes",
+                pair ? (resident ? ", CTA pairs, resident weights" : ", CTA pairs") : (resident ? ", resident weights" : ", streamed weights"));
     if (pair) {
         if (f4) return conv_halo_launch_t<128, true, true>(ctx, mapA, mapB, a, grid, smem);
         return bn == 256 ? conv_halo_launch_t<256, false, true>(ctx, mapA, mapB, a, grid, smem)
