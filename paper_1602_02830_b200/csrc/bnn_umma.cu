@@ -56,6 +56,7 @@ template <int BN> struct Warps {
 };
 constexpr uint32_t A_BYTES = BM * BK;
 constexpr int ACC_BUFS = 2;
+constexpr int ACC_MAX = 4;                      // accumulator buffers when 128-wide tiles are worked on by four epilogue teams
 template <int BN> struct Cfg {
     static constexpr uint32_t B_BYTES = BN * BK;
     static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
@@ -177,17 +178,22 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
 struct __align__(16) Control {
     uint64_t full[STAGES_MAX];
     uint64_t empty[STAGES_MAX];
-    uint64_t acc_full[ACC_BUFS];
-    uint64_t acc_empty[ACC_BUFS];
-    uint64_t started[ACC_BUFS];            // the tile's first (overwriting) K step has completed
+    uint64_t acc_full[ACC_MAX];
+    uint64_t acc_empty[ACC_MAX];
+    uint64_t started[ACC_MAX];             // the tile's first (overwriting) K step has completed
     uint64_t full_b[B_STAGES_MAX];         // k_umma_conv: its weight ring (full / empty above are its slab ring)
     uint64_t empty_b[B_STAGES_MAX];
     uint32_t tmem_base;
     uint32_t failed;
-    __align__(16) int32_t thr[ACC_BUFS][BN_MAX];   // staged thresholds: clamped int32, or float bits on the 4-bit engine
-    uint32_t flip[ACC_BUFS][BN_MAX / 32];
-    uint32_t poolw[BM][BN_MAX / 32 + 1];   // convolution with pooling: the sign words of every pixel of the tile
+    // Staged per accumulator buffer (slot s of a kernel with tiles BN wide): thresholds thr[s * BN ..] (clamped int32, or
+    // float bits on the 4-bit engine) and flip words flip[s * BN / 32 ..]; 2 x 256 = 4 x 128 columns.
+    __align__(16) int32_t thr[2 * BN_MAX];
+    uint32_t flip[2 * BN_MAX / 32];
+    // Convolution with pooling: the sign words of every pixel of a tile, [team][pixel][BN / 32 + 1] (up to two teams of
+    // 256-wide tiles or four teams of 128-wide ones).
+    uint32_t poolw[4 * BM * (128 / 32 + 1)];
 };
+static_assert(4 * BM * (128 / 32 + 1) >= 2 * BM * (BN_MAX / 32 + 1), "pooling buffer holds two teams of 256-wide tiles");
 
 // Relaxed for the same reason as mbar_arrive_cta0 below: the barrier hands back tensor memory only.
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
@@ -287,12 +293,13 @@ __device__ __forceinline__ void store_signs(const UmmaArgs &p, uint32_t word, in
 // One 32-column chunk of accumulators (r, one output row per thread) -> the requested outputs.
 template <int BN, bool F4 = is_f4(BN)>
 __device__ __forceinline__ void epilogue_chunk(Control *ctl, const UmmaArgs &p, uint32_t (&r)[32], uint32_t buf, int c, int64_t col0,
-                                               int64_t row, int lin, int role = 0, uint4 *hold = nullptr) {
+                                               int64_t row, int lin, uint32_t *poolw, int role = 0, uint4 *hold = nullptr) {
+    // buf: the slot whose staged thresholds apply; poolw: this team's pooling buffer, BN / 32 + 1 words per pixel
     if (row >= p.M) return;
     if (p.thr) {                                         // thresholded signs: packed words and/or the next layer's operand
         // bit j of the word = (acc[j] >= thr[j]) = NOT sign(acc[j] - thr[j]); the sign bits are shifted
         // into four independent 8-bit chains (funnel shift: one instruction per column after the subtract)
-        const int4 *tp = reinterpret_cast<const int4 *>(&ctl->thr[buf][32 * c]);
+        const int4 *tp = reinterpret_cast<const int4 *>(&ctl->thr[buf * BN + 32 * c]);
         uint32_t w4[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
         for (int g = 7; g >= 0; --g) {
@@ -307,9 +314,10 @@ __device__ __forceinline__ void epilogue_chunk(Control *ctl, const UmmaArgs &p, 
             }
         }
         const uint32_t lt = __byte_perm(__byte_perm(w4[0], w4[1], 0x0040), __byte_perm(w4[2], w4[3], 0x0040), 0x5410);
-        uint32_t word = ~lt ^ ctl->flip[buf][c];
+        const uint32_t flipw = ctl->flip[buf * (BN / 32) + c];
+        uint32_t word = ~lt ^ flipw;
         if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;      // columns beyond N stay 0
-        if (p.pool) ctl->poolw[lin][c] = word ^ ctl->flip[buf][c];   // un-flipped (dot >= thr) bits
+        if (p.pool) poolw[lin * (BN / 32 + 1) + c] = word ^ flipw;   // un-flipped (dot >= thr) bits
         else if (p.out) p.out[row * p.ldo + (col0 >> 5)] = word;
         if (p.out8 && !p.pool) store_signs(p, word, row, col0, role, hold);
     }
@@ -366,27 +374,35 @@ __device__ __forceinline__ int tile_lin(const UmmaArgs &p, int i) {
     return (b * p.TH + y) * p.W + x;
 }
 
-template <int BN, bool F4 = is_f4(BN), int EPI_WARPS = Warps<BN>::EPI_WARPS>
+// EPI_WARPS: the warps that work on this tile together.  A kernel may run several such teams (TEAM = 0 .. 3) on different
+// tiles at once, each with its own pooling buffer and pair of named barriers.  buf = the accumulator buffer (and slot of
+// staged thresholds) of this tile, acc_parity the phase of its "full" barrier, slot_next the slot that receives the
+// thresholds of the team's next tile (first column n0_next; -1 = none; same_next = they are the ones already staged);
+// `first` says that this is the team's first tile (it stages its own thresholds).
+template <int BN, bool F4 = is_f4(BN), int EPI_WARPS = Warps<BN>::EPI_WARPS, int TEAM = 0, bool PREFETCH = true>
 __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, uint32_t tmem_base, uint32_t buf, uint32_t tc,
-                                              int64_t m0, int64_t n0, int64_t n0_next, int q, int half, int lane, int et, bool &ok) {
+                                              int64_t m0, int64_t n0, int64_t n0_next, int q, int half, int lane, int et, bool &ok,
+                                              bool first, uint32_t acc_parity, uint32_t slot_next, bool same_next = false) {
     constexpr int EPW = EPI_WARPS / 4, EPI_THREADS = EPI_WARPS * 32;
+    constexpr int BAR_A = 1 + 2 * TEAM, BAR_B = 2 + 2 * TEAM;      // named barriers of this team
+    uint32_t *poolw = ctl->poolw + TEAM * BM * (BN / 32 + 1);
     static_assert(BN <= EPI_THREADS, "one staged threshold per epilogue thread");
     constexpr int CHUNKS = BN / 32, CPW = (CHUNKS + 1) / 2;   // 32-column chunks per tile and (at most) per warp with two warps per quadrant
     const int lin = tile_lin(p, 32 * q + lane);
     const int64_t row = m0 + lin;
-    if (p.thr && tc == 0) {                              // the first tile stages its own thresholds
-        if (et < BN) ctl->thr[buf][et] = staged_threshold<F4>((n0 + et < p.N) ? p.thr[n0 + et] : 0x7fffffff);
+    if (p.thr && first) {                                // the first tile stages its own thresholds
+        if (et < BN) ctl->thr[buf * BN + et] = staged_threshold<F4>((n0 + et < p.N) ? p.thr[n0 + et] : 0x7fffffff);
         if (et < BN / 32) {
             const int64_t w = (n0 >> 5) + et;
-            ctl->flip[buf][et] = (p.flip && w * 32 < p.N) ? p.flip[w] : 0u;
+            ctl->flip[buf * (BN / 32) + et] = (p.flip && w * 32 < p.N) ? p.flip[w] : 0u;
         }
     }
     const int tr_role = (et == 0) ? 3 : ((et == EPI_THREADS - 32) ? 4 : -1);
     if (tr_role >= 0) BNN_TR(tr_role, tc, 0);
     // the epilogue warps only: staged thresholds visible; previous tile's pooling words no longer read
-    if (p.thr) asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
+    if (p.thr) asm volatile("bar.sync %0, %1;" ::"n"(BAR_A), "n"(EPI_THREADS) : "memory");
     if (tr_role >= 0) BNN_TR(tr_role, tc, 1);
-    const bool have_next = p.thr && n0_next >= 0;
+    const bool have_next = p.thr && n0_next >= 0 && !same_next;      // (same_next: the thresholds already staged stay valid)
     int32_t next_thr = 0x7fffffff;
     uint32_t next_flip = 0u;
     if (have_next) {
@@ -400,8 +416,8 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
     // polling warp takes an issue slot on every turn of its loop, and with four of them on each scheduler the two
     // MMA-issuing threads, which share those schedulers, needed three times as long per instruction: a tile of nine
     // short K steps then ran at 40 % of the tensor pipe's rate.
-    if (et < 32 && ok && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->acc_full[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 3); ok = false; }
-    asm volatile("bar.sync 2, %0;" ::"n"(EPI_THREADS) : "memory");
+    if (et < 32 && ok && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->acc_full[buf]), acc_parity)) { fail(ctl, 3); ok = false; }
+    asm volatile("bar.sync %0, %1;" ::"n"(BAR_B), "n"(EPI_THREADS) : "memory");
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (tr_role >= 0) BNN_TR(tr_role, tc, 2);
     ok = ok && (ctl->failed == 0);
@@ -411,7 +427,7 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
     if (ok) {
 #endif
         const uint32_t tbase = tmem_base + ((uint32_t)(32 * q) << 16) + buf * BN;
-        if constexpr (EPW == 2) {
+        if constexpr (EPW == 2 && PREFETCH) {
             // two warps per quadrant, each a contiguous half of the columns (the first one chunk more when their number
             // is odd): chunk c+1 is fetched from tensor memory while chunk c is processed (unrolled, so both register
             // buffers are addressed statically)
@@ -427,14 +443,28 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                 uint32_t (&r)[32] = (cc & 1) ? rb : ra;
                 uint32_t (&rn)[32] = (cc & 1) ? ra : rb;
                 if (more) tmem_ld32(tbase + (uint32_t)(32 * (c + 1)), rn);
-                epilogue_chunk<BN, F4>(ctl, p, r, buf, c, col0, row, lin);
+                epilogue_chunk<BN, F4>(ctl, p, r, buf, c, col0, row, lin, poolw);
                 if (more) tmem_ld_wait(rn);
             }
         } else {
             // more warps per quadrant: chunks go round-robin over them, one register buffer, and the other warps of
             // the scheduler cover the load latency
             uint32_t r[32];
-            if constexpr (CHUNKS == 2 * EPW) {
+            if constexpr (EPW == 2) {
+                // two warps per quadrant, each a contiguous half of the columns, one chunk at a time (kernels whose thread
+                // count leaves no registers for a second chunk in flight); adjacent chunks pair up for whole-sector stores
+                const int c_first = half * CPW, c_end = half ? CHUNKS : CPW;
+                uint4 hold = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll 1
+                for (int c = c_first; c < c_end; ++c) {
+                    const int64_t col0 = n0 + 32 * c;
+                    if (col0 >= p.N) break;                  // uniform over the warp
+                    tmem_ld32(tbase + (uint32_t)(32 * c), r);
+                    tmem_ld_wait(r);
+                    const int role = (CPW % 2 == 0) ? 1 + ((c - c_first) & 1) : 0;
+                    epilogue_chunk<BN, F4>(ctl, p, r, buf, c, col0, row, lin, poolw, role, &hold);
+                }
+            } else if constexpr (CHUNKS == 2 * EPW) {
                 // two adjacent chunks per warp, so that nibble outputs leave as whole 32-byte sectors
                 uint4 hold = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll 1
@@ -444,16 +474,19 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                     if (col0 >= p.N) break;                  // uniform over the warp
                     tmem_ld32(tbase + (uint32_t)(32 * c), r);
                     tmem_ld_wait(r);
-                    epilogue_chunk<BN, F4>(ctl, p, r, buf, c, col0, row, lin, 1 + i, &hold);
+                    epilogue_chunk<BN, F4>(ctl, p, r, buf, c, col0, row, lin, poolw, 1 + i, &hold);
                 }
             } else {
+                uint4 hold = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll 1
                 for (int c = half; c < CHUNKS; c += EPW) {
                     const int64_t col0 = n0 + 32 * c;
                     if (col0 >= p.N) break;                  // uniform over the warp
                     tmem_ld32(tbase + (uint32_t)(32 * c), r);
                     tmem_ld_wait(r);
-                    epilogue_chunk<BN, F4>(ctl, p, r, buf, c, col0, row, lin);
+                    // one warp per quadrant walks all chunks: adjacent ones pair up for whole-sector nibble stores
+                    const int role = (EPW == 1 && CHUNKS % 2 == 0) ? 1 + (c & 1) : 0;
+                    epilogue_chunk<BN, F4>(ctl, p, r, buf, c, col0, row, lin, poolw, role, &hold);
                 }
             }
         }
@@ -466,7 +499,7 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
     if (p.pool) {
         // 2x2 max-pool then threshold == OR of the four thresholded bits, then flip.  The tile holds TB images
         // x TH rows x W columns (TH, W even), i.e. 32 whole windows; 256 (window, word) items for 128 threads.
-        asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
+        asm volatile("bar.sync %0, %1;" ::"n"(BAR_A), "n"(EPI_THREADS) : "memory");
         if (ok) {
             const int Wo = p.W >> 1, nwords = (int)((min((int64_t)BN, p.N - n0) + 31) >> 5);
             for (int e = et; e < (BM / 4) * (BN / 32); e += EPI_THREADS) {
@@ -476,8 +509,9 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                 const int r0 = (2 * wy) * p.W + 2 * wx;                 // top-left pixel of the window inside the tile
                 const int64_t pix = m0 + r0;                            // its linear pixel index b*H*W + y*W + x
                 if (pix >= p.M) continue;
-                uint32_t word = ctl->poolw[r0][c] | ctl->poolw[r0 + 1][c] | ctl->poolw[r0 + p.W][c] | ctl->poolw[r0 + p.W + 1][c];
-                word ^= ctl->flip[buf][c];
+                constexpr int PP = BN / 32 + 1;
+                uint32_t word = poolw[r0 * PP + c] | poolw[(r0 + 1) * PP + c] | poolw[(r0 + p.W) * PP + c] | poolw[(r0 + p.W + 1) * PP + c];
+                word ^= ctl->flip[buf * (BN / 32) + c];
                 const int64_t col0 = n0 + 32 * c;
                 if (col0 + 32 > p.N) word &= (1u << (p.N - col0)) - 1u;
                 // output pixel: same image, (y/2, x/2).  The tile starts at x = 0 of an even row and holds whole rows (of
@@ -492,10 +526,12 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
     }
     if (tr_role >= 0) BNN_TR(tr_role, tc, 4);
     if (have_next) {
+        // (a team that stays on one accumulator buffer restages that buffer's thresholds: only when all have finished reading)
+        if (slot_next == buf) asm volatile("bar.sync %0, %1;" ::"n"(BAR_A), "n"(EPI_THREADS) : "memory");
         // Every epilogue thread has passed this tile's barrier, so none still reads the other buffer's thresholds (they
         // belonged to the previous tile); the next tile's barrier makes these visible.
-        if (et < BN) ctl->thr[buf ^ 1u][et] = staged_threshold<F4>(next_thr);
-        if (et < BN / 32) ctl->flip[buf ^ 1u][et] = next_flip;
+        if (et < BN) ctl->thr[slot_next * BN + et] = staged_threshold<F4>(next_thr);
+        if (et < BN / 32) ctl->flip[slot_next * (BN / 32) + et] = next_flip;
     }
     if (tr_role >= 0) BNN_TR(tr_role, tc, 5);
 }
@@ -503,13 +539,18 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
 // Persistent: gridDim.x CTAs (one per SM) walk the tile list with stride gridDim.x.  The shared-memory ring
 // runs on across tiles; the accumulator is double-buffered in tensor memory (2 x 256 columns), so the
 // epilogue of tile i overlaps the main loop of tile i+1.
-template <int BN>
+// TEAMS > 1: the epilogue warps form that many teams, team k on the CTA's tiles k, k + TEAMS, ... with an accumulator
+// buffer of its own (TEAMS x BN columns of tensor memory).  For tiles with few K steps the epilogue, ~2500 clocks of
+// mostly latency per tile, is what the tile rate follows; with several tiles' epilogues in flight it is their throughput.
+template <int BN, int TEAMS = 1>
 __global__ void __launch_bounds__(Warps<BN>::NTHREADS, 1)
 k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const UmmaArgs p) {
     constexpr int STAGES = Cfg<BN>::STAGES;
     constexpr uint32_t STAGE_BYTES = Cfg<BN>::STAGE_BYTES;
     constexpr int EPI_WARPS = Warps<BN>::EPI_WARPS, MMA_WARP_B = Warps<BN>::MMA_WARP_B;
-    constexpr uint32_t TMEM_COLS = Cfg<BN>::TMEM_COLS;
+    constexpr int NBUF = TEAMS == 1 ? ACC_BUFS : TEAMS, TW = EPI_WARPS / TEAMS;      // accumulator buffers; warps per team
+    static_assert(TEAMS == 1 || (!is_f4(BN) && NBUF * BN <= 512 && TW % 4 == 0), "teams: byte tiles whose buffers fit tensor memory");
+    constexpr uint32_t TMEM_COLS = TEAMS == 1 ? Cfg<BN>::TMEM_COLS : (NBUF * BN <= 256 ? 256 : 512);
     extern __shared__ uint8_t smem_raw[];
     // operand tiles need 1024-byte alignment for the 128-byte swizzle pattern
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -522,9 +563,9 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
-        for (int b = 0; b < ACC_BUFS; ++b) {
+        for (int b = 0; b < NBUF; ++b) {
             mbar_init(smem_u32(&ctl->acc_full[b]), N_ISSUE);    // one commit from each MMA-issuing warp
-            mbar_init(smem_u32(&ctl->acc_empty[b]), EPI_WARPS);
+            mbar_init(smem_u32(&ctl->acc_empty[b]), TW);        // the warps of the team that reads this buffer
             mbar_init(smem_u32(&ctl->started[b]), 1);
         }
         ctl->failed = 0;
@@ -592,7 +633,9 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                 int cc = 0, tx = -1, ty = -1;            // channel slice and tap offsets of the current K step
                 for (int kit = 0; kit < p.k_iters; ++kit) {
                     const bool pre = first_tile && kit < npre;      // B already requested, bytes already expected
+                    if (kit == 0) BNN_TR(0, (t - blockIdx.x) / gridDim.x, 0);
                     if (ph > 0 && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->empty[s]), (ph - 1) & 1)) { fail(ctl, 1); ok = false; break; }
+                    if (kit == 0) BNN_TR(0, (t - blockIdx.x) / gridDim.x, 1);
                     const uint32_t bar = smem_u32(&ctl->full[s]);
                     if (!pre) mbar_expect_tx(bar, STAGE_BYTES);
                     const uint32_t dst = smem_u32(tiles + s * STAGE_BYTES);
@@ -624,15 +667,17 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
             uint32_t it0 = 0, tc = 0;                    // it0: K steps of this CTA before the current tile
             bool ok = true;
             for (int64_t t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++tc, it0 += (uint32_t)p.k_iters) {
-                const uint32_t buf = tc & 1;
-                if (tc >= ACC_BUFS && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->acc_empty[buf]), ((tc / ACC_BUFS) - 1) & 1)) { fail(ctl, 4); ok = false; break; }
+                const uint32_t buf = tc % NBUF, use = tc / NBUF;
+                if (use > 0 && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->acc_empty[buf]), (use - 1) & 1)) { fail(ctl, 4); ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                BNN_TR(1 + w, tc, 0);
                 const uint32_t tmem_d = tmem_base + buf * BN;
                 uint32_t s = (it0 + w) % STAGES, par = ((it0 + w) / STAGES) & 1;   // ring slot and phase of this warp's next step
                 for (int kit = w; kit < p.k_iters; kit += N_ISSUE) {
-                    if (w > 0 && kit == w && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->started[buf]), (tc / ACC_BUFS) & 1)) { fail(ctl, 5); ok = false; break; }
+                    if (w > 0 && kit == w && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->started[buf]), use & 1)) { fail(ctl, 5); ok = false; break; }
                     if (!mbar_wait(ctl, p.wait_ns, full0 + 8 * s, par)) { fail(ctl, 2); ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    if (kit < 2) BNN_TR(1 + w, tc, 1 + kit);
                     const uint64_t adesc = adesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
                     const uint64_t bdesc = bdesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
                     const int nk = (kit == p.k_iters - 1) ? p.k_last : BK / 32;   // the last step may end early (K not a multiple of BK)
@@ -648,6 +693,7 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                     if (s >= (uint32_t)STAGES) { s -= STAGES; par ^= 1u; }
                 }
                 umma_commit(smem_u32(&ctl->acc_full[buf]));     // this warp's share of the tile complete (also after a failure)
+                BNN_TR(1 + w, tc, 11);
             }
         }
     } else if (warp < 2 + EPI_WARPS) {
@@ -656,19 +702,34 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
         bnn_pdl_wait();
         bnn_pdl_launch_next();
         const int q = warp & 3;
-        const int half = (warp - 2) >> 2;
-        const int et = threadIdx.x - 64;                 // 0 .. EPI_THREADS-1 among the epilogue threads
-        uint32_t tc = 0;
+        const int team = (warp - 2) / TW;
+        const int half = ((warp - 2) % TW) >> 2;
+        const int et = (threadIdx.x - 64) % (32 * TW);   // 0 .. 32 * TW - 1 among the team's threads
         bool ok = true;
         // 32-bit tile arithmetic (the host checks the tile count)
         const uint32_t tn = (uint32_t)tiles_n, nt = (uint32_t)ntiles;
-        for (uint32_t t = blockIdx.x; t < nt; t += gridDim.x, ++tc) {
-            const uint32_t buf = tc & 1;
+        for (uint32_t tc = (uint32_t)team; ; tc += TEAMS) {
+            const uint32_t t = blockIdx.x + tc * gridDim.x;
+            if (t >= nt) break;
             const uint32_t tm_i = t / tn;
             const int64_t m0 = (int64_t)tm_i * BM, n0 = (int64_t)(t - tm_i * tn) * BN;
-            const uint32_t t2 = t + gridDim.x;
+            const uint32_t t2 = t + TEAMS * gridDim.x;
             const int64_t n0_next = (t2 < nt) ? (int64_t)(t2 % tn) * BN : -1;
-            epilogue_tile<BN>(ctl, p, tmem_base, buf, tc, m0, n0, n0_next, q, half, lane, et, ok);
+            uint32_t buf;
+            if constexpr (TEAMS == 1) {
+                buf = tc & 1;
+                epilogue_tile<BN>(ctl, p, tmem_base, buf, tc, m0, n0, n0_next, q, half, lane, et, ok, tc == 0, (tc / ACC_BUFS) & 1, buf ^ 1u);
+            } else {
+                buf = (uint32_t)team;
+                const bool first = tc < (uint32_t)TEAMS, same = n0_next == n0;
+                const uint32_t par = (tc / TEAMS) & 1u;
+#define BNN_EPI_TEAM(K) epilogue_tile<BN, false, TW, K, false>(ctl, p, tmem_base, buf, tc, m0, n0, n0_next, q, half, lane, et, ok, first, par, buf, same)
+                if (TEAMS > 3 && team == 3) BNN_EPI_TEAM((TEAMS > 3 ? 3 : 0));
+                else if (TEAMS > 2 && team == 2) BNN_EPI_TEAM((TEAMS > 2 ? 2 : 0));
+                else if (team == 1) BNN_EPI_TEAM(1);
+                else BNN_EPI_TEAM(0);
+#undef BNN_EPI_TEAM
+            }
             // hand the accumulator buffer back to the MMA warp
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
@@ -763,12 +824,15 @@ __device__ __forceinline__ void umma_mxf4_2sm(uint32_t tmem_d, uint64_t adesc, u
         ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(tmem_sf) : "memory");
 }
 
-template <int BN>
+template <int BN, int TEAMS = 1>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(Warps<BN>::NTHREADS, 1)
 k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const UmmaArgs p) {
     constexpr int STAGES2 = Cfg2<BN>::STAGES;
     constexpr uint32_t STAGE2_BYTES = Cfg2<BN>::STAGE_BYTES;
     constexpr int EPI_WARPS = Warps<BN>::EPI_WARPS, MMA_WARP_B = Warps<BN>::MMA_WARP_B;
+    constexpr int NBUF = TEAMS == 1 ? ACC_BUFS : TEAMS, TW = EPI_WARPS / TEAMS;      // see k_umma_i8
+    static_assert(TEAMS == 1 || (!is_f4(BN) && NBUF * BN <= 512 && TW % 4 == 0), "teams: byte tiles whose buffers fit tensor memory");
+    constexpr uint32_t TMEM_COLS2 = TEAMS == 1 ? Cfg<BN>::TMEM_COLS : (NBUF * BN <= 256 ? 256 : 512);
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     Control *ctl = reinterpret_cast<Control *>(tiles + STAGES2 * STAGE2_BYTES);
@@ -782,16 +846,16 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES2; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
-        for (int b = 0; b < ACC_BUFS; ++b) {
+        for (int b = 0; b < NBUF; ++b) {
             mbar_init(smem_u32(&ctl->acc_full[b]), N_ISSUE);    // one multicast commit from each of the leader's MMA warps
-            mbar_init(smem_u32(&ctl->acc_empty[b]), 2 * EPI_WARPS);
+            mbar_init(smem_u32(&ctl->acc_empty[b]), 2 * TW);    // the warps of the team that reads this buffer, in both CTAs
             mbar_init(smem_u32(&ctl->started[b]), 1);
         }
         ctl->failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(Cfg<BN>::TMEM_COLS) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(TMEM_COLS2) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -872,13 +936,13 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
             uint32_t it0 = 0, tc = 0;
             bool ok = true;
             for (int64_t t = pair; t < ntiles && ok; t += npairs, ++tc, it0 += (uint32_t)p.k_iters) {
-                const uint32_t buf = tc & 1;
-                if (tc >= ACC_BUFS && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->acc_empty[buf]), ((tc / ACC_BUFS) - 1) & 1)) { fail_pair(ctl, 14); ok = false; break; }
+                const uint32_t buf = tc % NBUF, use = tc / NBUF;
+                if (use > 0 && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->acc_empty[buf]), (use - 1) & 1)) { fail_pair(ctl, 14); ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tmem_d = tmem_base + buf * BN;
                 uint32_t s = (it0 + w) % STAGES2, par = ((it0 + w) / STAGES2) & 1;
                 for (int kit = w; kit < p.k_iters; kit += N_ISSUE) {
-                    if (w > 0 && kit == w && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->started[buf]), (tc / ACC_BUFS) & 1)) { fail_pair(ctl, 15); ok = false; break; }
+                    if (w > 0 && kit == w && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->started[buf]), use & 1)) { fail_pair(ctl, 15); ok = false; break; }
                     if (!mbar_wait(ctl, p.wait_ns, full0 + 8 * s, par)) { fail_pair(ctl, 12); ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint64_t adesc = adesc0 + (uint64_t)(s * (STAGE2_BYTES >> 4));
@@ -903,18 +967,33 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         bnn_pdl_wait();
         bnn_pdl_launch_next();
         const int q = warp & 3;
-        const int half = (warp - 2) >> 2;
-        const int et = threadIdx.x - 64;
-        uint32_t tc = 0;
+        const int team = (warp - 2) / TW;
+        const int half = ((warp - 2) % TW) >> 2;
+        const int et = (threadIdx.x - 64) % (32 * TW);
         bool ok = true;
         const uint32_t tn = (uint32_t)tiles_n, nt = (uint32_t)ntiles, np = (uint32_t)npairs;
-        for (uint32_t t = (uint32_t)pair; t < nt; t += np, ++tc) {
-            const uint32_t buf = tc & 1;
+        for (uint32_t tc = (uint32_t)team; ; tc += TEAMS) {
+            const uint32_t t = (uint32_t)pair + tc * np;
+            if (t >= nt) break;
             const uint32_t tm_i = t / tn;
             const int64_t m0 = (int64_t)tm_i * (2 * BM) + rank * BM, n0 = (int64_t)(t - tm_i * tn) * BN;
-            const uint32_t t2 = t + np;
+            const uint32_t t2 = t + TEAMS * np;
             const int64_t n0_next = (t2 < nt) ? (int64_t)(t2 % tn) * BN : -1;
-            epilogue_tile<BN>(ctl, p, tmem_base, buf, tc, m0, n0, n0_next, q, half, lane, et, ok);
+            uint32_t buf;
+            if constexpr (TEAMS == 1) {
+                buf = tc & 1;
+                epilogue_tile<BN>(ctl, p, tmem_base, buf, tc, m0, n0, n0_next, q, half, lane, et, ok, tc == 0, (tc / ACC_BUFS) & 1, buf ^ 1u);
+            } else {
+                buf = (uint32_t)team;
+                const bool first = tc < (uint32_t)TEAMS, same = n0_next == n0;
+                const uint32_t par = (tc / TEAMS) & 1u;
+#define BNN_EPI_TEAM(K) epilogue_tile<BN, false, TW, K, false>(ctl, p, tmem_base, buf, tc, m0, n0, n0_next, q, half, lane, et, ok, first, par, buf, same)
+                if (TEAMS > 3 && team == 3) BNN_EPI_TEAM((TEAMS > 3 ? 3 : 0));
+                else if (TEAMS > 2 && team == 2) BNN_EPI_TEAM((TEAMS > 2 ? 2 : 0));
+                else if (team == 1) BNN_EPI_TEAM(1);
+                else BNN_EPI_TEAM(0);
+#undef BNN_EPI_TEAM
+            }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive_cta0(smem_u32(&ctl->acc_empty[buf]));
@@ -926,7 +1005,7 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     cluster_sync_all();                                     // nobody leaves while the peer may still read its shared memory
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(Cfg<BN>::TMEM_COLS) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS2) : "memory");
     }
 }
 
@@ -1123,6 +1202,8 @@ static int umma_prepare(bnn_ctx *ctx) {
         BNN_CUDA_TRY(ctx, cudaFuncSetAttribute(k_umma_i8<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes<256>()));
         BNN_CUDA_TRY(ctx, cudaFuncSetAttribute(k_umma_i8<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes<128>()));
         BNN_CUDA_TRY(ctx, cudaFuncSetAttribute(k_umma_i8<192>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes<192>()));
+        BNN_CUDA_TRY(ctx, (cudaFuncSetAttribute(k_umma_i8<256, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes<256>())));
+        BNN_CUDA_TRY(ctx, (cudaFuncSetAttribute(k_umma_i8<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes<128>())));
         attr_set[ctx->device] = true;
     }
     return BNN_OK;
@@ -1136,7 +1217,7 @@ static int umma_tile_n(int64_t N, int64_t M = 0, int sm_count = 0) {
 }
 template <int BN> static size_t umma2_smem_bytes() { return (size_t)Cfg2<BN>::STAGES * Cfg2<BN>::STAGE_BYTES + sizeof(Control) + 1024; }
 // Pairs of CTAs that can be resident at once for the two-SM kernel on this device (0 = cannot be used).
-template <int BN>
+template <int BN, int TEAMS = 1>
 static int umma2_max_pairs(bnn_ctx *ctx) {
     static std::mutex m;
     static int cached[64];
@@ -1145,7 +1226,7 @@ static int umma2_max_pairs(bnn_ctx *ctx) {
     if (ctx->device < 0 || ctx->device >= 64) return 0;
     if (!have[ctx->device]) {
         int pairs = 0;
-        if (cudaFuncSetAttribute(k_umma_i8_2sm<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma2_smem_bytes<BN>()) == cudaSuccess) {
+        if (cudaFuncSetAttribute(k_umma_i8_2sm<BN, TEAMS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma2_smem_bytes<BN>()) == cudaSuccess) {
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3(2 * ctx->sm_count, 1, 1);
             cfg.blockDim = dim3(Warps<BN>::NTHREADS, 1, 1);
@@ -1154,13 +1235,19 @@ static int umma2_max_pairs(bnn_ctx *ctx) {
             attr.id = cudaLaunchAttributeClusterDimension;
             attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
             cfg.attrs = &attr; cfg.numAttrs = 1;
-            if (cudaOccupancyMaxActiveClusters(&pairs, k_umma_i8_2sm<BN>, &cfg) != cudaSuccess) pairs = 0;
+            if (cudaOccupancyMaxActiveClusters(&pairs, k_umma_i8_2sm<BN, TEAMS>, &cfg) != cudaSuccess) pairs = 0;
         }
         (void)cudaGetLastError();
         cached[ctx->device] = pairs;
         have[ctx->device] = true;
     }
     return cached[ctx->device];
+}
+// Epilogue teams (k_umma_i8<BN, TEAMS>) for byte-operand tiles whose K steps take less time than one tile's epilogue
+// (~2500-3500 clocks): 4 x 64 clocks per K step at 128 columns, 4 x 128 at 256.
+static bool umma_want_teams(const UmmaArgs &a, int bn) {
+    if (!a.thr || a.conv || is_f4(bn) || (bn != 128 && bn != 256)) return false;
+    return (int64_t)a.k_iters * 4 * (bn / 2) <= 4096;
 }
 static void note_kernel(bnn_ctx *ctx, const char *name, int bn, const char *operands, const char *extra = "") {
     snprintf(ctx->last_kernel, sizeof(ctx->last_kernel), "%s<%d> %s%s", name, bn, operands, extra);
@@ -1172,7 +1259,11 @@ static int umma_launch(bnn_ctx *ctx, const CUtensorMap &mapA, const CUtensorMap 
     if (tiles >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;      // the kernels count tiles in 32 bits
     const int64_t grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
     const dim3 g((unsigned)grid);
-    if (bn == 192) BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8<192>, g, dim3(Warps<192>::NTHREADS), umma_smem_bytes<192>(), ctx->stream, mapA, mapB, a));
+    const bool teams = umma_want_teams(a, bn);
+    if (teams) note_kernel(ctx, "k_umma_i8", bn, "128 x bn tiles, tcgen05 kind::i8 on bytes", bn == 128 ? ", 4 epilogue teams" : ", 2 epilogue teams");
+    if (teams && bn == 256) BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8<256, 2>, g, dim3(Warps<256>::NTHREADS), umma_smem_bytes<256>(), ctx->stream, mapA, mapB, a));
+    else if (teams) BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8<128, 4>, g, dim3(Warps<128>::NTHREADS), umma_smem_bytes<128>(), ctx->stream, mapA, mapB, a));
+    else if (bn == 192) BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8<192>, g, dim3(Warps<192>::NTHREADS), umma_smem_bytes<192>(), ctx->stream, mapA, mapB, a));
     else if (bn == 256) BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8<256>, g, dim3(Warps<256>::NTHREADS), umma_smem_bytes<256>(), ctx->stream, mapA, mapB, a));
     else BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8<128>, g, dim3(Warps<128>::NTHREADS), umma_smem_bytes<128>(), ctx->stream, mapA, mapB, a));
     return bnn_check_launch(ctx);
@@ -1301,6 +1392,12 @@ int bnn_umma_gemm(bnn_ctx *ctx, const void *A8, int64_t lda8, bool a_unsigned, c
         const int64_t tiles2 = ((M + 2 * BM - 1) / (2 * BM)) * ((N + 255) / 256);
         if (tiles2 >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;
         const int64_t use = tiles2 < pairs ? tiles2 : pairs;
+        if (umma_want_teams(a, 256) && umma2_max_pairs<256, 2>(ctx) >= pairs) {
+            note_kernel(ctx, "k_umma_i8_2sm", 256, "CTA pairs, 256 x bn tiles, tcgen05 cta_group::2 kind::i8 on bytes", ", 2 epilogue teams");
+            BNN_CUDA_TRY(ctx, (bnn_launch_dependent(k_umma_i8_2sm<256, 2>, dim3((unsigned)(2 * use)), dim3(Warps<256>::NTHREADS), umma2_smem_bytes<256>(),
+                                                    ctx->stream, mapA, mapB, a)));
+            return bnn_check_launch(ctx);
+        }
         note_kernel(ctx, "k_umma_i8_2sm", 256, "CTA pairs, 256 x bn tiles, tcgen05 cta_group::2 kind::i8 on bytes");
         BNN_CUDA_TRY(ctx, bnn_launch_dependent(k_umma_i8_2sm<256>, dim3((unsigned)(2 * use)), dim3(Warps<256>::NTHREADS), umma2_smem_bytes<256>(),
                                                ctx->stream, mapA, mapB, a));

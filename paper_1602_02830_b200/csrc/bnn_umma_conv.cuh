@@ -262,7 +262,7 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             const int64_t m0 = (int64_t)tm_i * TILE_M + rank * BM, n0 = (int64_t)(t - tm_i * tn) * BN;
             const uint32_t t2 = t + nunits;
             const int64_t n0_next = (t2 < nt) ? (int64_t)(t2 % tn) * BN : -1;
-            epilogue_tile<BN, F4, EPI_WARPS>(ctl, p, tmem_base, buf, tc, m0, n0, n0_next, q, half, lane, et, ok);
+            epilogue_tile<BN, F4, EPI_WARPS>(ctl, p, tmem_base, buf, tc, m0, n0, n0_next, q, half, lane, et, ok, tc == 0, (tc / ACC_BUFS) & 1, buf ^ 1u);
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) { if (PAIR) mbar_arrive_cta0(smem_u32(&ctl->acc_empty[buf])); else mbar_arrive(smem_u32(&ctl->acc_empty[buf])); }
