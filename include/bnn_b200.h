@@ -205,6 +205,21 @@ BNN_API int bnn_binary_conv2d(bnn_ctx *ctx, const uint32_t *act, const uint8_t *
                       const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, int32_t *out_sums);
 
 /* ---------------------------------------------------------------------------------------------
+ * Exploiting filter repetitions (Section 3.3).  A binary 3x3 filter over C_in channels consists of C_in two-dimensional
+ * 3x3 filters, of which only 2^9 exist -- 2^8 classes when a filter and its negation count as one.  With the switch on,
+ * bnn_binary_conv2d on a binary input classifies the layer's C_out x C_in 2-D filters, applies per input channel only the
+ * DISTINCT ones to the map (one XNOR-popcount on a 9-bit neighbourhood per distinct filter and pixel) and forms every
+ * filter's result as a signed sum of those responses.  Results are the same integers and bits as without the switch.
+ * It runs on the CUDA cores and needs a workspace of bnn_filter_repetition_workspace_bytes(C_in, C_out) for the class
+ * tables (BNN_ERR_WORKSPACE otherwise).  It shows the mechanism; on this GPU the full product on the tensor cores is faster.
+ * bnn_filter_repetition_count classifies the filters Wp ([C_out][3][3][C_in / 32] words) and returns, in *distinct (host),
+ * the number of distinct 2-D filters summed over the input channels (at most min(256, C_out) per channel, against
+ * C_out * C_in filter applications without the exploit); it uses the same workspace and synchronises the stream. */
+BNN_API int bnn_set_conv_filter_repetition(bnn_ctx *ctx, int on);
+BNN_API size_t bnn_filter_repetition_workspace_bytes(int64_t C_in, int64_t C_out);
+BNN_API int bnn_filter_repetition_count(bnn_ctx *ctx, const uint32_t *Wp, int64_t C_in, int64_t C_out, int64_t *distinct);
+
+/* ---------------------------------------------------------------------------------------------
  * Whole ConvNet forward: a stack of 3x3 / pad-1 layers, each  conv -> optional 2x2 max-pool -> threshold -> Sign
  * (Algorithm 4 with convolutions in place of the dense products, Section 3.3).  Layer 0 takes the 8-bit image
  * (9 * C_in <= 32, bit-plane layer of Section 1.6); every other layer takes the previous layer's binary map.

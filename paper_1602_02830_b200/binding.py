@@ -29,7 +29,8 @@ EXPORTS = (
     "bnn_expanded_bytes", "bnn_expand_signs", "bnn_baseline_gemm_f32", "bnn_convnet_workspace_bytes",
     "bnn_convnet_forward", "bnn_set_operand_bits", "bnn_expanded_ld_f4",
     "bnn_expanded_bytes_f4", "bnn_expand_signs_f4", "bnn_binary_dense_expanded", "bnn_set_wait_limit_ns",
-    "bnn_debug_drop_loads", "bnn_set_conv_form", "bnn_measure_pipe_rates", "bnn_last_tensor_kernel",
+    "bnn_debug_drop_loads", "bnn_set_conv_form", "bnn_measure_pipe_rates", "bnn_last_tensor_kernel", "bnn_set_conv_filter_repetition",
+    "bnn_filter_repetition_workspace_bytes", "bnn_filter_repetition_count",
 )
 
 
@@ -91,6 +92,10 @@ def lib() -> ctypes.CDLL:
         L.bnn_measure_pipe_rates.argtypes = [vp, vp, c_size_t, POINTER(c_double), POINTER(c_double), POINTER(c_double)]
         L.bnn_last_tensor_kernel.argtypes = [vp]
         L.bnn_last_tensor_kernel.restype = ctypes.c_char_p
+        L.bnn_set_conv_filter_repetition.argtypes = [vp, c_int]
+        L.bnn_filter_repetition_workspace_bytes.argtypes = [i64, i64]
+        L.bnn_filter_repetition_workspace_bytes.restype = c_size_t
+        L.bnn_filter_repetition_count.argtypes = [vp, vp, i64, i64, POINTER(c_int64)]
         L.bnn_expanded_ld_f4.argtypes = [i64]
         L.bnn_expanded_ld_f4.restype = i64
         L.bnn_expanded_bytes_f4.argtypes = [i64, i64]
@@ -244,6 +249,18 @@ class Context:
 
     def last_tensor_kernel(self) -> str:
         return lib().bnn_last_tensor_kernel(self._h).decode()
+
+    def set_conv_filter_repetition(self, on: bool):
+        self._ck(lib().bnn_set_conv_filter_repetition(self._h, int(on)), "bnn_set_conv_filter_repetition")
+
+    def filter_repetition_workspace_bytes(self, C_in: int, C_out: int) -> int:
+        return int(lib().bnn_filter_repetition_workspace_bytes(C_in, C_out))
+
+    def filter_repetition_count(self, Wp, C_in: int, C_out: int) -> int:
+        """bnn_filter_repetition_count: distinct 2-D filters (up to sign) summed over the input channels."""
+        out = c_int64()
+        self._ck(lib().bnn_filter_repetition_count(self._h, _ptr(Wp), C_in, C_out, ctypes.byref(out)), "bnn_filter_repetition_count")
+        return int(out.value)
 
     def set_conv_form(self, form: int):
         self._ck(lib().bnn_set_conv_form(self._h, form), "bnn_set_conv_form")

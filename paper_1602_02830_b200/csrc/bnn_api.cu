@@ -24,6 +24,7 @@ extern "C" int bnn_create(bnn_ctx **out, int device, void *cuda_stream) {
     c->wait_limit_ns = 2000000000ull;
     c->drop_loads = 0;
     c->conv_form = 0;
+    c->filter_repetition = 0;
     c->last_kernel[0] = 0;
     c->copy_stream = nullptr;
     c->copy_ready = false;
@@ -90,6 +91,12 @@ extern "C" int bnn_set_operand_bits(bnn_ctx *ctx, int bits) {
 extern "C" int bnn_set_wait_limit_ns(bnn_ctx *ctx, uint64_t ns) {
     if (!ctx || ns == 0 || ns > 60000000000ull) return BNN_ERR_INVALID_ARG;
     ctx->wait_limit_ns = ns;
+    return BNN_OK;
+}
+
+extern "C" int bnn_set_conv_filter_repetition(bnn_ctx *ctx, int on) {
+    if (!ctx || (on != 0 && on != 1)) return BNN_ERR_INVALID_ARG;
+    ctx->filter_repetition = on;
     return BNN_OK;
 }
 

@@ -22,6 +22,7 @@ struct bnn_ctx {
     int operand_bits; // tensor engine, +-1 x +-1 products: 4 = e2m1 nibbles (default), 8 = signed bytes
     int engine;    // 0 auto, 1 CUDA-core XOR-popcount kernels only, 2 tensor-core int8 engine where it applies
     unsigned long long wait_limit_ns;   // tensor engine: how long one of its device-side waits may last before it gives up
+    int filter_repetition;   // bnn_binary_conv2d on a binary input applies only the distinct 2-D filters per channel (Section 3.3)
     int conv_form;    // tensor engine, 3x3 convolutions: 0 = halo-tile kernel where the geometry allows, 1 = one operand box per tap
     char last_kernel[96];   // the tensor-core kernel launched last, for bnn_last_tensor_kernel
     int drop_loads;   // test hook: the tensor kernels' producer issues no loads, so that their waits run into the limit

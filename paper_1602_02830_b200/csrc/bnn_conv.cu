@@ -125,6 +125,8 @@ extern "C" int bnn_binary_conv2d(bnn_ctx *ctx, const uint32_t *act, const uint8_
     if (!bnn_aligned16(act) && (Cw % 4) == 0) return BNN_ERR_ALIGNMENT;
     if (!bnn_aligned16(Wp) && (Cw % 4) == 0) return BNN_ERR_ALIGNMENT;
     if (out_bits && !bnn_aligned16(out_bits)) return BNN_ERR_ALIGNMENT;
+    if (ctx->filter_repetition)      // Section 3.3: apply only the distinct 2-D filters of every channel (CUDA cores)
+        return bnn_fr_conv(ctx, act, B, H, W, C_in, Wp, C_out, pool, thr, flip, out_bits, out_sums);
     {
         // tensor-core engine: activations and weights are expanded to +-1 bytes in the workspace and the convolution
         // runs as 9 * C_in/128 K steps of TMA 4-D loads whose out-of-image halo arrives as zeros

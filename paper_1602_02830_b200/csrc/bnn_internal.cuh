@@ -50,3 +50,8 @@ size_t bnn_planes_scratch_bytes(int64_t M, int64_t K);
 int bnn_first_layer_planes_pre(bnn_ctx *ctx, const uint8_t *X, int64_t ldx, const uint32_t *Wp, int64_t ldw_w, const int32_t *thr,
                                const uint32_t *flip, uint32_t *out_bits, int64_t ldo_w, int32_t *out_sums, int64_t lds, int64_t M,
                                int64_t N, int64_t K, void *scratch);
+
+// ---- filter repetitions (bnn_conv_fr.cu): only the distinct 2-D filters of every input channel are applied
+size_t bnn_fr_workspace_bytes(int64_t C_in, int64_t C_out);
+int bnn_fr_conv(bnn_ctx *ctx, const uint32_t *act, int64_t B, int64_t H, int64_t W, int64_t C_in, const uint32_t *Wp, int64_t C_out,
+                int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, int32_t *out_sums);

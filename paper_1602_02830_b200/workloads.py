@@ -89,3 +89,18 @@ def dense_case(batch: int, K: int = 4096, N: int = 4096, seed: int = 4):
     thr = rng.integers(-64, 65, size=N, dtype=np.int32)
     A = pm1(np.random.default_rng([seed, batch]), (batch, K))
     return {"A": A, "W": W, "thr": thr}
+
+
+def dictionary_conv_weights(rng: np.random.Generator, Cout: int, Cin: int, distinct_per_channel: int) -> np.ndarray:
+    """Cout x 3 x 3 x Cin +-1 weights with repeated 2-D filters (Section 3.3 reports that only 42 % of a trained network's
+    filters are distinct): in every input channel the Cout 3x3 slices are drawn from `distinct_per_channel` random patterns
+    (distinct even up to negation, each used at least once), with random signs.  Stands in for trained weights."""
+    wgt = np.empty((Cout, 3, 3, Cin), np.int8)
+    for c in range(Cin):
+        codes = rng.choice(256, size=distinct_per_channel, replace=False)      # classes up to sign: tap 0 = +1, 8 free taps
+        pats = np.array([[1] + [1 if (k >> b) & 1 else -1 for b in range(8)] for k in codes], np.int8)
+        pick = np.concatenate([np.arange(distinct_per_channel), rng.integers(0, distinct_per_channel, Cout - distinct_per_channel)])
+        rng.shuffle(pick)
+        sign = (2 * rng.integers(0, 2, Cout) - 1).astype(np.int8)
+        wgt[:, :, :, c] = (pats[pick] * sign[:, None]).reshape(Cout, 3, 3)
+    return wgt
