@@ -52,7 +52,8 @@ template <int BN> struct Warps {
     static constexpr int EPW = EPI_WARPS / 4;
     static constexpr int EPI_THREADS = EPI_WARPS * 32;
     static constexpr int MMA_WARP_B = 2 + EPI_WARPS;                 // the second MMA-issuing warp (the first is warp 1)
-    static constexpr int NTHREADS = 64 + EPI_THREADS + 32 * (N_ISSUE - 1);
+    static constexpr int PROD_WARP_B = MMA_WARP_B + N_ISSUE - 1;      // second producer warp (pair kernel: the B operand's loads)
+    static constexpr int NTHREADS = 64 + EPI_THREADS + 32 * (N_ISSUE - 1) + 32;
 };
 constexpr uint32_t A_BYTES = BM * BK;
 constexpr int ACC_BUFS = 2;
@@ -650,7 +651,7 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                 }
             }
         }
-    } else if (warp == 1 || warp >= MMA_WARP_B) {
+    } else if (warp == 1 || warp == MMA_WARP_B) {
         // ---------------- MMA issuers.  Issuing one K step (wait, four instructions, commit) costs the issuing thread
         // more clocks than the tensor core needs to execute it, so N_ISSUE warps on different schedulers share the work
         // round-robin over the K steps of every tile.  All products are exact integers, so the order in which the
@@ -879,20 +880,23 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     }
 
-    if (warp == 0) {
-        // ---------------- TMA producer (both CTAs): own A rows, own half of the tile's B rows
+    if (warp == 0 || warp == Warps<BN>::PROD_WARP_B) {
+        // ---------------- TMA producers (both CTAs): warp 0 requests this CTA's A rows, the second producer warp its half of
+        // the tile's B rows.  One thread needs ~500-700 clocks per K step for its barrier poll, the byte count and two loads
+        // -- more than the 512 clocks in which a 256-wide K step of bytes is multiplied -- so a tile of few K steps (the
+        // first MLP layer has seven) ran at the producer's pace; with the loads split each thread issues one per K step.
         if (lane == 0) {
+            const bool is_b = (warp != 0);
             bool ok = true;
             uint32_t s = 0, ph = 0;                      // ring slot, and the number of times the ring has wrapped
             const uint32_t tn32 = (uint32_t)tiles_n;
-            // the weights of the first ring fill are requested before the wait for the preceding kernel (see k_umma_i8)
-            const int npre = !p.b_static ? 0 : (p.k_iters < STAGES2 ? p.k_iters : STAGES2);
+            // the weights of the first ring fill are requested before the wait for the preceding kernel (see k_umma_i8);
+            // the bytes are expected by the A producer's arrival, which may come later
+            const int npre = (!p.b_static || !is_b) ? 0 : (p.k_iters < STAGES2 ? p.k_iters : STAGES2);
             {
                 const int nb0f = (int)(((uint32_t)pair % tn32) * BN + rank * (BN / 2));
-                for (int kit = 0; kit < npre; ++kit) {
-                    if (rank == 0) mbar_expect_tx(smem_u32(&ctl->full[kit]), 2 * STAGE2_BYTES);
+                for (int kit = 0; kit < npre; ++kit)
                     tma_load_2d_2sm(smem_u32(tiles + kit * STAGE2_BYTES + A_BYTES), &mapB, kit * BK, nb0f, smem_u32(&ctl->full[kit]) & PEER_MASK);
-                }
             }
             bnn_pdl_wait();
             for (uint32_t t = (uint32_t)pair; t < (uint32_t)ntiles && ok; t += (uint32_t)npairs) {
@@ -910,20 +914,26 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                 int cc = 0, tx = -1, ty = -1;
                 for (int kit = 0; kit < p.k_iters; ++kit) {
                     const bool pre = first_tile && kit < npre;
+                    if (kit < 4 && !is_b) BNN_TR(0, (t - (uint32_t)pair) / (uint32_t)npairs, 2 * kit);
                     if (ph > 0 && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->empty[s]), (ph - 1) & 1)) { fail_pair(ctl, 11); ok = false; break; }
-                    if (rank == 0 && !pre) mbar_expect_tx(smem_u32(&ctl->full[s]), 2 * STAGE2_BYTES);   // the bytes of both CTAs
+                    if (kit < 4 && !is_b) BNN_TR(0, (t - (uint32_t)pair) / (uint32_t)npairs, 2 * kit + 1);
                     const uint32_t bar0 = smem_u32(&ctl->full[s]) & PEER_MASK;
-                    if (p.conv) {
-                        tma_load_4d_2sm(smem_u32(tiles + s * STAGE2_BYTES), &mapA, cc * BK, tx, y0 + ty, b0, bar0);
-                        if (++cc == p.c_chunks) { cc = 0; if (++tx == 2) { tx = -1; ++ty; } }
-                    } else
-                    tma_load_2d_2sm(smem_u32(tiles + s * STAGE2_BYTES), &mapA, kit * BK, m0, bar0);
-                    if (!pre) tma_load_2d_2sm(smem_u32(tiles + s * STAGE2_BYTES + A_BYTES), &mapB, kit * BK, nb0, bar0);
+                    if (!is_b) {
+                        if (rank == 0) mbar_expect_tx(smem_u32(&ctl->full[s]), 2 * STAGE2_BYTES);   // the bytes of both CTAs, both operands
+                        if (p.conv) {
+                            tma_load_4d_2sm(smem_u32(tiles + s * STAGE2_BYTES), &mapA, cc * BK, tx, y0 + ty, b0, bar0);
+                            if (++cc == p.c_chunks) { cc = 0; if (++tx == 2) { tx = -1; ++ty; } }
+                        } else {
+                            tma_load_2d_2sm(smem_u32(tiles + s * STAGE2_BYTES), &mapA, kit * BK, m0, bar0);
+                        }
+                    } else if (!pre) {
+                        tma_load_2d_2sm(smem_u32(tiles + s * STAGE2_BYTES + A_BYTES), &mapB, kit * BK, nb0, bar0);
+                    }
                     if (++s == (uint32_t)STAGES2) { s = 0; ++ph; }
                 }
             }
         }
-    } else if (warp == 1 || warp >= MMA_WARP_B) {
+    } else if (warp == 1 || warp == MMA_WARP_B) {
         // ---------------- MMA issuers: two warps of the leader CTA only (even / odd K steps), for both tensor cores
         if (lane == 0 && rank == 0) {
             const int w = (warp == 1) ? 0 : warp - MMA_WARP_B + 1;
@@ -939,12 +949,14 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                 const uint32_t buf = tc % NBUF, use = tc / NBUF;
                 if (use > 0 && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->acc_empty[buf]), (use - 1) & 1)) { fail_pair(ctl, 14); ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                BNN_TR(1 + w, tc, 0);
                 const uint32_t tmem_d = tmem_base + buf * BN;
                 uint32_t s = (it0 + w) % STAGES2, par = ((it0 + w) / STAGES2) & 1;
                 for (int kit = w; kit < p.k_iters; kit += N_ISSUE) {
                     if (w > 0 && kit == w && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->started[buf]), use & 1)) { fail_pair(ctl, 15); ok = false; break; }
                     if (!mbar_wait(ctl, p.wait_ns, full0 + 8 * s, par)) { fail_pair(ctl, 12); ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    if (kit < 10) BNN_TR(1 + w, tc, 1 + kit);
                     const uint64_t adesc = adesc0 + (uint64_t)(s * (STAGE2_BYTES >> 4));
                     const uint64_t bdesc = bdesc0 + (uint64_t)(s * (STAGE2_BYTES >> 4));
                     const int nk = (kit == p.k_iters - 1) ? p.k_last : BK / 32;
@@ -960,6 +972,7 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                     if (s >= (uint32_t)STAGES2) { s -= STAGES2; par ^= 1u; }
                 }
                 umma_commit_2sm(smem_u32(&ctl->acc_full[buf]));
+                BNN_TR(1 + w, tc, 11);
             }
         }
     } else if (warp < 2 + EPI_WARPS) {
