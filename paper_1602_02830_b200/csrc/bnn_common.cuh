@@ -24,7 +24,7 @@ struct bnn_ctx {
     unsigned long long wait_limit_ns;   // tensor engine: how long one of its device-side waits may last before it gives up
     int filter_repetition;   // bnn_binary_conv2d on a binary input applies only the distinct 2-D filters per channel (Section 3.3)
     int conv_form;    // tensor engine, 3x3 convolutions: 0 = halo-tile kernel where the geometry allows, 1 = one operand box per tap
-    char last_kernel[96];   // the tensor-core kernel launched last, for bnn_last_tensor_kernel
+    char last_kernel[160];   // the tensor-core kernel launched last, for bnn_last_tensor_kernel
     int drop_loads;   // test hook: the tensor kernels' producer issues no loads, so that their waits run into the limit
 };
 

@@ -177,13 +177,13 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
 }
 
 struct __align__(16) Control {
-    uint64_t full[STAGES_MAX];
-    uint64_t empty[STAGES_MAX];
+    uint64_t full[2 * STAGES_MAX];         // two barrier pairs per ring slot, see RingCursor
+    uint64_t empty[2 * STAGES_MAX];
     uint64_t acc_full[ACC_MAX];
     uint64_t acc_empty[ACC_MAX];
     uint64_t started[ACC_MAX];             // the tile's first (overwriting) K step has completed
-    uint64_t full_b[B_STAGES_MAX];         // k_umma_conv: its weight ring (full / empty above are its slab ring)
-    uint64_t empty_b[B_STAGES_MAX];
+    uint64_t full_b[B_STAGES_MAX];         // k_umma_conv: its weight ring (full / empty above are its slab ring); resident
+    uint64_t empty_b[B_STAGES_MAX];        // weights use one pair per stage, a streamed ring two per slot
     uint32_t tmem_base;
     uint32_t failed;
     // Staged per accumulator buffer (slot s of a kernel with tiles BN wide): thresholds thr[s * BN ..] (clamped int32, or
@@ -226,6 +226,26 @@ __device__ __forceinline__ bool mbar_wait(const Control *ctl, unsigned long long
         }
     }
 }
+
+// Position in a ring of S operand slots that is guarded by 2 S barrier pairs: stage G of a CTA's sequence lives in slot
+// G % S and signals barrier pair G % 2S, phase G / 2S.
+// Why twice as many barriers as slots: a wait on a phase PARITY is only right while the waiter is at most one phase ahead
+// of the barrier.  Two issuing threads that take alternate stages of one ring keep that distance only when each barrier
+// belongs to one of them.  With one barrier per slot and an odd S the uses of a slot alternate between the threads, and a
+// thread can reach its next use while the other thread's use in between is still loading (loads complete out of
+// order): the parity it waits for then matches the phase before, the wait returns at once, and it multiplies a slot
+// that is being written and releases it a second time.  2 S is even, so every barrier pair has one consumer thread.
+struct RingCursor {
+    uint32_t b, lap;                 // barrier pair of the next stage; how often the barrier ring has wrapped
+    __device__ __forceinline__ void start(uint32_t G, uint32_t S) { b = G % (2 * S); lap = G / (2 * S); }
+    __device__ __forceinline__ uint32_t slot(uint32_t S) const { return b >= S ? b - S : b; }
+    __device__ __forceinline__ uint32_t parity() const { return lap & 1u; }
+    // the stage that used this slot before (S stages earlier): whether there is one, its barrier pair and phase parity
+    __device__ __forceinline__ bool reuses(uint32_t S) const { return lap > 0 || b >= S; }
+    __device__ __forceinline__ uint32_t prev_bar(uint32_t S) const { return b >= S ? b - S : b + S; }
+    __device__ __forceinline__ uint32_t prev_parity(uint32_t S) const { return (b >= S ? lap : lap - 1u) & 1u; }
+    __device__ __forceinline__ void advance(uint32_t n, uint32_t S) { b += n; if (b >= 2 * S) { b -= 2 * S; ++lap; } }   // n <= 2 S
+};
 
 // 8 sign bits -> 8 e2m1 nibbles (+1.0 = 0x2, -1.0 = 0xa); bit i lands in nibble i.
 __device__ __forceinline__ uint32_t nibbles_of_byte(uint32_t x) {
@@ -563,7 +583,7 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
     const int64_t ntiles = tiles_m * tiles_n;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
+        for (int s = 0; s < 2 * STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
         for (int b = 0; b < NBUF; ++b) {
             mbar_init(smem_u32(&ctl->acc_full[b]), N_ISSUE);    // one commit from each MMA-issuing warp
             mbar_init(smem_u32(&ctl->acc_empty[b]), TW);        // the warps of the team that reads this buffer
@@ -605,7 +625,7 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
             // The loop below runs once per K step in a single thread that shares its scheduler with epilogue warps:
             // everything per tile is computed once, ring slot / phase / tap advance incrementally (no divisions inside;
             // with them a 3x3 convolution's producer could not keep up: 128 -> 128 channels at 32 x 32, 88 -> 57 us).
-            uint32_t s = 0, ph = 0;                      // ring slot, and the number of times the ring has wrapped
+            RingCursor rc; rc.start(0, STAGES);
             const uint32_t tn32 = (uint32_t)tiles_n;
             // B is weights, not a product of the preceding kernel: its share of the first ring fill is requested before
             // the wait for that kernel, A's after it
@@ -635,11 +655,11 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                 for (int kit = 0; kit < p.k_iters; ++kit) {
                     const bool pre = first_tile && kit < npre;      // B already requested, bytes already expected
                     if (kit == 0) BNN_TR(0, (t - blockIdx.x) / gridDim.x, 0);
-                    if (ph > 0 && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->empty[s]), (ph - 1) & 1)) { fail(ctl, 1); ok = false; break; }
+                    if (rc.reuses(STAGES) && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->empty[rc.prev_bar(STAGES)]), rc.prev_parity(STAGES))) { fail(ctl, 1); ok = false; break; }
                     if (kit == 0) BNN_TR(0, (t - blockIdx.x) / gridDim.x, 1);
-                    const uint32_t bar = smem_u32(&ctl->full[s]);
+                    const uint32_t bar = smem_u32(&ctl->full[rc.b]);
                     if (!pre) mbar_expect_tx(bar, STAGE_BYTES);
-                    const uint32_t dst = smem_u32(tiles + s * STAGE_BYTES);
+                    const uint32_t dst = smem_u32(tiles + rc.slot(STAGES) * STAGE_BYTES);
                     if (p.conv) {
                         tma_load_4d(dst, &mapA, cc * BK, tx, y0 + ty, b0, bar);
                         if (++cc == p.c_chunks) { cc = 0; if (++tx == 2) { tx = -1; ++ty; } }
@@ -647,7 +667,7 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                         tma_load_2d(dst, &mapA, kit * BK, m0, bar);
                     }
                     if (!pre) tma_load_2d(dst + A_BYTES, &mapB, kit * BK, n0, bar);
-                    if (++s == (uint32_t)STAGES) { s = 0; ++ph; }
+                    rc.advance(1, STAGES);
                 }
             }
         }
@@ -673,10 +693,11 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 BNN_TR(1 + w, tc, 0);
                 const uint32_t tmem_d = tmem_base + buf * BN;
-                uint32_t s = (it0 + w) % STAGES, par = ((it0 + w) / STAGES) & 1;   // ring slot and phase of this warp's next step
+                RingCursor rc; rc.start(it0 + w, STAGES);            // this warp's next step
                 for (int kit = w; kit < p.k_iters; kit += N_ISSUE) {
                     if (w > 0 && kit == w && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->started[buf]), use & 1)) { fail(ctl, 5); ok = false; break; }
-                    if (!mbar_wait(ctl, p.wait_ns, full0 + 8 * s, par)) { fail(ctl, 2); ok = false; break; }
+                    if (!mbar_wait(ctl, p.wait_ns, full0 + 8 * rc.b, rc.parity())) { fail(ctl, 2); ok = false; break; }
+                    const uint32_t s = rc.slot(STAGES);
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     if (kit < 2) BNN_TR(1 + w, tc, 1 + kit);
                     const uint64_t adesc = adesc0 + (uint64_t)(s * (STAGE_BYTES >> 4));
@@ -688,10 +709,9 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                         if (is_f4(BN)) umma_mxf4(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u, tmem_base + SF_COL);
                         else umma_i8(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u);
                     }
-                    umma_commit(empty0 + 8 * s);                // stage may be refilled once these MMAs have read it
+                    umma_commit(empty0 + 8 * rc.b);             // stage may be refilled once these MMAs have read it
                     if (kit == 0) umma_commit(smem_u32(&ctl->started[buf]));
-                    s += N_ISSUE;
-                    if (s >= (uint32_t)STAGES) { s -= STAGES; par ^= 1u; }
+                    rc.advance(N_ISSUE, STAGES);
                 }
                 umma_commit(smem_u32(&ctl->acc_full[buf]));     // this warp's share of the tile complete (also after a failure)
                 BNN_TR(1 + w, tc, 11);
@@ -846,7 +866,7 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     const int64_t ntiles = tiles_m * tiles_n;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES2; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
+        for (int s = 0; s < 2 * STAGES2; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
         for (int b = 0; b < NBUF; ++b) {
             mbar_init(smem_u32(&ctl->acc_full[b]), N_ISSUE);    // one multicast commit from each of the leader's MMA warps
             mbar_init(smem_u32(&ctl->acc_empty[b]), 2 * TW);    // the warps of the team that reads this buffer, in both CTAs
@@ -888,7 +908,7 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         if (lane == 0) {
             const bool is_b = (warp != 0);
             bool ok = true;
-            uint32_t s = 0, ph = 0;                      // ring slot, and the number of times the ring has wrapped
+            RingCursor rc; rc.start(0, STAGES2);
             const uint32_t tn32 = (uint32_t)tiles_n;
             // the weights of the first ring fill are requested before the wait for the preceding kernel (see k_umma_i8);
             // the bytes are expected by the A producer's arrival, which may come later
@@ -915,11 +935,12 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                 for (int kit = 0; kit < p.k_iters; ++kit) {
                     const bool pre = first_tile && kit < npre;
                     if (kit < 4 && !is_b) BNN_TR(0, (t - (uint32_t)pair) / (uint32_t)npairs, 2 * kit);
-                    if (ph > 0 && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->empty[s]), (ph - 1) & 1)) { fail_pair(ctl, 11); ok = false; break; }
+                    if (rc.reuses(STAGES2) && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->empty[rc.prev_bar(STAGES2)]), rc.prev_parity(STAGES2))) { fail_pair(ctl, 11); ok = false; break; }
                     if (kit < 4 && !is_b) BNN_TR(0, (t - (uint32_t)pair) / (uint32_t)npairs, 2 * kit + 1);
-                    const uint32_t bar0 = smem_u32(&ctl->full[s]) & PEER_MASK;
+                    const uint32_t s = rc.slot(STAGES2);
+                    const uint32_t bar0 = smem_u32(&ctl->full[rc.b]) & PEER_MASK;
                     if (!is_b) {
-                        if (rank == 0) mbar_expect_tx(smem_u32(&ctl->full[s]), 2 * STAGE2_BYTES);   // the bytes of both CTAs, both operands
+                        if (rank == 0) mbar_expect_tx(smem_u32(&ctl->full[rc.b]), 2 * STAGE2_BYTES);   // the bytes of both CTAs, both operands
                         if (p.conv) {
                             tma_load_4d_2sm(smem_u32(tiles + s * STAGE2_BYTES), &mapA, cc * BK, tx, y0 + ty, b0, bar0);
                             if (++cc == p.c_chunks) { cc = 0; if (++tx == 2) { tx = -1; ++ty; } }
@@ -929,7 +950,7 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                     } else if (!pre) {
                         tma_load_2d_2sm(smem_u32(tiles + s * STAGE2_BYTES + A_BYTES), &mapB, kit * BK, nb0, bar0);
                     }
-                    if (++s == (uint32_t)STAGES2) { s = 0; ++ph; }
+                    rc.advance(1, STAGES2);
                 }
             }
         }
@@ -951,10 +972,11 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 BNN_TR(1 + w, tc, 0);
                 const uint32_t tmem_d = tmem_base + buf * BN;
-                uint32_t s = (it0 + w) % STAGES2, par = ((it0 + w) / STAGES2) & 1;
+                RingCursor rc; rc.start(it0 + w, STAGES2);
                 for (int kit = w; kit < p.k_iters; kit += N_ISSUE) {
                     if (w > 0 && kit == w && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->started[buf]), use & 1)) { fail_pair(ctl, 15); ok = false; break; }
-                    if (!mbar_wait(ctl, p.wait_ns, full0 + 8 * s, par)) { fail_pair(ctl, 12); ok = false; break; }
+                    if (!mbar_wait(ctl, p.wait_ns, full0 + 8 * rc.b, rc.parity())) { fail_pair(ctl, 12); ok = false; break; }
+                    const uint32_t s = rc.slot(STAGES2);
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     if (kit < 10) BNN_TR(1 + w, tc, 1 + kit);
                     const uint64_t adesc = adesc0 + (uint64_t)(s * (STAGE2_BYTES >> 4));
@@ -966,10 +988,9 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                         if (is_f4(BN)) umma_mxf4_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u, tmem_base + SF_COL);
                         else umma_i8_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u);
                     }
-                    umma_commit_2sm(empty0 + 8 * s);
+                    umma_commit_2sm(empty0 + 8 * rc.b);
                     if (kit == 0) umma_commit_2sm_local(smem_u32(&ctl->started[buf]));
-                    s += N_ISSUE;
-                    if (s >= (uint32_t)STAGES2) { s -= STAGES2; par ^= 1u; }
+                    rc.advance(N_ISSUE, STAGES2);
                 }
                 umma_commit_2sm(smem_u32(&ctl->acc_full[buf]));
                 BNN_TR(1 + w, tc, 11);

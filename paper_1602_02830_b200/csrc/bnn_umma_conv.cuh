@@ -63,10 +63,14 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     const int64_t tiles_n = (p.N + BN - 1) / BN;
     const int64_t ntiles = tiles_m * tiles_n;
     const int groups = p.k_iters / 3;                    // slabs per tile: 3 horizontal taps x channel slices
+    const int RB = p.b_resident ? NB : 3 * NB;           // barrier pairs of the weight stages
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < NA; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
-        for (int s = 0; s < NB; ++s) { mbar_init(smem_u32(&ctl->full_b[s]), 1); mbar_init(smem_u32(&ctl->empty_b[s]), 1); }
+        // every barrier pair of a ring must have ONE consuming thread (see RingCursor): the slabs alternate between the two
+        // issuing threads, so their ring has 2 NA pairs; streamed weight stages change hands every three (one slab's
+        // vertical taps), so that ring has RB = 3 NB pairs (NB is even: a multiple of 6 stages and of the NB slots)
+        for (int s = 0; s < 2 * NA; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
+        for (int s = 0; s < RB; ++s) { mbar_init(smem_u32(&ctl->full_b[s]), 1); mbar_init(smem_u32(&ctl->empty_b[s]), 1); }
         for (int b = 0; b < ACC_BUFS; ++b) {
             mbar_init(smem_u32(&ctl->acc_full[b]), N_ISSUE);                          // one commit from each issuing thread
             mbar_init(smem_u32(&ctl->acc_empty[b]), (PAIR ? 2 : 1) * EPI_WARPS);      // the leader's barrier counts both CTAs' warps
@@ -134,8 +138,8 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 b_loaded = true;
             }
             bnn_pdl_wait();
-            uint32_t sa = 0, pha = 0;                    // slab ring slot and the number of times that ring has wrapped
-            uint32_t sb = 0, phb = 0;                    // the same for the weight ring (streamed weights)
+            RingCursor ra; ra.start(0, (uint32_t)NA);    // slab ring
+            uint32_t sb = 0, bb_i = 0, lapb = 0;         // streamed weights: ring slot, barrier pair, wraps of the barrier ring
             for (uint32_t t = unit; t < (uint32_t)ntiles && ok; t += nunits) {
 #ifdef EXP_NO_LOADS
                 if (t != unit) break;                    // experiment: only the first tile's operands are ever loaded
@@ -153,13 +157,13 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 for (int cc = 0; cc < p.c_chunks && ok; ++cc) {
                     for (int dxi = 0; dxi < 3 && ok; ++dxi) {
                         if (cc == 0) BNN_TR(0, tr_tile, 2 * dxi);
-                        if (pha > 0 && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->empty[sa]), (pha - 1) & 1)) { conv_fail<PAIR>(ctl, 21); ok = false; break; }
+                        if (ra.reuses((uint32_t)NA) && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->empty[ra.prev_bar((uint32_t)NA)]), ra.prev_parity((uint32_t)NA))) { conv_fail<PAIR>(ctl, 21); ok = false; break; }
                         if (cc == 0) BNN_TR(0, tr_tile, 2 * dxi + 1);
-                        const uint32_t bar = smem_u32(&ctl->full[sa]);
+                        const uint32_t bar = smem_u32(&ctl->full[ra.b]);
                         if (rank == 0) mbar_expect_tx(bar, a_tx);
                         // dimensions of the map: channel byte, column, image, row
-                        load_a(smem_u32(slabs + (size_t)sa * A_STAGE), cc * BK, dxi - 1, b0, y0 - 1, bar);
-                        if (++sa == (uint32_t)NA) { sa = 0; ++pha; }
+                        load_a(smem_u32(slabs + (size_t)ra.slot((uint32_t)NA) * A_STAGE), cc * BK, dxi - 1, b0, y0 - 1, bar);
+                        ra.advance(1, (uint32_t)NA);
                         for (int dyi = 0; dyi < 3; ++dyi, ++kit) {
                             if (p.b_resident) {
                                 if (b_loaded) continue;
@@ -167,11 +171,16 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                                 if (rank == 0) mbar_expect_tx(bb, b_tx);
                                 load_b(smem_u32(wts + (size_t)kit * B_STAGE), (3 * dyi + dxi) * p.tap_bytes + cc * BK, n0, bb);
                             } else {
-                                if (phb > 0 && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->empty_b[sb]), (phb - 1) & 1)) { conv_fail<PAIR>(ctl, 22); ok = false; break; }
-                                const uint32_t bb = smem_u32(&ctl->full_b[sb]);
+                                if (lapb > 0 || bb_i >= (uint32_t)NB) {      // the stage NB earlier must have been multiplied
+                                    const uint32_t pb_i = bb_i >= (uint32_t)NB ? bb_i - (uint32_t)NB : bb_i + (uint32_t)(RB - NB);
+                                    const uint32_t pp = (bb_i >= (uint32_t)NB ? lapb : lapb - 1u) & 1u;
+                                    if (!mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->empty_b[pb_i]), pp)) { conv_fail<PAIR>(ctl, 22); ok = false; break; }
+                                }
+                                const uint32_t bb = smem_u32(&ctl->full_b[bb_i]);
                                 if (rank == 0) mbar_expect_tx(bb, b_tx);
                                 load_b(smem_u32(wts + (size_t)sb * B_STAGE), (3 * dyi + dxi) * p.tap_bytes + cc * BK, n0, bb);
-                                if (++sb == (uint32_t)NB) { sb = 0; ++phb; }
+                                if (++sb == (uint32_t)NB) sb = 0;
+                                if (++bb_i == (uint32_t)RB) { bb_i = 0; ++lapb; }
                             }
                         }
                     }
@@ -218,8 +227,9 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 BNN_TR(1 + w, tc, 0);
 #pragma unroll 1
                 for (uint32_t g = g_first; g < (uint32_t)groups && ok; g += 2) {
-                    const uint32_t a_seq = j + g, sa = a_seq % (uint32_t)NA, pa = (a_seq / (uint32_t)NA) & 1u;
-                    if (!mbar_wait(ctl, p.wait_ns, fullA0 + 8 * sa, pa)) { conv_fail<PAIR>(ctl, 26); ok = false; break; }
+                    RingCursor ra; ra.start(j + g, (uint32_t)NA);
+                    const uint32_t sa = ra.slot((uint32_t)NA);
+                    if (!mbar_wait(ctl, p.wait_ns, fullA0 + 8 * ra.b, ra.parity())) { conv_fail<PAIR>(ctl, 26); ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint64_t aslab = adesc0 + (uint64_t)(sa * a_step);
                     const uint32_t kit0 = 3u * g;
@@ -227,20 +237,23 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
 #pragma unroll
                     for (uint32_t dyi = 0; dyi < 3; ++dyi) {
                         const uint32_t kit = kit0 + dyi;
-                        uint32_t sb = kit, pb = 0;
-                        if (!p.b_resident) { const uint32_t b_seq = tc * (uint32_t)p.k_iters + kit; sb = b_seq % (uint32_t)NB; pb = (b_seq / (uint32_t)NB) & 1u; }
+                        uint32_t sb = kit, bb_i = kit, pb = 0;       // weight slot, its barrier pair, phase parity
+                        if (!p.b_resident) {
+                            const uint32_t b_seq = tc * (uint32_t)p.k_iters + kit;
+                            sb = b_seq % (uint32_t)NB; bb_i = b_seq % (uint32_t)RB; pb = (b_seq / (uint32_t)RB) & 1u;
+                        }
                         if (wait_b) {
-                            if (!mbar_wait(ctl, p.wait_ns, fullB0 + 8 * sb, pb)) { conv_fail<PAIR>(ctl, 27); ok = false; break; }
+                            if (!mbar_wait(ctl, p.wait_ns, fullB0 + 8 * bb_i, pb)) { conv_fail<PAIR>(ctl, 27); ok = false; break; }
                             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                         }
                         const uint64_t adesc = aslab + (uint64_t)(dyi * dy_step);
                         const uint64_t bdesc = bdesc0 + (uint64_t)(sb * b_step);
 #pragma unroll
                         for (int k = 0; k < BK / 32; ++k) mma(adesc + 2 * k, bdesc + 2 * k, tmem_d, (kit > 0 || k > 0) ? 1u : 0u);
-                        if (!p.b_resident) commit(emptyB0 + 8 * sb);
+                        if (!p.b_resident) commit(emptyB0 + 8 * bb_i);
                         if (kit == 0) { if (PAIR) umma_commit_2sm_local(smem_u32(&ctl->started[buf])); else umma_commit(smem_u32(&ctl->started[buf])); }
                     }
-                    commit(emptyA0 + 8 * sa);                   // the slab's three K steps have been issued
+                    commit(emptyA0 + 8 * ra.b);                 // the slab's three K steps have been issued
                 }
                 commit(smem_u32(&ctl->acc_full[buf]));          // this thread's share of the tile (also after a failure)
                 BNN_TR(1 + w, tc, 11);
