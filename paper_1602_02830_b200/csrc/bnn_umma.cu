@@ -176,12 +176,28 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
         :: "memory");
 }
 
+// Zeroes 32 accumulator columns of the calling warp's 32 lanes.  Every epilogue warp does this to the columns it has
+// read (and every buffer is zeroed once at kernel start), so that every MMA of a tile ACCUMULATES: with an overwriting
+// first MMA the second issuing thread had to wait at the start of every tile until that MMA had completed, and the tensor
+// pipe ran on one thread's issue rate meanwhile (a pair's MMA costs its issuing thread ~120 clocks, more than the pipe
+// needs to execute it): ~1200 clocks per tile.
+__device__ __forceinline__ void tmem_zero32(uint32_t taddr) {
+    const uint32_t z = 0u;
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1};"
+                 ::"r"(taddr), "r"(z) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// All `cols` accumulator columns (a multiple of 32) of the calling warp's lane quadrant.
+__device__ __forceinline__ void tmem_zero_all(uint32_t tmem_base, int warp, int cols) {
+    for (int c = 0; c < cols; c += 32) tmem_zero32(tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)c);
+    tmem_st_wait();
+}
+
 struct __align__(16) Control {
     uint64_t full[2 * STAGES_MAX];         // two barrier pairs per ring slot, see RingCursor
     uint64_t empty[2 * STAGES_MAX];
     uint64_t acc_full[ACC_MAX];
     uint64_t acc_empty[ACC_MAX];
-    uint64_t started[ACC_MAX];             // the tile's first (overwriting) K step has completed
     uint64_t full_b[B_STAGES_MAX];         // k_umma_conv: its weight ring (full / empty above are its slab ring); resident
     uint64_t empty_b[B_STAGES_MAX];        // weights use one pair per stage, a streamed ring two per slot
     uint32_t tmem_base;
@@ -237,14 +253,16 @@ __device__ __forceinline__ bool mbar_wait(const Control *ctl, unsigned long long
 // that is being written and releases it a second time.  2 S is even, so every barrier pair has one consumer thread.
 struct RingCursor {
     uint32_t b, lap;                 // barrier pair of the next stage; how often the barrier ring has wrapped
-    __device__ __forceinline__ void start(uint32_t G, uint32_t S) { b = G % (2 * S); lap = G / (2 * S); }
-    __device__ __forceinline__ uint32_t slot(uint32_t S) const { return b >= S ? b - S : b; }
+    // M: barrier pairs per slot (2 for two consumer threads that alternate; a multiple of the number of threads that
+    // take the stages in turn, so that G % (M S) fixes the thread)
+    __device__ __forceinline__ void start(uint32_t G, uint32_t S, uint32_t M = 2) { b = G % (M * S); lap = G / (M * S); }
+    __device__ __forceinline__ uint32_t slot(uint32_t S) const { uint32_t x = b; while (x >= S) x -= S; return x; }
     __device__ __forceinline__ uint32_t parity() const { return lap & 1u; }
     // the stage that used this slot before (S stages earlier): whether there is one, its barrier pair and phase parity
     __device__ __forceinline__ bool reuses(uint32_t S) const { return lap > 0 || b >= S; }
-    __device__ __forceinline__ uint32_t prev_bar(uint32_t S) const { return b >= S ? b - S : b + S; }
+    __device__ __forceinline__ uint32_t prev_bar(uint32_t S, uint32_t M = 2) const { return b >= S ? b - S : b + (M - 1) * S; }
     __device__ __forceinline__ uint32_t prev_parity(uint32_t S) const { return (b >= S ? lap : lap - 1u) & 1u; }
-    __device__ __forceinline__ void advance(uint32_t n, uint32_t S) { b += n; if (b >= 2 * S) { b -= 2 * S; ++lap; } }   // n <= 2 S
+    __device__ __forceinline__ void advance(uint32_t n, uint32_t S, uint32_t M = 2) { b += n; if (b >= M * S) { b -= M * S; ++lap; } }   // n <= M S
 };
 
 // 8 sign bits -> 8 e2m1 nibbles (+1.0 = 0x2, -1.0 = 0xa); bit i lands in nibble i.
@@ -442,11 +460,7 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (tr_role >= 0) BNN_TR(tr_role, tc, 2);
     ok = ok && (ctl->failed == 0);
-#ifdef EXP_NO_EPI
-    if (false) {                                         // experiment: the accumulators are never read
-#else
     if (ok) {
-#endif
         const uint32_t tbase = tmem_base + ((uint32_t)(32 * q) << 16) + buf * BN;
         if constexpr (EPW == 2 && PREFETCH) {
             // two warps per quadrant, each a contiguous half of the columns (the first one chunk more when their number
@@ -454,7 +468,7 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
             // buffers are addressed statically)
             uint32_t ra[32], rb[32];
             const int c_first = half * CPW, c_end = half ? CHUNKS : CPW;
-            if (n0 + 32 * c_first < p.N) { tmem_ld32(tbase + (uint32_t)(32 * c_first), ra); tmem_ld_wait(ra); }
+            if (n0 + 32 * c_first < p.N) { tmem_ld32(tbase + (uint32_t)(32 * c_first), ra); tmem_ld_wait(ra); tmem_zero32(tbase + (uint32_t)(32 * c_first)); }
 #pragma unroll
             for (int cc = 0; cc < CPW; ++cc) {
                 const int c = c_first + cc;
@@ -465,7 +479,7 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                 uint32_t (&rn)[32] = (cc & 1) ? ra : rb;
                 if (more) tmem_ld32(tbase + (uint32_t)(32 * (c + 1)), rn);
                 epilogue_chunk<BN, F4>(ctl, p, r, buf, c, col0, row, lin, poolw);
-                if (more) tmem_ld_wait(rn);
+                if (more) { tmem_ld_wait(rn); tmem_zero32(tbase + (uint32_t)(32 * (c + 1))); }
             }
         } else {
             // more warps per quadrant: chunks go round-robin over them, one register buffer, and the other warps of
@@ -482,6 +496,7 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                     if (col0 >= p.N) break;                  // uniform over the warp
                     tmem_ld32(tbase + (uint32_t)(32 * c), r);
                     tmem_ld_wait(r);
+                    tmem_zero32(tbase + (uint32_t)(32 * c));
                     const int role = (CPW % 2 == 0) ? 1 + ((c - c_first) & 1) : 0;
                     epilogue_chunk<BN, F4>(ctl, p, r, buf, c, col0, row, lin, poolw, role, &hold);
                 }
@@ -495,6 +510,7 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                     if (col0 >= p.N) break;                  // uniform over the warp
                     tmem_ld32(tbase + (uint32_t)(32 * c), r);
                     tmem_ld_wait(r);
+                    tmem_zero32(tbase + (uint32_t)(32 * c));
                     epilogue_chunk<BN, F4>(ctl, p, r, buf, c, col0, row, lin, poolw, 1 + i, &hold);
                 }
             } else {
@@ -505,12 +521,14 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
                     if (col0 >= p.N) break;                  // uniform over the warp
                     tmem_ld32(tbase + (uint32_t)(32 * c), r);
                     tmem_ld_wait(r);
+                    tmem_zero32(tbase + (uint32_t)(32 * c));
                     // one warp per quadrant walks all chunks: adjacent ones pair up for whole-sector nibble stores
                     const int role = (EPW == 1 && CHUNKS % 2 == 0) ? 1 + (c & 1) : 0;
                     epilogue_chunk<BN, F4>(ctl, p, r, buf, c, col0, row, lin, poolw, role, &hold);
                 }
             }
         }
+        tmem_st_wait();                                  // the zeroes are in place before the buffer is handed back
         // padding words of the packed output
         if (half == 0 && p.out && !p.pool && row < p.M && n0 + BN >= p.N) {
             for (int64_t w = (p.N + 31) >> 5; w < p.ldo; ++w) p.out[row * p.ldo + w] = 0u;
@@ -587,7 +605,6 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
         for (int b = 0; b < NBUF; ++b) {
             mbar_init(smem_u32(&ctl->acc_full[b]), N_ISSUE);    // one commit from each MMA-issuing warp
             mbar_init(smem_u32(&ctl->acc_empty[b]), TW);        // the warps of the team that reads this buffer
-            mbar_init(smem_u32(&ctl->started[b]), 1);
         }
         ctl->failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -604,14 +621,18 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
     // waits for it below (bnn_pdl_wait): the producer (after requesting weights that kernel does not write), the
     // epilogue warps at once; they also release this kernel's own successor.
 
-    if (is_f4(BN)) {
+    {
+        // Every accumulator buffer starts at zero (all MMAs accumulate, see tmem_zero32).
         // 4-bit engine: every value is exactly +-1, so every block scale is 2^0.  In UE8M0 that is the byte 0x7f, and
         // with all 32 scale-factor columns filled with it the instruction reads 1.0 wherever it looks.
         if (warp >= 2 && warp < 6) {
-            const uint32_t v = 0x7f7f7f7fu;
-            asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1};"
-                         ::"r"(tmem_base + SF_COL + ((uint32_t)(32 * (warp & 3)) << 16)), "r"(v) : "memory");
-            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            tmem_zero_all(tmem_base, warp, NBUF * BN);
+            if (is_f4(BN)) {
+                const uint32_t v = 0x7f7f7f7fu;
+                asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1};"
+                             ::"r"(tmem_base + SF_COL + ((uint32_t)(32 * (warp & 3)) << 16)), "r"(v) : "memory");
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            }
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
@@ -674,9 +695,8 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
     } else if (warp == 1 || warp == MMA_WARP_B) {
         // ---------------- MMA issuers.  Issuing one K step (wait, four instructions, commit) costs the issuing thread
         // more clocks than the tensor core needs to execute it, so N_ISSUE warps on different schedulers share the work
-        // round-robin over the K steps of every tile.  All products are exact integers, so the order in which the
-        // streams reach the accumulator does not matter, except that the overwriting first step must be there
-        // first: the other warps wait for its completion once per tile.
+        // round-robin over the K steps of every tile.  All products are exact integers and every MMA accumulates into a
+        // buffer that the epilogue left at zero, so the order in which the streams reach the accumulator does not matter.
         if (lane == 0) {
             const int w = (warp == 1) ? 0 : warp - MMA_WARP_B + 1;   // this warp takes K steps w, w + N_ISSUE, ...
             // e2m1 x e2m1 (format 1), UE8M0 scales (bit 23) on the 4-bit engine; N >> 3 at bit 17, M >> 4 at bit 24
@@ -695,7 +715,6 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
                 const uint32_t tmem_d = tmem_base + buf * BN;
                 RingCursor rc; rc.start(it0 + w, STAGES);            // this warp's next step
                 for (int kit = w; kit < p.k_iters; kit += N_ISSUE) {
-                    if (w > 0 && kit == w && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->started[buf]), use & 1)) { fail(ctl, 5); ok = false; break; }
                     if (!mbar_wait(ctl, p.wait_ns, full0 + 8 * rc.b, rc.parity())) { fail(ctl, 2); ok = false; break; }
                     const uint32_t s = rc.slot(STAGES);
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -706,11 +725,10 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k) {   // 32 bytes of K per instruction: start address advances by 32 B (>> 4 = 2)
                         if (k >= nk) break;
-                        if (is_f4(BN)) umma_mxf4(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u, tmem_base + SF_COL);
-                        else umma_i8(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u);
+                        if (is_f4(BN)) umma_mxf4(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, 1u, tmem_base + SF_COL);
+                        else umma_i8(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, 1u);
                     }
                     umma_commit(empty0 + 8 * rc.b);             // stage may be refilled once these MMAs have read it
-                    if (kit == 0) umma_commit(smem_u32(&ctl->started[buf]));
                     rc.advance(N_ISSUE, STAGES);
                 }
                 umma_commit(smem_u32(&ctl->acc_full[buf]));     // this warp's share of the tile complete (also after a failure)
@@ -811,10 +829,6 @@ __device__ __forceinline__ void umma_commit_2sm(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                  ::"r"(bar), "h"(mask) : "memory");
 }
-// The same for a barrier of the issuing CTA alone.
-__device__ __forceinline__ void umma_commit_2sm_local(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
 // Arrive on the barrier at the same offset in CTA 0 of the cluster.  Relaxed: the barrier hands back tensor memory, whose
 // reads are ordered by tcgen05.wait::ld and the tcgen05 fence before the arrival; nothing written to memory is passed
 // on through it.  (With release semantics at cluster scope the arrival waited for the epilogue's global stores to
@@ -852,6 +866,8 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     constexpr uint32_t STAGE2_BYTES = Cfg2<BN>::STAGE_BYTES;
     constexpr int EPI_WARPS = Warps<BN>::EPI_WARPS, MMA_WARP_B = Warps<BN>::MMA_WARP_B;
     constexpr int NBUF = TEAMS == 1 ? ACC_BUFS : TEAMS, TW = EPI_WARPS / TEAMS;      // see k_umma_i8
+    constexpr int NI2 = N_ISSUE;
+    constexpr uint32_t RM = 2;                              // barrier pairs per ring slot (see RingCursor)
     static_assert(TEAMS == 1 || (!is_f4(BN) && NBUF * BN <= 512 && TW % 4 == 0), "teams: byte tiles whose buffers fit tensor memory");
     constexpr uint32_t TMEM_COLS2 = TEAMS == 1 ? Cfg<BN>::TMEM_COLS : (NBUF * BN <= 256 ? 256 : 512);
     extern __shared__ uint8_t smem_raw[];
@@ -866,11 +882,10 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     const int64_t ntiles = tiles_m * tiles_n;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < 2 * STAGES2; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
+        for (int s = 0; s < (int)RM * STAGES2; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
         for (int b = 0; b < NBUF; ++b) {
-            mbar_init(smem_u32(&ctl->acc_full[b]), N_ISSUE);    // one multicast commit from each of the leader's MMA warps
+            mbar_init(smem_u32(&ctl->acc_full[b]), NI2);        // one multicast commit from each of the leader's MMA warps
             mbar_init(smem_u32(&ctl->acc_empty[b]), 2 * TW);    // the warps of the team that reads this buffer, in both CTAs
-            mbar_init(smem_u32(&ctl->started[b]), 1);
         }
         ctl->failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -885,14 +900,18 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = ctl->tmem_base;
 
-    if (is_f4(BN)) {
-        // 4-bit engine: unit block scales (byte 0x7f) in this CTA's scale-factor columns; the leader's MMAs read the
-        // columns of both CTAs, so the pair synchronises once more before the first one is issued
+    {
+        // Zero accumulators in this CTA's tensor memory (see tmem_zero32) and, on the 4-bit engine, unit block scales (byte
+        // 0x7f) in its scale-factor columns; the leader's MMAs write / read the columns of both CTAs, so the pair
+        // synchronises once more before the first one is issued
         if (warp >= 2 && warp < 6) {
-            const uint32_t v = 0x7f7f7f7fu;
-            asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1};"
-                         ::"r"(tmem_base + SF_COL + ((uint32_t)(32 * (warp & 3)) << 16)), "r"(v) : "memory");
-            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            tmem_zero_all(tmem_base, warp, NBUF * BN);
+            if (is_f4(BN)) {
+                const uint32_t v = 0x7f7f7f7fu;
+                asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1};"
+                             ::"r"(tmem_base + SF_COL + ((uint32_t)(32 * (warp & 3)) << 16)), "r"(v) : "memory");
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            }
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
@@ -901,25 +920,27 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     }
 
     if (warp == 0 || warp == Warps<BN>::PROD_WARP_B) {
-        // ---------------- TMA producers (both CTAs): warp 0 requests this CTA's A rows, the second producer warp its half of
-        // the tile's B rows.  One thread needs ~500-700 clocks per K step for its barrier poll, the byte count and two loads
-        // -- more than the 512 clocks in which a 256-wide K step of bytes is multiplied -- so a tile of few K steps (the
-        // first MLP layer has seven) ran at the producer's pace; with the loads split each thread issues one per K step.
+        // ---------------- TMA producers (both CTAs): two threads, alternate K steps.  One thread needs ~500-700 clocks per K
+        // step for its barrier poll, the byte count and two loads -- more than the 448-512 clocks in which the step is
+        // multiplied -- so with one producer a tile ran at the producer's pace; each of two has twice the time.
         if (lane == 0) {
-            const bool is_b = (warp != 0);
+            // each producer thread takes every other K step of the pair's sequence, with both operands
+            const uint32_t wp = (warp == 0) ? 0u : 1u;
             bool ok = true;
-            RingCursor rc; rc.start(0, STAGES2);
+            RingCursor rc; rc.start(wp, STAGES2, RM);
             const uint32_t tn32 = (uint32_t)tiles_n;
-            // the weights of the first ring fill are requested before the wait for the preceding kernel (see k_umma_i8);
-            // the bytes are expected by the A producer's arrival, which may come later
-            const int npre = (!p.b_static || !is_b) ? 0 : (p.k_iters < STAGES2 ? p.k_iters : STAGES2);
+            uint32_t it0 = 0;                            // K steps of this pair before the current tile
+            // the weights of the first ring fill are requested before the wait for the preceding kernel (see k_umma_i8)
+            const int npre = !p.b_static ? 0 : (p.k_iters < STAGES2 ? p.k_iters : STAGES2);
             {
                 const int nb0f = (int)(((uint32_t)pair % tn32) * BN + rank * (BN / 2));
-                for (int kit = 0; kit < npre; ++kit)
+                for (int kit = (int)wp; kit < npre; kit += 2) {
+                    if (rank == 0) mbar_expect_tx(smem_u32(&ctl->full[kit]), 2 * STAGE2_BYTES);
                     tma_load_2d_2sm(smem_u32(tiles + kit * STAGE2_BYTES + A_BYTES), &mapB, kit * BK, nb0f, smem_u32(&ctl->full[kit]) & PEER_MASK);
+                }
             }
             bnn_pdl_wait();
-            for (uint32_t t = (uint32_t)pair; t < (uint32_t)ntiles && ok; t += (uint32_t)npairs) {
+            for (uint32_t t = (uint32_t)pair; t < (uint32_t)ntiles && ok; t += (uint32_t)npairs, it0 += (uint32_t)p.k_iters) {
                 const bool first_tile = (t == (uint32_t)pair);
                 const uint32_t tm = t / tn32;
                 const int m0 = (int)(tm * (2 * BM) + rank * BM);
@@ -931,33 +952,31 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                     b0 = (p.TB > 1) ? tm128 * p.TB : tm128 / tiles_per_img;
                     y0 = (p.TB > 1) ? 0 : (tm128 % tiles_per_img) * p.TH;
                 }
-                int cc = 0, tx = -1, ty = -1;
-                for (int kit = 0; kit < p.k_iters; ++kit) {
+                for (int kit = (int)((wp + it0) & 1u); kit < p.k_iters; kit += 2) {
                     const bool pre = first_tile && kit < npre;
-                    if (kit < 4 && !is_b) BNN_TR(0, (t - (uint32_t)pair) / (uint32_t)npairs, 2 * kit);
-                    if (rc.reuses(STAGES2) && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->empty[rc.prev_bar(STAGES2)]), rc.prev_parity(STAGES2))) { fail_pair(ctl, 11); ok = false; break; }
-                    if (kit < 4 && !is_b) BNN_TR(0, (t - (uint32_t)pair) / (uint32_t)npairs, 2 * kit + 1);
-                    const uint32_t s = rc.slot(STAGES2);
+                    if (kit < 8) BNN_TR(0, (t - (uint32_t)pair) / (uint32_t)npairs, kit);
+                    if (rc.reuses(STAGES2) && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->empty[rc.prev_bar(STAGES2, RM)]), rc.prev_parity(STAGES2))) { fail_pair(ctl, 11); ok = false; break; }
+                    const uint32_t dst = smem_u32(tiles + rc.slot(STAGES2) * STAGE2_BYTES);
                     const uint32_t bar0 = smem_u32(&ctl->full[rc.b]) & PEER_MASK;
-                    if (!is_b) {
-                        if (rank == 0) mbar_expect_tx(smem_u32(&ctl->full[rc.b]), 2 * STAGE2_BYTES);   // the bytes of both CTAs, both operands
-                        if (p.conv) {
-                            tma_load_4d_2sm(smem_u32(tiles + s * STAGE2_BYTES), &mapA, cc * BK, tx, y0 + ty, b0, bar0);
-                            if (++cc == p.c_chunks) { cc = 0; if (++tx == 2) { tx = -1; ++ty; } }
-                        } else {
-                            tma_load_2d_2sm(smem_u32(tiles + s * STAGE2_BYTES), &mapA, kit * BK, m0, bar0);
-                        }
-                    } else if (!pre) {
-                        tma_load_2d_2sm(smem_u32(tiles + s * STAGE2_BYTES + A_BYTES), &mapB, kit * BK, nb0, bar0);
+                    if (!pre && rank == 0) mbar_expect_tx(smem_u32(&ctl->full[rc.b]), 2 * STAGE2_BYTES);   // the bytes of both CTAs, both operands
+                    if (p.conv) {
+                        const int tap = kit / p.c_chunks, cc = kit - tap * p.c_chunks, ty = tap / 3;
+                        tma_load_4d_2sm(dst, &mapA, cc * BK, tap - 3 * ty - 1, y0 + ty - 1, b0, bar0);
+                    } else {
+                        tma_load_2d_2sm(dst, &mapA, kit * BK, m0, bar0);
                     }
-                    rc.advance(1, STAGES2);
+                    if (!pre) tma_load_2d_2sm(dst + A_BYTES, &mapB, kit * BK, nb0, bar0);
+                    rc.advance(2, STAGES2, RM);
                 }
             }
         }
     } else if (warp == 1 || warp == MMA_WARP_B) {
-        // ---------------- MMA issuers: two warps of the leader CTA only (even / odd K steps), for both tensor cores
+        // ---------------- MMA issuers: two warps of the leader CTA only (even / odd K steps), for both tensor cores.  A pair's
+        // MMA costs the thread that issues it ~120 clocks, more than the tensor cores need for most shapes, so one thread
+        // cannot keep them busy; two reach the pipe's rate in a loop of nothing else (measured: 112 clocks per 256 x 224
+        // x 64 nibble MMA, 128 per 256 x 256 x 32 byte MMA, on one accumulator or two).
         if (lane == 0 && rank == 0) {
-            const int w = (warp == 1) ? 0 : warp - MMA_WARP_B + 1;
+            const int w = (warp == 1) ? 0 : 1;
             // the host's descriptor carries M = 128 in bits [24,29); the pair multiplies M = 256
             const uint32_t idesc = is_f4(BN)
                 ? ((1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (1u << 23) | ((uint32_t)((2 * BM) >> 4) << 24))
@@ -972,12 +991,15 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 BNN_TR(1 + w, tc, 0);
                 const uint32_t tmem_d = tmem_base + buf * BN;
-                RingCursor rc; rc.start(it0 + w, STAGES2);
-                for (int kit = w; kit < p.k_iters; kit += N_ISSUE) {
-                    if (w > 0 && kit == w && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->started[buf]), use & 1)) { fail_pair(ctl, 15); ok = false; break; }
+                RingCursor rc; rc.start(it0 + w, STAGES2, RM);
+                for (int kit = w; kit < p.k_iters; kit += NI2) {
+                    const bool fine = (kit == 4 + w);         // instrumented builds: one steady-state K step per tile in detail
+                    if (fine) BNN_TR(5 + w, tc, 0);
                     if (!mbar_wait(ctl, p.wait_ns, full0 + 8 * rc.b, rc.parity())) { fail_pair(ctl, 12); ok = false; break; }
+                    if (fine) BNN_TR(5 + w, tc, 1);
                     const uint32_t s = rc.slot(STAGES2);
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    if (fine) BNN_TR(5 + w, tc, 2);
                     if (kit < 10) BNN_TR(1 + w, tc, 1 + kit);
                     const uint64_t adesc = adesc0 + (uint64_t)(s * (STAGE2_BYTES >> 4));
                     const uint64_t bdesc = bdesc0 + (uint64_t)(s * (STAGE2_BYTES >> 4));
@@ -985,12 +1007,13 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k) {
                         if (k >= nk) break;
-                        if (is_f4(BN)) umma_mxf4_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u, tmem_base + SF_COL);
-                        else umma_i8_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kit > 0 || k > 0) ? 1u : 0u);
+                        if (is_f4(BN)) umma_mxf4_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, 1u, tmem_base + SF_COL);
+                        else umma_i8_2sm(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, 1u);
+                        if (fine) BNN_TR(5 + w, tc, 3 + k);
                     }
                     umma_commit_2sm(empty0 + 8 * rc.b);
-                    if (kit == 0) umma_commit_2sm_local(smem_u32(&ctl->started[buf]));
-                    rc.advance(N_ISSUE, STAGES2);
+                    if (fine) BNN_TR(5 + w, tc, 7);
+                    rc.advance(NI2, STAGES2, RM);
                 }
                 umma_commit_2sm(smem_u32(&ctl->acc_full[buf]));
                 BNN_TR(1 + w, tc, 11);

@@ -74,7 +74,6 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         for (int b = 0; b < ACC_BUFS; ++b) {
             mbar_init(smem_u32(&ctl->acc_full[b]), N_ISSUE);                          // one commit from each issuing thread
             mbar_init(smem_u32(&ctl->acc_empty[b]), (PAIR ? 2 : 1) * EPI_WARPS);      // the leader's barrier counts both CTAs' warps
-            mbar_init(smem_u32(&ctl->started[b]), 1);
         }
         ctl->failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -94,16 +93,19 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = ctl->tmem_base;
 
-    if (F4) {   // unit block scales for the 4-bit instruction (see k_umma_i8)
+    {   // zero accumulators (every MMA accumulates, see tmem_zero32); unit block scales for the 4-bit instruction (see k_umma_i8)
         if (warp >= 2 && warp < 6) {
-            const uint32_t v = 0x7f7f7f7fu;
-            asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1};"
-                         ::"r"(tmem_base + SF_COL + ((uint32_t)(32 * (warp & 3)) << 16)), "r"(v) : "memory");
-            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            tmem_zero_all(tmem_base, warp, ACC_BUFS * BN);
+            if (F4) {
+                const uint32_t v = 0x7f7f7f7fu;
+                asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1};"
+                             ::"r"(tmem_base + SF_COL + ((uint32_t)(32 * (warp & 3)) << 16)), "r"(v) : "memory");
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            }
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
-        if (PAIR) cluster_sync_all();                    // the leader's MMAs read the scale columns of both CTAs
+        if (PAIR) cluster_sync_all();                    // the leader's MMAs write the accumulators and read the scale columns of both CTAs
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     }
 
@@ -141,9 +143,6 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             RingCursor ra; ra.start(0, (uint32_t)NA);    // slab ring
             uint32_t sb = 0, bb_i = 0, lapb = 0;         // streamed weights: ring slot, barrier pair, wraps of the barrier ring
             for (uint32_t t = unit; t < (uint32_t)ntiles && ok; t += nunits) {
-#ifdef EXP_NO_LOADS
-                if (t != unit) break;                    // experiment: only the first tile's operands are ever loaded
-#endif
                 const uint32_t tm = t / tn32;
                 const int n0 = (int)((t - tm * tn32) * BN) + n_own;
                 const int tm128 = PAIR ? 2 * (int)tm + (int)rank : (int)tm;      // this CTA's 128 pixels
@@ -193,9 +192,8 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         // does besides the MMAs themselves -- barrier polls, fences, commits: ~250 clocks per slab -- is not hidden by the
         // tensor pipe's queue, it adds to the pipe's time; with a second thread issuing the next slab's twelve MMAs
         // meanwhile it is.  All products are exact, so the order in which the two streams reach the accumulator does not
-        // matter, except that the tile's first (overwriting) K step must be there first: the thread that does not own the
-        // tile's first slab waits once per tile for that step's completion.  In a pair the leader's two threads issue for
-        // both tensor cores (M = 256).
+        // matter: every MMA accumulates into a buffer that the epilogue left at zero.  In a pair the leader's two threads
+        // issue for both tensor cores (M = 256).
         if (lane == 0 && rank == 0) {
             const uint32_t w = (warp == 1) ? 0u : 1u;    // this thread takes the slabs whose running number is w mod 2
             const uint32_t idesc = F4
@@ -218,11 +216,8 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 const uint32_t tmem_d = tmem_base + buf * BN;
                 const bool wait_b = !p.b_resident || tc == 0;
                 const uint32_t g_first = (j + w) & 1u;   // first slab of this tile that is this thread's: 0 or 1
-                if (g_first == 0) {                      // owner of the tile's first slab: the accumulator buffer must be free
-                    if (tc >= ACC_BUFS && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->acc_empty[buf]), ((tc / ACC_BUFS) - 1) & 1)) { conv_fail<PAIR>(ctl, 24); ok = false; break; }
-                } else {
-                    if (!mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->started[buf]), (tc / ACC_BUFS) & 1)) { conv_fail<PAIR>(ctl, 25); ok = false; break; }
-                }
+                // the accumulator buffer must have been read (and zeroed) by the epilogue of the tile before the last
+                if (tc >= ACC_BUFS && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->acc_empty[buf]), ((tc / ACC_BUFS) - 1) & 1)) { conv_fail<PAIR>(ctl, 24); ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 BNN_TR(1 + w, tc, 0);
 #pragma unroll 1
@@ -249,9 +244,8 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                         const uint64_t adesc = aslab + (uint64_t)(dyi * dy_step);
                         const uint64_t bdesc = bdesc0 + (uint64_t)(sb * b_step);
 #pragma unroll
-                        for (int k = 0; k < BK / 32; ++k) mma(adesc + 2 * k, bdesc + 2 * k, tmem_d, (kit > 0 || k > 0) ? 1u : 0u);
+                        for (int k = 0; k < BK / 32; ++k) mma(adesc + 2 * k, bdesc + 2 * k, tmem_d, 1u);
                         if (!p.b_resident) commit(emptyB0 + 8 * bb_i);
-                        if (kit == 0) { if (PAIR) umma_commit_2sm_local(smem_u32(&ctl->started[buf])); else umma_commit(smem_u32(&ctl->started[buf])); }
                     }
                     commit(emptyA0 + 8 * ra.b);                 // the slab's three K steps have been issued
                 }
