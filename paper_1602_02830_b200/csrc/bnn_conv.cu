@@ -282,9 +282,15 @@ extern "C" int bnn_convnet_forward(bnn_ctx *ctx, const bnn_convnet_desc *net, co
         return st;
     }
 
-    // A layer with a multiple of 256 input channels runs on 4-bit operands (e2m1 nibbles, twice the MMA rate and half
-    // the operand bytes; a K step is one tap and 256 channels); the layer before it then writes nibbles instead of bytes.
-    auto on_nibbles = [&](int k) { return k > 0 && k < L && ctx->operand_bits != 8 && (net->layers[k].C_in % 256) == 0; };
+    // A layer with a multiple of 256 input channels, or with exactly 128 where the halo-tile kernel takes it, runs on 4-bit
+    // operands (e2m1 nibbles, twice the MMA rate and half the operand bytes; a K step is one tap and 256 or 128 channels);
+    // the layer before it then writes nibbles instead of bytes.
+    auto on_nibbles = [&](int k) {
+        if (k <= 0 || k >= L || ctx->operand_bits == 8) return false;
+        int64_t hk = H, wk = W;                                      // the layer's input size
+        for (int i = 0; i < k; ++i) if (net->layers[i].pool) { hk /= 2; wk /= 2; }
+        return bnn_umma_conv_f4_takes(ctx, hk, wk, net->layers[k].pool, net->layers[k].C_in);
+    };
     const int8_t *cur8 = nullptr;
     for (int k = 0; k < L; ++k) {
         const bnn_conv_layer_desc &D = net->layers[k];

@@ -41,6 +41,7 @@ int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B,
                   int64_t C_out, int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, int32_t *out_sums,
                   int8_t *out8 = nullptr, int64_t ldo8 = 0, int out_f4 = 0,   // out_f4: out8 receives e2m1 nibbles (ldo8 bytes per pixel)
                   int b_static = 0);                                          // b_static: W8 is not written by the kernel launched just before
+bool bnn_umma_conv_f4_takes(const bnn_ctx *ctx, int64_t H, int64_t W, int pool, int64_t C_in);
 int bnn_umma_conv_f4(bnn_ctx *ctx, const uint8_t *act4, const uint8_t *W4, int64_t B, int64_t H, int64_t W, int64_t C_in,
                      int64_t C_out, int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, uint8_t *out4,
                      int64_t ldo4, int32_t *out_sums = nullptr, int b_static = 0);

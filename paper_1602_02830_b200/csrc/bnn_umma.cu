@@ -73,8 +73,10 @@ __device__ int g_umma_error;                    // 0 = fine; otherwise a code sa
 // Instrumented builds only: clock stamps of CTA 0, [role][tile][slot].
 __device__ long long g_trace[8 * 16 * 16];
 #define BNN_TR(role, tile, slot) do { if (blockIdx.x == 0 && (tile) < 16) g_trace[((role) * 16 + (tile)) * 16 + (slot)] = clock64(); } while (0)
+#define BNN_TR_CLK(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) { g_trace[7 * 256 + 2 * (i)] = clock64(); unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_trace[7 * 256 + 2 * (i) + 1] = (long long)t_; } } while (0)
 #else
 #define BNN_TR(role, tile, slot) do { } while (0)
+#define BNN_TR_CLK(i) do { } while (0)
 #endif
 
 struct UmmaArgs {
@@ -94,8 +96,9 @@ struct UmmaArgs {
     int pool;               // 2x2 max-pool (as OR of the sign bits) before the packed store
     int b_static;           // B (weights) is not written by the kernel launched just before this one
     // halo-tile convolution kernel (k_umma_conv): A stages hold a (TH + 2)-row slab of the input per horizontal tap
-    int a_stage_bytes, n_a_stages;   // bytes of one slab = (TH + 2) * TB * W * 128; slabs in the ring
-    int n_b_stages;         // weight stages of BN x 128 bytes
+    int kbytes;             // k_umma_conv: bytes of channels per pixel and K step: 128 (128-byte swizzle) or 64 (64-byte swizzle)
+    int a_stage_bytes, n_a_stages;   // bytes of one slab = (TH + 2) * TB * W * kbytes; slabs in the ring
+    int n_b_stages;         // weight stages of BN x kbytes bytes
     int b_resident;         // all k_iters weight stages stay in shared memory (this CTA's tiles share their filters)
     int dy_bytes;           // one image row of the slab: TB * W * 128 bytes
     int tap_bytes;          // bytes of one tap in a filter row of the weight matrix (C_in bytes, or C_in / 2 for nibbles)
@@ -134,6 +137,14 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
     d |= (uint64_t)(1024u >> 4) << 32;   // stride byte offset
     d |= 1ull << 46;                      // descriptor version of sm_100
     d |= 2ull << 61;                      // SWIZZLE_128B
+    return d;
+}
+// The same for rows of 64 bytes with the 64-byte swizzle: groups of eight rows 512 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t addr) {
+    uint64_t d = (uint64_t)((addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)(512u >> 4) << 32;
+    d |= 1ull << 46;
+    d |= 4ull << 61;                      // SWIZZLE_64B
     return d;
 }
 __device__ __forceinline__ void umma_i8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
@@ -877,6 +888,7 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();                // 0 = leader of the pair
     const int64_t pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+    BNN_TR_CLK(0);
     const int64_t tiles_m = (p.M + 2 * BM - 1) / (2 * BM);  // 256-row tiles
     const int64_t tiles_n = (p.N + BN - 1) / BN;
     const int64_t ntiles = tiles_m * tiles_n;
@@ -1059,6 +1071,7 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    BNN_TR_CLK(1);
     cluster_sync_all();                                     // nobody leaves while the peer may still read its shared memory
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -1232,16 +1245,17 @@ int get_encode(bnn_ctx *ctx, encode_fn_t *out) {
 }
 
 // 2-D byte tensor rows x kbytes (row pitch ld bytes), box 128 bytes x box_rows, 128-byte swizzle, zero fill outside.
-int make_map(bnn_ctx *ctx, CUtensorMap *map, const void *base, int64_t rows, int64_t kbytes, int64_t ld, int box_rows) {
+// box_k = 64: boxes of 64 bytes with the 64-byte swizzle (the halo-tile convolution's half-width K steps).
+int make_map(bnn_ctx *ctx, CUtensorMap *map, const void *base, int64_t rows, int64_t kbytes, int64_t ld, int box_rows, int box_k = BK) {
     encode_fn_t enc;
     if (int st = get_encode(ctx, &enc)) return st;
     cuuint64_t dims[2] = {(cuuint64_t)kbytes, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)ld};
-    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    cuuint32_t box[2] = {(cuuint32_t)box_k, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, box_k == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { ctx->last_cuda_error = (int)r; return BNN_ERR_CUDA; }
     return BNN_OK;
 }
@@ -1515,16 +1529,16 @@ namespace {
 constexpr size_t SMEM_OPT_IN = 227 * 1024;      // dynamic shared memory a CTA can opt in to on sm_100
 // Activation map with the dimensions ordered (channel byte, column, image, row): a box of {128, W, TB, TH + 2} lands in
 // shared memory as [row][image][column] rows of 128 bytes.  cb = bytes of channels per pixel.
-int make_map_slab(bnn_ctx *ctx, CUtensorMap *map, const void *base, int64_t B, int64_t H, int64_t W, int64_t cb, int TH, int TB) {
+int make_map_slab(bnn_ctx *ctx, CUtensorMap *map, const void *base, int64_t B, int64_t H, int64_t W, int64_t cb, int TH, int TB, int kb) {
     encode_fn_t enc;
     if (int st = get_encode(ctx, &enc)) return st;
     cuuint64_t dims[4] = {(cuuint64_t)cb, (cuuint64_t)W, (cuuint64_t)B, (cuuint64_t)H};
     cuuint64_t strides[3] = {(cuuint64_t)cb, (cuuint64_t)(H * W * cb), (cuuint64_t)(W * cb)};
-    cuuint32_t box[4] = {(cuuint32_t)BK, (cuuint32_t)W, (cuuint32_t)TB, (cuuint32_t)(TH + 2)};
+    cuuint32_t box[4] = {(cuuint32_t)kb, (cuuint32_t)W, (cuuint32_t)TB, (cuuint32_t)(TH + 2)};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(base), dims, strides, box, estr,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, kb == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { ctx->last_cuda_error = (int)r; return BNN_ERR_CUDA; }
     return BNN_OK;
 }
@@ -1579,17 +1593,19 @@ int conv_halo_launch_t(bnn_ctx *ctx, const CUtensorMap &mapA, const CUtensorMap 
 }  // namespace
 
 // Whether the halo-tile kernel takes this layer: slabs of whole 1024-byte swizzle periods per image row of the tile.
-static bool conv_halo_ok(const bnn_ctx *ctx, int64_t W, int TH, int TB) {
+static bool conv_halo_ok(const bnn_ctx *ctx, int64_t W, int TH, int TB, int kb = BK) {
     if (ctx->conv_form == 1 || ctx->drop_loads) return false;
-    return ((TB * W) % 8) == 0 && W <= 256 && TB <= 256 && TH + 2 <= 256 && (size_t)(TH + 2) * TB * W * BK <= 48 * 1024;
+    return ((TB * W) % 8) == 0 && W <= 256 && TB <= 256 && TH + 2 <= 256 && (size_t)(TH + 2) * TB * W * kb <= 48 * 1024;
 }
 
 // act: [B][H][W][cb] bytes (cb = C_in bytes, or C_in / 2 for nibbles; a multiple of 128), Wt: [C_out][9 * cb].  `a` arrives
 // with the outputs, thresholds, pooling and tile geometry filled in.
-static int conv_halo_launch(bnn_ctx *ctx, bool f4, const void *act, const void *Wt, int64_t B, int64_t H, int64_t W, int64_t cb,
-                            int64_t C_out, int TH, int TB, UmmaArgs a, int b_static) {
-    const int c_chunks = (int)(cb / BK);
-    const size_t a_stage = (size_t)(TH + 2) * TB * W * BK;
+// w_pitch: bytes between the filters' rows of Wt.  cb = 64 (128 channels as nibbles): K steps of 64 bytes.
+static int conv_halo_launch(bnn_ctx *ctx, bool f4, const void *act, const void *Wt, int64_t w_pitch, int64_t B, int64_t H, int64_t W,
+                            int64_t cb, int64_t C_out, int TH, int TB, UmmaArgs a, int b_static) {
+    const int kb = cb == 64 ? 64 : BK;
+    const int c_chunks = (int)(cb / kb);
+    const size_t a_stage = (size_t)(TH + 2) * TB * W * kb;
     const size_t avail = SMEM_OPT_IN - 1024 - sizeof(Control);
     // 1. CTA pairs with the tile's filters resident, half of them in each CTA: 256 filters per tile on bytes, 128 on nibbles
     //    (two accumulator buffers and the scale columns must fit the 512 columns of tensor memory).
@@ -1604,12 +1620,12 @@ static int conv_halo_launch(bnn_ctx *ctx, bool f4, const void *act, const void *
         else st = conv_kernel_prepare<128, false, true>(ctx, &max_pairs);
         if (st) return st;
         const int64_t tn = (C_out + bn - 1) / bn;
-        pair = resident = max_pairs > 0 && nb <= B_STAGES_MAX && (size_t)nb * (bn / 2) * BK + 2 * a_stage <= avail && tn <= max_pairs;
+        pair = resident = max_pairs > 0 && nb <= B_STAGES_MAX && (size_t)nb * (bn / 2) * kb + 2 * a_stage <= avail && tn <= max_pairs;
     }
     // 2. otherwise one CTA per tile: resident weights where 128 filters fit, else streamed through a ring
     if (!pair) {
         bn = 128;
-        resident = c_chunks == 1 && 9 * (size_t)128 * BK + 2 * a_stage <= avail && (C_out + 127) / 128 <= ctx->sm_count;
+        resident = c_chunks == 1 && 9 * (size_t)128 * kb + 2 * a_stage <= avail && (C_out + 127) / 128 <= ctx->sm_count;
         if (!resident && C_out > 128) bn = f4 ? 192 : 256;
         nb = resident ? 9 : 4;
         int st = BNN_OK;
@@ -1617,17 +1633,17 @@ static int conv_halo_launch(bnn_ctx *ctx, bool f4, const void *act, const void *
         else st = bn == 128 ? conv_kernel_prepare<128, false, false>(ctx, nullptr) : conv_kernel_prepare<256, false, false>(ctx, nullptr);
         if (st) return st;
     }
-    const size_t b_stage = (size_t)(pair ? bn / 2 : bn) * BK, b_bytes = (size_t)nb * b_stage;
+    const size_t b_stage = (size_t)(pair ? bn / 2 : bn) * kb, b_bytes = (size_t)nb * b_stage;
     int na = (int)((avail - b_bytes) / a_stage);
     na = na > 4 ? 4 : na;
     if (na < 2) return BNN_ERR_INVALID_ARG;
     CUtensorMap mapA, mapB;
-    if (int st = make_map_slab(ctx, &mapA, act, B, H, W, cb, TH, TB)) return st;
-    if (int st = make_map(ctx, &mapB, Wt, C_out, 9 * cb, 9 * cb, (int)(b_stage / BK))) return st;
+    if (int st = make_map_slab(ctx, &mapA, act, B, H, W, cb, TH, TB, kb)) return st;
+    if (int st = make_map(ctx, &mapB, Wt, C_out, 9 * cb, w_pitch, (int)(b_stage / kb), kb)) return st;
     a.conv = 1; a.H = (int)H; a.W = (int)W; a.TH = TH; a.TB = TB; a.c_chunks = c_chunks;
-    a.k_iters = 9 * c_chunks; a.k_last = BK / 32;
+    a.k_iters = 9 * c_chunks; a.k_last = kb / 32; a.kbytes = kb;
     a.a_stage_bytes = (int)a_stage; a.n_a_stages = na; a.n_b_stages = nb; a.b_resident = resident ? 1 : 0;
-    a.dy_bytes = (int)(TB * W * BK); a.tap_bytes = (int)cb; a.perm = TB > 1 ? 1 : 0; a.b_static = b_static;
+    a.dy_bytes = (int)(TB * W * kb); a.tap_bytes = (int)cb; a.perm = TB > 1 ? 1 : 0; a.b_static = b_static;
     const int64_t tn = (C_out + bn - 1) / bn;
     const int64_t tile_m = pair ? 2 * BM : BM, tiles = ((a.M + tile_m - 1) / tile_m) * tn;
     if (tiles >= (int64_t(1) << 31)) return BNN_ERR_INVALID_ARG;
@@ -1663,7 +1679,7 @@ int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B,
         h.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BM >> 4) << 24);
         h.C = out_sums; h.ldc = C_out; h.out = out_bits; h.ldo = (C_out + 31) / 32; h.thr = thr; h.flip = flip;
         h.out8 = out8; h.ldo8 = ldo8; h.out_f4 = out_f4; h.pool = pool;
-        return conv_halo_launch(ctx, false, act8, W8, B, H, W, C_in, C_out, TH, TB, h, b_static);
+        return conv_halo_launch(ctx, false, act8, W8, bnn_umma_operand_ld(9 * C_in), B, H, W, C_in, C_out, TH, TB, h, b_static);
     }
     CUtensorMap mapA, mapB;
     const int bn = umma_tile_n(C_out);
@@ -1697,21 +1713,29 @@ int bnn_umma_conv(bnn_ctx *ctx, const int8_t *act8, const int8_t *W8, int64_t B,
 // (C_in % 256 == 0, so that a K step is one tap and 256 channels = 128 bytes per pixel); pixels outside the image arrive
 // as zero nibbles (+0.0).  Outputs: packed signs and / or nibbles for the next layer (out4, pitch ldo4 bytes per pixel),
 // or the int32 sums (not with pooling).
+// Whether the 4-bit engine takes a layer with C_in input maps: whole 128-byte channel slices (256 maps) in either form
+// of the kernel, or exactly 128 maps (64 bytes per pixel) as half-width K steps of the halo-tile kernel.
+bool bnn_umma_conv_f4_takes(const bnn_ctx *ctx, int64_t H, int64_t W, int pool, int64_t C_in) {
+    if (C_in > 0 && (C_in % (2 * BK)) == 0) return true;
+    int TH, TB;
+    return C_in == BK && bnn_umma_conv_tiling(H, W, pool, &TH, &TB) && conv_halo_ok(ctx, W, TH, TB, 64);
+}
+
 int bnn_umma_conv_f4(bnn_ctx *ctx, const uint8_t *act4, const uint8_t *W4, int64_t B, int64_t H, int64_t W, int64_t C_in,
                      int64_t C_out, int pool, const int32_t *thr, const uint32_t *flip, uint32_t *out_bits, uint8_t *out4,
                      int64_t ldo4, int32_t *out_sums, int b_static) {
     int TH, TB;
-    if (!bnn_umma_conv_tiling(H, W, pool, &TH, &TB) || (C_in % (2 * BK)) != 0 || (pool && (out_sums || !out_bits)) ||
+    if (!bnn_umma_conv_tiling(H, W, pool, &TH, &TB) || !bnn_umma_conv_f4_takes(ctx, H, W, pool, C_in) || (pool && (out_sums || !out_bits)) ||
         (!out_bits && !out4 && !out_sums) || ((out_bits || out4) && !thr))
         return BNN_ERR_INVALID_ARG;
     if (!bnn_aligned16(act4) || !bnn_aligned16(W4)) return BNN_ERR_ALIGNMENT;
-    if (conv_halo_ok(ctx, W, TH, TB)) {
+    if (conv_halo_ok(ctx, W, TH, TB, C_in == BK ? 64 : BK)) {
         UmmaArgs h{};
         h.wait_ns = ctx->wait_limit_ns;
         h.M = B * H * W; h.N = C_out;
         h.C = out_sums; h.ldc = C_out; h.out = out_bits; h.ldo = (C_out + 31) / 32; h.thr = thr; h.flip = flip;
         h.out8 = reinterpret_cast<int8_t *>(out4); h.ldo8 = ldo4; h.out_f4 = 1; h.pool = pool;
-        return conv_halo_launch(ctx, true, act4, W4, B, H, W, C_in / 2, C_out, TH, TB, h, b_static);
+        return conv_halo_launch(ctx, true, act4, W4, bnn_umma_operand_ld_f4(9 * C_in), B, H, W, C_in / 2, C_out, TH, TB, h, b_static);
     }
     CUtensorMap mapA, mapB;
     // CTA pairs (each CTA its own 128 pixels and half of the tile's filters) cut the operand bytes per CTA by 30 %, but

@@ -37,7 +37,7 @@ template <int BN, bool F4, bool PAIR> struct ConvCfg {
     static constexpr int EPI_WARPS = (BN == 192) ? 8 : 16;
     static constexpr int MMA_WARP_B = 2 + EPI_WARPS;                    // the second MMA-issuing warp (the first is warp 1)
     static constexpr int NTHREADS = 64 + 32 * EPI_WARPS + 32;
-    static constexpr uint32_t B_STAGE = (PAIR ? BN / 2 : BN) * BK;      // a CTA of a pair keeps half of the tile's filters
+    static constexpr uint32_t B_ROWS = PAIR ? BN / 2 : BN;              // a CTA of a pair keeps half of the tile's filters
     static constexpr uint32_t TMEM_COLS = F4 ? 512 : (2 * BN <= 256 ? 256 : 512);
 };
 
@@ -46,7 +46,11 @@ __global__ void __launch_bounds__((ConvCfg<BN, F4, PAIR>::NTHREADS), 1)
 k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const UmmaArgs p) {
     using C = ConvCfg<BN, F4, PAIR>;
     constexpr int EPI_WARPS = C::EPI_WARPS, MMA_WARP_B = C::MMA_WARP_B;
-    constexpr uint32_t B_STAGE = C::B_STAGE, TMEM_COLS = C::TMEM_COLS;
+    constexpr uint32_t TMEM_COLS = C::TMEM_COLS;
+    // K step: 128 bytes of channels per pixel (128-byte swizzle), or 64 bytes (64-byte swizzle: 128 maps as nibbles, two
+    // MMAs per step); the vertical-tap offset TB * W * KB is a whole number of swizzle periods (8 rows) in both
+    const int KB = p.kbytes;
+    const uint32_t B_STAGE = C::B_ROWS * (uint32_t)KB;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *slabs = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t A_STAGE = (uint32_t)p.a_stage_bytes;
@@ -63,6 +67,7 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     const int64_t tiles_n = (p.N + BN - 1) / BN;
     const int64_t ntiles = tiles_m * tiles_n;
     const int groups = p.k_iters / 3;                    // slabs per tile: 3 horizontal taps x channel slices
+    BNN_TR_CLK(0);
     const int RB = p.b_resident ? NB : 3 * NB;           // barrier pairs of the weight stages
 
     if (threadIdx.x == 0) {
@@ -135,7 +140,7 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                         for (int dyi = 0; dyi < 3; ++dyi, ++kit) {
                             const uint32_t bar = smem_u32(&ctl->full_b[kit]);
                             if (rank == 0) mbar_expect_tx(bar, b_tx);
-                            load_b(smem_u32(wts + (size_t)kit * B_STAGE), (3 * dyi + dxi) * p.tap_bytes + cc * BK, n0_first, bar);
+                            load_b(smem_u32(wts + (size_t)kit * B_STAGE), (3 * dyi + dxi) * p.tap_bytes + cc * KB, n0_first, bar);
                         }
                 b_loaded = true;
             }
@@ -161,14 +166,14 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                         const uint32_t bar = smem_u32(&ctl->full[ra.b]);
                         if (rank == 0) mbar_expect_tx(bar, a_tx);
                         // dimensions of the map: channel byte, column, image, row
-                        load_a(smem_u32(slabs + (size_t)ra.slot((uint32_t)NA) * A_STAGE), cc * BK, dxi - 1, b0, y0 - 1, bar);
+                        load_a(smem_u32(slabs + (size_t)ra.slot((uint32_t)NA) * A_STAGE), cc * KB, dxi - 1, b0, y0 - 1, bar);
                         ra.advance(1, (uint32_t)NA);
                         for (int dyi = 0; dyi < 3; ++dyi, ++kit) {
                             if (p.b_resident) {
                                 if (b_loaded) continue;
                                 const uint32_t bb = smem_u32(&ctl->full_b[kit]);
                                 if (rank == 0) mbar_expect_tx(bb, b_tx);
-                                load_b(smem_u32(wts + (size_t)kit * B_STAGE), (3 * dyi + dxi) * p.tap_bytes + cc * BK, n0, bb);
+                                load_b(smem_u32(wts + (size_t)kit * B_STAGE), (3 * dyi + dxi) * p.tap_bytes + cc * KB, n0, bb);
                             } else {
                                 if (lapb > 0 || bb_i >= (uint32_t)NB) {      // the stage NB earlier must have been multiplied
                                     const uint32_t pb_i = bb_i >= (uint32_t)NB ? bb_i - (uint32_t)NB : bb_i + (uint32_t)(RB - NB);
@@ -177,7 +182,7 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                                 }
                                 const uint32_t bb = smem_u32(&ctl->full_b[bb_i]);
                                 if (rank == 0) mbar_expect_tx(bb, b_tx);
-                                load_b(smem_u32(wts + (size_t)sb * B_STAGE), (3 * dyi + dxi) * p.tap_bytes + cc * BK, n0, bb);
+                                load_b(smem_u32(wts + (size_t)sb * B_STAGE), (3 * dyi + dxi) * p.tap_bytes + cc * KB, n0, bb);
                                 if (++sb == (uint32_t)NB) sb = 0;
                                 if (++bb_i == (uint32_t)RB) { bb_i = 0; ++lapb; }
                             }
@@ -206,7 +211,9 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             auto commit = [&](uint32_t bar) { if (PAIR) umma_commit_2sm(bar); else umma_commit(bar); };   // in a pair: to both CTAs
             const uint32_t fullA0 = smem_u32(&ctl->full[0]), emptyA0 = smem_u32(&ctl->empty[0]);
             const uint32_t fullB0 = smem_u32(&ctl->full_b[0]), emptyB0 = smem_u32(&ctl->empty_b[0]);
-            const uint64_t adesc0 = smem_desc_sw128(smem_u32(slabs)), bdesc0 = smem_desc_sw128(smem_u32(wts));
+            const uint64_t adesc0 = KB == 64 ? smem_desc_sw64(smem_u32(slabs)) : smem_desc_sw128(smem_u32(slabs));
+            const uint64_t bdesc0 = KB == 64 ? smem_desc_sw64(smem_u32(wts)) : smem_desc_sw128(smem_u32(wts));
+            const int n_mma = KB >> 5;                   // MMAs (32 bytes of K each) per K step
             const uint32_t a_step = A_STAGE >> 4, b_step = B_STAGE >> 4, dy_step = (uint32_t)p.dy_bytes >> 4;
             uint32_t tc = 0;
             uint32_t j = 0;                              // running number of the tile's first slab (over all tiles of this CTA)
@@ -244,7 +251,7 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                         const uint64_t adesc = aslab + (uint64_t)(dyi * dy_step);
                         const uint64_t bdesc = bdesc0 + (uint64_t)(sb * b_step);
 #pragma unroll
-                        for (int k = 0; k < BK / 32; ++k) mma(adesc + 2 * k, bdesc + 2 * k, tmem_d, 1u);
+                        for (int k = 0; k < BK / 32; ++k) { if (k >= n_mma) break; mma(adesc + 2 * k, bdesc + 2 * k, tmem_d, 1u); }
                         if (!p.b_resident) commit(emptyB0 + 8 * bb_i);
                     }
                     commit(emptyA0 + 8 * ra.b);                 // the slab's three K steps have been issued
@@ -279,6 +286,7 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    BNN_TR_CLK(1);
     if (PAIR) cluster_sync_all();                        // nobody leaves while the partner may still signal its barriers
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");

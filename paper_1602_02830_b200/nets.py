@@ -72,7 +72,7 @@ def prepare_convnet(ctx, layers, expand_weights: bool = True):
             # the same bits viewed as Cout rows of 9*Cin: re-pack with a legal leading dimension, then expand
             rows = ctx.pack_signs(_dev(ctx, flat, torch.int8), pack_along=0)
             d["W8"] = ctx.expand_signs(rows, Cout, 9 * Cin)
-            if i > 0 and Cin % 256 == 0:                       # layers the library runs on 4-bit operands
+            if i > 0 and Cin % 128 == 0:                       # layers the library may run on 4-bit operands
                 d["W4"] = ctx.expand_signs_f4(rows, Cout, 9 * Cin)
         out.append(d)
     return out
