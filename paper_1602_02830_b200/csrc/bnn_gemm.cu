@@ -100,6 +100,14 @@ __global__ void __launch_bounds__(256, (RSMAX <= 16) ? 3 : 1) k_skinny(const Ski
             *reinterpret_cast<uint4 *>(Ss + (int64_t)r * Kw4 + 4 * q) = v;
         }
     }
+    // thresholds and flip word of the CTA's 32 outputs: requested now, in parallel, so that the packing loop at the end
+    // reads shared memory (as 32 dependent global loads of one thread they were half of a batch-1 call's time)
+    __shared__ int32_t thr_s[32];
+    __shared__ uint32_t flip_s;
+    if (MODE == 0 && p.out) {
+        if (tid < 32) thr_s[tid] = (l0 + tid < p.RL) ? p.thr[l0 + tid] : 0;
+        if (tid == 32) flip_s = p.flip ? p.flip[blockIdx.x] : 0u;
+    }
     // output scores: per output s the affine form of BatchNorm, a = gamma / sqrt(var + eps), b = beta - mean * a, once
     // per CTA in double (the square root and the division are the expensive part)
     __shared__ double bn_a[32], bn_b[32];
@@ -168,10 +176,11 @@ __global__ void __launch_bounds__(256, (RSMAX <= 16) ? 3 : 1) k_skinny(const Ski
         if (p.out) {
             if (tid < p.RS) {
                 uint32_t word = 0u;
-                const uint32_t fw = p.flip ? p.flip[blockIdx.x] : 0u;
+                const uint32_t fw = flip_s;
+#pragma unroll
                 for (int lc = 0; lc < 32; ++lc) {
                     if (l0 + lc < p.RL) {
-                        const uint32_t q = res[lc * RSMAX + tid] >= p.thr[l0 + lc];
+                        const uint32_t q = res[lc * RSMAX + tid] >= thr_s[lc];
                         word |= ((q ^ (fw >> lc)) & 1u) << lc;
                     }
                 }
