@@ -386,7 +386,7 @@ def main():
                                                     "operands already in the tensor engine's format, as inside the step)" % kernel_name,
                       "achieved": dense_ops / (kernel_ms / 1e3) / 1e12, "peak": tensor_peak, "unit": "TFLOP/s",
                       "frac": dense_ops / (kernel_ms / 1e3) / 1e12 / tensor_peak,
-                      "traffic": 28962048 if args.operand_bits == 4 else 60967424,
+                      "traffic": 28969984 if args.operand_bits == 4 else 60967424,
                       "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of this kernel, one launch: "
                                         "profiles/k_umma_i8_mlp_batch10000.md (not re-measured by this run)",
                       "peak_kind": "2 ops per MAC; peak = %.0f x measured bf16 burst %.1f TFLOP/s (NOMINAL %s:bf16 ratio, not a "
