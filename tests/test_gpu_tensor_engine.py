@@ -272,13 +272,15 @@ def test_mlp_forward_unaligned_input_falls_back_cleanly(ctx):
     del ws
 
 
-@pytest.mark.parametrize("channels", [(128, 128, 256, 128), (128, 256, 256, 512, 256)])
+@pytest.mark.parametrize("channels,hw,B", [((128, 128, 256, 128), 32, 20), ((128, 256, 256, 512, 256), 32, 20),
+                                           ((128, 128, 256, 128), 16, 256), ((128, 128, 128, 128, 256, 256), 16, 256)])
 @pytest.mark.parametrize("pre_expanded", [True, False])
-def test_convnet_forward_chained_on_tensor_engine(ctx, pre_expanded, channels):
+def test_convnet_forward_chained_on_tensor_engine(ctx, pre_expanded, channels, hw, B):
     """bnn_convnet_forward with every layer on the tensor engine: +-1 values handed from layer to layer (pooled and not)
-    as bytes, or as 4-bit nibbles into layers with a multiple of 256 input channels (the second list has three of
-    those in a row: not pooled, pooled, not pooled)."""
-    B, hw = 20, 32
+    as 4-bit nibbles: into layers with a multiple of 256 input channels (the second list has three of those in a row: not
+    pooled, pooled, not pooled) and into layers with 128 (half-width K steps, rows of 64 bytes; the third list has them at
+    every image size down to 4 x 4, where one tile holds several images).  The batches keep every layer above the sizes
+    from which the engine takes it."""
     case = wl.convnet_case(batch=B, hw=hw, channels=channels, seed=9)
     want = oracle.convnet_forward(case["X"], case["layers"])
     net = nets.prepare_convnet(ctx, case["layers"], expand_weights=pre_expanded)
