@@ -449,8 +449,6 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
     }
     const int tr_role = (et == 0) ? 3 : ((et == EPI_THREADS - 32) ? 4 : -1);
     if (tr_role >= 0) BNN_TR(tr_role, tc, 0);
-    // the epilogue warps only: staged thresholds visible; previous tile's pooling words no longer read
-    if (p.thr) asm volatile("bar.sync %0, %1;" ::"n"(BAR_A), "n"(EPI_THREADS) : "memory");
     if (tr_role >= 0) BNN_TR(tr_role, tc, 1);
     const bool have_next = p.thr && n0_next >= 0 && !same_next;      // (same_next: the thresholds already staged stay valid)
     int32_t next_thr = 0x7fffffff;
@@ -467,6 +465,7 @@ __device__ __forceinline__ void epilogue_tile(Control *ctl, const UmmaArgs &p, u
     // MMA-issuing threads, which share those schedulers, needed three times as long per instruction: a tile of nine
     // short K steps then ran at 40 % of the tensor pipe's rate.
     if (et < 32 && ok && !mbar_wait(ctl, p.wait_ns, smem_u32(&ctl->acc_full[buf]), acc_parity)) { fail(ctl, 3); ok = false; }
+    // (the same barrier makes the staged thresholds visible and says that nobody reads the previous tile's pooling words)
     asm volatile("bar.sync %0, %1;" ::"n"(BAR_B), "n"(EPI_THREADS) : "memory");
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (tr_role >= 0) BNN_TR(tr_role, tc, 2);

@@ -270,13 +270,18 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         uint32_t tc = 0;
         bool ok = true;
         const uint32_t tn = (uint32_t)tiles_n, nt = (uint32_t)ntiles;
+        int64_t n0_prev = -2;                            // filter block whose thresholds the other slot holds
         for (uint32_t t = unit; t < nt; t += nunits, ++tc) {
             const uint32_t buf = tc & 1;
             const uint32_t tm_i = t / tn;
             const int64_t m0 = (int64_t)tm_i * TILE_M + rank * BM, n0 = (int64_t)(t - tm_i * tn) * BN;
             const uint32_t t2 = t + nunits;
             const int64_t n0_next = (t2 < nt) ? (int64_t)(t2 % tn) * BN : -1;
-            epilogue_tile<BN, F4, EPI_WARPS>(ctl, p, tmem_base, buf, tc, m0, n0, n0_next, q, half, lane, et, ok, tc == 0, (tc / ACC_BUFS) & 1, buf ^ 1u);
+            // the other slot was staged for the tile before this one: with resident weights every tile of a CTA has the same
+            // filters, and nothing is fetched or staged after the first two tiles
+            epilogue_tile<BN, F4, EPI_WARPS>(ctl, p, tmem_base, buf, tc, m0, n0, n0_next, q, half, lane, et, ok, tc == 0, (tc / ACC_BUFS) & 1, buf ^ 1u,
+                                             n0_next == n0_prev);
+            n0_prev = n0;
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) { if (PAIR) mbar_arrive_cta0(smem_u32(&ctl->acc_empty[buf])); else mbar_arrive(smem_u32(&ctl->acc_empty[buf])); }
