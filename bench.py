@@ -236,6 +236,7 @@ def main():
     sampler = ClockSampler(local) if rank == 0 else None
     if sampler:
         sampler.start()
+        time.sleep(0.15)                     # nvidia-smi needs ~0.1 s before its first sample
     times = timed_steps(step_fn, args.steps, args.warmup)
     total_ms = sum(times)
     # the clock record belongs to the timed region above; the poller is stopped before the end-to-end loop because its
@@ -260,6 +261,11 @@ def main():
         soak = {"steps": n_soak, "seconds": e0.elapsed_time(e1) / 1e3, "ms_per_step": soak_ms,
                 "images_per_s": BATCH / (soak_ms / 1e3), "clocks": sampler2.stop(),
                 "note": "back to back, working set stays in L2 (no flush between steps)"}
+
+    if clocks is not None and clocks.get("sm_mhz") is None and soak is not None and soak["clocks"].get("sm_mhz") is not None:
+        # the counted region (a few milliseconds) fell between two samples: the record of the soak (the same step, back to
+        # back, right after it) stands in and says so
+        clocks = dict(soak["clocks"], source="soak: the counted region was shorter than one sampling period")
 
     # ---- end to end: pinned host buffers, copies inside the timed region
     Xh = torch.from_numpy(case["X"]).pin_memory()
