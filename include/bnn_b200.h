@@ -137,6 +137,17 @@ BNN_API int bnn_set_wait_limit_ns(bnn_ctx *ctx, uint64_t ns);
  * launched through this context run in their single-SM form with a producer that requests no operands, so their
  * consumers' waits run into the limit.  Outputs of such calls are undefined.  on = 0 restores normal operation. */
 BNN_API int bnn_debug_drop_loads(bnn_ctx *ctx, int on);
+/* Test hook, host only (no context, no GPU): where stage number `stage` (0, 1, 2, ... in the order a CTA's producer fills
+ * them) of a tensor-engine operand ring of `slots` slots lives.  The kernels guard every slot with TWO barrier pairs, used
+ * alternately, so that each barrier has a single consuming thread when two threads issue alternate stages: stage G uses
+ * slot G mod slots, barrier pair G mod (2 slots), and waits for phase parity (G div (2 slots)) mod 2.
+ * Outputs: the stage's slot, barrier pair and parity; whether an earlier stage used the slot (reuses) and, if so, the
+ * barrier pair and parity of that stage (stage - slots), which the producer waits for before refilling; and the barrier
+ * pair and parity after advancing by `step` stages (1 <= step <= 2 slots), as a thread that takes every step-th stage does.
+ * BNN_ERR_INVALID_ARG for slots = 0, step out of range or a null pointer. */
+BNN_API int bnn_debug_ring_position(uint32_t stage, uint32_t slots, uint32_t step, uint32_t *slot, uint32_t *barrier,
+                                    uint32_t *parity, int32_t *reuses, uint32_t *prev_barrier, uint32_t *prev_parity,
+                                    uint32_t *next_barrier, uint32_t *next_parity);
 /* Synchronises the context's stream and returns BNN_ERR_DEVICE_STATUS if a kernel gave up on one of its
  * bounded waits since the last call (its outputs are then undefined), BNN_OK otherwise. */
 BNN_API int bnn_device_status(bnn_ctx *ctx);

@@ -29,7 +29,7 @@ EXPORTS = (
     "bnn_expanded_bytes", "bnn_expand_signs", "bnn_baseline_gemm_f32", "bnn_convnet_workspace_bytes",
     "bnn_convnet_forward", "bnn_set_operand_bits", "bnn_expanded_ld_f4",
     "bnn_expanded_bytes_f4", "bnn_expand_signs_f4", "bnn_binary_dense_expanded", "bnn_set_wait_limit_ns",
-    "bnn_debug_drop_loads", "bnn_set_conv_form", "bnn_measure_pipe_rates", "bnn_last_tensor_kernel", "bnn_set_conv_filter_repetition",
+    "bnn_debug_drop_loads", "bnn_debug_ring_position", "bnn_set_conv_form", "bnn_measure_pipe_rates", "bnn_last_tensor_kernel", "bnn_set_conv_filter_repetition",
     "bnn_filter_repetition_workspace_bytes", "bnn_filter_repetition_count",
 )
 
@@ -88,6 +88,8 @@ def lib() -> ctypes.CDLL:
         L.bnn_set_operand_bits.argtypes = [vp, c_int]
         L.bnn_set_wait_limit_ns.argtypes = [vp, ctypes.c_uint64]
         L.bnn_debug_drop_loads.argtypes = [vp, c_int]
+        L.bnn_debug_ring_position.argtypes = [ctypes.c_uint32] * 3 + [vp] * 8
+        L.bnn_debug_ring_position.restype = c_int
         L.bnn_set_conv_form.argtypes = [vp, c_int]
         L.bnn_measure_pipe_rates.argtypes = [vp, vp, c_size_t, POINTER(c_double), POINTER(c_double), POINTER(c_double)]
         L.bnn_last_tensor_kernel.argtypes = [vp]
@@ -404,6 +406,16 @@ class Context:
         self._ck(lib().bnn_mlp_forward_host(self._h, ctypes.byref(desc), _ptr(X_host), X_host.stride(0), batch,
                                             _ptr(scores_host), n_out), "bnn_mlp_forward_host")
         return scores_host
+
+
+def debug_ring_position(stage: int, slots: int, step: int = 1) -> dict:
+    """bnn_debug_ring_position: host-only view of the operand-ring arithmetic of the tensor-engine kernels."""
+    o = [ctypes.c_uint32() for _ in range(3)] + [ctypes.c_int32()] + [ctypes.c_uint32() for _ in range(4)]
+    st = lib().bnn_debug_ring_position(stage, slots, step, *[ctypes.byref(x) for x in o])
+    if st:
+        raise BnnError(st, "bnn_debug_ring_position")
+    keys = ("slot", "barrier", "parity", "reuses", "prev_barrier", "prev_parity", "next_barrier", "next_parity")
+    return {k: int(v.value) for k, v in zip(keys, o)}
 
 
 def fold_batchnorm(gamma, beta, mean, var, eps: float, x_max: int):

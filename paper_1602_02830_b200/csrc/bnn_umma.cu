@@ -266,14 +266,14 @@ struct RingCursor {
     uint32_t b, lap;                 // barrier pair of the next stage; how often the barrier ring has wrapped
     // M: barrier pairs per slot (2 for two consumer threads that alternate; a multiple of the number of threads that
     // take the stages in turn, so that G % (M S) fixes the thread)
-    __device__ __forceinline__ void start(uint32_t G, uint32_t S, uint32_t M = 2) { b = G % (M * S); lap = G / (M * S); }
-    __device__ __forceinline__ uint32_t slot(uint32_t S) const { uint32_t x = b; while (x >= S) x -= S; return x; }
-    __device__ __forceinline__ uint32_t parity() const { return lap & 1u; }
+    __host__ __device__ __forceinline__ void start(uint32_t G, uint32_t S, uint32_t M = 2) { b = G % (M * S); lap = G / (M * S); }
+    __host__ __device__ __forceinline__ uint32_t slot(uint32_t S) const { uint32_t x = b; while (x >= S) x -= S; return x; }
+    __host__ __device__ __forceinline__ uint32_t parity() const { return lap & 1u; }
     // the stage that used this slot before (S stages earlier): whether there is one, its barrier pair and phase parity
-    __device__ __forceinline__ bool reuses(uint32_t S) const { return lap > 0 || b >= S; }
-    __device__ __forceinline__ uint32_t prev_bar(uint32_t S, uint32_t M = 2) const { return b >= S ? b - S : b + (M - 1) * S; }
-    __device__ __forceinline__ uint32_t prev_parity(uint32_t S) const { return (b >= S ? lap : lap - 1u) & 1u; }
-    __device__ __forceinline__ void advance(uint32_t n, uint32_t S, uint32_t M = 2) { b += n; if (b >= M * S) { b -= M * S; ++lap; } }   // n <= M S
+    __host__ __device__ __forceinline__ bool reuses(uint32_t S) const { return lap > 0 || b >= S; }
+    __host__ __device__ __forceinline__ uint32_t prev_bar(uint32_t S, uint32_t M = 2) const { return b >= S ? b - S : b + (M - 1) * S; }
+    __host__ __device__ __forceinline__ uint32_t prev_parity(uint32_t S) const { return (b >= S ? lap : lap - 1u) & 1u; }
+    __host__ __device__ __forceinline__ void advance(uint32_t n, uint32_t S, uint32_t M = 2) { b += n; if (b >= M * S) { b -= M * S; ++lap; } }   // n <= M S
 };
 
 // 8 sign bits -> 8 e2m1 nibbles (+1.0 = 0x2, -1.0 = 0xa); bit i lands in nibble i.
@@ -1804,6 +1804,24 @@ extern "C" BNN_API int bnn_trace_read(long long *host, int clear) {
     return BNN_OK;
 }
 #endif
+
+// Host-side view of the ring arithmetic the kernels use (RingCursor), for tests without a GPU.
+extern "C" int bnn_debug_ring_position(uint32_t stage, uint32_t slots, uint32_t step, uint32_t *slot, uint32_t *barrier,
+                                       uint32_t *parity, int32_t *reuses, uint32_t *prev_barrier, uint32_t *prev_parity,
+                                       uint32_t *next_barrier, uint32_t *next_parity) {
+    if (slots == 0 || step == 0 || step > 2 * slots || !slot || !barrier || !parity || !reuses || !prev_barrier || !prev_parity ||
+        !next_barrier || !next_parity)
+        return BNN_ERR_INVALID_ARG;
+    RingCursor rc;
+    rc.start(stage, slots);
+    *slot = rc.slot(slots); *barrier = rc.b; *parity = rc.parity();
+    *reuses = rc.reuses(slots) ? 1 : 0;
+    *prev_barrier = rc.reuses(slots) ? rc.prev_bar(slots) : 0u;
+    *prev_parity = rc.reuses(slots) ? rc.prev_parity(slots) : 0u;
+    rc.advance(step, slots);
+    *next_barrier = rc.b; *next_parity = rc.parity();
+    return BNN_OK;
+}
 
 extern "C" int bnn_device_status(bnn_ctx *ctx) {
     if (!ctx) return BNN_ERR_INVALID_ARG;

@@ -144,3 +144,44 @@ def test_test_side_packer_roundtrip():
     p = np_pack_pm1(x, 4)
     assert p.shape == (5, 4) and np.array_equal(np_unpack_pm1(p, 70), x) and padding_is_zero(p, 70)
     assert np_pack_pm1(np.array([[1, -1, 1]]))[0, 0] == 0b101
+
+
+@pytest.mark.parametrize("slots", [2, 3, 4, 5, 6, 7])
+def test_operand_ring_gives_every_barrier_one_consumer(slots):
+    """Ring arithmetic of the tensor-engine kernels, on the host.  Two threads take alternate stages; a wait on a phase
+    parity is only right while the waiter is at most one phase ahead of its barrier, which holds when every barrier is
+    waited on by ONE thread in phase order (that thread's own previous use is the phase before).  With one barrier per
+    slot and an odd number of slots the uses of a barrier alternate between the threads; with two barrier pairs per slot
+    they never do."""
+    build.build()
+    consumer_of, producer_of, last_phase = {}, {}, {}
+    for G in range(0, 20 * slots + 3):
+        r = binding.debug_ring_position(G, slots, 2)
+        assert r["slot"] == G % slots
+        assert r["barrier"] == G % (2 * slots) and r["parity"] == (G // (2 * slots)) % 2
+        # one consuming thread (stage parity) per barrier, phases in order
+        assert consumer_of.setdefault(r["barrier"], G % 2) == G % 2
+        phase = G // (2 * slots)
+        assert last_phase.get(r["barrier"], -1) == phase - 1
+        last_phase[r["barrier"]] = phase
+        # the producer refills a slot after the stage `slots` earlier was consumed: that stage's barrier and parity
+        assert r["reuses"] == (1 if G >= slots else 0)
+        if G >= slots:
+            e = binding.debug_ring_position(G - slots, slots, 1)
+            assert (r["prev_barrier"], r["prev_parity"]) == (e["barrier"], e["parity"])
+            # with two producer threads on alternate stages, each "empty" barrier also has one waiting thread
+            assert producer_of.setdefault(r["prev_barrier"], G % 2) == G % 2
+        # advancing by the thread's stride lands where a fresh start would
+        n = binding.debug_ring_position(G + 2, slots, 1)
+        assert (r["next_barrier"], r["next_parity"]) == (n["barrier"], n["parity"])
+    # the flawed layout for comparison: one barrier per slot, odd ring -> consecutive uses of a barrier change hands
+    if slots % 2 == 1:
+        users = [G % 2 for G in range(0, 4 * slots) if G % slots == 0]
+        assert users[0] != users[1]
+
+
+def test_operand_ring_position_rejects_bad_arguments():
+    build.build()
+    for args in ((0, 0, 1), (0, 3, 0), (0, 3, 7)):
+        with pytest.raises(binding.BnnError):
+            binding.debug_ring_position(*args)
