@@ -298,7 +298,7 @@ def main():
                                                        out=act_out), min(args.steps, 50), 3)
     # ... and the tensor kernel of that layer by itself, on operands that are already expanded (what runs inside the step,
     # where the weights were expanded once and the previous layer wrote the activations in operand format)
-    kernel_ms, kernel_name = None, None
+    kernel_ms, kernel_name, kernel_clock = None, None, (None, None)
     if tensor_step:
         bits = args.operand_bits
         expand = ctx.expand_signs_f4 if bits == 4 else ctx.expand_signs
@@ -308,6 +308,7 @@ def main():
                                                               SIZES[2], SIZES[1]), min(args.steps, 50), 3)
         kernel_ms = sum(kernel_times) / len(kernel_times)
         kernel_name = ctx.last_tensor_kernel()
+        kernel_clock = ctx.last_tensor_kernel_clock()      # (SM MHz inside the last launch, us its first CTA lived)
         del A_exp, W_exp
     first = net["layers"][0]
     first_times = timed_steps(lambda: ctx.first_layer_bitplanes(X, first["Wp"], BATCH, SIZES[1], SIZES[0], thr=first["thr"],
@@ -402,6 +403,9 @@ def main():
                       "probe_rate_note": "8857 TOPS = kind::mxf4 with resident operands, all SMs, measured once on this pool "
                                          "(profiles/pipe_rates_sm100.md)",
                       "ms_per_launch": kernel_ms,
+                      "sm_mhz_in_kernel": kernel_clock[0], "us_in_kernel_cta0": kernel_clock[1],
+                      "sm_mhz_note": "clock64 against %globaltimer inside the last timed launch (bnn_last_tensor_kernel_clock): the "
+                                     "clock the kernel ran at, as opposed to the maximum that nvidia-smi samples around it",
                       "fused_call": {"what": "bnn_binary_dense from packed operands: two expansion kernels + the same kernel",
                                      "ms": dense_ms, "achieved": dense_ach, "frac": dense_ach / tensor_peak}}
                      if tensor_step else

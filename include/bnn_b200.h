@@ -313,6 +313,11 @@ BNN_API int bnn_measure_pipe_rates(bnn_ctx *ctx, void *scratch, size_t scratch_b
 /* Name and tile shape of the tensor-core kernel this context launched last ("" if none yet): lets a benchmark label its
  * numbers with what actually ran.  The string is owned by the context and valid until its next call. */
 BNN_API const char *bnn_last_tensor_kernel(const bnn_ctx *ctx);
+/* The SM clock the tensor-core kernel launched last on this device really ran at, and how long its first CTA lived:
+ * the kernel's CTA 0 reads the SM cycle counter and the nanosecond timer when it starts and when it ends.  (This part
+ * holds tensor-heavy kernels well below the maximum SM clock that nvidia-smi samples around them.)  Synchronises the
+ * context's stream.  sm_mhz, microseconds: host pointers, written.  0.0 MHz if no such kernel has run. */
+BNN_API int bnn_last_tensor_kernel_clock(bnn_ctx *ctx, double *sm_mhz, double *microseconds);
 
 /* ---------------------------------------------------------------------------------------------
  * Context only (Section 4, Fig. 3): the paper's comparison point, a deliberately unoptimized matrix product of the

@@ -29,7 +29,7 @@ EXPORTS = (
     "bnn_expanded_bytes", "bnn_expand_signs", "bnn_baseline_gemm_f32", "bnn_convnet_workspace_bytes",
     "bnn_convnet_forward", "bnn_set_operand_bits", "bnn_expanded_ld_f4",
     "bnn_expanded_bytes_f4", "bnn_expand_signs_f4", "bnn_binary_dense_expanded", "bnn_set_wait_limit_ns",
-    "bnn_debug_drop_loads", "bnn_debug_ring_position", "bnn_set_conv_form", "bnn_measure_pipe_rates", "bnn_last_tensor_kernel", "bnn_set_conv_filter_repetition",
+    "bnn_debug_drop_loads", "bnn_debug_ring_position", "bnn_set_conv_form", "bnn_measure_pipe_rates", "bnn_last_tensor_kernel", "bnn_last_tensor_kernel_clock", "bnn_set_conv_filter_repetition",
     "bnn_filter_repetition_workspace_bytes", "bnn_filter_repetition_count",
 )
 
@@ -94,6 +94,7 @@ def lib() -> ctypes.CDLL:
         L.bnn_measure_pipe_rates.argtypes = [vp, vp, c_size_t, POINTER(c_double), POINTER(c_double), POINTER(c_double)]
         L.bnn_last_tensor_kernel.argtypes = [vp]
         L.bnn_last_tensor_kernel.restype = ctypes.c_char_p
+        L.bnn_last_tensor_kernel_clock.argtypes = [vp, POINTER(c_double), POINTER(c_double)]
         L.bnn_set_conv_filter_repetition.argtypes = [vp, c_int]
         L.bnn_filter_repetition_workspace_bytes.argtypes = [i64, i64]
         L.bnn_filter_repetition_workspace_bytes.restype = c_size_t
@@ -251,6 +252,12 @@ class Context:
 
     def last_tensor_kernel(self) -> str:
         return lib().bnn_last_tensor_kernel(self._h).decode()
+
+    def last_tensor_kernel_clock(self):
+        """(SM MHz inside the tensor-core kernel that ran last, microseconds its first CTA lived)."""
+        mhz, us = c_double(), c_double()
+        self._ck(lib().bnn_last_tensor_kernel_clock(self._h, ctypes.byref(mhz), ctypes.byref(us)), "bnn_last_tensor_kernel_clock")
+        return mhz.value, us.value
 
     def set_conv_filter_repetition(self, on: bool):
         self._ck(lib().bnn_set_conv_filter_repetition(self._h, int(on)), "bnn_set_conv_filter_repetition")

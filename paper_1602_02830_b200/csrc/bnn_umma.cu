@@ -69,14 +69,17 @@ constexpr int STAGES_MAX = 7;
 constexpr int B_STAGES_MAX = 18;                // weight stages of the halo-tile convolution kernel (9 taps x 2 channel slices resident)
 
 __device__ int g_umma_error;                    // 0 = fine; otherwise a code saying which wait gave up
+// SM clock count and wall-clock nanoseconds at the start [0, 1] and the end [2, 3] of CTA 0 of the tensor-engine kernel that
+// ran last: the clock the kernel really ran at (this part runs tensor-heavy kernels well below the maximum that
+// nvidia-smi reports around them).  Two register reads and two stores by one thread per kernel.
+__device__ long long g_umma_clock[4];
+#define BNN_CLK_REC(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) { g_umma_clock[2 * (i)] = clock64(); unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_umma_clock[2 * (i) + 1] = (long long)t_; } } while (0)
 #ifdef BNN_TRACE
 // Instrumented builds only: clock stamps of CTA 0, [role][tile][slot].
 __device__ long long g_trace[8 * 16 * 16];
 #define BNN_TR(role, tile, slot) do { if (blockIdx.x == 0 && (tile) < 16) g_trace[((role) * 16 + (tile)) * 16 + (slot)] = clock64(); } while (0)
-#define BNN_TR_CLK(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) { g_trace[7 * 256 + 2 * (i)] = clock64(); unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_trace[7 * 256 + 2 * (i) + 1] = (long long)t_; } } while (0)
 #else
 #define BNN_TR(role, tile, slot) do { } while (0)
-#define BNN_TR_CLK(i) do { } while (0)
 #endif
 
 struct UmmaArgs {
@@ -609,6 +612,7 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
     const int64_t tiles_m = (p.M + BM - 1) / BM;
     const int64_t tiles_n = (p.N + BN - 1) / BN;
     const int64_t ntiles = tiles_m * tiles_n;
+    BNN_CLK_REC(0);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 2 * STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
@@ -788,6 +792,7 @@ k_umma_i8(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUte
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    BNN_CLK_REC(1);
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
@@ -887,7 +892,7 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();                // 0 = leader of the pair
     const int64_t pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
-    BNN_TR_CLK(0);
+    BNN_CLK_REC(0);
     const int64_t tiles_m = (p.M + 2 * BM - 1) / (2 * BM);  // 256-row tiles
     const int64_t tiles_n = (p.N + BN - 1) / BN;
     const int64_t ntiles = tiles_m * tiles_n;
@@ -1070,7 +1075,7 @@ k_umma_i8_2sm(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    BNN_TR_CLK(1);
+    BNN_CLK_REC(1);
     cluster_sync_all();                                     // nobody leaves while the peer may still read its shared memory
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -1820,6 +1825,19 @@ extern "C" int bnn_debug_ring_position(uint32_t stage, uint32_t slots, uint32_t 
     *prev_parity = rc.reuses(slots) ? rc.prev_parity(slots) : 0u;
     rc.advance(step, slots);
     *next_barrier = rc.b; *next_parity = rc.parity();
+    return BNN_OK;
+}
+
+extern "C" int bnn_last_tensor_kernel_clock(bnn_ctx *ctx, double *sm_mhz, double *microseconds) {
+    if (!ctx || !sm_mhz || !microseconds) return BNN_ERR_INVALID_ARG;
+    bnn_device_guard guard(ctx);
+    if (!guard.ok) return BNN_ERR_CUDA;
+    BNN_CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream));
+    long long c[4] = {0, 0, 0, 0};
+    BNN_CUDA_TRY(ctx, cudaMemcpyFromSymbol(c, g_umma_clock, sizeof(c)));
+    const double ns = (double)(c[3] - c[1]);
+    *microseconds = ns / 1e3;
+    *sm_mhz = ns > 0 ? (double)(c[2] - c[0]) / ns * 1e3 : 0.0;
     return BNN_OK;
 }
 

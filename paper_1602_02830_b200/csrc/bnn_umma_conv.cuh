@@ -67,7 +67,7 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     const int64_t tiles_n = (p.N + BN - 1) / BN;
     const int64_t ntiles = tiles_m * tiles_n;
     const int groups = p.k_iters / 3;                    // slabs per tile: 3 horizontal taps x channel slices
-    BNN_TR_CLK(0);
+    BNN_CLK_REC(0);
     const int RB = p.b_resident ? NB : 3 * NB;           // barrier pairs of the weight stages
 
     if (threadIdx.x == 0) {
@@ -291,7 +291,7 @@ k_umma_conv(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    BNN_TR_CLK(1);
+    BNN_CLK_REC(1);
     if (PAIR) cluster_sync_all();                        // nobody leaves while the partner may still signal its barriers
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");

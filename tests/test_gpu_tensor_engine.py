@@ -360,3 +360,20 @@ def test_back_to_back_calls_without_synchronisation(ctx):
         assert (np.abs(got - want_s[k]) <= tol).all()
     ctx.set_workspace(None)
     del ws, ws2
+
+
+def test_last_tensor_kernel_clock_reports_a_plausible_sm_clock(ctx):
+    """The kernel's own record of the SM clock it ran at (cycle counter against the nanosecond timer in its first CTA)."""
+    M, N, K = 4096, 4096, 4096
+    A, B = wl.gemm_case(M, N, K, seed=5)
+    Ap = ctx.pack_signs(dev(A))
+    Bp = ctx.pack_signs(dev(B), pack_along=1)
+    ws = with_ws(ctx, ctx.gemm_workspace_bytes(M, N, K))
+    C = torch.empty(M, N, dtype=torch.int32, device="cuda")
+    for _ in range(3):
+        ctx.xnor_gemm(Ap, Bp, M, N, K, C=C)
+    mhz, us = ctx.last_tensor_kernel_clock()
+    assert 300.0 < mhz < 2300.0, mhz
+    assert 1.0 < us < 1000.0, us
+    ctx.set_workspace(None)
+    del ws
